@@ -1,0 +1,137 @@
+/*
+ * bcjr_b200 -- C ABI of the B200 (sm_100a) BCJR soft-quantisation library.
+ *
+ * One weight block w[0..n) is encoded by a path through a bitshift trellis with S = 2^Lb
+ * states: from state s the k input bits b lead to s' = ((s << k) | b) mod S, and state s
+ * emits the scalar codebook[s]  (paper Section 3.1).  All calls treat `num_blocks`
+ * independent blocks stored back to back (block i = W[i*n .. i*n+n), i.e. a row-major
+ * matrix whose rows are cut into consecutive blocks of n).
+ *
+ * Conventions shared by every entry point
+ *   - "device" pointers are CUDA device memory of the context's device, caller-owned; the
+ *     library never frees or reallocates them.  "host" pointers are ordinary host memory.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) unless stated otherwise.  The context owns its scratch memory; it
+ *     grows on demand (cudaMalloc on the calling thread) and is reused by later calls, so
+ *     two calls on one context must not overlap on the GPU.
+ *   - Every call returns a bcjr_status; nothing throws, aborts or traps.
+ *   - The first state is free and the last state is free (no tail biting); the
+ *     log-potential of state s at step t is  -(w_t - codebook[s])^2 / (2 T)  (Eq. 4).
+ */
+#ifndef BCJR_B200_H
+#define BCJR_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bcjr_ctx bcjr_ctx;
+
+typedef enum {
+    BCJR_OK = 0,
+    BCJR_EINVAL = -1,        /* bad argument (NULL pointer, dims out of range, T <= 0, ...) */
+    BCJR_ENOMEM = -2,        /* scratch allocation failed */
+    BCJR_ECUDA = -3,         /* a CUDA runtime call failed; see bcjr_last_cuda_error */
+    BCJR_ESTATE = -4,        /* bcjr_backward without a preceding bcjr_soft_quantize */
+    BCJR_EUNSUPPORTED = -5,  /* (Lb, k) combination the kernels do not cover */
+    BCJR_ETIMEOUT = -6,      /* a bounded device-side wait gave up (reported by bcjr_sync_status) */
+    BCJR_ENUMERIC = -7       /* non-finite values met on the device */
+} bcjr_status;
+
+/* Diagnostics gathered on the device since the last bcjr_sync_status. */
+typedef struct {
+    int32_t device_status;        /* BCJR_OK or the first device-side error */
+    float max_posterior_defect;   /* max over blocks and steps of |sum_s gamma_t(s) - 1| (Eq. 6) */
+    float max_logz_mismatch;      /* max |log Z (alpha side) - log Z (beta side)|, natural log */
+    int32_t kernel_launches;      /* kernels launched by this context since creation */
+    int32_t last_path;            /* 0 = generic kernels, 1 = cluster kernels used by the last call */
+} bcjr_diag;
+
+/* Limits: 1 <= k <= 4, k <= Lb <= 16, Lb - k <= 14, n >= 1, T > 0 and finite. */
+
+/* Creates a context bound to CUDA device `device_ordinal`.  *out is owned by the caller
+ * and released with bcjr_destroy.  Synchronous. */
+bcjr_status bcjr_create(bcjr_ctx **out, int device_ordinal);
+
+/* Frees the context and its scratch memory (synchronises the device first). */
+bcjr_status bcjr_destroy(bcjr_ctx *ctx);
+
+/* Tuning / test hooks.  name = "path": 0 auto, 1 force generic kernels, 2 force cluster
+ * kernels (EUNSUPPORTED at call time when they do not cover the shape);
+ * name = "max_ctas": cap on resident thread blocks (0 = fill the GPU). */
+bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value);
+
+/*
+ * Soft codeword (Eq. 3 / Eq. 7): soft[t] = sum_s codebook[s] * p_T(s_t = s | w), with the
+ * marginals from the temperature-T forward-backward recursions of Eq. 5-6 carried in the
+ * log domain.
+ *   W         device in   [num_blocks * n] float32
+ *   codebook  device in   [2^Lb] float32
+ *   soft      device out  [num_blocks * n] float32
+ *   logZ      device out  [num_blocks] float32, natural log of Z_T per block (sum over legal
+ *                         paths of exp(-E/T), no prior constant); may be NULL
+ * Saves, for bcjr_backward: the W and codebook POINTERS (borrowed: keep them valid and
+ * unchanged until the matching bcjr_backward has been enqueued), the dims, T, and a private
+ * copy of `soft`.
+ */
+bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codebook,
+                               int Lb, int k, int n, int64_t num_blocks, float T,
+                               float *soft, float *logZ, void *cuda_stream);
+
+/*
+ * Backward pass of the autograd node of Section 3.5 for l = sum(grad_soft * soft), T held
+ * constant: the exact derivative of Eq. 7 through both recursions.
+ *   grad_soft      device in   [num_blocks * n]
+ *   grad_W         device out  [num_blocks * n]
+ *   grad_codebook  device out  [2^Lb], OVERWRITTEN with the sum over all blocks (direct term
+ *                  through the emitted value plus the term through the energies); may be NULL
+ * Uses the state saved by the last bcjr_soft_quantize on this context; BCJR_ESTATE if none.
+ */
+bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft,
+                          float *grad_W, float *grad_codebook, void *cuda_stream);
+
+/*
+ * Viterbi hard code (Section 3.2): the legal path minimising sum_t (w_t - codebook[s_t])^2.
+ * Path metrics are accumulated in IEEE double, d = (double)w - (double)c, m += d*d, without
+ * fused multiply-add; ties go to the lowest predecessor and the lowest final state.
+ *   path_bits  device out  [num_blocks * path_stride_bytes]; per block Lb + k(n-1) bits, most
+ *              significant first: s_1 in Lb bits, then the k input bits of every later step;
+ *              bit i is stored in byte i>>3 at bit position 7-(i&7); padding bits are zero.
+ *              path_stride_bytes >= ceil((Lb + k(n-1)) / 8).  May be NULL.
+ *   states     device out  [num_blocks * n] uint16 state sequence; may be NULL
+ *   hard       device out  [num_blocks * n] float32, exact copies of codebook entries; may be NULL
+ */
+bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook,
+                         int Lb, int k, int n, int64_t num_blocks,
+                         uint8_t *path_bits, int64_t path_stride_bytes,
+                         uint16_t *states, float *hard, void *cuda_stream);
+
+/*
+ * One training-style step with HOST buffers (pinned or pageable): copies W, codebook and
+ * grad_soft to the device, runs bcjr_soft_quantize and bcjr_backward, and copies soft,
+ * grad_W and grad_codebook back, all on `cuda_stream`; returns after the stream has been
+ * synchronised.  Any of soft / grad_W / grad_codebook may be NULL (not copied back).
+ */
+bcjr_status bcjr_step_host(bcjr_ctx *ctx, const float *W_host, const float *codebook_host,
+                           const float *grad_soft_host, int Lb, int k, int n, int64_t num_blocks,
+                           float T, float *soft_host, float *grad_W_host, float *grad_codebook_host,
+                           void *cuda_stream);
+
+/* Synchronises `cuda_stream`, then reports and clears the device-side status and
+ * diagnostics.  Returns the device status (BCJR_OK when clean). */
+bcjr_status bcjr_sync_status(bcjr_ctx *ctx, void *cuda_stream, bcjr_diag *out);
+
+/* Scratch bytes currently held by the context. */
+int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx);
+
+/* Text of the last CUDA error seen by this context ("" if none). Owned by the context. */
+const char *bcjr_last_cuda_error(const bcjr_ctx *ctx);
+
+const char *bcjr_status_string(bcjr_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCJR_B200_H */

@@ -1,0 +1,193 @@
+"""Thin ctypes binding of the C ABI in include/bcjr_b200.h.
+
+Argument marshalling only: every step of the method runs in the CUDA kernels behind the
+shared library.  torch is used for device memory and streams.  There is no CPU fallback:
+a missing library raises at load time, a failing call raises BcjrError.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libbcjr_b200.so"
+
+EXPORTS = ["bcjr_create", "bcjr_destroy", "bcjr_set_option", "bcjr_soft_quantize", "bcjr_backward",
+           "viterbi_hard", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
+           "bcjr_last_cuda_error", "bcjr_status_string"]
+
+
+class BcjrError(RuntimeError):
+    def __init__(self, code, where, detail=""):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code}){(' - ' + detail) if detail else ''}")
+
+
+class Diag(ctypes.Structure):
+    _fields_ = [("device_status", ctypes.c_int32), ("max_posterior_defect", ctypes.c_float),
+                ("max_logz_mismatch", ctypes.c_float), ("kernel_launches", ctypes.c_int32),
+                ("last_path", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the in-tree CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB_PATH.exists():
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2605_10655_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(str(LIB_PATH))
+    vp, i, i64, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
+    lib.bcjr_create.restype = i; lib.bcjr_create.argtypes = [ctypes.POINTER(vp), i]
+    lib.bcjr_destroy.restype = i; lib.bcjr_destroy.argtypes = [vp]
+    lib.bcjr_set_option.restype = i; lib.bcjr_set_option.argtypes = [vp, ctypes.c_char_p, i64]
+    lib.bcjr_soft_quantize.restype = i
+    lib.bcjr_soft_quantize.argtypes = [vp, vp, vp, i, i, i, i64, f, vp, vp, vp]
+    lib.bcjr_backward.restype = i; lib.bcjr_backward.argtypes = [vp, vp, vp, vp, vp]
+    lib.viterbi_hard.restype = i; lib.viterbi_hard.argtypes = [vp, vp, vp, i, i, i, i64, vp, i64, vp, vp, vp]
+    lib.bcjr_step_host.restype = i
+    lib.bcjr_step_host.argtypes = [vp, vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
+    lib.bcjr_sync_status.restype = i; lib.bcjr_sync_status.argtypes = [vp, vp, ctypes.POINTER(Diag)]
+    lib.bcjr_workspace_bytes.restype = i64; lib.bcjr_workspace_bytes.argtypes = [vp]
+    lib.bcjr_last_cuda_error.restype = ctypes.c_char_p; lib.bcjr_last_cuda_error.argtypes = [vp]
+    lib.bcjr_status_string.restype = ctypes.c_char_p; lib.bcjr_status_string.argtypes = [i]
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().bcjr_status_string(int(code)).decode()
+
+
+def path_bytes(Lb: int, k: int, n: int) -> int:
+    return (Lb + k * (n - 1) + 7) // 8
+
+
+def _stream_ptr(stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dev(t, dtype, numel=None, name="tensor"):
+    import torch
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    if numel is not None and t.numel() != numel:
+        raise ValueError(f"{name}: expected {numel} elements, got {t.numel()}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+class Context:
+    """Owns one bcjr_ctx (scratch memory + the state saved between forward and backward)."""
+
+    def __init__(self, device: int = 0):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        rc = self._lib.bcjr_create(ctypes.byref(self._h), int(device))
+        if rc != 0:
+            raise BcjrError(rc, "bcjr_create")
+        self.device = int(device)
+        self._saved = None
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.bcjr_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc, where):
+        if rc != 0:
+            raise BcjrError(rc, where, self._lib.bcjr_last_cuda_error(self._h).decode())
+
+    def set_option(self, name: str, value: int):
+        self._check(self._lib.bcjr_set_option(self._h, name.encode(), int(value)), "bcjr_set_option")
+
+    def bcjr_soft_quantize(self, W, codebook, Lb, k, n, T, soft=None, logZ=None, stream=None):
+        """W: [num_blocks*n] (any shape with that many elements) float32 CUDA.  Returns (soft, logZ)."""
+        import torch
+        B = W.numel() // n
+        if B * n != W.numel():
+            raise ValueError("W.numel() must be a multiple of n")
+        if soft is None:
+            soft = torch.empty_like(W)
+        if logZ is None:
+            logZ = torch.empty(B, dtype=torch.float32, device=W.device)
+        rc = self._lib.bcjr_soft_quantize(self._h, _dev(W, torch.float32, name="W"),
+                                          _dev(codebook, torch.float32, 1 << Lb, "codebook"), Lb, k, n, B,
+                                          float(T), _dev(soft, torch.float32, B * n, "soft"),
+                                          _dev(logZ, torch.float32, B, "logZ"), _stream_ptr(stream))
+        self._check(rc, "bcjr_soft_quantize")
+        self._saved = (W, codebook, Lb, B * n)       # keep the borrowed tensors alive
+        return soft, logZ
+
+    def bcjr_backward(self, grad_soft, grad_W=None, grad_codebook=None, stream=None):
+        import torch
+        if self._saved is None:
+            raise BcjrError(-4, "bcjr_backward")
+        W, codebook, Lb, numel = self._saved
+        if grad_W is None:
+            grad_W = torch.empty_like(W)
+        if grad_codebook is None:
+            grad_codebook = torch.empty(1 << Lb, dtype=torch.float32, device=W.device)
+        rc = self._lib.bcjr_backward(self._h, _dev(grad_soft, torch.float32, numel, "grad_soft"),
+                                     _dev(grad_W, torch.float32, numel, "grad_W"),
+                                     _dev(grad_codebook, torch.float32, 1 << Lb, "grad_codebook"),
+                                     _stream_ptr(stream))
+        self._check(rc, "bcjr_backward")
+        return grad_W, grad_codebook
+
+    def viterbi_hard(self, W, codebook, Lb, k, n, want_states=True, want_hard=True, stream=None):
+        """Returns (path_bits [B, nbytes] uint8, states [B, n] int16-as-uint16 bits or None, hard [B, n] or None)."""
+        import torch
+        B = W.numel() // n
+        nb = path_bytes(Lb, k, n)
+        bits = torch.empty((B, nb), dtype=torch.uint8, device=W.device)
+        states = torch.empty((B, n), dtype=torch.int16, device=W.device) if want_states else None
+        hard = torch.empty((B, n), dtype=torch.float32, device=W.device) if want_hard else None
+        rc = self._lib.viterbi_hard(self._h, _dev(W, torch.float32, name="W"),
+                                    _dev(codebook, torch.float32, 1 << Lb, "codebook"), Lb, k, n, B,
+                                    ctypes.c_void_p(bits.data_ptr()), nb,
+                                    ctypes.c_void_p(states.data_ptr()) if want_states else None,
+                                    ctypes.c_void_p(hard.data_ptr()) if want_hard else None, _stream_ptr(stream))
+        self._check(rc, "viterbi_hard")
+        return bits, states, hard
+
+    def bcjr_step_host(self, W, codebook, grad_soft, Lb, k, n, T, soft=None, grad_W=None, grad_codebook=None,
+                       stream=None):
+        """Host (CPU, ideally pinned) float32 tensors in, host tensors out; synchronous."""
+        import torch
+
+        def hp(t, name):
+            if t is None:
+                return None
+            if t.is_cuda or not t.is_contiguous() or t.dtype != torch.float32:
+                raise TypeError(f"{name}: expected a contiguous float32 CPU tensor")
+            return ctypes.c_void_p(t.data_ptr())
+        B = W.numel() // n
+        rc = self._lib.bcjr_step_host(self._h, hp(W, "W"), hp(codebook, "codebook"), hp(grad_soft, "grad_soft"),
+                                      Lb, k, n, B, float(T), hp(soft, "soft"), hp(grad_W, "grad_W"),
+                                      hp(grad_codebook, "grad_codebook"), _stream_ptr(stream))
+        self._check(rc, "bcjr_step_host")
+        self._saved = None
+
+    def sync_status(self, stream=None, check=True) -> Diag:
+        d = Diag()
+        rc = self._lib.bcjr_sync_status(self._h, _stream_ptr(stream), ctypes.byref(d))
+        if check:
+            self._check(rc, "bcjr_sync_status")
+        return d
+
+    def workspace_bytes(self) -> int:
+        return int(self._lib.bcjr_workspace_bytes(self._h))

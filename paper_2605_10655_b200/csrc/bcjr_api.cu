@@ -1,0 +1,444 @@
+// Host side of the C ABI declared in include/bcjr_b200.h: argument checks, scratch
+// management, kernel selection and launches.  No compute happens on the host.
+#include "../../include/bcjr_b200.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "bcjr_common.cuh"
+#include "bcjr_generic.cuh"
+#ifndef BCJR_NO_CLUSTER
+#include "bcjr_cluster.cuh"
+#endif
+
+using namespace bcjr;
+
+namespace {
+
+struct Buffer {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace
+
+struct bcjr_ctx {
+    int device = 0;
+    int num_sms = 0;
+    int max_smem_optin = 0;
+    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, staging[6];
+    DeviceDiag *diag = nullptr;
+    // saved by bcjr_soft_quantize for bcjr_backward
+    bool have_fwd = false;
+    const float *W = nullptr, *cb = nullptr;
+    int Lb = 0, k = 0, n = 0;
+    int64_t B = 0;
+    float T = 0.f;
+    // options
+    int opt_path = 0;
+    int opt_max_ctas = 0;
+    int launches = 0;
+    int last_path = 0;
+    std::string cuda_error;
+};
+
+namespace {
+
+bcjr_status cuda_fail(bcjr_ctx *ctx, cudaError_t e, const char *what)
+{
+    ctx->cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? BCJR_ENOMEM : BCJR_ECUDA;
+}
+
+#define CU(call)                                                        \
+    do {                                                                \
+        cudaError_t e__ = (call);                                       \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call);      \
+    } while (0)
+
+bcjr_status ensure(bcjr_ctx *ctx, Buffer &b, size_t bytes)
+{
+    if (bytes <= b.bytes) return BCJR_OK;
+    if (b.ptr) { CU(cudaFree(b.ptr)); b.ptr = nullptr; b.bytes = 0; }
+    CU(cudaMalloc(&b.ptr, bytes));
+    b.bytes = bytes;
+    return BCJR_OK;
+}
+
+bcjr_status check_dims(int Lb, int k, int n, int64_t B)
+{
+    if (k < 1 || k > 4 || Lb < k || Lb > 16 || n < 1 || B < 0) return BCJR_EINVAL;
+    if (Lb - k > 14) return BCJR_EUNSUPPORTED;
+    if ((int64_t)n * (int64_t)(1 << (Lb - k)) > ((int64_t)1 << 31)) return BCJR_EUNSUPPORTED;
+    return BCJR_OK;
+}
+
+int generic_threads(int Q)
+{
+    int t = (Q + 31) / 32 * 32;
+    if (t < 32) t = 32;
+    return t > GEN_MAX_THREADS ? GEN_MAX_THREADS : t;
+}
+
+struct GenericLaunch {
+    int threads, grid;
+    size_t smem;
+    bool msg_global;
+};
+
+template <typename Kern>
+bcjr_status plan_generic(bcjr_ctx *ctx, Kern kern, int Q, size_t msg_bytes, int64_t B, GenericLaunch *out)
+{
+    out->threads = generic_threads(Q);
+    const size_t header = GEN_SMEM_HEADER * sizeof(float);
+    const size_t budget = (size_t)ctx->max_smem_optin - 1024;
+    out->msg_global = header + msg_bytes > budget;
+    out->smem = out->msg_global ? header : header + msg_bytes;
+    CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)out->smem));
+    int occ = 0;
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, out->threads, out->smem));
+    if (occ < 1) occ = 1;
+    int64_t grid = (int64_t)occ * ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    if (grid > B) grid = B;
+    if (grid < 1) grid = 1;
+    out->grid = (int)grid;
+    return BCJR_OK;
+}
+
+template <int KB>
+bcjr_status launch_fwd_generic(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    const int Q = 1 << (p.Lb - KB);
+    GenericLaunch gl;
+    bcjr_status rc = plan_generic(ctx, fwd_generic_kernel<KB>, Q, (size_t)2 * Q * 4, p.B, &gl);
+    if (rc) return rc;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)gl.grid * p.n * Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, (size_t)gl.grid * (p.n + 2) * 4))) return rc;
+    if (gl.msg_global && (rc = ensure(ctx, ctx->msg, (size_t)gl.grid * 2 * Q * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    p.msg = gl.msg_global ? (float *)ctx->msg.ptr : nullptr;
+    fwd_generic_kernel<KB><<<gl.grid, gl.threads, gl.smem, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+template <int KB>
+bcjr_status launch_bwd_generic(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    const int S = 1 << p.Lb, Q = S >> KB;
+    GenericLaunch gl;
+    bcjr_status rc = plan_generic(ctx, bwd_generic_kernel<KB>, Q, (size_t)4 * Q * 4, p.B, &gl);
+    if (rc) return rc;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)gl.grid * 2 * p.n * Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, (size_t)gl.grid * (p.n + 2) * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->gc_part, (size_t)gl.grid * S * 4))) return rc;
+    if (gl.msg_global && (rc = ensure(ctx, ctx->msg, (size_t)gl.grid * 4 * Q * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    p.gc_part = (float *)ctx->gc_part.ptr;
+    p.msg = gl.msg_global ? (float *)ctx->msg.ptr : nullptr;
+    bwd_generic_kernel<KB><<<gl.grid, gl.threads, gl.smem, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    if (grad_codebook) {
+        reduce_gc_kernel<<<(S + 255) / 256, 256, 0, st>>>(p.gc_part, gl.grid, S, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
+template <int KB>
+bcjr_status launch_vit_generic(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
+{
+    const int Q = 1 << (p.Lb - KB);
+    GenericLaunch gl;
+    bcjr_status rc = plan_generic(ctx, viterbi_generic_kernel<KB>, Q, (size_t)2 * Q * 8, p.B, &gl);
+    if (rc) return rc;
+    if ((rc = ensure(ctx, ctx->bp, (size_t)gl.grid * p.n * Q))) return rc;
+    if ((rc = ensure(ctx, ctx->path_ws, (size_t)gl.grid * p.n * 4))) return rc;
+    if (gl.msg_global && (rc = ensure(ctx, ctx->msg, (size_t)gl.grid * 2 * Q * 8))) return rc;
+    p.bp = (uint8_t *)ctx->bp.ptr;
+    p.path_ws = (int *)ctx->path_ws.ptr;
+    p.msg = gl.msg_global ? (double *)ctx->msg.ptr : nullptr;
+    viterbi_generic_kernel<KB><<<gl.grid, gl.threads, gl.smem, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess && (prev == dev || cudaSetDevice(dev) == cudaSuccess)) ok = true;
+    }
+    ~DeviceGuard() { if (ok && prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+bcjr_status bcjr_create(bcjr_ctx **out, int device_ordinal)
+{
+    if (!out) return BCJR_EINVAL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device_ordinal < 0 || device_ordinal >= count) {
+        cudaGetLastError();
+        return BCJR_ECUDA;
+    }
+    bcjr_ctx *ctx = new (std::nothrow) bcjr_ctx();
+    if (!ctx) return BCJR_ENOMEM;
+    ctx->device = device_ordinal;
+    DeviceGuard guard(device_ordinal);
+    cudaDeviceProp prop;
+    if (!guard.ok || cudaGetDeviceProperties(&prop, device_ordinal) != cudaSuccess ||
+        cudaMalloc((void **)&ctx->diag, sizeof(DeviceDiag)) != cudaSuccess ||
+        cudaMemset(ctx->diag, 0, sizeof(DeviceDiag)) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return BCJR_ECUDA;
+    }
+    ctx->num_sms = prop.multiProcessorCount;
+    ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    *out = ctx;
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_destroy(bcjr_ctx *ctx)
+{
+    if (!ctx) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp, &ctx->path_ws,
+                     &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
+                     &ctx->staging[5]};
+    for (Buffer *b : all)
+        if (b->ptr) cudaFree(b->ptr);
+    if (ctx->diag) cudaFree(ctx->diag);
+    cudaGetLastError();
+    delete ctx;
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
+{
+    if (!ctx || !name) return BCJR_EINVAL;
+    if (!strcmp(name, "path")) {
+        if (value < 0 || value > 2) return BCJR_EINVAL;
+        ctx->opt_path = (int)value;
+        return BCJR_OK;
+    }
+    if (!strcmp(name, "max_ctas")) {
+        if (value < 0 || value > (1 << 20)) return BCJR_EINVAL;
+        ctx->opt_max_ctas = (int)value;
+        return BCJR_OK;
+    }
+    return BCJR_EINVAL;
+}
+
+bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codebook, int Lb, int k, int n,
+                               int64_t num_blocks, float T, float *soft, float *logZ, void *cuda_stream)
+{
+    if (!ctx) return BCJR_EINVAL;
+    if (!(T > 0.f) || !std::isfinite(T)) return BCJR_EINVAL;
+    bcjr_status rc = check_dims(Lb, k, n, num_blocks);
+    if (rc) return rc;
+    if (num_blocks > 0 && (!W || !codebook || !soft)) return BCJR_EINVAL;   // empty input: pointers unused
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    ctx->have_fwd = false;
+    if (num_blocks == 0) {
+        ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = 0; ctx->T = T;
+        ctx->have_fwd = true;
+        return BCJR_OK;
+    }
+    if ((rc = ensure(ctx, ctx->soft_copy, (size_t)num_blocks * n * 4))) return rc;
+    FwdParams p{};
+    p.W = W; p.cb = codebook; p.soft = soft; p.soft_copy = (float *)ctx->soft_copy.ptr; p.logZ = logZ;
+    p.diag = ctx->diag; p.B = num_blocks; p.Lb = Lb; p.n = n;
+    p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)T));
+    bool use_cluster = false;
+#ifndef BCJR_NO_CLUSTER
+    use_cluster = ctx->opt_path != 1 && cluster_supported(Lb, k);
+    if (ctx->opt_path == 2 && !use_cluster) return BCJR_EUNSUPPORTED;
+    if (use_cluster) rc = launch_fwd_cluster(ctx, p, k, st);
+#else
+    if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
+#endif
+    if (!use_cluster) {
+        switch (k) {
+            case 1: rc = launch_fwd_generic<1>(ctx, p, st); break;
+            case 2: rc = launch_fwd_generic<2>(ctx, p, st); break;
+            case 3: rc = launch_fwd_generic<3>(ctx, p, st); break;
+            default: rc = launch_fwd_generic<4>(ctx, p, st); break;
+        }
+    }
+    if (rc) return rc;
+    ctx->last_path = use_cluster ? 1 : 0;
+    ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = num_blocks; ctx->T = T;
+    ctx->have_fwd = true;
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, float *grad_codebook,
+                          void *cuda_stream)
+{
+    if (!ctx) return BCJR_EINVAL;
+    if (!ctx->have_fwd) return BCJR_ESTATE;
+    if (ctx->B > 0 && (!grad_soft || !grad_W)) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int S = 1 << ctx->Lb;
+    if (ctx->B == 0) {
+        if (grad_codebook) CU(cudaMemsetAsync(grad_codebook, 0, (size_t)S * 4, st));
+        return BCJR_OK;
+    }
+    BwdParams p{};
+    p.W = ctx->W; p.cb = ctx->cb; p.g = grad_soft; p.soft = (const float *)ctx->soft_copy.ptr; p.gW = grad_W;
+    p.diag = ctx->diag; p.B = ctx->B; p.Lb = ctx->Lb; p.n = ctx->n;
+    p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)ctx->T));
+    p.invT = (float)(1.0 / (double)ctx->T);
+    bcjr_status rc = BCJR_OK;
+    bool use_cluster = false;
+#ifndef BCJR_NO_CLUSTER
+    use_cluster = ctx->opt_path != 1 && cluster_supported(ctx->Lb, ctx->k);
+    if (ctx->opt_path == 2 && !use_cluster) return BCJR_EUNSUPPORTED;
+    if (use_cluster) rc = launch_bwd_cluster(ctx, p, ctx->k, grad_codebook, st);
+#else
+    if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
+#endif
+    if (!use_cluster) {
+        switch (ctx->k) {
+            case 1: rc = launch_bwd_generic<1>(ctx, p, grad_codebook, st); break;
+            case 2: rc = launch_bwd_generic<2>(ctx, p, grad_codebook, st); break;
+            case 3: rc = launch_bwd_generic<3>(ctx, p, grad_codebook, st); break;
+            default: rc = launch_bwd_generic<4>(ctx, p, grad_codebook, st); break;
+        }
+    }
+    if (rc) return rc;
+    ctx->last_path = use_cluster ? 1 : 0;
+    return BCJR_OK;
+}
+
+bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook, int Lb, int k, int n,
+                         int64_t num_blocks, uint8_t *path_bits, int64_t path_stride_bytes, uint16_t *states,
+                         float *hard, void *cuda_stream)
+{
+    if (!ctx) return BCJR_EINVAL;
+    bcjr_status rc = check_dims(Lb, k, n, num_blocks);
+    if (rc) return rc;
+    if (num_blocks > 0 && (!W || !codebook)) return BCJR_EINVAL;
+    const int64_t nbits = Lb + (int64_t)k * (n - 1);
+    if (path_bits && path_stride_bytes < (nbits + 7) / 8) return BCJR_EINVAL;
+    if (num_blocks == 0) return BCJR_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    VitParams p{};
+    p.W = W; p.cb = codebook; p.path_bits = path_bits; p.path_stride = path_stride_bytes;
+    p.states = states; p.hard = hard; p.B = num_blocks; p.Lb = Lb; p.n = n;
+    switch (k) {
+        case 1: rc = launch_vit_generic<1>(ctx, p, st); break;
+        case 2: rc = launch_vit_generic<2>(ctx, p, st); break;
+        case 3: rc = launch_vit_generic<3>(ctx, p, st); break;
+        default: rc = launch_vit_generic<4>(ctx, p, st); break;
+    }
+    if (rc) return rc;
+    ctx->last_path = 0;
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_step_host(bcjr_ctx *ctx, const float *W_host, const float *codebook_host,
+                           const float *grad_soft_host, int Lb, int k, int n, int64_t num_blocks, float T,
+                           float *soft_host, float *grad_W_host, float *grad_codebook_host, void *cuda_stream)
+{
+    if (!ctx || !W_host || !codebook_host || !grad_soft_host) return BCJR_EINVAL;
+    bcjr_status rc = check_dims(Lb, k, n, num_blocks);
+    if (rc) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t wbytes = (size_t)num_blocks * n * 4, cbytes = ((size_t)1 << Lb) * 4;
+    const size_t sizes[6] = {wbytes, cbytes, wbytes, wbytes, wbytes, cbytes};
+    for (int i = 0; i < 6; ++i)
+        if ((rc = ensure(ctx, ctx->staging[i], sizes[i] ? sizes[i] : 4))) return rc;
+    float *dW = (float *)ctx->staging[0].ptr, *dcb = (float *)ctx->staging[1].ptr;
+    float *dg = (float *)ctx->staging[2].ptr, *dsoft = (float *)ctx->staging[3].ptr;
+    float *dgW = (float *)ctx->staging[4].ptr, *dgc = (float *)ctx->staging[5].ptr;
+    if (wbytes) CU(cudaMemcpyAsync(dW, W_host, wbytes, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(dcb, codebook_host, cbytes, cudaMemcpyHostToDevice, st));
+    if (wbytes) CU(cudaMemcpyAsync(dg, grad_soft_host, wbytes, cudaMemcpyHostToDevice, st));
+    if ((rc = bcjr_soft_quantize(ctx, dW, dcb, Lb, k, n, num_blocks, T, dsoft, nullptr, cuda_stream))) return rc;
+    if ((rc = bcjr_backward(ctx, dg, dgW, dgc, cuda_stream))) return rc;
+    if (soft_host && wbytes) CU(cudaMemcpyAsync(soft_host, dsoft, wbytes, cudaMemcpyDeviceToHost, st));
+    if (grad_W_host && wbytes) CU(cudaMemcpyAsync(grad_W_host, dgW, wbytes, cudaMemcpyDeviceToHost, st));
+    if (grad_codebook_host) CU(cudaMemcpyAsync(grad_codebook_host, dgc, cbytes, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_sync_status(bcjr_ctx *ctx, void *cuda_stream, bcjr_diag *out)
+{
+    if (!ctx) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CU(cudaStreamSynchronize(st));
+    DeviceDiag h;
+    CU(cudaMemcpy(&h, ctx->diag, sizeof(h), cudaMemcpyDeviceToHost));
+    CU(cudaMemset(ctx->diag, 0, sizeof(DeviceDiag)));
+    if (out) {
+        out->device_status = h.status;
+        float f;
+        memcpy(&f, &h.max_defect, 4);
+        out->max_posterior_defect = f;
+        memcpy(&f, &h.max_logz_gap, 4);
+        out->max_logz_mismatch = f * 0.6931472f;
+        out->kernel_launches = ctx->launches;
+        out->last_path = ctx->last_path;
+    }
+    return (bcjr_status)h.status;
+}
+
+int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx)
+{
+    if (!ctx) return 0;
+    const Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp,
+                           &ctx->path_ws, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
+                           &ctx->staging[4], &ctx->staging[5]};
+    int64_t tot = 0;
+    for (const Buffer *b : all) tot += (int64_t)b->bytes;
+    return tot;
+}
+
+const char *bcjr_last_cuda_error(const bcjr_ctx *ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
+
+const char *bcjr_status_string(bcjr_status s)
+{
+    switch (s) {
+        case BCJR_OK: return "ok";
+        case BCJR_EINVAL: return "invalid argument";
+        case BCJR_ENOMEM: return "out of device memory";
+        case BCJR_ECUDA: return "CUDA runtime error";
+        case BCJR_ESTATE: return "bcjr_backward called without a saved forward pass";
+        case BCJR_EUNSUPPORTED: return "unsupported (Lb, k, n) combination";
+        case BCJR_ETIMEOUT: return "device-side wait timed out";
+        case BCJR_ENUMERIC: return "non-finite values on the device";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,106 @@
+// Shared device helpers and parameter blocks of the BCJR kernels (sm_100a).
+//
+// Notation (paper Section 3, with the state vector compressed by the trellis structure):
+//   S = 2^Lb states, K = 2^k branches, Q = S / K groups.
+//   The K states q*K + b (b < K) share one predecessor set {q + j*Q : j < K}; so
+//     log alpha_t(s) = e_t(s) + L_t(s >> k),   L_{t+1}(q) = LSE_j [ L_t((q + jQ) >> k) + e_t(q + jQ) ]
+//     log beta_t(s)  = M_t(s & (Q-1)),         M_{t-1}(q) = LSE_b [ M_t((qK + b) & (Q-1)) + e_t(qK + b) ]
+//   with e_t(s) = -(w_t - c[s])^2 / (2T)  (Eq. 4-5).  Only L and M (Q values each) are carried.
+//   All kernels work in base 2: every log-domain value is a log2, lam2 = log2(e) / (2T).
+//   Each step an integer "gauge" offset is subtracted from L (and M) so that magnitudes stay
+//   small; the integer sums O_t, P_t are exact, so log Z and the posterior normaliser
+//   D_t = log2 Z - O_t - P_t are recovered without loss.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bcjr {
+
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2f(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcpf(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Device-side status / diagnostics block (one per context, in global memory).
+struct DeviceDiag {
+    int status;                  // first non-zero bcjr_status raised on the device
+    unsigned int max_defect;     // float bits of max |sum gamma - 1|
+    unsigned int max_logz_gap;   // float bits of max |log2 Z(alpha) - log2 Z(beta)|
+    int pad;
+};
+
+__device__ __forceinline__ void diag_max(unsigned int *slot, float v) {
+    // v >= 0: float ordering equals unsigned ordering of the bit patterns
+    if (!(v >= 0.0f)) v = __int_as_float(0x7f800000);   // NaN or negative -> +inf so it is seen
+    atomicMax(slot, __float_as_uint(v));
+}
+
+struct FwdParams {
+    const float *W;          // [B*n]
+    const float *cb;         // [S]
+    float *soft;             // [B*n]
+    float *soft_copy;        // [B*n] context-owned copy, read again by the backward pass
+    float *logZ;             // [B] or null (natural log)
+    float *hist;             // [grid][n*Q] gauge-fixed L_t, t = 1..n
+    int *stepO;              // [grid][n+2] cumulative integer offsets O_t
+    float *msg;              // [grid][2*Q] message ping-pong in global memory, or null (shared)
+    DeviceDiag *diag;
+    int64_t B;
+    int Lb, n;
+    float lam2;              // log2(e) / (2T)
+};
+
+struct BwdParams {
+    const float *W;
+    const float *cb;
+    const float *g;          // upstream gradient [B*n]
+    const float *soft;       // saved soft codeword [B*n]
+    float *gW;               // [B*n]
+    float *gc_part;          // [grid][S] per-CTA partial of grad_codebook
+    float *hist;             // [grid][2*n*Q]: L_t then Atilde_t
+    int *stepO;
+    float *msg;              // [grid][4*Q] or null
+    DeviceDiag *diag;
+    int64_t B;
+    int Lb, n;
+    float lam2;
+    float invT;              // 1/T
+};
+
+struct VitParams {
+    const float *W;
+    const float *cb;
+    uint8_t *path_bits;      // or null
+    int64_t path_stride;
+    uint16_t *states;        // or null
+    float *hard;             // or null
+    uint8_t *bp;             // [grid][n*Q] best branch per group per step
+    double *msg;             // [grid][2*Q] or null (shared)
+    int *path_ws;            // [grid][n] state sequence scratch
+    int64_t B;
+    int Lb, n;
+};
+
+}  // namespace bcjr

@@ -1,0 +1,45 @@
+"""The C-ABI library loads without a GPU and exports every symbol the public header declares."""
+import ctypes
+import re
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parents[1]
+
+
+def _declared_functions():
+    names = []
+    for h in sorted((ROOT / "include").glob("*.h")):
+        text = re.sub(r"/\*.*?\*/", "", h.read_text(), flags=re.S)
+        names += re.findall(r"\b([A-Za-z_][A-Za-z0-9_]*)\s*\([^;{]*\)\s*;", text)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2605_10655_b200 import binding, build
+    build.build()
+    lib = ctypes.CDLL(str(binding.LIB_PATH))
+    declared = _declared_functions()
+    assert {"bcjr_soft_quantize", "bcjr_backward", "viterbi_hard", "bcjr_create", "bcjr_destroy"} <= set(declared)
+    for name in declared:
+        assert hasattr(lib, name), f"{name} is declared in include/ but not exported"
+    assert set(binding.EXPORTS) == set(declared)
+
+
+def test_status_strings_and_host_side_argument_checks():
+    from paper_2605_10655_b200 import binding
+    lib = binding.load_library()
+    assert binding.status_string(0) == "ok"
+    assert "unsupported" in binding.status_string(-5)
+    # NULL context / NULL pointers are rejected on the host before any CUDA call
+    assert lib.bcjr_soft_quantize(None, None, None, 8, 2, 64, 1, 0.5, None, None, None) == -1
+    assert lib.bcjr_backward(None, None, None, None, None) == -1
+    assert lib.viterbi_hard(None, None, None, 8, 2, 64, 1, None, 0, None, None, None) == -1
+    assert lib.bcjr_destroy(None) == -1
+    assert binding.path_bytes(16, 2, 256) == 66 and binding.path_bytes(16, 3, 256) == 98
+
+
+def test_no_product_module_imports_the_oracle():
+    pkg = ROOT / "paper_2605_10655_b200"
+    for f in list(pkg.rglob("*.py")) + list(pkg.rglob("*.cu")) + list(pkg.rglob("*.cuh")):
+        text = f.read_text()
+        assert "import oracle" not in text and "from oracle" not in text and "bcjr_oracle" not in text, f

@@ -1,0 +1,185 @@
+"""GPU parity: the CUDA path (called through the C ABI) against the float64 CPU oracle,
+element by element, on the same seeded inputs."""
+import json
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import bruteforce as bf
+import oracle
+import parity
+from paper_2605_10655_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+GENERIC, CLUSTER = 1, 2
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2605_10655_b200 import Context
+    c = Context(0)
+    yield c
+    c.close()
+
+
+def _rand(n, Lb, B, seed, student=False):
+    rng = np.random.default_rng(seed)
+    c = rng.standard_normal(1 << Lb).astype(np.float32)
+    W = (rng.standard_t(4, size=(B, n)) / np.sqrt(2.0)).astype(np.float32) if student \
+        else rng.standard_normal((B, n)).astype(np.float32)
+    g = rng.standard_normal((B, n)).astype(np.float32)
+    return W, c, g
+
+
+def _check_all(ctx, W, c, g, Lb, k, T, what, viterbi=True):
+    got = parity.gpu_forward_backward(ctx, W, c, g, Lb, k, T)
+    ref_f = oracle.soft_quantize(W, c, Lb, k, T)
+    ref_b = oracle.backward(W, c, g, Lb, k, T)
+    parity.assert_forward_backward(got, ref_f, ref_b, what)
+    assert got["diag"].max_posterior_defect < 1e-3, what
+    if viterbi:
+        parity.assert_viterbi(parity.gpu_viterbi(ctx, W, c, Lb, k), oracle.viterbi(W, c, Lb, k), what)
+    return got
+
+
+# ------------------------------------------------------------------ tiny workload, all blocks
+def test_tiny_workload_all_blocks(ctx):
+    ctx.set_option("path", 0)
+    wl = synth.tiny()
+    W, c, g = wl.weights(), wl.codebook(), wl.upstream()
+    got = _check_all(ctx, W, c, g, wl.Lb, wl.k, wl.T, "tiny")
+    gold = json.loads((Path(__file__).parent / "golden" / "tiny_expected.json").read_text())
+    assert parity.rel_inf(got["soft"][0], gold["soft_block0"]) <= parity.SOFT_TOL
+    assert parity.rel_inf(got["grad_codebook"], gold["grad_codebook"]) <= parity.GRAD_TOL
+
+
+def test_enumerable_case_against_every_path(ctx):
+    wl = synth.brute()
+    W, c, g = wl.weights(), wl.codebook(), wl.upstream()
+    got = parity.gpu_forward_backward(ctx, W, c, g, wl.Lb, wl.k, wl.T)
+    vit = parity.gpu_viterbi(ctx, W, c, wl.Lb, wl.k)
+    for b in range(W.shape[0]):
+        soft, logZ, _ = bf.soft_codeword(W[b], c, wl.Lb, wl.k, wl.T)
+        assert parity.rel_inf(got["soft"][b], soft) <= parity.SOFT_TOL
+        assert abs(got["logZ"][b] - logZ) < 1e-4
+        states, _, gap = bf.best_path(W[b], c, wl.Lb, wl.k)
+        assert gap > 1e-6
+        np.testing.assert_array_equal(vit["states"][b], states)
+        np.testing.assert_array_equal(vit["path_bits"][b], bf.pack_path_bits(states, wl.Lb, wl.k))
+    gw, gc = bf.fd_gradients(W[0], c, g[0].astype(np.float64), wl.Lb, wl.k, wl.T)
+    one = parity.gpu_forward_backward(ctx, W[:1], c, g[:1], wl.Lb, wl.k, wl.T)
+    assert parity.rel_inf(one["grad_W"][0], gw) <= parity.GRAD_TOL
+    assert parity.rel_inf(one["grad_codebook"], gc) <= parity.GRAD_TOL
+
+
+# ------------------------------------------------------------------ shapes, ragged sizes, edge cases
+SHAPES = [  # (Lb, k, n, B, T)
+    (4, 2, 6, 5, 0.5), (2, 2, 7, 3, 0.3), (3, 2, 9, 4, 0.4), (5, 3, 11, 3, 0.2), (4, 4, 5, 2, 1.0),
+    (6, 1, 33, 7, 0.1), (8, 2, 64, 301, 0.5), (9, 3, 40, 10, 0.05), (10, 4, 17, 9, 0.2), (7, 1, 1, 6, 0.3),
+    (8, 2, 2, 4, 0.2), (11, 2, 100, 13, 0.02), (13, 3, 30, 5, 0.1), (15, 1, 12, 2, 0.3),
+]
+
+
+@pytest.mark.parametrize("Lb,k,n,B,T", SHAPES)
+def test_shapes_generic_path(ctx, Lb, k, n, B, T):
+    ctx.set_option("path", GENERIC)
+    try:
+        W, c, g = _rand(n, Lb, B, seed=1000 + Lb * 10 + k)
+        _check_all(ctx, W, c, g, Lb, k, T, f"Lb={Lb} k={k} n={n}")
+    finally:
+        ctx.set_option("path", 0)
+
+
+def test_more_blocks_than_resident_ctas(ctx):
+    # the persistent loop must visit every block exactly once, whatever the grid size
+    Lb, k, n, T = 8, 2, 16, 0.3
+    W, c, g = _rand(n, Lb, 37, seed=77)
+    ref = parity.gpu_forward_backward(ctx, W, c, g, Lb, k, T)
+    ctx.set_option("max_ctas", 5)
+    try:
+        got = parity.gpu_forward_backward(ctx, W, c, g, Lb, k, T)
+        vit = parity.gpu_viterbi(ctx, W, c, Lb, k)
+    finally:
+        ctx.set_option("max_ctas", 0)
+    np.testing.assert_array_equal(got["soft"], ref["soft"])
+    np.testing.assert_array_equal(got["grad_W"], ref["grad_W"])
+    assert parity.rel_inf(got["grad_codebook"], ref["grad_codebook"]) < 1e-5
+    parity.assert_viterbi(vit, oracle.viterbi(W, c, Lb, k), "max_ctas=5")
+
+
+def test_empty_input_and_argument_errors(ctx):
+    import torch
+    from paper_2605_10655_b200 import BcjrError, Context
+    dev = torch.device("cuda", 0)
+    c = torch.zeros(256, device=dev)
+    W = torch.zeros((0, 64), device=dev)
+    soft, logZ = ctx.bcjr_soft_quantize(W, c, 8, 2, 64, 0.5)
+    assert soft.numel() == 0
+    gW, gc = ctx.bcjr_backward(torch.zeros((0, 64), device=dev))
+    ctx.sync_status()
+    assert float(gc.abs().max()) == 0.0
+    W = torch.zeros((2, 64), device=dev)
+    for bad in [dict(Lb=8, k=2, T=0.0), dict(Lb=8, k=2, T=float("nan")), dict(Lb=8, k=5, T=1.0),
+                dict(Lb=8, k=0, T=1.0)]:
+        with pytest.raises(BcjrError) as ei:
+            ctx.bcjr_soft_quantize(W, c, bad["Lb"], bad["k"], 64, bad["T"])
+        assert ei.value.code == -1
+    with pytest.raises(BcjrError) as ei:
+        ctx.bcjr_soft_quantize(torch.zeros((1, 4), device=dev), torch.zeros(1 << 16, device=dev), 16, 1, 4, 1.0)
+    assert ei.value.code == -5
+    fresh = Context(0)
+    try:
+        rc = fresh._lib.bcjr_backward(fresh._h, W.data_ptr(), W.data_ptr(), None, None)  # noqa
+        assert rc == -4                                 # backward before any forward
+    finally:
+        fresh.close()
+
+
+# ------------------------------------------------------------------ mid trellis (S = 4096)
+@pytest.mark.parametrize("T", [1.0, 0.1, 0.01])
+def test_mid_trellis_temperature_sweep(ctx, T):
+    wl = synth.mid()
+    idx = synth.sample_blocks(wl.num_blocks(), 24)
+    W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
+    _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"mid T={T}", viterbi=(T == 1.0))
+
+
+def test_mid_trellis_cold_limit_matches_viterbi(ctx):
+    # Section 3.3, identity 1: as T -> 0 the soft codeword tends to the hard Viterbi output.
+    # Compared where the float64 oracle itself has converged (its argmax equals its Viterbi).
+    wl = synth.mid()
+    idx = synth.sample_blocks(wl.num_blocks(), 16, seed=5)
+    W, c = wl.weights()[idx], wl.codebook()
+    T = 1e-4
+    got = parity.gpu_forward_backward(ctx, W, c, None, wl.Lb, wl.k, T)
+    ref = oracle.soft_quantize(W, c, wl.Lb, wl.k, T)
+    vit = oracle.viterbi(W, c, wl.Lb, wl.k)
+    assert parity.rel_inf(got["soft"], ref["soft"]) <= parity.SOFT_TOL
+    c64 = c.astype(np.float64)
+    # nearest table entry to the soft value = the state the posterior has collapsed onto
+    conv = np.abs(ref["soft"] - vit["hard"]) < 1e-3
+    assert conv.mean() > 0.9
+    assert np.abs(got["soft"][conv] - vit["hard"][conv]).max() < 2e-3
+    gvit = parity.gpu_viterbi(ctx, W, c, wl.Lb, wl.k)
+    parity.assert_viterbi(gvit, vit, "mid viterbi")
+
+
+# ------------------------------------------------------------------ S = 2^16
+def test_q_proj_shape_sampled_blocks(ctx):
+    wl = synth.q_proj()
+    idx = synth.sample_blocks(wl.num_blocks(), 6)
+    W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
+    _check_all(ctx, W, c, g, wl.Lb, wl.k, wl.T, "q_proj sample")
+
+
+@pytest.mark.parametrize("T", [0.01, 0.001])
+def test_three_bit_student_t_low_temperature(ctx, T):
+    wl = synth.gate_k3()
+    idx = synth.sample_blocks(wl.num_blocks(), 4)
+    W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
+    got = _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"k=3 student-t T={T}", viterbi=(T == 0.01))
+    assert np.all(np.isfinite(got["soft"])) and np.all(np.isfinite(got["grad_W"]))
+    tot = got["grad_W"].astype(np.float64).sum() + got["grad_codebook"].astype(np.float64).sum()
+    assert abs(tot - g.astype(np.float64).sum()) < 1e-2 * np.abs(g).sum()
