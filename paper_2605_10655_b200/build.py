@@ -15,7 +15,7 @@ SOURCES = [CSRC / "bcjr_api.cu"]
 HEADERS = sorted(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "bcjr_b200.h"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-DBCJR_NO_CLUSTER"]
+              "-shared", "-Xcompiler", "-fPIC", "-cudart", "static"]
 
 
 def needs_build() -> bool:

@@ -174,6 +174,60 @@ bcjr_status launch_vit_generic(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
     return BCJR_OK;
 }
 
+#ifndef BCJR_NO_CLUSTER
+// One cluster of CL CTAs per weight block in flight; the grid is the number of clusters the
+// GPU can hold at once (persistent loop over blocks inside the kernel).
+template <typename Kern>
+bcjr_status plan_cluster(bcjr_ctx *ctx, Kern kern, int CL, int threads, size_t smem, int64_t B,
+                         cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attr, cudaStream_t st)
+{
+    CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg->gridDim = dim3(CL * ctx->num_sms, 1, 1);
+    cfg->blockDim = dim3(threads, 1, 1);
+    cfg->dynamicSmemBytes = smem;
+    cfg->stream = st;
+    cfg->attrs = attr;
+    cfg->numAttrs = 1;
+    int ncl = 0;
+    CU(cudaOccupancyMaxActiveClusters(&ncl, kern, cfg));
+    if (ncl < 1) return BCJR_EUNSUPPORTED;
+    if (ctx->opt_max_ctas > 0 && ncl > ctx->opt_max_ctas / CL) ncl = ctx->opt_max_ctas / CL > 0 ? ctx->opt_max_ctas / CL : 1;
+    if (ncl > B) ncl = (int)B;
+    cfg->gridDim = dim3(CL * ncl, 1, 1);
+    return BCJR_OK;
+}
+
+template <int LB, int KB, int CL, int THREADS>
+bcjr_status launch_fwd_cluster_t(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    using C = ClusterCfg<LB, KB, CL, THREADS>;
+    if (p.n > C::MAX_N) return BCJR_EUNSUPPORTED;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    auto kern = fwd_cluster_kernel<LB, KB, CL, THREADS>;
+    bcjr_status rc = plan_cluster(ctx, kern, CL, THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    if (rc) return rc;
+    const int ncl = cfg.gridDim.x / CL;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * p.n * C::Q * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    CU(cudaLaunchKernelEx(&cfg, kern, p));
+    ctx->launches += 1;
+    return BCJR_OK;
+}
+
+bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
+{
+    if (p.Lb != 16) return BCJR_EUNSUPPORTED;
+    if (k == 2) return launch_fwd_cluster_t<16, 2, 2, 512>(ctx, p, st);
+    if (k == 3) return launch_fwd_cluster_t<16, 3, 2, 512>(ctx, p, st);
+    return BCJR_EUNSUPPORTED;
+}
+#endif
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = false;
@@ -314,9 +368,7 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
     bcjr_status rc = BCJR_OK;
     bool use_cluster = false;
 #ifndef BCJR_NO_CLUSTER
-    use_cluster = ctx->opt_path != 1 && cluster_supported(ctx->Lb, ctx->k);
-    if (ctx->opt_path == 2 && !use_cluster) return BCJR_EUNSUPPORTED;
-    if (use_cluster) rc = launch_bwd_cluster(ctx, p, ctx->k, grad_codebook, st);
+    use_cluster = false;   // the backward pass has no cluster kernel yet
 #else
     if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
 #endif

@@ -1,0 +1,422 @@
+// Cluster kernels for the large trellis (S = 2^LB states, LB >= 2k): one weight block per
+// thread-block cluster, the state vector spread over the cluster's shared memories.
+//
+// Butterfly form of the recursions.  Write a state as s = [j | x | l] with j and l of k bits
+// and x of LB-2k bits.  One trellis step couples, for fixed x, the K inputs L_t([j|x]) with the
+// K outputs L_{t+1}([x|l]) through the K*K states [j|x|l]:
+//     L_{t+1}([x|l]) = LSE_j ( L_t([j|x]) + e_t([j|x|l]) )
+//     M_{t-1}([j|x]) = LSE_b ( M_t([x|b]) + e_t([j|x|b]) )
+// and the posterior of state [j|x|b] at step t is proportional to
+//     exp( L_t([j|x]) + e_t([j|x|b]) + M_t([x|b]) ).
+// A thread owns the same butterflies x for every step, both sweeps and every block, so the
+// K*K codebook entries of each of its butterflies stay in registers for the whole kernel.
+// Each output has exactly one consumer butterfly; it is pushed straight into the consumer
+// CTA's shared memory (st.shared::cluster), and one cluster barrier closes the step.
+//
+// History: the beta sweep needs L_t([j|x]) again.  The input buffer of alpha step t is exactly
+// that data in the layout the owner reads it, so one elected thread streams the whole buffer
+// to a per-cluster history in global memory with a bulk copy (TMA, shared -> global), and the
+// beta sweep prefetches it back two steps ahead (global -> shared, mbarrier completion).
+#pragma once
+#include "bcjr_common.cuh"
+
+namespace bcjr {
+
+// ---------------------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v)
+{
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d)
+{
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+                 : "memory");
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_sync() { cluster_arrive(); cluster_wait(); }
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_count_x()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store(void *gdst, uint32_t ssrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_load(uint32_t sdst, const void *gsrc, uint32_t bytes, uint32_t mbar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(sdst),
+                 "l"(gsrc), "r"(bytes), "r"(mbar)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~2^20 polls, raises BCJR_ETIMEOUT (-6) in the diagnostics and
+// sets the CTA-wide abort flag so that later waits return at once; the kernel then runs to its
+// end (with meaningless numbers) instead of hanging.
+__device__ __forceinline__ void mbar_wait_bounded(uint32_t mbar, uint32_t parity, volatile int *abort_flag, DeviceDiag *diag)
+{
+    if (*abort_flag) return;
+    for (int i = 0; i < (1 << 20); ++i)
+        if (mbar_try_wait(mbar, parity)) return;
+    *abort_flag = 1;
+    atomicCAS(&diag->status, 0, -6);
+}
+
+template <int LB, int KB, int CL, int THREADS>
+struct ClusterCfg {
+    static constexpr int K = 1 << KB;
+    static constexpr int S = 1 << LB;
+    static constexpr int Q = S >> KB;                 // groups = message length
+    static constexpr int NB = S >> (2 * KB);          // butterflies
+    static constexpr int NBC = NB / CL;               // butterflies per CTA
+    static constexpr int BPT = NBC / THREADS;         // butterflies per thread
+    static constexpr int QC = Q / CL;                 // message entries held per CTA
+    static constexpr int NWARP = THREADS / 32;
+    static constexpr int NSTAGE = 3;
+    static constexpr int MAX_N = 2048;
+    static_assert(LB >= 2 * KB, "butterfly form needs LB >= 2k");
+    static_assert(NBC % THREADS == 0 && BPT >= 1, "butterflies must divide evenly");
+    static_assert(CL * NWARP <= 32, "one partial per lane");
+    static_assert(NBC % K == 0 || CL == 1, "vector pushes must stay inside one CTA");
+    // shared memory carve-up (floats unless noted)
+    static constexpr int OFF_MSG = 0;                         // [2][QC]
+    static constexpr int OFF_STAGE = OFF_MSG + 2 * QC;        // [NSTAGE][QC]
+    static constexpr int OFF_W = OFF_STAGE + NSTAGE * QC;     // [MAX_N]
+    static constexpr int OFF_O = OFF_W + MAX_N;               // int [MAX_N + 2]
+    static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;    // [2][32]
+    static constexpr int OFF_PART = OFF_WMAX + 64;            // [2][32][4]
+    static constexpr int OFF_LZ = OFF_PART + 256;             // [2][32]
+    static constexpr int OFF_MBAR = OFF_LZ + 64;              // uint64 [NSTAGE] (8-byte aligned: even offset)
+    static constexpr int OFF_FLAG = OFF_MBAR + 2 * NSTAGE + 2;
+    static constexpr int SMEM_FLOATS = OFF_FLAG + 4;
+    static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
+    static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
+    static_assert((QC * 4) % 16 == 0, "bulk copies move multiples of 16 bytes");
+};
+
+// Per-thread constants of one owned butterfly.
+struct ButterflyAddr {
+    uint32_t push_alpha;   // cluster address (buffer 0) where the K alpha outputs go, contiguous
+    uint32_t push_beta[16];
+};
+
+// --------------------------------------------------------------------------------------
+// Forward call on a cluster: alpha sweep, log Z, beta sweep fused with Eq. 6-7.
+// --------------------------------------------------------------------------------------
+template <int LB, int KB, int CL, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
+{
+    using C = ClusterCfg<LB, KB, CL, THREADS>;
+    constexpr int K = C::K, NB = C::NB, NBC = C::NBC, BPT = C::BPT, QC = C::QC, NWARP = C::NWARP;
+    extern __shared__ __align__(16) float smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t cid = cluster_id_x(), ncl = cluster_count_x();
+    const int n = p.n;
+    const float NEG_INF = __int_as_float(0xff800000);
+    const float nlam = -p.lam2;
+
+    float *msg = smem + C::OFF_MSG;
+    float *stage = smem + C::OFF_STAGE;
+    float *w_s = smem + C::OFF_W;
+    int *O_s = reinterpret_cast<int *>(smem + C::OFF_O);
+    float *wmax = smem + C::OFF_WMAX;
+    float *part = smem + C::OFF_PART;
+    float *lz = smem + C::OFF_LZ;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
+    const uint32_t mbar0 = smem_u32(smem + C::OFF_MBAR);
+    const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage);
+    const uint32_t wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
+
+    // history of this cluster: [n][CL][QC]
+    float *hist = p.hist + (size_t)cid * n * C::Q;
+
+    // ---- codebook of the owned butterflies -> registers; push addresses
+    float cb[BPT][K][K];
+    uint32_t push_a[BPT];          // alpha: K contiguous outputs (cluster address, buffer 0)
+    uint32_t push_b[BPT][K];       // beta: K scalar outputs
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        const int xl = i * THREADS + tid;               // local butterfly
+        const int x = (int)rank * NBC + xl;             // global butterfly
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+#pragma unroll
+            for (int l = 0; l < K; ++l) cb[i][j][l] = __ldg(p.cb + (size_t)j * C::Q + (size_t)x * K + l);
+        // alpha outputs L([x|l]) = index x*K + l; consumer butterfly x2 = (x*K + l) mod NB with
+        // input slot j2 = (x*K) / NB; it lives in CTA x2 / NBC at [j2][x2 - r2*NBC]
+        {
+            const int q2 = x * K;
+            const int j2 = q2 / NB, x2 = q2 % NB;
+            const int r2 = x2 / NBC, xl2 = x2 % NBC;
+            push_a[i] = mapa_u32(msg_u32 + (uint32_t)(j2 * NBC + xl2) * 4u, (uint32_t)r2);
+        }
+        // beta outputs M([j|x]) = index j*NB + x; consumer butterfly x1 = (j*NB + x) / K reads it
+        // as its input b1 = x mod K; it lives in CTA x1 / NBC at [(x1 - r1*NBC)*K + b1]
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            const int q1 = j * NB + x;
+            const int x1 = q1 / K, b1 = q1 % K;
+            const int r1 = x1 / NBC, xl1 = x1 % NBC;
+            push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(xl1 * K + b1) * 4u, (uint32_t)r1);
+        }
+    }
+    // partial-result slots: every warp of every CTA writes one entry into every CTA's array
+    uint32_t wmax_dst[CL], lz_dst[CL];
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+        wmax_dst[r] = mapa_u32(wmax_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+        lz_dst[r] = mapa_u32(lz_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+    }
+    const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 16u, 0u);
+
+    if (tid == 0) {
+        for (int s = 0; s < C::NSTAGE; ++s) mbar_init(mbar0 + 8u * s, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    uint32_t loads_done = 0;       // bulk loads consumed so far (stage = count % NSTAGE, parity = (count / NSTAGE) & 1)
+    uint32_t loads_issued = 0;
+    float defect = 0.f, zgap = 0.f;
+
+    for (int64_t blk = cid; blk < p.B; blk += ncl) {
+        const float *w = p.W + blk * n;
+        for (int t = tid; t < n; t += THREADS) w_s[t] = __ldg(w + t);
+        for (int q = tid; q < QC; q += THREADS) msg[q] = 0.f;        // L_1 = 0 (buffer 0)
+        if (tid == 0) O_s[1] = 0;
+        int O = 0;
+        float off = 0.f, cmax = 0.f;
+        cluster_sync();
+        // ================= alpha sweep: step t maps L_t (buffer (t-1)&1) to L_{t+1} (buffer t&1)
+        for (int t = 1; t <= n; ++t) {
+            const int cur = (t - 1) & 1;
+            const float *Lin = msg + cur * QC;
+            const uint32_t nxt_off = (uint32_t)((t & 1) * QC) * 4u;
+            if (tid == 0) {                                          // spill L_t for the beta sweep
+                fence_proxy_async();
+                bulk_store(hist + ((size_t)(t - 1) * CL + rank) * QC, msg_u32 + (uint32_t)(cur * QC) * 4u, QC * 4u);
+                bulk_commit();
+            }
+            const float wt = w_s[t - 1];
+            float tmax = NEG_INF;
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                const int xl = i * THREADS + tid;
+                float Lj[K];
+#pragma unroll
+                for (int j = 0; j < K; ++j) Lj[j] = Lin[j * NBC + xl];
+                float out[K];
+#pragma unroll
+                for (int l = 0; l < K; ++l) {
+                    float a[K], m = NEG_INF;
+#pragma unroll
+                    for (int j = 0; j < K; ++j) {
+                        const float d = wt - cb[i][j][l];
+                        a[j] = fmaf(d * d, nlam, Lj[j]);
+                        m = fmaxf(m, a[j]);
+                    }
+                    float sum = 0.f;
+#pragma unroll
+                    for (int j = 0; j < K; ++j) sum += ex2f(a[j] - m);
+                    out[l] = (m - off) + lg2f(sum);
+                    tmax = fmaxf(tmax, out[l]);
+                }
+#pragma unroll
+                for (int l = 0; l < K; l += 4)
+                    st_cluster_v4(push_a[i] + nxt_off + 4u * l, out[l], out[l + 1], out[l + 2], out[l + 3]);
+            }
+            tmax = warp_max(tmax);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
+            }
+            O += (int)off;
+            if (tid == 0) {
+                O_s[t + 1] = O;
+                bulk_wait_read0();                                   // buffer `cur` may be overwritten next step
+            }
+            cluster_sync();
+            cmax = warp_max(lane < CL * NWARP ? wmax[(t & 1) * 32 + lane] : NEG_INF);
+            off = rintf(cmax);
+        }
+        // ================= log2 Z = O_{n+1} + LSE_q L_{n+1}(q); L_{n+1} sits in buffer n&1
+        {
+            const float *Lfin = msg + (n & 1) * QC;
+            float ssum = 0.f;
+            for (int q = tid; q < QC; q += THREADS) ssum += ex2f(Lfin[q] - cmax);
+            ssum = warp_sum(ssum);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
+            }
+            if (tid == 0) bulk_wait_all0();                          // history fully written
+            cluster_sync();
+        }
+        float lsefin;
+        {
+            float v = lane < CL * NWARP ? lz[lane] : 0.f;
+            v = warp_sum(v);
+            lsefin = cmax + lg2f(v);
+        }
+        const int Ofin = O;
+        if (tid == 0 && rank == 0 && p.logZ)
+            p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
+        // ================= beta sweep: step t maps M_t (buffer (n-t)&1) to M_{t-1}
+        for (int q = tid; q < QC; q += THREADS) msg[q] = 0.f;        // M_n = 0 (buffer 0)
+        if (tid == 0) {                                              // prefetch L_n and L_{n-1}
+            fence_proxy_async();
+            for (int d = 0; d < 2 && n - d >= 1; ++d) {
+                const uint32_t s = loads_issued % C::NSTAGE;
+                mbar_expect_tx(mbar0 + 8u * s, QC * 4u);
+                bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(n - d - 1) * CL + rank) * QC, QC * 4u, mbar0 + 8u * s);
+                ++loads_issued;
+            }
+        }
+        int P = 0;
+        float offM = 0.f;
+        cluster_sync();
+        for (int t = n; t >= 1; --t) {
+            const int cur = (n - t) & 1;
+            const float *Min = msg + cur * QC;
+            const uint32_t nxt_off = (uint32_t)((cur ^ 1) * QC) * 4u;
+            if (tid == 0 && t - 2 >= 1) {                            // prefetch L_{t-2}
+                fence_proxy_async();
+                const uint32_t s = loads_issued % C::NSTAGE;
+                mbar_expect_tx(mbar0 + 8u * s, QC * 4u);
+                bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(t - 3) * CL + rank) * QC, QC * 4u, mbar0 + 8u * s);
+                ++loads_issued;
+            }
+            const uint32_t st = loads_done % C::NSTAGE;
+            mbar_wait_bounded(mbar0 + 8u * st, (loads_done / C::NSTAGE) & 1u, abort_flag, p.diag);
+            ++loads_done;
+            const float *Lh = stage + st * QC;
+            const float wt = w_s[t - 1];
+            const float D = (float)(Ofin - O_s[t] - P) + lsefin;
+            float num = 0.f, den = 0.f, tmax = NEG_INF;
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                const int xl = i * THREADS + tid;
+                float Mb[K];
+#pragma unroll
+                for (int b = 0; b < K; b += 4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(Min + xl * K + b);
+                    Mb[b] = v.x; Mb[b + 1] = v.y; Mb[b + 2] = v.z; Mb[b + 3] = v.w;
+                }
+#pragma unroll
+                for (int j = 0; j < K; ++j) {
+                    float u[K], m = NEG_INF;
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        const float d = wt - cb[i][j][b];
+                        u[b] = fmaf(d * d, nlam, Mb[b]);
+                        m = fmaxf(m, u[b]);
+                    }
+                    float sum = 0.f, craw = 0.f;
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        const float pb = ex2f(u[b] - m);
+                        sum += pb;
+                        craw = fmaf(pb, cb[i][j][b], craw);
+                    }
+                    const float out = (m - offM) + lg2f(sum);
+                    tmax = fmaxf(tmax, out);
+                    st_cluster_f32(push_b[i][j] + nxt_off, out);
+                    const float f = ex2f(m + Lh[j * NBC + xl] - D);
+                    den = fmaf(f, sum, den);
+                    num = fmaf(f, craw, num);
+                }
+            }
+            num = warp_sum(num); den = warp_sum(den); tmax = warp_max(tmax);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
+                st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u, num);
+                st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u + 4u, den);
+            }
+            P += (int)offM;
+            cluster_sync();
+            cmax = warp_max(lane < CL * NWARP ? wmax[(t & 1) * 32 + lane] : NEG_INF);
+            offM = rintf(cmax);
+            if (rank == 0 && warp == 0) {
+                float a = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4] : 0.f;
+                float b = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4 + 1] : 0.f;
+                a = warp_sum(a); b = warp_sum(b);
+                if (lane == 0) {
+                    const float sw = a / b;
+                    p.soft[blk * n + t - 1] = sw;
+                    if (p.soft_copy) p.soft_copy[blk * n + t - 1] = sw;
+                    defect = fmaxf(defect, fabsf(b - 1.f));
+                }
+            }
+        }
+        // ================= consistency: P_0 + LSE_q M_0(q) against log2 Z (M_0 in buffer n&1)
+        {
+            const float *Mfin = msg + (n & 1) * QC;
+            float ssum = 0.f;
+            for (int q = tid; q < QC; q += THREADS) ssum += ex2f(Mfin[q] - cmax);
+            ssum = warp_sum(ssum);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r] + 32u * 4u, ssum);
+            }
+            cluster_sync();
+            float v = lane < CL * NWARP ? lz[32 + lane] : 0.f;
+            v = warp_sum(v);
+            const float lz_beta = cmax + lg2f(v);
+            zgap = fmaxf(zgap, fabsf((float)(P - Ofin) + (lz_beta - lsefin)));
+            cluster_sync();     // nobody still reads this block's buffers when the next block starts
+        }
+    }
+    if (tid == 0 && rank == 0) {
+        diag_max(&p.diag->max_defect, defect);
+        diag_max(&p.diag->max_logz_gap, zgap);
+    }
+    cluster_sync();             // no CTA leaves while a peer may still address its shared memory
+}
+
+// ---------------------------------------------------------------------------- host side
+inline bool cluster_supported(int Lb, int k) { return Lb == 16 && (k == 2 || k == 3); }
+
+}  // namespace bcjr
