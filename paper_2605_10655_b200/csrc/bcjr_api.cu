@@ -219,6 +219,40 @@ bcjr_status launch_fwd_cluster_t(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
     return BCJR_OK;
 }
 
+template <int LB, int KB, int CL, int THREADS>
+bcjr_status launch_bwd_cluster_t(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    using C = ClusterCfg<LB, KB, CL, THREADS>;
+    using BC = BwdClusterCfg<LB, KB, CL, THREADS>;
+    if (p.n > BC::MAX_N) return BCJR_EUNSUPPORTED;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    auto kern = bwd_cluster_kernel<LB, KB, CL, THREADS>;
+    bcjr_status rc = plan_cluster(ctx, kern, CL, THREADS, BC::SMEM_BYTES, p.B, &cfg, attr, st);
+    if (rc) return rc;
+    const int ncl = cfg.gridDim.x / CL;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * p.n * 2 * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * C::S * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.gc_part = (float *)ctx->gc_part.ptr;
+    CU(cudaLaunchKernelEx(&cfg, kern, p));
+    ctx->launches += 1;
+    if (grad_codebook) {
+        reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, C::S, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
+bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_codebook, cudaStream_t st)
+{
+    if (p.Lb != 16) return BCJR_EUNSUPPORTED;
+    if (k == 2) return launch_bwd_cluster_t<16, 2, 4, 512>(ctx, p, grad_codebook, st);
+    if (k == 3) return launch_bwd_cluster_t<16, 3, 4, 256>(ctx, p, grad_codebook, st);
+    return BCJR_EUNSUPPORTED;
+}
+
 bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
@@ -368,7 +402,9 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
     bcjr_status rc = BCJR_OK;
     bool use_cluster = false;
 #ifndef BCJR_NO_CLUSTER
-    use_cluster = false;   // the backward pass has no cluster kernel yet
+    use_cluster = ctx->opt_path != 1 && cluster_supported(ctx->Lb, ctx->k);
+    if (ctx->opt_path == 2 && !use_cluster) return BCJR_EUNSUPPORTED;
+    if (use_cluster) rc = launch_bwd_cluster(ctx, p, ctx->k, grad_codebook, st);
 #else
     if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
 #endif

@@ -103,6 +103,14 @@ __device__ __forceinline__ void mbar_wait_bounded(uint32_t mbar, uint32_t parity
     atomicCAS(&diag->status, 0, -6);
 }
 
+// max over up to 64 per-warp slots, two per lane
+__device__ __forceinline__ float slot_max(const float *slots, int lane, int count)
+{
+    float v = lane < count ? slots[lane] : __int_as_float(0xff800000);
+    if (lane + 32 < count) v = fmaxf(v, slots[lane + 32]);
+    return v;
+}
+
 template <int LB, int KB, int CL, int THREADS>
 struct ClusterCfg {
     static constexpr int K = 1 << KB;
@@ -117,7 +125,7 @@ struct ClusterCfg {
     static constexpr int MAX_N = 2048;
     static_assert(LB >= 2 * KB, "butterfly form needs LB >= 2k");
     static_assert(NBC % THREADS == 0 && BPT >= 1, "butterflies must divide evenly");
-    static_assert(CL * NWARP <= 32, "one partial per lane");
+    static_assert(CL * NWARP <= 64, "at most two partials per lane");
     static_assert(NBC % K == 0 || CL == 1, "vector pushes must stay inside one CTA");
     // shared memory carve-up (floats unless noted)
     static constexpr int OFF_MSG = 0;                         // [2][QC]
@@ -133,12 +141,6 @@ struct ClusterCfg {
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
     static_assert((QC * 4) % 16 == 0, "bulk copies move multiples of 16 bytes");
-};
-
-// Per-thread constants of one owned butterfly.
-struct ButterflyAddr {
-    uint32_t push_alpha;   // cluster address (buffer 0) where the K alpha outputs go, contiguous
-    uint32_t push_beta[16];
 };
 
 // --------------------------------------------------------------------------------------
@@ -414,6 +416,320 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
         diag_max(&p.diag->max_logz_gap, zgap);
     }
     cluster_sync();             // no CTA leaves while a peer may still address its shared memory
+}
+
+
+// --------------------------------------------------------------------------------------
+// Backward call on a cluster.  Same butterflies; each message now carries a second value, the
+// conditional expectation of the centred emitted sum (At on the alpha side, Bt on the beta
+// side, see bcjr_generic.cuh for the recursions).  The codebook gradient of a state is owned
+// by the thread that owns the state, for every step and every block, so it accumulates in
+// registers and is written once, at the end, to this cluster's partial sum.
+// --------------------------------------------------------------------------------------
+template <int LB, int KB, int CL, int THREADS>
+struct BwdClusterCfg {
+    using F = ClusterCfg<LB, KB, CL, THREADS>;
+    static constexpr int QC = F::QC;
+    static constexpr int NSTAGE = 3;
+    static constexpr int MAX_N = 2048;
+    static constexpr int OFF_MSG = 0;                          // [2 parity][2 arrays][QC]
+    static constexpr int OFF_STAGE = OFF_MSG + 4 * QC;         // [NSTAGE][2][QC]
+    static constexpr int OFF_W = OFF_STAGE + NSTAGE * 2 * QC;  // w, g, soft: [3][MAX_N]
+    static constexpr int OFF_O = OFF_W + 3 * MAX_N;            // int [MAX_N + 4]
+    static constexpr int OFF_WMAX = OFF_O + MAX_N + 4;         // [2][64]
+    static constexpr int OFF_PART = OFF_WMAX + 128;            // [2][64][4]
+    static constexpr int OFF_LZ = OFF_PART + 512;              // [64]
+    static constexpr int OFF_MBAR = OFF_LZ + 64;               // uint64 [NSTAGE]
+    static constexpr int OFF_FLAG = OFF_MBAR + 2 * NSTAGE + 2;
+    static constexpr int SMEM_FLOATS = OFF_FLAG + 4;
+    static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
+    static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
+};
+
+template <int LB, int KB, int CL, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
+{
+    using C = ClusterCfg<LB, KB, CL, THREADS>;
+    using BC = BwdClusterCfg<LB, KB, CL, THREADS>;
+    constexpr int K = C::K, NB = C::NB, NBC = C::NBC, BPT = C::BPT, QC = C::QC, NWARP = C::NWARP;
+    extern __shared__ __align__(16) float smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t cid = cluster_id_x(), ncl = cluster_count_x();
+    const int n = p.n;
+    const float NEG_INF = __int_as_float(0xff800000);
+    const float nlam = -p.lam2, invT = p.invT;
+
+    float *msg = smem + BC::OFF_MSG;
+    float *stage = smem + BC::OFF_STAGE;
+    float *w_s = smem + BC::OFF_W, *g_s = w_s + BC::MAX_N, *sf_s = g_s + BC::MAX_N;
+    int *O_s = reinterpret_cast<int *>(smem + BC::OFF_O);
+    float *wmax = smem + BC::OFF_WMAX;
+    float *part = smem + BC::OFF_PART;
+    float *lz = smem + BC::OFF_LZ;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + BC::OFF_FLAG);
+    const uint32_t mbar0 = smem_u32(smem + BC::OFF_MBAR);
+    const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage);
+    const uint32_t wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
+    constexpr uint32_t STEP_BYTES = 2u * QC * 4u;            // both arrays of one parity / one stage
+
+    float *hist = p.hist + (size_t)cid * n * 2 * C::Q;       // [n][CL][2][QC]
+
+    float cb[BPT][K][K], acc[BPT][K][K];
+    uint32_t push_a[BPT], push_b[BPT][K];
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        const int xl = i * THREADS + tid;
+        const int x = (int)rank * NBC + xl;
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+#pragma unroll
+            for (int l = 0; l < K; ++l) {
+                cb[i][j][l] = __ldg(p.cb + (size_t)j * C::Q + (size_t)x * K + l);
+                acc[i][j][l] = 0.f;
+            }
+        {
+            const int q2 = x * K;
+            const int j2 = q2 / NB, x2 = q2 % NB;
+            const int r2 = x2 / NBC, xl2 = x2 % NBC;
+            push_a[i] = mapa_u32(msg_u32 + (uint32_t)(j2 * NBC + xl2) * 4u, (uint32_t)r2);
+        }
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            const int q1 = j * NB + x;
+            const int x1 = q1 / K, b1 = q1 % K;
+            const int r1 = x1 / NBC, xl1 = x1 % NBC;
+            push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(xl1 * K + b1) * 4u, (uint32_t)r1);
+        }
+    }
+    uint32_t wmax_dst[CL], lz_dst[CL];
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+        wmax_dst[r] = mapa_u32(wmax_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+        lz_dst[r] = mapa_u32(lz_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+    }
+    const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 16u, 0u);
+
+    if (tid == 0) {
+        for (int s = 0; s < BC::NSTAGE; ++s) mbar_init(mbar0 + 8u * s, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    uint32_t loads_done = 0, loads_issued = 0;
+    float defect = 0.f;
+
+    for (int64_t blk = cid; blk < p.B; blk += ncl) {
+        for (int t = tid; t < n; t += THREADS) {
+            w_s[t] = __ldg(p.W + blk * n + t);
+            g_s[t] = __ldg(p.g + blk * n + t);
+            sf_s[t] = __ldg(p.soft + blk * n + t);
+        }
+        for (int q = tid; q < 2 * QC; q += THREADS) msg[q] = 0.f;    // L_1 = 0, At_1 = 0 (parity 0)
+        if (tid == 0) O_s[1] = 0;
+        int O = 0;
+        float off = 0.f, cmax = 0.f;
+        cluster_sync();
+        // ================= alpha sweep
+        for (int t = 1; t <= n; ++t) {
+            const int cur = (t - 1) & 1;
+            const float *Lin = msg + cur * 2 * QC, *Ain = Lin + QC;
+            const uint32_t nxt_off = (uint32_t)((t & 1) * 2 * QC) * 4u;
+            if (tid == 0) {
+                fence_proxy_async();
+                bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)(cur * 2 * QC) * 4u, STEP_BYTES);
+                bulk_commit();
+            }
+            const float wt = w_s[t - 1], gt = g_s[t - 1];
+            const float gsh = -gt * sf_s[t - 1];                      // centring: h = g c - g soft
+            float tmax = NEG_INF;
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                const int xl = i * THREADS + tid;
+                float Lj[K], Aj[K];
+#pragma unroll
+                for (int j = 0; j < K; ++j) { Lj[j] = Lin[j * NBC + xl]; Aj[j] = Ain[j * NBC + xl] + gsh; }
+                float outL[K], outA[K];
+#pragma unroll
+                for (int l = 0; l < K; ++l) {
+                    float a[K], m = NEG_INF;
+#pragma unroll
+                    for (int j = 0; j < K; ++j) {
+                        const float d = wt - cb[i][j][l];
+                        a[j] = fmaf(d * d, nlam, Lj[j]);
+                        m = fmaxf(m, a[j]);
+                    }
+                    float sum = 0.f, ax = 0.f;
+#pragma unroll
+                    for (int j = 0; j < K; ++j) {
+                        const float pj = ex2f(a[j] - m);
+                        sum += pj;
+                        ax = fmaf(pj, fmaf(gt, cb[i][j][l], Aj[j]), ax);
+                    }
+                    outL[l] = (m - off) + lg2f(sum);
+                    outA[l] = ax * rcpf(sum);
+                    tmax = fmaxf(tmax, outL[l]);
+                }
+#pragma unroll
+                for (int l = 0; l < K; l += 4) {
+                    st_cluster_v4(push_a[i] + nxt_off + 4u * l, outL[l], outL[l + 1], outL[l + 2], outL[l + 3]);
+                    st_cluster_v4(push_a[i] + nxt_off + QC * 4u + 4u * l, outA[l], outA[l + 1], outA[l + 2], outA[l + 3]);
+                }
+            }
+            tmax = warp_max(tmax);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 64) * 4u, tmax);
+            }
+            O += (int)off;
+            if (tid == 0) {
+                O_s[t + 1] = O;
+                bulk_wait_read0();
+            }
+            cluster_sync();
+            cmax = warp_max(slot_max(wmax + (t & 1) * 64, lane, CL * NWARP));
+            off = rintf(cmax);
+        }
+        // ================= log2 Z
+        {
+            const float *Lfin = msg + (n & 1) * 2 * QC;
+            float ssum = 0.f;
+            for (int q = tid; q < QC; q += THREADS) ssum += ex2f(Lfin[q] - cmax);
+            ssum = warp_sum(ssum);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
+            }
+            if (tid == 0) bulk_wait_all0();
+            cluster_sync();
+        }
+        float lsefin;
+        {
+            float v = (lane < CL * NWARP ? lz[lane] : 0.f) + (lane + 32 < CL * NWARP ? lz[lane + 32] : 0.f);
+            v = warp_sum(v);
+            lsefin = cmax + lg2f(v);
+        }
+        const int Ofin = O;
+        // ================= beta sweep with the gradient contraction
+        for (int q = tid; q < 2 * QC; q += THREADS) msg[q] = 0.f;    // M_n = 0, Bt_n = 0 (parity 0)
+        if (tid == 0) {
+            fence_proxy_async();
+            for (int d = 0; d < 2 && n - d >= 1; ++d) {
+                const uint32_t s = loads_issued % BC::NSTAGE;
+                mbar_expect_tx(mbar0 + 8u * s, STEP_BYTES);
+                bulk_load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(n - d - 1) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
+                ++loads_issued;
+            }
+        }
+        int P = 0;
+        float offM = 0.f;
+        cluster_sync();
+        for (int t = n; t >= 1; --t) {
+            const int cur = (n - t) & 1;
+            const float *Min = msg + cur * 2 * QC, *Bin = Min + QC;
+            const uint32_t nxt_off = (uint32_t)((cur ^ 1) * 2 * QC) * 4u;
+            if (tid == 0 && t - 2 >= 1) {
+                fence_proxy_async();
+                const uint32_t s = loads_issued % BC::NSTAGE;
+                mbar_expect_tx(mbar0 + 8u * s, STEP_BYTES);
+                bulk_load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(t - 3) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
+                ++loads_issued;
+            }
+            const uint32_t st = loads_done % BC::NSTAGE;
+            mbar_wait_bounded(mbar0 + 8u * st, (loads_done / BC::NSTAGE) & 1u, abort_flag, p.diag);
+            ++loads_done;
+            const float *Lh = stage + st * 2 * QC, *Ah = Lh + QC;
+            const float wt = w_s[t - 1], gt = g_s[t - 1], sft = sf_s[t - 1];
+            const float gsh = -gt * sft;
+            const float D = (float)(Ofin - O_s[t] - P) + lsefin;
+            float S0 = 0.f, S1 = 0.f, S2 = 0.f, S3 = 0.f, tmax = NEG_INF;
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                const int xl = i * THREADS + tid;
+                float Mb[K], Yb[K];
+#pragma unroll
+                for (int b = 0; b < K; b += 4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(Min + xl * K + b);
+                    Mb[b] = v.x; Mb[b + 1] = v.y; Mb[b + 2] = v.z; Mb[b + 3] = v.w;
+                    const float4 y = *reinterpret_cast<const float4 *>(Bin + xl * K + b);
+                    Yb[b] = y.x + gsh; Yb[b + 1] = y.y + gsh; Yb[b + 2] = y.z + gsh; Yb[b + 3] = y.w + gsh;
+                }
+#pragma unroll
+                for (int j = 0; j < K; ++j) {
+                    float u[K], d[K], m = NEG_INF;
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        d[b] = wt - cb[i][j][b];
+                        u[b] = fmaf(d[b] * d[b], nlam, Mb[b]);
+                        m = fmaxf(m, u[b]);
+                    }
+                    const float Lhj = Lh[j * NBC + xl], Ahj = Ah[j * NBC + xl];
+                    const float f = ex2f(m + Lhj - D);
+                    const float fg = f * gt, fi = f * invT;
+                    float sum = 0.f, craw = 0.f, yacc = 0.f, ycc = 0.f;
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        const float pb = ex2f(u[b] - m);
+                        const float y = fmaf(gt, cb[i][j][b], Yb[b]);        // h + Bt
+                        const float pc = pb * cb[i][j][b];
+                        sum += pb;
+                        craw += pc;
+                        yacc = fmaf(pb, y, yacc);
+                        ycc = fmaf(pc, y, ycc);
+                        const float r = y + Ahj;
+                        acc[i][j][b] = fmaf(pb, fmaf(fi * d[b], r, fg), acc[i][j][b]);
+                    }
+                    const float outM = (m - offM) + lg2f(sum);
+                    tmax = fmaxf(tmax, outM);
+                    st_cluster_f32(push_b[i][j] + nxt_off, outM);
+                    st_cluster_f32(push_b[i][j] + nxt_off + QC * 4u, yacc * rcpf(sum));
+                    // sums over the posterior: gamma = f * p_b
+                    const float s2 = fmaf(Ahj, sum, yacc);                    // sum_b p_b r_b
+                    S0 = fmaf(f, sum, S0);
+                    S1 = fmaf(f, fmaf(-sft, sum, craw), S1);                  // sum gamma (c - soft)
+                    S2 = fmaf(f, s2, S2);                                     // sum gamma r
+                    S3 = fmaf(f, fmaf(-sft, s2, fmaf(Ahj, craw, ycc)), S3);   // sum gamma r (c - soft)
+                }
+            }
+            S0 = warp_sum(S0); S1 = warp_sum(S1); S2 = warp_sum(S2); S3 = warp_sum(S3);
+            tmax = warp_max(tmax);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 64) * 4u, tmax);
+                const uint32_t pd = part_dst + (uint32_t)((t & 1) * 256) * 4u;
+                st_cluster_f32(pd, S0); st_cluster_f32(pd + 4u, S1); st_cluster_f32(pd + 8u, S2); st_cluster_f32(pd + 12u, S3);
+            }
+            P += (int)offM;
+            cluster_sync();
+            cmax = warp_max(slot_max(wmax + (t & 1) * 64, lane, CL * NWARP));
+            offM = rintf(cmax);
+            if (rank == 0 && warp == 0) {
+                const float *pp = part + (t & 1) * 256 + lane * 4;
+                const bool on = lane < CL * NWARP, on2 = lane + 32 < CL * NWARP;
+                float a0 = on ? pp[0] : 0.f, a1 = on ? pp[1] : 0.f, a2 = on ? pp[2] : 0.f, a3 = on ? pp[3] : 0.f;
+                if (on2) { a0 += pp[128]; a1 += pp[129]; a2 += pp[130]; a3 += pp[131]; }
+                a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+                if (lane == 0) {
+                    const float i0 = 1.f / a0;
+                    p.gW[blk * n + t - 1] = invT * (a3 * i0 - (a2 * i0) * (a1 * i0));
+                    defect = fmaxf(defect, fabsf(a0 - 1.f));
+                }
+            }
+        }
+        cluster_sync();
+    }
+    // this cluster's partial of grad_codebook: state [j|x|b] = j*Q + x*K + b
+    float *gc = p.gc_part + (size_t)cid * C::S;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        const int x = (int)rank * NBC + i * THREADS + tid;
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+#pragma unroll
+            for (int b = 0; b < K; ++b) gc[(size_t)j * C::Q + (size_t)x * K + b] = acc[i][j][b];
+    }
+    if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
+    cluster_sync();
 }
 
 // ---------------------------------------------------------------------------- host side
