@@ -37,7 +37,8 @@ typedef enum {
     BCJR_ESTATE = -4,        /* bcjr_backward without a preceding bcjr_soft_quantize */
     BCJR_EUNSUPPORTED = -5,  /* (Lb, k) combination the kernels do not cover */
     BCJR_ETIMEOUT = -6,      /* a bounded device-side wait gave up (reported by bcjr_sync_status) */
-    BCJR_ENUMERIC = -7       /* non-finite values met on the device */
+    BCJR_ENUMERIC = -7,      /* non-finite values met on the device */
+    BCJR_ETOOLARGE = -8      /* problem does not fit the fixed scratch of bcjr_soft_quantize_static */
 } bcjr_status;
 
 /* Diagnostics gathered on the device since the last bcjr_sync_status. */
@@ -130,6 +131,44 @@ int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx);
 const char *bcjr_last_cuda_error(const bcjr_ctx *ctx);
 
 const char *bcjr_status_string(bcjr_status status);
+
+/*
+ * bcjr_soft_quantize_static -- the forward call for callers that cannot allocate.
+ * (The paper has no counterpart: this is a packaging of bcjr_soft_quantize, not a step of the
+ * method.)
+ *
+ * Some callers may not call cudaMalloc or cudaFree at all: a latency-critical host loop that
+ * cannot afford the device-wide synchronisation those calls imply, a process whose device
+ * memory was handed to another allocator up front, a plug-in that may only launch work on the
+ * buffers it is given.  This entry point computes exactly what bcjr_soft_quantize computes
+ * (same kernel, same results) but needs no context and never allocates or frees: its scratch
+ * is a fixed array of BCJR_STATIC_SCRATCH_BYTES that is part of the library image on every
+ * GPU that loads the library, for the life of the process.
+ *
+ *   W, codebook, soft, logZ, cuda_stream: as for bcjr_soft_quantize (device pointers of the
+ *   CURRENT device; logZ may be NULL).  Nothing is saved for a backward pass.
+ *
+ * Limits: the messages must fit shared memory (Lb - k <= 14) and one block's history must fit
+ * the scratch: n * 2^(Lb-k) * 4 + (n+2) * 4 bytes (rounded up to 256) <= BCJR_STATIC_SCRATCH_BYTES
+ * - 256.  Larger problems are refused with BCJR_ETOOLARGE before anything is launched.  The
+ * number of blocks is unlimited; fewer thread blocks run at once when the scratch is tight.
+ *
+ * Set-up: the first call on each device looks up the device address of the scratch array
+ * (once, under a lock; that device must be current, as it is for the call itself).  Make that
+ * first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same scratch, and it keeps the previous call's
+ * contents (the part that must start from zero is cleared on the stream at each call).  Calls
+ * whose kernels could overlap on the GPU -- different streams, or different host threads
+ * without ordering -- race on it: order them on one stream or with events.
+ */
+#define BCJR_STATIC_SCRATCH_BYTES (32u << 20)
+bcjr_status bcjr_soft_quantize_static(const float *W, const float *codebook, int Lb, int k, int n,
+                                      int64_t num_blocks, float T, float *soft, float *logZ,
+                                      void *cuda_stream);
+
+/* Size in bytes of the fixed scratch array behind bcjr_soft_quantize_static. */
+int64_t bcjr_static_scratch_bytes(void);
 
 #ifdef __cplusplus
 }

@@ -9,4 +9,5 @@ pass and the Viterbi hard code, behind the C ABI of include/bcjr_b200.h.
 
 The CUDA library is loaded on first use; there is no CPU fallback.
 """
-from .binding import BcjrError, Context, Diag, load_library, path_bytes, status_string  # noqa: F401
+from .binding import (BcjrError, Context, Diag, bcjr_soft_quantize_static, load_library,  # noqa: F401
+                      path_bytes, status_string)

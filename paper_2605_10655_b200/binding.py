@@ -14,7 +14,8 @@ LIB_PATH = _PKG / "libbcjr_b200.so"
 
 EXPORTS = ["bcjr_create", "bcjr_destroy", "bcjr_set_option", "bcjr_soft_quantize", "bcjr_backward",
            "viterbi_hard", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
-           "bcjr_last_cuda_error", "bcjr_status_string"]
+           "bcjr_last_cuda_error", "bcjr_status_string", "bcjr_soft_quantize_static",
+           "bcjr_static_scratch_bytes"]
 
 
 class BcjrError(RuntimeError):
@@ -55,6 +56,9 @@ def load_library() -> ctypes.CDLL:
     lib.bcjr_workspace_bytes.restype = i64; lib.bcjr_workspace_bytes.argtypes = [vp]
     lib.bcjr_last_cuda_error.restype = ctypes.c_char_p; lib.bcjr_last_cuda_error.argtypes = [vp]
     lib.bcjr_status_string.restype = ctypes.c_char_p; lib.bcjr_status_string.argtypes = [i]
+    lib.bcjr_soft_quantize_static.restype = i
+    lib.bcjr_soft_quantize_static.argtypes = [vp, vp, i, i, i, i64, f, vp, vp, vp]
+    lib.bcjr_static_scratch_bytes.restype = i64; lib.bcjr_static_scratch_bytes.argtypes = []
     _lib = lib
     return lib
 
@@ -82,6 +86,30 @@ def _dev(t, dtype, numel=None, name="tensor"):
     if numel is not None and t.numel() != numel:
         raise ValueError(f"{name}: expected {numel} elements, got {t.numel()}")
     return ctypes.c_void_p(t.data_ptr())
+
+
+def bcjr_soft_quantize_static(W, codebook, Lb, k, n, T, soft=None, logZ=None, stream=None):
+    """Forward call for callers that may not allocate device memory: no context, no cudaMalloc;
+    the scratch is a fixed array inside the library (see include/bcjr_b200.h for the limits).
+    The output tensors are the caller's: pass `soft` / `logZ` to avoid torch allocating them here.
+    All calls on a device share that scratch, so keep them ordered on one stream."""
+    import torch
+    lib = load_library()
+    B = W.numel() // n
+    if B * n != W.numel():
+        raise ValueError("W.numel() must be a multiple of n")
+    if soft is None:
+        soft = torch.empty_like(W)
+    if logZ is None:
+        logZ = torch.empty(B, dtype=torch.float32, device=W.device)
+    with torch.cuda.device(W.device):
+        rc = lib.bcjr_soft_quantize_static(_dev(W, torch.float32, name="W"),
+                                           _dev(codebook, torch.float32, 1 << Lb, "codebook"), Lb, k, n, B,
+                                           float(T), _dev(soft, torch.float32, B * n, "soft"),
+                                           _dev(logZ, torch.float32, B, "logZ"), _stream_ptr(stream))
+    if rc != 0:
+        raise BcjrError(rc, "bcjr_soft_quantize_static")
+    return soft, logZ
 
 
 class Context:

@@ -11,7 +11,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libbcjr_b200.so"
-SOURCES = [CSRC / "bcjr_api.cu"]
+SOURCES = [CSRC / "bcjr_api.cu", CSRC / "bcjr_static.cu"]
 HEADERS = sorted(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "bcjr_b200.h"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -525,6 +525,7 @@ const char *bcjr_status_string(bcjr_status s)
         case BCJR_EUNSUPPORTED: return "unsupported (Lb, k, n) combination";
         case BCJR_ETIMEOUT: return "device-side wait timed out";
         case BCJR_ENUMERIC: return "non-finite values on the device";
+        case BCJR_ETOOLARGE: return "problem exceeds the fixed scratch of bcjr_soft_quantize_static";
     }
     return "unknown status";
 }

@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams 
 }
 
 // Deterministic (fixed-order) sum of the per-CTA partial codebook gradients.
-__global__ void reduce_gc_kernel(const float *part, int nparts, int S, float *out)
+static __global__ void reduce_gc_kernel(const float *part, int nparts, int S, float *out)
 {
     const int u = blockIdx.x * blockDim.x + threadIdx.x;
     if (u >= S) return;
