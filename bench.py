@@ -26,7 +26,7 @@ import numpy as np
 ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
-from paper_2605_10655_b200 import synth  # noqa: E402
+from paper_2605_10655_b200 import shard, synth  # noqa: E402
 
 METRIC = "bcjr_fwd_bwd_trellis_edge_updates_per_s"
 UNIT = "edges/s"
@@ -99,10 +99,10 @@ def cpu_baseline(wl, seconds_hint: float = 20.0):
     sample of blocks of the same workload (one block per core)."""
     import oracle
     cores = oracle.host_cores()
-    nblk = max(1, min(cores, wl.num_blocks()))
-    # one block per core at S = 2^16 is ~25 core-seconds; smaller trellises take more blocks
+    # ~5 core-seconds per block at S = 2^16, n = 256 (forward + backward); four blocks per core
+    # keep the sample near 20 s; smaller trellises take proportionally more blocks
     scale = max(1, int((1 << 16) * 256 / (wl.S * wl.n)))
-    nblk = min(wl.num_blocks(), nblk * min(scale, 64))
+    nblk = max(1, min(wl.num_blocks(), 4 * cores * min(scale, 64)))
     W, c, g = wl.weights(0)[:nblk], wl.codebook(), wl.upstream(0)[:nblk]
     t0 = time.time()
     oracle.soft_quantize(W, c, wl.Lb, wl.k, wl.T)
@@ -217,8 +217,7 @@ def main():
             if ev is not None:
                 ev["b1"].append(torch.cuda.Event(enable_timing=True)); ev["b1"][-1].record()
             gc_total.add_(gc)
-        if world > 1:
-            dist.all_reduce(gc_total)
+        shard.allreduce_grad_codebook(gc_total)          # the one exchange of the data-parallel path
 
     for s in range(args.warmup):
         fresh_g(s); flush.zero_()
