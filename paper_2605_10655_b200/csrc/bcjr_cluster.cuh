@@ -103,6 +103,61 @@ __device__ __forceinline__ void mbar_wait_bounded(uint32_t mbar, uint32_t parity
     atomicCAS(&diag->status, 0, -6);
 }
 
+// ---------------------------------------------------------------------------- packed fp32 pairs
+// sm_100 executes add/mul/fma on two packed fp32 values per instruction (f32x2): the kernels
+// keep every per-state quantity as a pair so that the FP32 instruction count per state halves
+// and the special-function unit, not instruction issue, is the binding pipe.
+__device__ __forceinline__ float2 add2(float2 a, float2 b)
+{
+    float2 d;
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; add.rn.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b)
+{
+    float2 d;
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; sub.rn.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b)
+{
+    float2 d;
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; mul.rn.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
+{
+    float2 d;
+    asm("{ .reg .b64 ra, rb, rc, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; mov.b64 rc, {%6, %7}; "
+        "fma.rn.f32x2 rd, ra, rb, rc; mov.b64 {%0, %1}, rd; }"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+__device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
+__device__ __forceinline__ float2 lg2f2(float2 a) { return make_float2(lg2f(a.x), lg2f(a.y)); }
+__device__ __forceinline__ float2 rcpf2(float2 a) { return make_float2(rcpf(a.x), rcpf(a.y)); }
+__device__ __forceinline__ float max3f(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// elementwise max over N pairs
+template <int N>
+__device__ __forceinline__ float2 max_pairs(const float2 (&a)[N])
+{
+    float2 m = a[0];
+    int j = 1;
+#pragma unroll
+    for (; j + 1 < N; j += 2) { m.x = max3f(m.x, a[j].x, a[j + 1].x); m.y = max3f(m.y, a[j].y, a[j + 1].y); }
+    if (j < N) { m.x = fmaxf(m.x, a[j].x); m.y = fmaxf(m.y, a[j].y); }
+    return m;
+}
+
 // max over up to 64 per-warp slots, two per lane
 __device__ __forceinline__ float slot_max(const float *slots, int lane, int count)
 {
@@ -121,6 +176,7 @@ struct ClusterCfg {
     static constexpr int BPT = NBC / THREADS;         // butterflies per thread
     static constexpr int QC = Q / CL;                 // message entries held per CTA
     static constexpr int NWARP = THREADS / 32;
+    static constexpr int THREADS_ = THREADS;
     static constexpr int NSTAGE = 3;
     static constexpr int MAX_N = 2048;
     static_assert(LB >= 2 * KB, "butterfly form needs LB >= 2k");
@@ -146,6 +202,49 @@ struct ClusterCfg {
 // --------------------------------------------------------------------------------------
 // Forward call on a cluster: alpha sweep, log Z, beta sweep fused with Eq. 6-7.
 // --------------------------------------------------------------------------------------
+
+// Codebook of the owned butterflies, in the pairing a sweep wants.  Alpha pairs neighbouring
+// outputs l: A[i][j][h] = (c[j|x|2h], c[j|x|2h+1]);  beta pairs neighbouring inputs j:
+// B[i][jh][b] = (c[2jh|x|b], c[2jh+1|x|b]).  Reloaded (from L2) at the start of each sweep.
+template <typename C>
+__device__ __forceinline__ void load_cb_alpha(float2 (&A)[C::BPT][C::K][C::K / 2], const float *cbk, int rank, int tid)
+{
+#pragma unroll
+    for (int i = 0; i < C::BPT; ++i) {
+        const int x = rank * C::NBC + i * C::THREADS_ + tid;
+#pragma unroll
+        for (int j = 0; j < C::K; ++j)
+#pragma unroll
+            for (int h = 0; h < C::K / 2; h += 2) {
+                const float4 v = __ldg(reinterpret_cast<const float4 *>(cbk + (size_t)j * C::Q + (size_t)x * C::K) + h / 2);
+                A[i][j][h] = make_float2(v.x, v.y);
+                A[i][j][h + 1] = make_float2(v.z, v.w);
+            }
+    }
+}
+template <typename C>
+__device__ __forceinline__ void load_cb_beta(float2 (&B)[C::BPT][C::K / 2][C::K], const float *cbk, int rank, int tid)
+{
+#pragma unroll
+    for (int i = 0; i < C::BPT; ++i) {
+        const int x = rank * C::NBC + i * C::THREADS_ + tid;
+#pragma unroll
+        for (int jh = 0; jh < C::K / 2; ++jh)
+#pragma unroll
+            for (int b = 0; b < C::K; b += 4) {
+                const float4 v0 = __ldg(reinterpret_cast<const float4 *>(cbk + (size_t)(2 * jh) * C::Q + (size_t)x * C::K) + b / 4);
+                const float4 v1 = __ldg(reinterpret_cast<const float4 *>(cbk + (size_t)(2 * jh + 1) * C::Q + (size_t)x * C::K) + b / 4);
+                B[i][jh][b] = make_float2(v0.x, v1.x);
+                B[i][jh][b + 1] = make_float2(v0.y, v1.y);
+                B[i][jh][b + 2] = make_float2(v0.z, v1.z);
+                B[i][jh][b + 3] = make_float2(v0.w, v1.w);
+            }
+    }
+}
+
+// --------------------------------------------------------------------------------------
+// Forward call on a cluster: alpha sweep, log Z, beta sweep fused with Eq. 6-7.
+// --------------------------------------------------------------------------------------
 template <int LB, int KB, int CL, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
 {
@@ -157,7 +256,7 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
     const uint32_t cid = cluster_id_x(), ncl = cluster_count_x();
     const int n = p.n;
     const float NEG_INF = __int_as_float(0xff800000);
-    const float nlam = -p.lam2;
+    const float2 nl2 = splat2(-p.lam2);
 
     float *msg = smem + C::OFF_MSG;
     float *stage = smem + C::OFF_STAGE;
@@ -171,21 +270,13 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
     const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage);
     const uint32_t wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
 
-    // history of this cluster: [n][CL][QC]
-    float *hist = p.hist + (size_t)cid * n * C::Q;
+    float *hist = p.hist + (size_t)cid * n * C::Q;      // history of this cluster: [n][CL][QC]
 
-    // ---- codebook of the owned butterflies -> registers; push addresses
-    float cb[BPT][K][K];
     uint32_t push_a[BPT];          // alpha: K contiguous outputs (cluster address, buffer 0)
     uint32_t push_b[BPT][K];       // beta: K scalar outputs
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
-        const int xl = i * THREADS + tid;               // local butterfly
-        const int x = (int)rank * NBC + xl;             // global butterfly
-#pragma unroll
-        for (int j = 0; j < K; ++j)
-#pragma unroll
-            for (int l = 0; l < K; ++l) cb[i][j][l] = __ldg(p.cb + (size_t)j * C::Q + (size_t)x * K + l);
+        const int x = (int)rank * NBC + i * THREADS + tid;
         // alpha outputs L([x|l]) = index x*K + l; consumer butterfly x2 = (x*K + l) mod NB with
         // input slot j2 = (x*K) / NB; it lives in CTA x2 / NBC at [j2][x2 - r2*NBC]
         {
@@ -232,56 +323,63 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
         float off = 0.f, cmax = 0.f;
         cluster_sync();
         // ================= alpha sweep: step t maps L_t (buffer (t-1)&1) to L_{t+1} (buffer t&1)
-        for (int t = 1; t <= n; ++t) {
-            const int cur = (t - 1) & 1;
-            const float *Lin = msg + cur * QC;
-            const uint32_t nxt_off = (uint32_t)((t & 1) * QC) * 4u;
-            if (tid == 0) {                                          // spill L_t for the beta sweep
-                fence_proxy_async();
-                bulk_store(hist + ((size_t)(t - 1) * CL + rank) * QC, msg_u32 + (uint32_t)(cur * QC) * 4u, QC * 4u);
-                bulk_commit();
-            }
-            const float wt = w_s[t - 1];
-            float tmax = NEG_INF;
-#pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                const int xl = i * THREADS + tid;
-                float Lj[K];
-#pragma unroll
-                for (int j = 0; j < K; ++j) Lj[j] = Lin[j * NBC + xl];
-                float out[K];
-#pragma unroll
-                for (int l = 0; l < K; ++l) {
-                    float a[K], m = NEG_INF;
-#pragma unroll
-                    for (int j = 0; j < K; ++j) {
-                        const float d = wt - cb[i][j][l];
-                        a[j] = fmaf(d * d, nlam, Lj[j]);
-                        m = fmaxf(m, a[j]);
-                    }
-                    float sum = 0.f;
-#pragma unroll
-                    for (int j = 0; j < K; ++j) sum += ex2f(a[j] - m);
-                    out[l] = (m - off) + lg2f(sum);
-                    tmax = fmaxf(tmax, out[l]);
+        {
+            float2 cbA[BPT][K][K / 2];
+            load_cb_alpha<C>(cbA, p.cb, (int)rank, tid);
+            for (int t = 1; t <= n; ++t) {
+                const int cur = (t - 1) & 1;
+                const float *Lin = msg + cur * QC;
+                const uint32_t nxt_off = (uint32_t)((t & 1) * QC) * 4u;
+                if (tid == 0) {                                          // spill L_t for the beta sweep
+                    fence_proxy_async();
+                    bulk_store(hist + ((size_t)(t - 1) * CL + rank) * QC, msg_u32 + (uint32_t)(cur * QC) * 4u, QC * 4u);
+                    bulk_commit();
                 }
+                const float2 w2 = splat2(w_s[t - 1]);
+                const float2 off2 = splat2(off);
+                float tmax = NEG_INF;
 #pragma unroll
-                for (int l = 0; l < K; l += 4)
-                    st_cluster_v4(push_a[i] + nxt_off + 4u * l, out[l], out[l + 1], out[l + 2], out[l + 3]);
-            }
-            tmax = warp_max(tmax);
-            if (lane == 0) {
+                for (int i = 0; i < BPT; ++i) {
+                    const int xl = i * THREADS + tid;
+                    float2 Lj[K];
 #pragma unroll
-                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
+                    for (int j = 0; j < K; ++j) Lj[j] = splat2(Lin[j * NBC + xl]);
+                    float2 out[K / 2];
+#pragma unroll
+                    for (int h = 0; h < K / 2; ++h) {
+                        float2 a[K];
+#pragma unroll
+                        for (int j = 0; j < K; ++j) {
+                            const float2 d = sub2(cbA[i][j][h], w2);
+                            a[j] = fma2(mul2(d, d), nl2, Lj[j]);
+                        }
+                        const float2 m = max_pairs<K>(a);
+                        float2 sum = ex2f2(sub2(a[0], m));
+#pragma unroll
+                        for (int j = 1; j < K; ++j) sum = add2(sum, ex2f2(sub2(a[j], m)));
+                        out[h] = add2(sub2(m, off2), lg2f2(sum));
+                        tmax = max3f(tmax, m.x, m.y);
+                    }
+#pragma unroll
+                    for (int h = 0; h < K / 2; h += 2)
+                        st_cluster_v4(push_a[i] + nxt_off + 8u * h, out[h].x, out[h].y, out[h + 1].x, out[h + 1].y);
+                }
+                tmax = warp_max(tmax);
+                if (lane == 0) {
+#pragma unroll
+                    for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
+                }
+                O += (int)off;
+                if (tid == 0) {
+                    O_s[t + 1] = O;
+                    bulk_wait_read0();                                   // buffer `cur` may be overwritten next step
+                }
+                cluster_sync();
+                // gauge for the next step: the rounded maximum of the group maxima just seen
+                // (within log2 K of the true maximum of L_{t+1}, which is all a gauge needs)
+                cmax = warp_max(slot_max(wmax + (t & 1) * 32, lane, CL * NWARP)) - off;
+                off = rintf(cmax);
             }
-            O += (int)off;
-            if (tid == 0) {
-                O_s[t + 1] = O;
-                bulk_wait_read0();                                   // buffer `cur` may be overwritten next step
-            }
-            cluster_sync();
-            cmax = warp_max(lane < CL * NWARP ? wmax[(t & 1) * 32 + lane] : NEG_INF);
-            off = rintf(cmax);
         }
         // ================= log2 Z = O_{n+1} + LSE_q L_{n+1}(q); L_{n+1} sits in buffer n&1
         {
@@ -319,77 +417,88 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
         int P = 0;
         float offM = 0.f;
         cluster_sync();
-        for (int t = n; t >= 1; --t) {
-            const int cur = (n - t) & 1;
-            const float *Min = msg + cur * QC;
-            const uint32_t nxt_off = (uint32_t)((cur ^ 1) * QC) * 4u;
-            if (tid == 0 && t - 2 >= 1) {                            // prefetch L_{t-2}
-                fence_proxy_async();
-                const uint32_t s = loads_issued % C::NSTAGE;
-                mbar_expect_tx(mbar0 + 8u * s, QC * 4u);
-                bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(t - 3) * CL + rank) * QC, QC * 4u, mbar0 + 8u * s);
-                ++loads_issued;
-            }
-            const uint32_t st = loads_done % C::NSTAGE;
-            mbar_wait_bounded(mbar0 + 8u * st, (loads_done / C::NSTAGE) & 1u, abort_flag, p.diag);
-            ++loads_done;
-            const float *Lh = stage + st * QC;
-            const float wt = w_s[t - 1];
-            const float D = (float)(Ofin - O_s[t] - P) + lsefin;
-            float num = 0.f, den = 0.f, tmax = NEG_INF;
-#pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                const int xl = i * THREADS + tid;
-                float Mb[K];
-#pragma unroll
-                for (int b = 0; b < K; b += 4) {
-                    const float4 v = *reinterpret_cast<const float4 *>(Min + xl * K + b);
-                    Mb[b] = v.x; Mb[b + 1] = v.y; Mb[b + 2] = v.z; Mb[b + 3] = v.w;
+        {
+            float2 cbB[BPT][K / 2][K];
+            load_cb_beta<C>(cbB, p.cb, (int)rank, tid);
+            for (int t = n; t >= 1; --t) {
+                const int cur = (n - t) & 1;
+                const float *Min = msg + cur * QC;
+                const uint32_t nxt_off = (uint32_t)((cur ^ 1) * QC) * 4u;
+                if (tid == 0 && t - 2 >= 1) {                            // prefetch L_{t-2}
+                    fence_proxy_async();
+                    const uint32_t s = loads_issued % C::NSTAGE;
+                    mbar_expect_tx(mbar0 + 8u * s, QC * 4u);
+                    bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(t - 3) * CL + rank) * QC, QC * 4u, mbar0 + 8u * s);
+                    ++loads_issued;
                 }
+                const uint32_t st = loads_done % C::NSTAGE;
+                mbar_wait_bounded(mbar0 + 8u * st, (loads_done / C::NSTAGE) & 1u, abort_flag, p.diag);
+                ++loads_done;
+                const float *Lh = stage + st * QC;
+                const float2 w2 = splat2(w_s[t - 1]);
+                // the outputs are gauge-shifted by offM; fold the shift into the inputs and into D
+                const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
+                float2 num2 = make_float2(0.f, 0.f), den2 = make_float2(0.f, 0.f);
+                float tmax = NEG_INF;
 #pragma unroll
-                for (int j = 0; j < K; ++j) {
-                    float u[K], m = NEG_INF;
+                for (int i = 0; i < BPT; ++i) {
+                    const int xl = i * THREADS + tid;
+                    float2 Mb[K];
 #pragma unroll
-                    for (int b = 0; b < K; ++b) {
-                        const float d = wt - cb[i][j][b];
-                        u[b] = fmaf(d * d, nlam, Mb[b]);
-                        m = fmaxf(m, u[b]);
+                    for (int b = 0; b < K; b += 4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(Min + xl * K + b);
+                        Mb[b] = splat2(v.x - offM); Mb[b + 1] = splat2(v.y - offM);
+                        Mb[b + 2] = splat2(v.z - offM); Mb[b + 3] = splat2(v.w - offM);
                     }
-                    float sum = 0.f, craw = 0.f;
 #pragma unroll
-                    for (int b = 0; b < K; ++b) {
-                        const float pb = ex2f(u[b] - m);
-                        sum += pb;
-                        craw = fmaf(pb, cb[i][j][b], craw);
+                    for (int jh = 0; jh < K / 2; ++jh) {
+                        float2 u[K];
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+                            const float2 d = sub2(cbB[i][jh][b], w2);
+                            u[b] = fma2(mul2(d, d), nl2, Mb[b]);
+                        }
+                        const float2 m = max_pairs<K>(u);
+                        const float2 LhD = make_float2(Lh[(2 * jh) * NBC + xl] - Dm, Lh[(2 * jh + 1) * NBC + xl] - Dm);
+                        const float2 f = ex2f2(add2(m, LhD));
+                        float2 pb = ex2f2(sub2(u[0], m));
+                        float2 sum = pb, craw = mul2(pb, cbB[i][jh][0]);
+#pragma unroll
+                        for (int b = 1; b < K; ++b) {
+                            pb = ex2f2(sub2(u[b], m));
+                            sum = add2(sum, pb);
+                            craw = fma2(pb, cbB[i][jh][b], craw);
+                        }
+                        const float2 out = add2(m, lg2f2(sum));
+                        tmax = max3f(tmax, m.x, m.y);
+                        st_cluster_f32(push_b[i][2 * jh] + nxt_off, out.x);
+                        st_cluster_f32(push_b[i][2 * jh + 1] + nxt_off, out.y);
+                        num2 = fma2(f, craw, num2);
+                        den2 = fma2(f, sum, den2);
                     }
-                    const float out = (m - offM) + lg2f(sum);
-                    tmax = fmaxf(tmax, out);
-                    st_cluster_f32(push_b[i][j] + nxt_off, out);
-                    const float f = ex2f(m + Lh[j * NBC + xl] - D);
-                    den = fmaf(f, sum, den);
-                    num = fmaf(f, craw, num);
                 }
-            }
-            num = warp_sum(num); den = warp_sum(den); tmax = warp_max(tmax);
-            if (lane == 0) {
-#pragma unroll
-                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
-                st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u, num);
-                st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u + 4u, den);
-            }
-            P += (int)offM;
-            cluster_sync();
-            cmax = warp_max(lane < CL * NWARP ? wmax[(t & 1) * 32 + lane] : NEG_INF);
-            offM = rintf(cmax);
-            if (rank == 0 && warp == 0) {
-                float a = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4] : 0.f;
-                float b = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4 + 1] : 0.f;
-                a = warp_sum(a); b = warp_sum(b);
+                float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
+                tmax = warp_max(tmax);
                 if (lane == 0) {
-                    const float sw = a / b;
-                    p.soft[blk * n + t - 1] = sw;
-                    if (p.soft_copy) p.soft_copy[blk * n + t - 1] = sw;
-                    defect = fmaxf(defect, fabsf(b - 1.f));
+#pragma unroll
+                    for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
+                    st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u, num);
+                    st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u + 4u, den);
+                }
+                P += (int)offM;
+                cluster_sync();
+                cmax = warp_max(slot_max(wmax + (t & 1) * 32, lane, CL * NWARP));
+                offM = rintf(cmax);
+                if (rank == 0 && warp == 0) {
+                    float a = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4] : 0.f;
+                    float b = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4 + 1] : 0.f;
+                    a = warp_sum(a); b = warp_sum(b);
+                    if (lane == 0) {
+                        const float sw = a / b;
+                        p.soft[blk * n + t - 1] = sw;
+                        if (p.soft_copy) p.soft_copy[blk * n + t - 1] = sw;
+                        defect = fmaxf(defect, fabsf(b - 1.f));
+                    }
                 }
             }
         }
@@ -418,13 +527,17 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
     cluster_sync();             // no CTA leaves while a peer may still address its shared memory
 }
 
-
 // --------------------------------------------------------------------------------------
 // Backward call on a cluster.  Same butterflies; each message now carries a second value, the
 // conditional expectation of the centred emitted sum (At on the alpha side, Bt on the beta
 // side, see bcjr_generic.cuh for the recursions).  The codebook gradient of a state is owned
 // by the thread that owns the state, for every step and every block, so it accumulates in
 // registers and is written once, at the end, to this cluster's partial sum.
+//
+// Per step the beta sweep hands three sums over the posterior to rank 0:
+//   S0 = sum gamma,   S2 = sum gamma r,   ZS = sum gamma (g_t + (w_t - c) r / T)
+// (ZS is the sum over states of exactly what is added to the codebook-gradient accumulators)
+// and  grad_W[t] = -(1/T) Cov(r, w_t - c) = g_t - ZS/S0 + (S2/S0) (w_t - soft_t) / T.
 // --------------------------------------------------------------------------------------
 template <int LB, int KB, int CL, int THREADS>
 struct BwdClusterCfg {
@@ -458,7 +571,8 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
     const uint32_t cid = cluster_id_x(), ncl = cluster_count_x();
     const int n = p.n;
     const float NEG_INF = __int_as_float(0xff800000);
-    const float nlam = -p.lam2, invT = p.invT;
+    const float invT = p.invT;
+    const float2 nl2 = splat2(-p.lam2);
 
     float *msg = smem + BC::OFF_MSG;
     float *stage = smem + BC::OFF_STAGE;
@@ -475,19 +589,15 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
 
     float *hist = p.hist + (size_t)cid * n * 2 * C::Q;       // [n][CL][2][QC]
 
-    float cb[BPT][K][K], acc[BPT][K][K];
+    float2 acc[BPT][K / 2][K];                               // grad_codebook of the owned states, paired like cbB
     uint32_t push_a[BPT], push_b[BPT][K];
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
-        const int xl = i * THREADS + tid;
-        const int x = (int)rank * NBC + xl;
+        const int x = (int)rank * NBC + i * THREADS + tid;
 #pragma unroll
-        for (int j = 0; j < K; ++j)
+        for (int jh = 0; jh < K / 2; ++jh)
 #pragma unroll
-            for (int l = 0; l < K; ++l) {
-                cb[i][j][l] = __ldg(p.cb + (size_t)j * C::Q + (size_t)x * K + l);
-                acc[i][j][l] = 0.f;
-            }
+            for (int b = 0; b < K; ++b) acc[i][jh][b] = make_float2(0.f, 0.f);
         {
             const int q2 = x * K;
             const int j2 = q2 / NB, x2 = q2 % NB;
@@ -530,65 +640,71 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
         int O = 0;
         float off = 0.f, cmax = 0.f;
         cluster_sync();
-        // ================= alpha sweep
-        for (int t = 1; t <= n; ++t) {
-            const int cur = (t - 1) & 1;
-            const float *Lin = msg + cur * 2 * QC, *Ain = Lin + QC;
-            const uint32_t nxt_off = (uint32_t)((t & 1) * 2 * QC) * 4u;
-            if (tid == 0) {
-                fence_proxy_async();
-                bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)(cur * 2 * QC) * 4u, STEP_BYTES);
-                bulk_commit();
-            }
-            const float wt = w_s[t - 1], gt = g_s[t - 1];
-            const float gsh = -gt * sf_s[t - 1];                      // centring: h = g c - g soft
-            float tmax = NEG_INF;
-#pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                const int xl = i * THREADS + tid;
-                float Lj[K], Aj[K];
-#pragma unroll
-                for (int j = 0; j < K; ++j) { Lj[j] = Lin[j * NBC + xl]; Aj[j] = Ain[j * NBC + xl] + gsh; }
-                float outL[K], outA[K];
-#pragma unroll
-                for (int l = 0; l < K; ++l) {
-                    float a[K], m = NEG_INF;
-#pragma unroll
-                    for (int j = 0; j < K; ++j) {
-                        const float d = wt - cb[i][j][l];
-                        a[j] = fmaf(d * d, nlam, Lj[j]);
-                        m = fmaxf(m, a[j]);
-                    }
-                    float sum = 0.f, ax = 0.f;
-#pragma unroll
-                    for (int j = 0; j < K; ++j) {
-                        const float pj = ex2f(a[j] - m);
-                        sum += pj;
-                        ax = fmaf(pj, fmaf(gt, cb[i][j][l], Aj[j]), ax);
-                    }
-                    outL[l] = (m - off) + lg2f(sum);
-                    outA[l] = ax * rcpf(sum);
-                    tmax = fmaxf(tmax, outL[l]);
+        // ================= alpha sweep carrying (L, At)
+        {
+            float2 cbA[BPT][K][K / 2];
+            load_cb_alpha<C>(cbA, p.cb, (int)rank, tid);
+            for (int t = 1; t <= n; ++t) {
+                const int cur = (t - 1) & 1;
+                const float *Lin = msg + cur * 2 * QC, *Ain = Lin + QC;
+                const uint32_t nxt_off = (uint32_t)((t & 1) * 2 * QC) * 4u;
+                if (tid == 0) {
+                    fence_proxy_async();
+                    bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)(cur * 2 * QC) * 4u, STEP_BYTES);
+                    bulk_commit();
                 }
+                const float gt = g_s[t - 1];
+                const float gsh = -gt * sf_s[t - 1];                      // centring: h = g c - g soft
+                const float2 w2 = splat2(w_s[t - 1]), g2 = splat2(gt), off2 = splat2(off);
+                float tmax = NEG_INF;
 #pragma unroll
-                for (int l = 0; l < K; l += 4) {
-                    st_cluster_v4(push_a[i] + nxt_off + 4u * l, outL[l], outL[l + 1], outL[l + 2], outL[l + 3]);
-                    st_cluster_v4(push_a[i] + nxt_off + QC * 4u + 4u * l, outA[l], outA[l + 1], outA[l + 2], outA[l + 3]);
+                for (int i = 0; i < BPT; ++i) {
+                    const int xl = i * THREADS + tid;
+                    float2 Lj[K], Aj[K];
+#pragma unroll
+                    for (int j = 0; j < K; ++j) { Lj[j] = splat2(Lin[j * NBC + xl]); Aj[j] = splat2(Ain[j * NBC + xl] + gsh); }
+                    float2 outL[K / 2], outA[K / 2];
+#pragma unroll
+                    for (int h = 0; h < K / 2; ++h) {
+                        float2 a[K];
+#pragma unroll
+                        for (int j = 0; j < K; ++j) {
+                            const float2 d = sub2(cbA[i][j][h], w2);
+                            a[j] = fma2(mul2(d, d), nl2, Lj[j]);
+                        }
+                        const float2 m = max_pairs<K>(a);
+                        float2 pj = ex2f2(sub2(a[0], m));
+                        float2 sum = pj, ax = mul2(pj, fma2(g2, cbA[i][0][h], Aj[0]));
+#pragma unroll
+                        for (int j = 1; j < K; ++j) {
+                            pj = ex2f2(sub2(a[j], m));
+                            sum = add2(sum, pj);
+                            ax = fma2(pj, fma2(g2, cbA[i][j][h], Aj[j]), ax);
+                        }
+                        outL[h] = add2(sub2(m, off2), lg2f2(sum));
+                        outA[h] = mul2(ax, rcpf2(sum));
+                        tmax = max3f(tmax, m.x, m.y);
+                    }
+#pragma unroll
+                    for (int h = 0; h < K / 2; h += 2) {
+                        st_cluster_v4(push_a[i] + nxt_off + 8u * h, outL[h].x, outL[h].y, outL[h + 1].x, outL[h + 1].y);
+                        st_cluster_v4(push_a[i] + nxt_off + QC * 4u + 8u * h, outA[h].x, outA[h].y, outA[h + 1].x, outA[h + 1].y);
+                    }
                 }
-            }
-            tmax = warp_max(tmax);
-            if (lane == 0) {
+                tmax = warp_max(tmax);
+                if (lane == 0) {
 #pragma unroll
-                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 64) * 4u, tmax);
+                    for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 64) * 4u, tmax);
+                }
+                O += (int)off;
+                if (tid == 0) {
+                    O_s[t + 1] = O;
+                    bulk_wait_read0();
+                }
+                cluster_sync();
+                cmax = warp_max(slot_max(wmax + (t & 1) * 64, lane, CL * NWARP)) - off;
+                off = rintf(cmax);
             }
-            O += (int)off;
-            if (tid == 0) {
-                O_s[t + 1] = O;
-                bulk_wait_read0();
-            }
-            cluster_sync();
-            cmax = warp_max(slot_max(wmax + (t & 1) * 64, lane, CL * NWARP));
-            off = rintf(cmax);
         }
         // ================= log2 Z
         {
@@ -610,7 +726,7 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
             lsefin = cmax + lg2f(v);
         }
         const int Ofin = O;
-        // ================= beta sweep with the gradient contraction
+        // ================= beta sweep carrying (M, Bt), with the gradient contraction
         for (int q = tid; q < 2 * QC; q += THREADS) msg[q] = 0.f;    // M_n = 0, Bt_n = 0 (parity 0)
         if (tid == 0) {
             fence_proxy_async();
@@ -624,95 +740,102 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
         int P = 0;
         float offM = 0.f;
         cluster_sync();
-        for (int t = n; t >= 1; --t) {
-            const int cur = (n - t) & 1;
-            const float *Min = msg + cur * 2 * QC, *Bin = Min + QC;
-            const uint32_t nxt_off = (uint32_t)((cur ^ 1) * 2 * QC) * 4u;
-            if (tid == 0 && t - 2 >= 1) {
-                fence_proxy_async();
-                const uint32_t s = loads_issued % BC::NSTAGE;
-                mbar_expect_tx(mbar0 + 8u * s, STEP_BYTES);
-                bulk_load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(t - 3) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
-                ++loads_issued;
-            }
-            const uint32_t st = loads_done % BC::NSTAGE;
-            mbar_wait_bounded(mbar0 + 8u * st, (loads_done / BC::NSTAGE) & 1u, abort_flag, p.diag);
-            ++loads_done;
-            const float *Lh = stage + st * 2 * QC, *Ah = Lh + QC;
-            const float wt = w_s[t - 1], gt = g_s[t - 1], sft = sf_s[t - 1];
-            const float gsh = -gt * sft;
-            const float D = (float)(Ofin - O_s[t] - P) + lsefin;
-            float S0 = 0.f, S1 = 0.f, S2 = 0.f, S3 = 0.f, tmax = NEG_INF;
-#pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                const int xl = i * THREADS + tid;
-                float Mb[K], Yb[K];
-#pragma unroll
-                for (int b = 0; b < K; b += 4) {
-                    const float4 v = *reinterpret_cast<const float4 *>(Min + xl * K + b);
-                    Mb[b] = v.x; Mb[b + 1] = v.y; Mb[b + 2] = v.z; Mb[b + 3] = v.w;
-                    const float4 y = *reinterpret_cast<const float4 *>(Bin + xl * K + b);
-                    Yb[b] = y.x + gsh; Yb[b + 1] = y.y + gsh; Yb[b + 2] = y.z + gsh; Yb[b + 3] = y.w + gsh;
+        {
+            float2 cbB[BPT][K / 2][K];
+            load_cb_beta<C>(cbB, p.cb, (int)rank, tid);
+            for (int t = n; t >= 1; --t) {
+                const int cur = (n - t) & 1;
+                const float *Min = msg + cur * 2 * QC, *Bin = Min + QC;
+                const uint32_t nxt_off = (uint32_t)((cur ^ 1) * 2 * QC) * 4u;
+                if (tid == 0 && t - 2 >= 1) {
+                    fence_proxy_async();
+                    const uint32_t s = loads_issued % BC::NSTAGE;
+                    mbar_expect_tx(mbar0 + 8u * s, STEP_BYTES);
+                    bulk_load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(t - 3) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
+                    ++loads_issued;
                 }
+                const uint32_t st = loads_done % BC::NSTAGE;
+                mbar_wait_bounded(mbar0 + 8u * st, (loads_done / BC::NSTAGE) & 1u, abort_flag, p.diag);
+                ++loads_done;
+                const float *Lh = stage + st * 2 * QC, *Ah = Lh + QC;
+                const float wt = w_s[t - 1], gt = g_s[t - 1], sft = sf_s[t - 1];
+                const float gsh = -gt * sft;
+                const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT);
+                const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
+                float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
+                float tmax = NEG_INF;
 #pragma unroll
-                for (int j = 0; j < K; ++j) {
-                    float u[K], d[K], m = NEG_INF;
+                for (int i = 0; i < BPT; ++i) {
+                    const int xl = i * THREADS + tid;
+                    float2 Mb[K], Yb[K];
 #pragma unroll
-                    for (int b = 0; b < K; ++b) {
-                        d[b] = wt - cb[i][j][b];
-                        u[b] = fmaf(d[b] * d[b], nlam, Mb[b]);
-                        m = fmaxf(m, u[b]);
+                    for (int b = 0; b < K; b += 4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(Min + xl * K + b);
+                        Mb[b] = splat2(v.x - offM); Mb[b + 1] = splat2(v.y - offM);
+                        Mb[b + 2] = splat2(v.z - offM); Mb[b + 3] = splat2(v.w - offM);
+                        const float4 y = *reinterpret_cast<const float4 *>(Bin + xl * K + b);
+                        Yb[b] = splat2(y.x + gsh); Yb[b + 1] = splat2(y.y + gsh);
+                        Yb[b + 2] = splat2(y.z + gsh); Yb[b + 3] = splat2(y.w + gsh);
                     }
-                    const float Lhj = Lh[j * NBC + xl], Ahj = Ah[j * NBC + xl];
-                    const float f = ex2f(m + Lhj - D);
-                    const float fg = f * gt, fi = f * invT;
-                    float sum = 0.f, craw = 0.f, yacc = 0.f, ycc = 0.f;
 #pragma unroll
-                    for (int b = 0; b < K; ++b) {
-                        const float pb = ex2f(u[b] - m);
-                        const float y = fmaf(gt, cb[i][j][b], Yb[b]);        // h + Bt
-                        const float pc = pb * cb[i][j][b];
-                        sum += pb;
-                        craw += pc;
-                        yacc = fmaf(pb, y, yacc);
-                        ycc = fmaf(pc, y, ycc);
-                        const float r = y + Ahj;
-                        acc[i][j][b] = fmaf(pb, fmaf(fi * d[b], r, fg), acc[i][j][b]);
+                    for (int jh = 0; jh < K / 2; ++jh) {
+                        float2 u[K], d[K];
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+                            d[b] = sub2(w2, cbB[i][jh][b]);
+                            u[b] = fma2(mul2(d[b], d[b]), nl2, Mb[b]);
+                        }
+                        const float2 m = max_pairs<K>(u);
+                        const float2 Ahj = make_float2(Ah[(2 * jh) * NBC + xl], Ah[(2 * jh + 1) * NBC + xl]);
+                        const float2 LhD = make_float2(Lh[(2 * jh) * NBC + xl] - Dm, Lh[(2 * jh + 1) * NBC + xl] - Dm);
+                        const float2 f = ex2f2(add2(m, LhD));
+                        const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
+                        float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+                            const float2 pb = ex2f2(sub2(u[b], m));
+                            const float2 y = fma2(g2, cbB[i][jh][b], Yb[b]);            // h + Bt
+                            const float2 z = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);      // f (g + (w - c) r / T)
+                            sum = add2(sum, pb);
+                            ya = fma2(pb, y, ya);
+                            zs = fma2(pb, z, zs);
+                            acc[i][jh][b] = fma2(pb, z, acc[i][jh][b]);
+                        }
+                        const float2 outM = add2(m, lg2f2(sum));
+                        const float2 outB = mul2(ya, rcpf2(sum));
+                        tmax = max3f(tmax, m.x, m.y);
+                        st_cluster_f32(push_b[i][2 * jh] + nxt_off, outM.x);
+                        st_cluster_f32(push_b[i][2 * jh + 1] + nxt_off, outM.y);
+                        st_cluster_f32(push_b[i][2 * jh] + nxt_off + QC * 4u, outB.x);
+                        st_cluster_f32(push_b[i][2 * jh + 1] + nxt_off + QC * 4u, outB.y);
+                        S0 = fma2(f, sum, S0);
+                        S2 = fma2(f, fma2(Ahj, sum, ya), S2);
+                        ZS = add2(ZS, zs);
                     }
-                    const float outM = (m - offM) + lg2f(sum);
-                    tmax = fmaxf(tmax, outM);
-                    st_cluster_f32(push_b[i][j] + nxt_off, outM);
-                    st_cluster_f32(push_b[i][j] + nxt_off + QC * 4u, yacc * rcpf(sum));
-                    // sums over the posterior: gamma = f * p_b
-                    const float s2 = fmaf(Ahj, sum, yacc);                    // sum_b p_b r_b
-                    S0 = fmaf(f, sum, S0);
-                    S1 = fmaf(f, fmaf(-sft, sum, craw), S1);                  // sum gamma (c - soft)
-                    S2 = fmaf(f, s2, S2);                                     // sum gamma r
-                    S3 = fmaf(f, fmaf(-sft, s2, fmaf(Ahj, craw, ycc)), S3);   // sum gamma r (c - soft)
                 }
-            }
-            S0 = warp_sum(S0); S1 = warp_sum(S1); S2 = warp_sum(S2); S3 = warp_sum(S3);
-            tmax = warp_max(tmax);
-            if (lane == 0) {
-#pragma unroll
-                for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 64) * 4u, tmax);
-                const uint32_t pd = part_dst + (uint32_t)((t & 1) * 256) * 4u;
-                st_cluster_f32(pd, S0); st_cluster_f32(pd + 4u, S1); st_cluster_f32(pd + 8u, S2); st_cluster_f32(pd + 12u, S3);
-            }
-            P += (int)offM;
-            cluster_sync();
-            cmax = warp_max(slot_max(wmax + (t & 1) * 64, lane, CL * NWARP));
-            offM = rintf(cmax);
-            if (rank == 0 && warp == 0) {
-                const float *pp = part + (t & 1) * 256 + lane * 4;
-                const bool on = lane < CL * NWARP, on2 = lane + 32 < CL * NWARP;
-                float a0 = on ? pp[0] : 0.f, a1 = on ? pp[1] : 0.f, a2 = on ? pp[2] : 0.f, a3 = on ? pp[3] : 0.f;
-                if (on2) { a0 += pp[128]; a1 += pp[129]; a2 += pp[130]; a3 += pp[131]; }
-                a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+                const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), zz = warp_sum(ZS.x + ZS.y);
+                tmax = warp_max(tmax);
                 if (lane == 0) {
-                    const float i0 = 1.f / a0;
-                    p.gW[blk * n + t - 1] = invT * (a3 * i0 - (a2 * i0) * (a1 * i0));
-                    defect = fmaxf(defect, fabsf(a0 - 1.f));
+#pragma unroll
+                    for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 64) * 4u, tmax);
+                    const uint32_t pd = part_dst + (uint32_t)((t & 1) * 256) * 4u;
+                    st_cluster_f32(pd, s0); st_cluster_f32(pd + 4u, s2); st_cluster_f32(pd + 8u, zz);
+                }
+                P += (int)offM;
+                cluster_sync();
+                cmax = warp_max(slot_max(wmax + (t & 1) * 64, lane, CL * NWARP));
+                offM = rintf(cmax);
+                if (rank == 0 && warp == 0) {
+                    const float *pp = part + (t & 1) * 256 + lane * 4;
+                    const bool on = lane < CL * NWARP, on2 = lane + 32 < CL * NWARP;
+                    float a0 = on ? pp[0] : 0.f, a2 = on ? pp[1] : 0.f, az = on ? pp[2] : 0.f;
+                    if (on2) { a0 += pp[128]; a2 += pp[129]; az += pp[130]; }
+                    a0 = warp_sum(a0); a2 = warp_sum(a2); az = warp_sum(az);
+                    if (lane == 0) {
+                        const float i0 = 1.f / a0;
+                        p.gW[blk * n + t - 1] = (gt - az * i0) + (a2 * i0) * (wt - sft) * invT;
+                        defect = fmaxf(defect, fabsf(a0 - 1.f));
+                    }
                 }
             }
         }
@@ -724,9 +847,12 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
     for (int i = 0; i < BPT; ++i) {
         const int x = (int)rank * NBC + i * THREADS + tid;
 #pragma unroll
-        for (int j = 0; j < K; ++j)
+        for (int jh = 0; jh < K / 2; ++jh)
 #pragma unroll
-            for (int b = 0; b < K; ++b) gc[(size_t)j * C::Q + (size_t)x * K + b] = acc[i][j][b];
+            for (int b = 0; b < K; ++b) {
+                gc[(size_t)(2 * jh) * C::Q + (size_t)x * K + b] = acc[i][jh][b].x;
+                gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[i][jh][b].y;
+            }
     }
     if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
     cluster_sync();
