@@ -175,6 +175,12 @@ bcjr_status launch_vit_generic(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
 }
 
 #ifndef BCJR_NO_CLUSTER
+#ifndef FWD_THREADS_K2
+#define FWD_THREADS_K2 512
+#endif
+#ifndef FWD_CL_K2
+#define FWD_CL_K2 2
+#endif
 // One cluster of CL CTAs per weight block in flight; the grid is the number of clusters the
 // GPU can hold at once (persistent loop over blocks inside the kernel).
 template <typename Kern>
@@ -256,7 +262,7 @@ bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_co
 bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
-    if (k == 2) return launch_fwd_cluster_t<16, 2, 2, 512>(ctx, p, st);
+    if (k == 2) return launch_fwd_cluster_t<16, 2, FWD_CL_K2, FWD_THREADS_K2>(ctx, p, st);
     if (k == 3) return launch_fwd_cluster_t<16, 3, 2, 512>(ctx, p, st);
     return BCJR_EUNSUPPORTED;
 }

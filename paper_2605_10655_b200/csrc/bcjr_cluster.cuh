@@ -39,6 +39,26 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, f
     asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
                  : "memory");
 }
+// Asynchronous remote stores: the data lands in the destination CTA's shared memory and the
+// destination's mbarrier is credited with the bytes, so the consumer learns that its inputs are
+// complete from the mbarrier alone -- no cluster-wide barrier and no fence on the producer side.
+__device__ __forceinline__ void st_async_f32(uint32_t addr, float v, uint32_t mbar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(addr), "f"(v), "r"(mbar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_v2(uint32_t addr, float a, float b, uint32_t mbar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(addr), "f"(a),
+                 "f"(b), "r"(mbar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_v4(uint32_t addr, float a, float b, float c, float d, uint32_t mbar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+                 "f"(a), "f"(b), "f"(c), "f"(d), "r"(mbar)
+                 : "memory");
+}
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_sync() { cluster_arrive(); cluster_wait(); }
@@ -184,24 +204,21 @@ struct ClusterCfg {
     static_assert(CL * NWARP <= 64, "at most two partials per lane");
     static_assert(NBC % K == 0 || CL == 1, "vector pushes must stay inside one CTA");
     // shared memory carve-up (floats unless noted)
-    static constexpr int OFF_MSG = 0;                         // [2][QC]
-    static constexpr int OFF_STAGE = OFF_MSG + 2 * QC;        // [NSTAGE][QC]
+    static constexpr int NBUF = 3;                            // message buffers (see the step protocol)
+    static constexpr int OFF_MSG = 0;                         // [NBUF][QC]
+    static constexpr int OFF_STAGE = OFF_MSG + NBUF * QC;     // [NSTAGE][QC]
     static constexpr int OFF_W = OFF_STAGE + NSTAGE * QC;     // [MAX_N]
     static constexpr int OFF_O = OFF_W + MAX_N;               // int [MAX_N + 2]
-    static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;    // [2][32]
-    static constexpr int OFF_PART = OFF_WMAX + 64;            // [2][32][4]
-    static constexpr int OFF_LZ = OFF_PART + 256;             // [2][32]
-    static constexpr int OFF_MBAR = OFF_LZ + 64;              // uint64 [NSTAGE] (8-byte aligned: even offset)
-    static constexpr int OFF_FLAG = OFF_MBAR + 2 * NSTAGE + 2;
+    static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;    // [NBUF][64]
+    static constexpr int OFF_PART = OFF_WMAX + 192;           // [NBUF][64][2]
+    static constexpr int OFF_LZ = OFF_PART + 384;             // [2][64]
+    static constexpr int OFF_MBAR = OFF_LZ + 128;             // uint64 [NSTAGE] history ring, then [NBUF] message buffers
+    static constexpr int OFF_FLAG = OFF_MBAR + 2 * (NSTAGE + NBUF) + 2;
     static constexpr int SMEM_FLOATS = OFF_FLAG + 4;
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
     static_assert((QC * 4) % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
-
-// --------------------------------------------------------------------------------------
-// Forward call on a cluster: alpha sweep, log Z, beta sweep fused with Eq. 6-7.
-// --------------------------------------------------------------------------------------
 
 // Codebook of the owned butterflies, in the pairing a sweep wants.  Alpha pairs neighbouring
 // outputs l: A[i][j][h] = (c[j|x|2h], c[j|x|2h+1]);  beta pairs neighbouring inputs j:
@@ -244,12 +261,25 @@ __device__ __forceinline__ void load_cb_beta(float2 (&B)[C::BPT][C::K / 2][C::K]
 
 // --------------------------------------------------------------------------------------
 // Forward call on a cluster: alpha sweep, log Z, beta sweep fused with Eq. 6-7.
+//
+// Step protocol (no per-step barrier).  The messages live in three buffers.  Step s reads
+// buffer s%3 and every thread pushes its outputs, with st.async, into buffer (s+1)%3 of the
+// consumer's CTA, crediting that CTA's mbarrier full[(s+1)%3].  A thread starts step s+1 when
+// full[(s+1)%3] of its own CTA completes, i.e. when every input of its CTA has landed.
+// Three buffers make this safe without any further handshake: a thread can only be writing
+// buffer b again (step s+3) after every thread of the cluster has finished step s+2, hence
+// has long finished reading b (step s+1).  The per-warp partial results (gauge maximum,
+// posterior sums) travel the same way into small slot arrays.  One thread per CTA arms each
+// phase (arrive.expect_tx) and moves the history with bulk copies.
 // --------------------------------------------------------------------------------------
 template <int LB, int KB, int CL, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
 {
     using C = ClusterCfg<LB, KB, CL, THREADS>;
     constexpr int K = C::K, NB = C::NB, NBC = C::NBC, BPT = C::BPT, QC = C::QC, NWARP = C::NWARP;
+    constexpr int NBUF = C::NBUF, SLOTS = CL * NWARP;
+    constexpr uint32_t TX_MSG = QC * 4u + SLOTS * 4u;            // messages + gauge slots per phase
+    constexpr uint32_t TX_PART = SLOTS * 8u;                     // posterior partial sums (rank 0 only)
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = cluster_ctarank();
@@ -266,27 +296,30 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
     float *part = smem + C::OFF_PART;
     float *lz = smem + C::OFF_LZ;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
-    const uint32_t mbar0 = smem_u32(smem + C::OFF_MBAR);
+    const uint32_t mbar_stage = smem_u32(smem + C::OFF_MBAR);
+    const uint32_t mbar_full = mbar_stage + 8u * C::NSTAGE;
     const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage);
     const uint32_t wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
 
     float *hist = p.hist + (size_t)cid * n * C::Q;      // history of this cluster: [n][CL][QC]
 
-    uint32_t push_a[BPT];          // alpha: K contiguous outputs (cluster address, buffer 0)
-    uint32_t push_b[BPT][K];       // beta: K scalar outputs
+    // Destinations.  alpha: the K outputs of butterfly x are L([x|l]) = index x*K + l; their
+    // consumer is butterfly (x*K) mod NB, input slot (x*K) / NB, one CTA, contiguous.  beta: the
+    // output M([j|x]) = index j*NB + x goes to butterfly (j*NB + x) / K as its input x mod K;
+    // its CTA is floor(j*CL/K), a compile-time function of j.
+    uint32_t push_a[BPT], push_a_mbar[BPT], push_b[BPT][K], full_of[CL];
+#pragma unroll
+    for (int r = 0; r < CL; ++r) full_of[r] = mapa_u32(mbar_full, (uint32_t)r);
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
         const int x = (int)rank * NBC + i * THREADS + tid;
-        // alpha outputs L([x|l]) = index x*K + l; consumer butterfly x2 = (x*K + l) mod NB with
-        // input slot j2 = (x*K) / NB; it lives in CTA x2 / NBC at [j2][x2 - r2*NBC]
         {
             const int q2 = x * K;
             const int j2 = q2 / NB, x2 = q2 % NB;
             const int r2 = x2 / NBC, xl2 = x2 % NBC;
             push_a[i] = mapa_u32(msg_u32 + (uint32_t)(j2 * NBC + xl2) * 4u, (uint32_t)r2);
+            push_a_mbar[i] = mapa_u32(mbar_full, (uint32_t)r2);
         }
-        // beta outputs M([j|x]) = index j*NB + x; consumer butterfly x1 = (j*NB + x) / K reads it
-        // as its input b1 = x mod K; it lives in CTA x1 / NBC at [(x1 - r1*NBC)*K + b1]
 #pragma unroll
         for (int j = 0; j < K; ++j) {
             const int q1 = j * NB + x;
@@ -295,6 +328,7 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
             push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(xl1 * K + b1) * 4u, (uint32_t)r1);
         }
     }
+    static_assert(K % CL == 0, "beta destinations: CTA of output j is j*CL/K");
     // partial-result slots: every warp of every CTA writes one entry into every CTA's array
     uint32_t wmax_dst[CL], lz_dst[CL];
 #pragma unroll
@@ -302,37 +336,54 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
         wmax_dst[r] = mapa_u32(wmax_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
         lz_dst[r] = mapa_u32(lz_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
     }
-    const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 16u, 0u);
+    const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 8u, 0u);
 
     if (tid == 0) {
-        for (int s = 0; s < C::NSTAGE; ++s) mbar_init(mbar0 + 8u * s, 1);
+        for (int s = 0; s < C::NSTAGE + NBUF; ++s) mbar_init(mbar_stage + 8u * s, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     uint32_t loads_done = 0;       // bulk loads consumed so far (stage = count % NSTAGE, parity = (count / NSTAGE) & 1)
     uint32_t loads_issued = 0;
+    uint32_t full_phase = 0;       // bit b = parity to wait for on full[b]
+    int ib = 0;                    // buffer holding the inputs of the next step
     float defect = 0.f, zgap = 0.f;
+
+    // wait until every input of this CTA for the coming step has landed in buffer b
+    auto wait_inputs = [&](int b) {
+        mbar_wait_bounded(mbar_full + 8u * b, (full_phase >> b) & 1u, abort_flag, p.diag);
+        full_phase ^= 1u << b;
+    };
 
     for (int64_t blk = cid; blk < p.B; blk += ncl) {
         const float *w = p.W + blk * n;
         for (int t = tid; t < n; t += THREADS) w_s[t] = __ldg(w + t);
-        for (int q = tid; q < QC; q += THREADS) msg[q] = 0.f;        // L_1 = 0 (buffer 0)
+        for (int q = tid; q < QC; q += THREADS) msg[ib * QC + q] = 0.f;      // L_1 = 0
         if (tid == 0) O_s[1] = 0;
         int O = 0;
         float off = 0.f, cmax = 0.f;
         cluster_sync();
-        // ================= alpha sweep: step t maps L_t (buffer (t-1)&1) to L_{t+1} (buffer t&1)
+        // ================= alpha sweep: step t maps L_t to L_{t+1}
         {
             float2 cbA[BPT][K][K / 2];
             load_cb_alpha<C>(cbA, p.cb, (int)rank, tid);
             for (int t = 1; t <= n; ++t) {
-                const int cur = (t - 1) & 1;
-                const float *Lin = msg + cur * QC;
-                const uint32_t nxt_off = (uint32_t)((t & 1) * QC) * 4u;
-                if (tid == 0) {                                          // spill L_t for the beta sweep
+                const int ob = ib == NBUF - 1 ? 0 : ib + 1;
+                if (t > 1) {
+                    wait_inputs(ib);
+                    // gauge: rounded maximum of the group maxima of the previous step (within
+                    // log2 K of the maximum of L_t, which is all a gauge needs)
+                    cmax = warp_max(slot_max(wmax + ib * 64, lane, SLOTS)) - off;
+                    off = rintf(cmax);
+                }
+                const float *Lin = msg + ib * QC;
+                const uint32_t ob_off = (uint32_t)(ob * QC) * 4u, ob_mbar = 8u * ob;
+                if (tid == 0) {
+                    mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
+                    bulk_wait_read0();                                   // previous spill has left its buffer
                     fence_proxy_async();
-                    bulk_store(hist + ((size_t)(t - 1) * CL + rank) * QC, msg_u32 + (uint32_t)(cur * QC) * 4u, QC * 4u);
+                    bulk_store(hist + ((size_t)(t - 1) * CL + rank) * QC, msg_u32 + (uint32_t)(ib * QC) * 4u, QC * 4u);
                     bulk_commit();
                 }
                 const float2 w2 = splat2(w_s[t - 1]);
@@ -362,28 +413,24 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
                     }
 #pragma unroll
                     for (int h = 0; h < K / 2; h += 2)
-                        st_cluster_v4(push_a[i] + nxt_off + 8u * h, out[h].x, out[h].y, out[h + 1].x, out[h + 1].y);
+                        st_async_v4(push_a[i] + ob_off + 8u * h, out[h].x, out[h].y, out[h + 1].x, out[h + 1].y,
+                                    push_a_mbar[i] + ob_mbar);
                 }
                 tmax = warp_max(tmax);
                 if (lane == 0) {
 #pragma unroll
-                    for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
+                    for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 64) * 4u, tmax, full_of[r] + ob_mbar);
                 }
                 O += (int)off;
-                if (tid == 0) {
-                    O_s[t + 1] = O;
-                    bulk_wait_read0();                                   // buffer `cur` may be overwritten next step
-                }
-                cluster_sync();
-                // gauge for the next step: the rounded maximum of the group maxima just seen
-                // (within log2 K of the true maximum of L_{t+1}, which is all a gauge needs)
-                cmax = warp_max(slot_max(wmax + (t & 1) * 32, lane, CL * NWARP)) - off;
-                off = rintf(cmax);
+                if (tid == 0) O_s[t + 1] = O;
+                ib = ob;
             }
         }
-        // ================= log2 Z = O_{n+1} + LSE_q L_{n+1}(q); L_{n+1} sits in buffer n&1
+        // ================= log2 Z = O_{n+1} + LSE_q L_{n+1}(q); L_{n+1} sits in buffer ib
+        wait_inputs(ib);
+        cmax = warp_max(slot_max(wmax + ib * 64, lane, SLOTS)) - off;
         {
-            const float *Lfin = msg + (n & 1) * QC;
+            const float *Lfin = msg + ib * QC;
             float ssum = 0.f;
             for (int q = tid; q < QC; q += THREADS) ssum += ex2f(Lfin[q] - cmax);
             ssum = warp_sum(ssum);
@@ -396,21 +443,21 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
         }
         float lsefin;
         {
-            float v = lane < CL * NWARP ? lz[lane] : 0.f;
+            float v = (lane < SLOTS ? lz[lane] : 0.f) + (lane + 32 < SLOTS ? lz[lane + 32] : 0.f);
             v = warp_sum(v);
             lsefin = cmax + lg2f(v);
         }
         const int Ofin = O;
         if (tid == 0 && rank == 0 && p.logZ)
             p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
-        // ================= beta sweep: step t maps M_t (buffer (n-t)&1) to M_{t-1}
-        for (int q = tid; q < QC; q += THREADS) msg[q] = 0.f;        // M_n = 0 (buffer 0)
+        // ================= beta sweep: step t maps M_t to M_{t-1}
+        for (int q = tid; q < QC; q += THREADS) msg[ib * QC + q] = 0.f;      // M_n = 0
         if (tid == 0) {                                              // prefetch L_n and L_{n-1}
             fence_proxy_async();
             for (int d = 0; d < 2 && n - d >= 1; ++d) {
                 const uint32_t s = loads_issued % C::NSTAGE;
-                mbar_expect_tx(mbar0 + 8u * s, QC * 4u);
-                bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(n - d - 1) * CL + rank) * QC, QC * 4u, mbar0 + 8u * s);
+                mbar_expect_tx(mbar_stage + 8u * s, QC * 4u);
+                bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(n - d - 1) * CL + rank) * QC, QC * 4u, mbar_stage + 8u * s);
                 ++loads_issued;
             }
         }
@@ -420,19 +467,44 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
         {
             float2 cbB[BPT][K / 2][K];
             load_cb_beta<C>(cbB, p.cb, (int)rank, tid);
+            // rank 0, warp 0: turn the partial sums of step t (slots of buffer b) into soft[t]
+            auto finish_step = [&](int t, int b) {
+                if (rank == 0 && warp == 0) {
+                    float a = lane < SLOTS ? part[(b * 64 + lane) * 2] : 0.f;
+                    float c = lane < SLOTS ? part[(b * 64 + lane) * 2 + 1] : 0.f;
+                    if (lane + 32 < SLOTS) { a += part[(b * 64 + lane + 32) * 2]; c += part[(b * 64 + lane + 32) * 2 + 1]; }
+                    a = warp_sum(a); c = warp_sum(c);
+                    if (lane == 0) {
+                        const float sw = a / c;
+                        p.soft[blk * n + t - 1] = sw;
+                        if (p.soft_copy) p.soft_copy[blk * n + t - 1] = sw;
+                        defect = fmaxf(defect, fabsf(c - 1.f));
+                    }
+                }
+            };
             for (int t = n; t >= 1; --t) {
-                const int cur = (n - t) & 1;
-                const float *Min = msg + cur * QC;
-                const uint32_t nxt_off = (uint32_t)((cur ^ 1) * QC) * 4u;
-                if (tid == 0 && t - 2 >= 1) {                            // prefetch L_{t-2}
-                    fence_proxy_async();
-                    const uint32_t s = loads_issued % C::NSTAGE;
-                    mbar_expect_tx(mbar0 + 8u * s, QC * 4u);
-                    bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(t - 3) * CL + rank) * QC, QC * 4u, mbar0 + 8u * s);
-                    ++loads_issued;
+                const int ob = ib == NBUF - 1 ? 0 : ib + 1;
+                if (t < n) {
+                    wait_inputs(ib);
+                    cmax = warp_max(slot_max(wmax + ib * 64, lane, SLOTS));
+                    P += (int)offM;                                      // P_t
+                    offM = rintf(cmax);
+                    finish_step(t + 1, ib);
+                }
+                const float *Min = msg + ib * QC;
+                const uint32_t ob_off = (uint32_t)(ob * QC) * 4u, ob_mbar = 8u * ob;
+                if (tid == 0) {
+                    mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
+                    if (t - 2 >= 1) {                                    // prefetch L_{t-2}
+                        fence_proxy_async();
+                        const uint32_t s = loads_issued % C::NSTAGE;
+                        mbar_expect_tx(mbar_stage + 8u * s, QC * 4u);
+                        bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(t - 3) * CL + rank) * QC, QC * 4u, mbar_stage + 8u * s);
+                        ++loads_issued;
+                    }
                 }
                 const uint32_t st = loads_done % C::NSTAGE;
-                mbar_wait_bounded(mbar0 + 8u * st, (loads_done / C::NSTAGE) & 1u, abort_flag, p.diag);
+                mbar_wait_bounded(mbar_stage + 8u * st, (loads_done / C::NSTAGE) & 1u, abort_flag, p.diag);
                 ++loads_done;
                 const float *Lh = stage + st * QC;
                 const float2 w2 = splat2(w_s[t - 1]);
@@ -471,49 +543,38 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
                         }
                         const float2 out = add2(m, lg2f2(sum));
                         tmax = max3f(tmax, m.x, m.y);
-                        st_cluster_f32(push_b[i][2 * jh] + nxt_off, out.x);
-                        st_cluster_f32(push_b[i][2 * jh + 1] + nxt_off, out.y);
+                        st_async_f32(push_b[i][2 * jh] + ob_off, out.x, full_of[(2 * jh) * CL / K] + ob_mbar);
+                        st_async_f32(push_b[i][2 * jh + 1] + ob_off, out.y, full_of[(2 * jh + 1) * CL / K] + ob_mbar);
                         num2 = fma2(f, craw, num2);
                         den2 = fma2(f, sum, den2);
                     }
                 }
-                float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
+                const float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
                 tmax = warp_max(tmax);
                 if (lane == 0) {
 #pragma unroll
-                    for (int r = 0; r < CL; ++r) st_cluster_f32(wmax_dst[r] + (uint32_t)((t & 1) * 32) * 4u, tmax);
-                    st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u, num);
-                    st_cluster_f32(part_dst + (uint32_t)((t & 1) * 128) * 4u + 4u, den);
+                    for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 64) * 4u, tmax, full_of[r] + ob_mbar);
+                    st_async_v2(part_dst + (uint32_t)(ob * 128) * 4u, num, den, full_of[0] + ob_mbar);
                 }
-                P += (int)offM;
-                cluster_sync();
-                cmax = warp_max(slot_max(wmax + (t & 1) * 32, lane, CL * NWARP));
-                offM = rintf(cmax);
-                if (rank == 0 && warp == 0) {
-                    float a = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4] : 0.f;
-                    float b = lane < CL * NWARP ? part[(t & 1) * 128 + lane * 4 + 1] : 0.f;
-                    a = warp_sum(a); b = warp_sum(b);
-                    if (lane == 0) {
-                        const float sw = a / b;
-                        p.soft[blk * n + t - 1] = sw;
-                        if (p.soft_copy) p.soft_copy[blk * n + t - 1] = sw;
-                        defect = fmaxf(defect, fabsf(b - 1.f));
-                    }
-                }
+                ib = ob;
             }
+            wait_inputs(ib);                                             // M_0 and the sums of step 1
+            cmax = warp_max(slot_max(wmax + ib * 64, lane, SLOTS));
+            P += (int)offM;                                              // P_0
+            finish_step(1, ib);
         }
-        // ================= consistency: P_0 + LSE_q M_0(q) against log2 Z (M_0 in buffer n&1)
+        // ================= consistency: P_0 + LSE_q M_0(q) against log2 Z (M_0 in buffer ib)
         {
-            const float *Mfin = msg + (n & 1) * QC;
+            const float *Mfin = msg + ib * QC;
             float ssum = 0.f;
             for (int q = tid; q < QC; q += THREADS) ssum += ex2f(Mfin[q] - cmax);
             ssum = warp_sum(ssum);
             if (lane == 0) {
 #pragma unroll
-                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r] + 32u * 4u, ssum);
+                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r] + 64u * 4u, ssum);
             }
             cluster_sync();
-            float v = lane < CL * NWARP ? lz[32 + lane] : 0.f;
+            float v = (lane < SLOTS ? lz[64 + lane] : 0.f) + (lane + 32 < SLOTS ? lz[96 + lane] : 0.f);
             v = warp_sum(v);
             const float lz_beta = cmax + lg2f(v);
             zgap = fmaxf(zgap, fabsf((float)(P - Ofin) + (lz_beta - lsefin)));
