@@ -12,6 +12,7 @@
 #include "bcjr_generic.cuh"
 #ifndef BCJR_NO_CLUSTER
 #include "bcjr_cluster.cuh"
+#include "bcjr_solo.cuh"
 #endif
 
 using namespace bcjr;
@@ -40,6 +41,7 @@ struct bcjr_ctx {
     // options
     int opt_path = 0;
     int opt_max_ctas = 0;
+    int opt_fwd_variant = 0;   // 0 = TMEM single-CTA forward kernel where it applies, 1 = cluster forward kernel
     int launches = 0;
     int last_path = 0;
     std::string cuda_error;
@@ -259,9 +261,28 @@ bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_co
     return BCJR_EUNSUPPORTED;
 }
 
+// Forward call, one CTA per block with the codebook in tensor memory (Lb = 16, k = 2).
+bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    using C = SoloCfg;
+    if (p.n > C::MAX_N) return BCJR_EUNSUPPORTED;
+    CU(cudaFuncSetAttribute(fwd_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    int64_t grid = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    if (grid > p.B) grid = p.B;
+    bcjr_status rc = ensure(ctx, ctx->hist, (size_t)grid * p.n * C::Q * 4);
+    if (rc) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    fwd_solo_kernel<<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
 bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
+    if (k == 2 && ctx->opt_fwd_variant != 1) return launch_fwd_solo(ctx, p, st);
     if (k == 2) return launch_fwd_cluster_t<16, 2, FWD_CL_K2, FWD_THREADS_K2>(ctx, p, st);
     if (k == 3) return launch_fwd_cluster_t<16, 3, 2, 512>(ctx, p, st);
     return BCJR_EUNSUPPORTED;
@@ -331,6 +352,11 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
     if (!strcmp(name, "path")) {
         if (value < 0 || value > 2) return BCJR_EINVAL;
         ctx->opt_path = (int)value;
+        return BCJR_OK;
+    }
+    if (!strcmp(name, "fwd_variant")) {
+        if (value < 0 || value > 1) return BCJR_EINVAL;
+        ctx->opt_fwd_variant = (int)value;
         return BCJR_OK;
     }
     if (!strcmp(name, "max_ctas")) {

@@ -1,0 +1,398 @@
+// Forward call, one CTA per weight block, for the 2^16-state trellis (k = 2).
+//
+// The whole codebook (2^16 floats = 256 KB) does not fit one SM's registers next to anything
+// else, and not its shared memory either -- but it is exactly the size of the SM's tensor
+// memory (TMEM, 512 columns x 128 lanes x 32 bit), which this path does not otherwise use.
+// TMEM is lane-private (a warp reaches only the 32 lanes of its sub-partition) and that is
+// precisely the access pattern here: a thread owns the same butterflies for the whole kernel
+// (see bcjr_cluster.cuh for the butterfly form), so the K*K codebook entries of each of its
+// butterflies sit in "its" TMEM lane and are fetched with tcgen05.ld, sixteen columns at a
+// time, one butterfly ahead of the arithmetic.  With the codebook out of the register file and
+// the compressed message vector (64 KB) double-buffered in shared memory, one SM handles a
+// block alone: the per-step exchange is a CTA barrier instead of a cluster-wide handshake.
+//
+// Warp roles: 16 compute warps (512 threads, 8 butterflies each) and one copy warp that moves
+// the history with bulk copies -- alpha: shared -> global, one 64 KB message buffer per step;
+// beta: global -> shared in 8 KB chunks (one butterfly slot of all threads), through a ring of
+// 8 chunks with full/empty mbarriers.
+#pragma once
+#include "bcjr_cluster.cuh"
+
+namespace bcjr {
+
+// ---------------------------------------------------------------------------- TMEM helpers
+__device__ __forceinline__ void tmem_alloc_512(uint32_t smem_dst)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_dst) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_512(uint32_t taddr)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(taddr) : "memory");
+}
+// wait for this thread's outstanding tcgen05.ld; the loaded registers are operands so that no
+// use of them can be scheduled ahead of the wait
+__device__ __forceinline__ void tmem_wait_ld(float2 (&v)[8])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+f"(v[0].x), "+f"(v[0].y), "+f"(v[1].x), "+f"(v[1].y), "+f"(v[2].x), "+f"(v[2].y), "+f"(v[3].x), "+f"(v[3].y),
+                   "+f"(v[4].x), "+f"(v[4].y), "+f"(v[5].x), "+f"(v[5].y), "+f"(v[6].x), "+f"(v[6].y), "+f"(v[7].x), "+f"(v[7].y)
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// sixteen consecutive columns of the calling thread's lane, as eight packed pairs
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float2 (&v)[8])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "f"(v[0].x), "f"(v[0].y), "f"(v[1].x), "f"(v[1].y), "f"(v[2].x), "f"(v[2].y), "f"(v[3].x), "f"(v[3].y), "f"(v[4].x),
+        "f"(v[4].y), "f"(v[5].x), "f"(v[5].y), "f"(v[6].x), "f"(v[6].y), "f"(v[7].x), "f"(v[7].y)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float2 (&v)[8])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=f"(v[0].x), "=f"(v[0].y), "=f"(v[1].x), "=f"(v[1].y), "=f"(v[2].x), "=f"(v[2].y), "=f"(v[3].x), "=f"(v[3].y),
+          "=f"(v[4].x), "=f"(v[4].y), "=f"(v[5].x), "=f"(v[5].y), "=f"(v[6].x), "=f"(v[6].y), "=f"(v[7].x), "=f"(v[7].y)
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t mbar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+}
+__device__ __forceinline__ void compute_barrier(int nthreads)
+{
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+
+struct SoloCfg {
+    static constexpr int LB = 16, KB = 2, K = 4, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
+    static constexpr int CTHREADS = 512;                       // compute threads
+    static constexpr int THREADS = CTHREADS + 32;              // + the copy warp
+    static constexpr int NWARP = CTHREADS / 32;
+    static constexpr int BPT = NB / CTHREADS;                  // 8 butterflies per thread
+    static constexpr int CH = K * CTHREADS;                    // floats per history chunk (one slot of all threads)
+    static constexpr int RD = BPT;                             // ring depth: one step of chunks
+    static constexpr int MAX_N = 2048;
+    static constexpr int OFF_MSG = 0;                          // [2][Q]
+    static constexpr int OFF_RING = OFF_MSG + 2 * Q;           // [RD][CH]
+    static constexpr int OFF_W = OFF_RING + RD * CH;           // [MAX_N]
+    static constexpr int OFF_O = OFF_W + MAX_N;                // int [MAX_N + 2]
+    static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;     // [2][32]
+    static constexpr int OFF_PART = OFF_WMAX + 64;             // [2][32][2]
+    static constexpr int OFF_LZ = OFF_PART + 128;              // [32]
+    static constexpr int OFF_MBAR = OFF_LZ + 32;               // uint64: full[RD], empty[RD], ready[2], freed[2]
+    static constexpr int NMBAR = 2 * RD + 4;
+    static constexpr int OFF_TMEM = OFF_MBAR + 2 * NMBAR;      // uint32 TMEM base
+    static constexpr int OFF_FLAG = OFF_TMEM + 2;
+    static constexpr int SMEM_FLOATS = OFF_FLAG + 2;
+    static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
+    static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
+    static_assert(BPT * K * K == 128, "a thread's codebook slice fills its 128 TMEM columns");
+};
+
+__global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams p)
+{
+    using C = SoloCfg;
+    constexpr int K = C::K, NB = C::NB, Q = C::Q, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, CH = C::CH, RD = C::RD;
+    extern __shared__ __align__(16) float smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = p.n;
+    const float NEG_INF = __int_as_float(0xff800000);
+    const float2 nl2 = splat2(-p.lam2);
+
+    float *msg = smem + C::OFF_MSG;
+    float *ring = smem + C::OFF_RING;
+    float *w_s = smem + C::OFF_W;
+    int *O_s = reinterpret_cast<int *>(smem + C::OFF_O);
+    float *wmax = smem + C::OFF_WMAX;
+    float *part = smem + C::OFF_PART;
+    float *lz = smem + C::OFF_LZ;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
+    const uint32_t mbar_full = smem_u32(smem + C::OFF_MBAR);
+    const uint32_t mbar_empty = mbar_full + 8u * RD;
+    const uint32_t mbar_ready = mbar_empty + 8u * RD;          // [2] compute -> copy warp: buffer holds L_t
+    const uint32_t mbar_freed = mbar_ready + 16u;              // [2] copy warp -> compute: buffer has been read
+    const uint32_t msg_u32 = smem_u32(msg), ring_u32 = smem_u32(ring);
+
+    float *hist = p.hist + (size_t)blockIdx.x * n * Q;         // [n][Q], layout of the alpha input buffer
+
+    if (tid == 0) {
+        for (int s = 0; s < RD; ++s) { mbar_init(mbar_full + 8u * s, 1); mbar_init(mbar_empty + 8u * s, NWARP); }
+        for (int s = 0; s < 2; ++s) { mbar_init(mbar_ready + 8u * s, 1); mbar_init(mbar_freed + 8u * s, 1); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc_512(smem_u32(const_cast<uint32_t *>(tmem_slot)));
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == NWARP) {
+        // ============================ copy warp (one elected lane) ============================
+        if (lane == 0) {
+            uint32_t use_ready[2] = {0u, 0u}, chunk = 0;      // completed phases per mbarrier
+            for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
+                for (int t = 1; t <= n; ++t) {                 // alpha: spill L_t once the buffer is complete
+                    const uint32_t b = (uint32_t)(t - 1) & 1u;
+                    mbar_wait_bounded(mbar_ready + 8u * b, use_ready[b] & 1u, abort_flag, p.diag);
+                    ++use_ready[b];
+                    fence_proxy_async();
+                    bulk_store(hist + (size_t)(t - 1) * Q, msg_u32 + b * Q * 4u, Q * 4u);
+                    bulk_commit();
+                    bulk_wait_read0();
+                    mbar_arrive(mbar_freed + 8u * b);
+                }
+                bulk_wait_all0();                              // history written before it is read back
+                for (int t = n; t >= 1; --t)                   // beta: stream L_t back, one slot chunk at a time
+                    for (int i = 0; i < BPT; ++i, ++chunk) {
+                        const uint32_t s = chunk % RD;
+                        mbar_wait_bounded(mbar_empty + 8u * s, ((chunk / RD) & 1u) ^ 1u, abort_flag, p.diag);
+                        mbar_expect_tx(mbar_full + 8u * s, CH * 4u);
+                        bulk_load(ring_u32 + s * CH * 4u, hist + (size_t)(t - 1) * Q + (size_t)i * CH, CH * 4u, mbar_full + 8u * s);
+                    }
+            }
+        }
+    } else {
+        // ============================ compute warps ============================
+        // TMEM: lanes of this warp's sub-partition, 128 columns per thread
+        const uint32_t tm = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
+        // destinations of the outputs (floats from the start of a message buffer)
+        //   alpha: L([x|l]) -> butterfly x2 = (x*K) mod NB, input j2 = (x*K) / NB: [(i2*K + j2)*CT + tid2 .. +K)
+        //   beta : M([j|x]) -> butterfly x1 = (j*NB + x) / K, input b1 = x mod K:  [(x1*K + b1)]
+        int push_a[BPT];
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) {
+            const int x = i * CT + tid;
+            const int q2 = x * K, j2 = q2 / NB, x2 = q2 % NB;
+            push_a[i] = ((x2 / CT) * K + j2) * CT + (x2 % CT);
+        }
+        const int push_b0 = (tid / K) * K + (tid % K);         // + (j*(NB/K) + i*CT/K) * K per (i, j)
+        uint32_t use_freed[2] = {0u, 0u}, chunk = 0;          // completed phases per mbarrier
+        float defect = 0.f, zgap = 0.f;
+
+        for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
+            const float *w = p.W + blk * n;
+            for (int t = tid; t < n; t += CT) w_s[t] = __ldg(w + t);
+            for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // L_1 = 0 in buffer 0
+            if (tid == 0) O_s[1] = 0;
+            // codebook -> TMEM in the alpha pairing: column 16 i + 4 j + l = c[j | x_i | l]
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                float2 v[8];
+#pragma unroll
+                for (int j = 0; j < K; ++j) {
+                    const float4 c4 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)j * Q + (size_t)(i * CT + tid) * K));
+                    v[2 * j] = make_float2(c4.x, c4.y);
+                    v[2 * j + 1] = make_float2(c4.z, c4.w);
+                }
+                tmem_st16(tm + 16u * i, v);
+            }
+            tmem_wait_st();
+            int O = 0;
+            float off = 0.f, cmax = 0.f;
+            compute_barrier(CT);
+            // ================= alpha sweep
+            for (int t = 1; t <= n; ++t) {
+                const int cur = (t - 1) & 1;
+                const float *Lin = msg + cur * Q;
+                float *Lout = msg + (cur ^ 1) * Q;
+                if (tid == 0) mbar_arrive(mbar_ready + 8u * cur);                // L_t complete: spill it
+                if (t > 1) {
+                    cmax = warp_max(lane < NWARP ? wmax[cur * 32 + lane] : NEG_INF) - off;
+                    off = rintf(cmax);
+                    // the buffer written now was spilled during the previous step: wait until read
+                    mbar_wait_bounded(mbar_freed + 8u * (cur ^ 1), use_freed[cur ^ 1] & 1u, abort_flag, p.diag);
+                    ++use_freed[cur ^ 1];
+                }
+                const float2 w2 = splat2(w_s[t - 1]);
+                const float2 off2 = splat2(off);
+                float tmax = NEG_INF;
+                float2 cb[2][8];
+                tmem_ld16(tm, cb[0]);
+#pragma unroll
+                for (int i = 0; i < BPT; ++i) {
+                    tmem_wait_ld(cb[i & 1]);
+                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
+                    float2 Lj[K];
+#pragma unroll
+                    for (int j = 0; j < K; ++j) Lj[j] = splat2(Lin[(i * K + j) * CT + tid]);
+                    float2 out[K / 2];
+#pragma unroll
+                    for (int h = 0; h < K / 2; ++h) {
+                        float2 a[K];
+#pragma unroll
+                        for (int j = 0; j < K; ++j) {
+                            const float2 d = sub2(cb[i & 1][2 * j + h], w2);
+                            a[j] = fma2(mul2(d, d), nl2, Lj[j]);
+                        }
+                        const float2 m = max_pairs<K>(a);
+                        float2 sum = ex2f2(sub2(a[0], m));
+#pragma unroll
+                        for (int j = 1; j < K; ++j) sum = add2(sum, ex2f2(sub2(a[j], m)));
+                        out[h] = add2(sub2(m, off2), lg2f2(sum));
+                        tmax = max3f(tmax, m.x, m.y);
+                    }
+                    *reinterpret_cast<float4 *>(Lout + push_a[i]) = make_float4(out[0].x, out[0].y, out[1].x, out[1].y);
+                }
+                tmax = warp_max(tmax);
+                if (lane == 0) wmax[(cur ^ 1) * 32 + warp] = tmax;
+                O += (int)off;
+                if (tid == 0) O_s[t + 1] = O;
+                compute_barrier(CT);
+            }
+            // ================= log2 Z = O_{n+1} + LSE_q L_{n+1}(q); L_{n+1} sits in buffer n&1
+            cmax = warp_max(lane < NWARP ? wmax[(n & 1) * 32 + lane] : NEG_INF) - off;
+            {
+                const float *Lfin = msg + (n & 1) * Q;
+                float ssum = 0.f;
+                for (int q = tid; q < Q; q += CT) ssum += ex2f(Lfin[q] - cmax);
+                ssum = warp_sum(ssum);
+                if (lane == 0) lz[warp] = ssum;
+                compute_barrier(CT);
+            }
+            const float lsefin = cmax + lg2f(warp_sum(lane < NWARP ? lz[lane] : 0.f));
+            const int Ofin = O;
+            if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
+            // the last spill (L_n, buffer (n-1)&1) must have left its buffer before it is reused
+            mbar_wait_bounded(mbar_freed + 8u * ((n - 1) & 1), use_freed[(n - 1) & 1] & 1u, abort_flag, p.diag);
+            ++use_freed[(n - 1) & 1];
+            // ================= beta sweep
+            for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // M_n = 0 in buffer 0
+            // codebook -> TMEM in the beta pairing: column 16 i + 8 jh + 2 b + e = c[2jh+e | x_i | b]
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                float2 v[8];
+#pragma unroll
+                for (int jh = 0; jh < K / 2; ++jh) {
+                    const float4 c0 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh) * Q + (size_t)(i * CT + tid) * K));
+                    const float4 c1 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh + 1) * Q + (size_t)(i * CT + tid) * K));
+                    v[4 * jh] = make_float2(c0.x, c1.x); v[4 * jh + 1] = make_float2(c0.y, c1.y);
+                    v[4 * jh + 2] = make_float2(c0.z, c1.z); v[4 * jh + 3] = make_float2(c0.w, c1.w);
+                }
+                tmem_st16(tm + 16u * i, v);
+            }
+            tmem_wait_st();
+            int P = 0;
+            float offM = 0.f;
+            compute_barrier(CT);
+            for (int t = n; t >= 1; --t) {
+                const int cur = (n - t) & 1;
+                const float *Min = msg + cur * Q;
+                float *Mout = msg + (cur ^ 1) * Q;
+                if (t < n) {
+                    cmax = warp_max(lane < NWARP ? wmax[cur * 32 + lane] : NEG_INF);
+                    P += (int)offM;
+                    offM = rintf(cmax);
+                    if (warp == 0) {                                             // soft[t+1] from the partial sums
+                        float a = lane < NWARP ? part[(cur * 32 + lane) * 2] : 0.f;
+                        float c = lane < NWARP ? part[(cur * 32 + lane) * 2 + 1] : 0.f;
+                        a = warp_sum(a); c = warp_sum(c);
+                        if (lane == 0) {
+                            const float sw = a / c;
+                            p.soft[blk * n + t] = sw;
+                            if (p.soft_copy) p.soft_copy[blk * n + t] = sw;
+                            defect = fmaxf(defect, fabsf(c - 1.f));
+                        }
+                    }
+                }
+                const float2 w2 = splat2(w_s[t - 1]);
+                const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
+                float2 num2 = make_float2(0.f, 0.f), den2 = make_float2(0.f, 0.f);
+                float tmax = NEG_INF;
+                float2 cb[2][8];
+                tmem_ld16(tm, cb[0]);
+#pragma unroll
+                for (int i = 0; i < BPT; ++i, ++chunk) {
+                    tmem_wait_ld(cb[i & 1]);
+                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
+                    const uint32_t s = chunk % RD;
+                    mbar_wait_bounded(mbar_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
+                    const float *Lh = ring + s * CH;
+                    float2 Mb[K];
+                    {
+                        const float4 v = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K);
+                        Mb[0] = splat2(v.x - offM); Mb[1] = splat2(v.y - offM);
+                        Mb[2] = splat2(v.z - offM); Mb[3] = splat2(v.w - offM);
+                    }
+#pragma unroll
+                    for (int jh = 0; jh < K / 2; ++jh) {
+                        float2 u[K];
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+                            const float2 d = sub2(cb[i & 1][4 * jh + b], w2);
+                            u[b] = fma2(mul2(d, d), nl2, Mb[b]);
+                        }
+                        const float2 m = max_pairs<K>(u);
+                        const float2 LhD = make_float2(Lh[(2 * jh) * CT + tid] - Dm, Lh[(2 * jh + 1) * CT + tid] - Dm);
+                        const float2 f = ex2f2(add2(m, LhD));
+                        float2 pb = ex2f2(sub2(u[0], m));
+                        float2 sum = pb, craw = mul2(pb, cb[i & 1][4 * jh]);
+#pragma unroll
+                        for (int b = 1; b < K; ++b) {
+                            pb = ex2f2(sub2(u[b], m));
+                            sum = add2(sum, pb);
+                            craw = fma2(pb, cb[i & 1][4 * jh + b], craw);
+                        }
+                        const float2 out = add2(m, lg2f2(sum));
+                        tmax = max3f(tmax, m.x, m.y);
+                        Mout[push_b0 + ((2 * jh) * (NB / K) + i * (CT / K)) * K] = out.x;
+                        Mout[push_b0 + ((2 * jh + 1) * (NB / K) + i * (CT / K)) * K] = out.y;
+                        num2 = fma2(f, craw, num2);
+                        den2 = fma2(f, sum, den2);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(mbar_empty + 8u * s);             // this warp is done with the chunk
+                }
+                const float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
+                tmax = warp_max(tmax);
+                if (lane == 0) {
+                    wmax[(cur ^ 1) * 32 + warp] = tmax;
+                    part[((cur ^ 1) * 32 + warp) * 2] = num;
+                    part[((cur ^ 1) * 32 + warp) * 2 + 1] = den;
+                }
+                compute_barrier(CT);
+            }
+            {
+                const int fin = n & 1;                                           // M_0 and the sums of step 1
+                cmax = warp_max(lane < NWARP ? wmax[fin * 32 + lane] : NEG_INF);
+                P += (int)offM;
+                if (warp == 0) {
+                    float a = lane < NWARP ? part[(fin * 32 + lane) * 2] : 0.f;
+                    float c = lane < NWARP ? part[(fin * 32 + lane) * 2 + 1] : 0.f;
+                    a = warp_sum(a); c = warp_sum(c);
+                    if (lane == 0) {
+                        const float sw = a / c;
+                        p.soft[blk * n] = sw;
+                        if (p.soft_copy) p.soft_copy[blk * n] = sw;
+                        defect = fmaxf(defect, fabsf(c - 1.f));
+                    }
+                }
+                // consistency: P_0 + LSE_q M_0(q) against log2 Z
+                const float *Mfin = msg + fin * Q;
+                float ssum = 0.f;
+                for (int q = tid; q < Q; q += CT) ssum += ex2f(Mfin[q] - cmax);
+                ssum = warp_sum(ssum);
+                compute_barrier(CT);                                             // lz is free again
+                if (lane == 0) lz[warp] = ssum;
+                compute_barrier(CT);
+                const float lz_beta = cmax + lg2f(warp_sum(lane < NWARP ? lz[lane] : 0.f));
+                zgap = fmaxf(zgap, fabsf((float)(P - Ofin) + (lz_beta - lsefin)));
+                compute_barrier(CT);
+            }
+        }
+        if (tid == 0) {
+            diag_max(&p.diag->max_defect, defect);
+            diag_max(&p.diag->max_logz_gap, zgap);
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) tmem_dealloc_512(tmem_base);
+}
+
+}  // namespace bcjr
