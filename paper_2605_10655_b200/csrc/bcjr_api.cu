@@ -13,6 +13,7 @@
 #ifndef BCJR_NO_CLUSTER
 #include "bcjr_cluster.cuh"
 #include "bcjr_solo.cuh"
+#include "bcjr_duo.cuh"
 #endif
 
 using namespace bcjr;
@@ -41,6 +42,7 @@ struct bcjr_ctx {
     // options
     int opt_path = 0;
     int opt_max_ctas = 0;
+    int opt_bwd_variant = 0;   // 0 = TMEM two-CTA backward kernel where it applies, 1 = register-accumulator cluster kernel
     int opt_fwd_variant = 0;   // 0 = TMEM single-CTA forward kernel where it applies, 1 = cluster forward kernel
     int launches = 0;
     int last_path = 0;
@@ -253,9 +255,33 @@ bcjr_status launch_bwd_cluster_t(bcjr_ctx *ctx, BwdParams p, float *grad_codeboo
     return BCJR_OK;
 }
 
+// Backward call, clusters of two with codebook and accumulators in tensor memory (Lb = 16, k = 2).
+bcjr_status launch_bwd_duo(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    using C = DuoCfg;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    bcjr_status rc = plan_cluster(ctx, bwd_duo_kernel, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    if (rc) return rc;
+    const int ncl = cfg.gridDim.x / C::CL;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * p.n * 2 * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * C::S * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.gc_part = (float *)ctx->gc_part.ptr;
+    CU(cudaLaunchKernelEx(&cfg, bwd_duo_kernel, p));
+    ctx->launches += 1;
+    if (grad_codebook) {
+        reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, C::S, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
 bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_codebook, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
+    if (k == 2 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg::MAX_N) return launch_bwd_duo(ctx, p, grad_codebook, st);
     if (k == 2) return launch_bwd_cluster_t<16, 2, 4, 512>(ctx, p, grad_codebook, st);
     if (k == 3) return launch_bwd_cluster_t<16, 3, 4, 256>(ctx, p, grad_codebook, st);
     return BCJR_EUNSUPPORTED;
@@ -352,6 +378,11 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
     if (!strcmp(name, "path")) {
         if (value < 0 || value > 2) return BCJR_EINVAL;
         ctx->opt_path = (int)value;
+        return BCJR_OK;
+    }
+    if (!strcmp(name, "bwd_variant")) {
+        if (value < 0 || value > 1) return BCJR_EINVAL;
+        ctx->opt_bwd_variant = (int)value;
         return BCJR_OK;
     }
     if (!strcmp(name, "fwd_variant")) {
