@@ -114,17 +114,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity)
 // Bounded wait: gives up after ~2^20 polls, raises BCJR_ETIMEOUT (-6) in the diagnostics and
 // sets the CTA-wide abort flag so that later waits return at once; the kernel then runs to its
 // end (with meaningless numbers) instead of hanging.
-__device__ __noinline__ void mbar_wait_slow(uint32_t mbar, uint32_t parity, volatile int *abort_flag, DeviceDiag *diag)
+__device__ __forceinline__ void mbar_wait_bounded(uint32_t mbar, uint32_t parity, volatile int *abort_flag, DeviceDiag *diag)
 {
+    if (mbar_try_wait(mbar, parity)) return;                     // fast path: one probe
     if (*abort_flag) return;
     for (int i = 0; i < (1 << 20); ++i)
         if (mbar_try_wait(mbar, parity)) return;
     *abort_flag = 1;
     atomicCAS(&diag->status, 0, -6);
 }
-__device__ __forceinline__ void mbar_wait_bounded(uint32_t mbar, uint32_t parity, volatile int *abort_flag, DeviceDiag *diag)
+// non-blocking probe of a phase
+__device__ __forceinline__ bool mbar_test(uint32_t mbar, uint32_t parity)
 {
-    if (!mbar_try_wait(mbar, parity)) mbar_wait_slow(mbar, parity, abort_flag, diag);   // fast path: one probe
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+    return ok != 0;
 }
 
 // ---------------------------------------------------------------------------- packed fp32 pairs

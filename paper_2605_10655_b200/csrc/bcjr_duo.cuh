@@ -12,10 +12,10 @@
 //
 // Step protocol.  Messages are double-buffered.  Every output is pushed with st.async into the
 // consumer CTA's buffer `ob` and credits that CTA's mbarrier full[ob] with its bytes; a phase of
-// full[ob] completes when (a) all bytes have landed, (b) every compute warp of the cluster has
-// arrived on it after its last butterfly of the step -- so nobody still reads the other buffer
-// when the next step starts overwriting it -- and (c) every CTA's copy warp has arrived, after
-// the bulk copy that spills that other buffer to the history has finished reading it.
+// full[ob] completes when (a) all bytes have landed and (b) every CTA of the cluster has
+// arrived on it, which a CTA does once all its warps have finished the step and the bulk copy
+// that spills its input buffer to the history has finished reading it -- so nobody still
+// reads the other buffer when the next step starts overwriting it.
 #pragma once
 #include "bcjr_solo.cuh"
 
@@ -30,13 +30,13 @@ struct DuoCfg {
     static constexpr int LB = 16, KB = 2, K = 4, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
     static constexpr int CL = 2;
     static constexpr int NBC = NB / CL, QC = Q / CL;
-    static constexpr int CTHREADS = 512, THREADS = CTHREADS + 32, NWARP = CTHREADS / 32;
-    static constexpr int BPT = NBC / CTHREADS;                 // 4 butterflies per thread
+    static constexpr int THREADS = 512, NWARP = THREADS / 32;
+    static constexpr int BPT = NBC / THREADS;                  // 4 butterflies per thread
     static constexpr int SLOTS = CL * NWARP;                   // 32 per-warp partial slots
-    static constexpr int CH = K * CTHREADS;                    // floats per array per history chunk
+    static constexpr int CH = K * THREADS;                     // floats per array per history chunk
     static constexpr int RD = BPT;                             // ring depth: one step of chunks
     static constexpr int MAX_N = 1024;
-    static constexpr int ARRIVALS = 1 + SLOTS + CL;            // armer + compute warps + copy warps
+    static constexpr int ARRIVALS = 1 + CL;                    // armer + one arrival per CTA of the cluster
     static constexpr int OFF_MSG = 0;                          // [2 parity][2 arrays][QC]
     static constexpr int OFF_RING = OFF_MSG + 4 * QC;          // [RD][2 arrays][CH]
     static constexpr int OFF_W = OFF_RING + RD * 2 * CH;       // w, g, soft: [3][MAX_N]
@@ -58,7 +58,7 @@ struct DuoCfg {
 __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p)
 {
     using C = DuoCfg;
-    constexpr int K = C::K, NB = C::NB, NBC = C::NBC, QC = C::QC, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS;
+    constexpr int K = C::K, NB = C::NB, NBC = C::NBC, QC = C::QC, BPT = C::BPT, NWARP = C::NWARP, CT = C::THREADS;
     constexpr int CL = C::CL, SLOTS = C::SLOTS, CH = C::CH, RD = C::RD;
     constexpr uint32_t BUF_BYTES = 2u * QC * 4u;                 // (L, At) of one parity
     constexpr uint32_t TX_MSG = BUF_BYTES + SLOTS * 4u;          // messages + gauge slots
@@ -109,349 +109,318 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
         full_phase ^= 1u << b;
     };
 
-    if (warp == NWARP) {
-        // ============================ copy warp ============================
-        // All 32 lanes follow the control flow (the cluster barriers are warp-wide); lane 0 issues.
-        uint32_t chunk = 0;
-        for (int64_t blk = cid; blk < p.B; blk += ncl) {
-            int ib = 0;
-            cluster_sync();                                      // block start (inputs zero-filled)
-            for (int t = 1; t <= n; ++t) {                       // alpha: spill (L_t, At_t)
-                const int ob = ib ^ 1;
-                if (t > 1) wait_inputs(ib);
-                if (lane == 0) {
-                    fence_proxy_async();
-                    bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)ib * BUF_BYTES, BUF_BYTES);
-                    bulk_commit();
-                    bulk_wait_read0();
+    const uint32_t tm_cb = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
+    const uint32_t tm_acc = tm_cb + 64u;
+    uint32_t push_a[BPT], push_b[BPT][K];
 #pragma unroll
-                    for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + 8u * ob);
-                }
-                __syncwarp();
-                ib = ob;
-            }
-            wait_inputs(ib);
-            if (lane == 0) bulk_wait_all0();                     // history written before it is read back
-            cluster_sync();                                      // log Z exchange
-            cluster_sync();                                      // beta start (inputs zero-filled)
-            for (int t = n; t >= 1; --t) {
-                const int ob = ib ^ 1;
-                if (t < n) wait_inputs(ib);
-                if (lane == 0) {
-#pragma unroll
-                    for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + 8u * ob);
-                    for (int i = 0; i < BPT; ++i, ++chunk) {
-                        const uint32_t s = chunk % RD;
-                        mbar_wait_bounded(ring_empty + 8u * s, ((chunk / RD) & 1u) ^ 1u, abort_flag, p.diag);
-                        mbar_expect_tx(ring_full + 8u * s, 2u * CH * 4u);
-                        const float *src = hist + ((size_t)(t - 1) * CL + rank) * 2 * QC + (size_t)i * CH;
-                        bulk_load(ring_u32 + s * 2u * CH * 4u, src, CH * 4u, ring_full + 8u * s);
-                        bulk_load(ring_u32 + s * 2u * CH * 4u + CH * 4u, src + QC, CH * 4u, ring_full + 8u * s);
-                    }
-                }
-                __syncwarp();
-                ib = ob;
-            }
-            wait_inputs(ib);
-            cluster_sync();                                      // block end
+    for (int i = 0; i < BPT; ++i) {
+        const int x = (int)rank * NBC + i * CT + tid;
+        {
+            // L([x|l]) -> butterfly x2 = (x*K) mod NB, input j2 = (x*K) / NB, at [(i2*K + j2)*CT + tid2 .. +K);
+            // with 512 threads and clusters of two the destination CTA is i & 1
+            const int q2 = x * K, j2 = q2 / NB, x2 = q2 % NB;
+            const int r2 = x2 / NBC, xl2 = x2 % NBC;
+            push_a[i] = mapa_u32(msg_u32 + (uint32_t)(((xl2 / CT) * K + j2) * CT + xl2 % CT) * 4u, (uint32_t)r2);
         }
-    } else {
-        // ============================ compute warps ============================
-        const uint32_t tm_cb = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
-        const uint32_t tm_acc = tm_cb + 64u;
-        uint32_t push_a[BPT], push_a_mbar[BPT], push_b[BPT][K];
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            // M([j|x]) -> butterfly x1 = (j*NB + x) / K, input b1 = x mod K, at [xl1*K + b1], CTA j*CL/K
+            const int q1 = j * NB + x, x1 = q1 / K, b1 = q1 % K;
+            const int r1 = x1 / NBC, xl1 = x1 % NBC;
+            push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(xl1 * K + b1) * 4u, (uint32_t)r1);
+        }
+    }
+    static_assert(NBC / K == CT, "alpha destination CTA of butterfly slot i is i mod CL");
+    uint32_t wmax_dst[CL], lz_dst[CL];
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+        wmax_dst[r] = mapa_u32(wmax_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+        lz_dst[r] = mapa_u32(lz_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+    }
+    const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 16u, 0u);
+    // zero the accumulators (beta pairing: column 64 + 16 i + 8 jh + 2 b + e <-> state [2jh+e | x_i | b])
+    {
+        float2 z[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z[e] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) tmem_st16(tm_acc + 16u * i, z);
+        tmem_wait_st();
+    }
+    uint32_t chunk = 0;            // history chunks consumed so far (all threads count alike)
+    uint32_t issued = 0;           // history chunks requested so far (thread 0)
+    float defect = 0.f;
+
+    for (int64_t blk = cid; blk < p.B; blk += ncl) {
+        int ib = 0;
+        for (int t = tid; t < n; t += CT) {
+            w_s[t] = __ldg(p.W + blk * n + t);
+            g_s[t] = __ldg(p.g + blk * n + t);
+            sf_s[t] = __ldg(p.soft + blk * n + t);
+        }
+        for (int q = tid; q < 2 * QC; q += CT) msg[q] = 0.f;                   // L_1 = 0, At_1 = 0 (parity 0)
+        if (tid == 0) O_s[1] = 0;
+        // codebook -> TMEM, alpha pairing: column 16 i + 4 j + l = c[j | x_i | l]
 #pragma unroll
         for (int i = 0; i < BPT; ++i) {
+            float2 v[8];
             const int x = (int)rank * NBC + i * CT + tid;
-            {
-                // L([x|l]) -> butterfly x2 = (x*K) mod NB, input j2 = (x*K) / NB, at [(i2*K + j2)*CT + tid2 .. +K)
-                const int q2 = x * K, j2 = q2 / NB, x2 = q2 % NB;
-                const int r2 = x2 / NBC, xl2 = x2 % NBC;
-                push_a[i] = mapa_u32(msg_u32 + (uint32_t)(((xl2 / CT) * K + j2) * CT + xl2 % CT) * 4u, (uint32_t)r2);
-                push_a_mbar[i] = full_of[r2];
-            }
 #pragma unroll
             for (int j = 0; j < K; ++j) {
-                // M([j|x]) -> butterfly x1 = (j*NB + x) / K, input b1 = x mod K, at [xl1*K + b1], CTA j*CL/K
-                const int q1 = j * NB + x, x1 = q1 / K, b1 = q1 % K;
-                const int r1 = x1 / NBC, xl1 = x1 % NBC;
-                push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(xl1 * K + b1) * 4u, (uint32_t)r1);
+                const float4 c4 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)j * C::Q + (size_t)x * K));
+                v[2 * j] = make_float2(c4.x, c4.y);
+                v[2 * j + 1] = make_float2(c4.z, c4.w);
             }
+            tmem_st16(tm_cb + 16u * i, v);
         }
-        uint32_t wmax_dst[CL], lz_dst[CL];
-#pragma unroll
-        for (int r = 0; r < CL; ++r) {
-            wmax_dst[r] = mapa_u32(wmax_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
-            lz_dst[r] = mapa_u32(lz_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
-        }
-        const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 16u, 0u);
-        // zero the accumulators (beta pairing: column 64 + 16 i + 8 jh + 2 b + e <-> state [2jh+e | x_i | b])
-        {
-            float2 z[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) z[e] = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int i = 0; i < BPT; ++i) tmem_st16(tm_acc + 16u * i, z);
-            tmem_wait_st();
-        }
-        uint32_t chunk = 0;
-        float defect = 0.f;
-
-        for (int64_t blk = cid; blk < p.B; blk += ncl) {
-            int ib = 0;
-            for (int t = tid; t < n; t += CT) {
-                w_s[t] = __ldg(p.W + blk * n + t);
-                g_s[t] = __ldg(p.g + blk * n + t);
-                sf_s[t] = __ldg(p.soft + blk * n + t);
+        tmem_wait_st();
+        int O = 0;
+        float off = 0.f, cmax = 0.f;
+        cluster_sync();                                          // block start
+        // ================= alpha sweep carrying (L, At)
+        for (int t = 1; t <= n; ++t) {
+            const int ob = ib ^ 1;
+            if (t > 1) {
+                wait_inputs(ib);
+                cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
+                off = rintf(cmax);
             }
-            for (int q = tid; q < 2 * QC; q += CT) msg[q] = 0.f;               // L_1 = 0, At_1 = 0 (parity 0)
-            if (tid == 0) O_s[1] = 0;
-            // codebook -> TMEM, alpha pairing: column 16 i + 4 j + l = c[j | x_i | l]
+            const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
+            const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
+            if (tid == 0) {
+                mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
+                fence_proxy_async();                                           // spill (L_t, At_t)
+                bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)ib * BUF_BYTES, BUF_BYTES);
+                bulk_commit();
+            }
+            const float gt = g_s[t - 1];
+            const float gsh = -gt * sf_s[t - 1];                              // centring: h = g c - g soft
+            const float2 w2 = splat2(w_s[t - 1]), g2 = splat2(gt), off2 = splat2(off);
+            float tmax = NEG_INF;
+            float2 cb[2][8];
+            tmem_ld16(tm_cb, cb[0]);
 #pragma unroll
             for (int i = 0; i < BPT; ++i) {
-                float2 v[8];
-                const int x = (int)rank * NBC + i * CT + tid;
+                tmem_wait_ld(cb[i & 1]);
+                if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
+                float2 outL[K / 2], outA[K / 2];
 #pragma unroll
-                for (int j = 0; j < K; ++j) {
-                    const float4 c4 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)j * C::Q + (size_t)x * K));
-                    v[2 * j] = make_float2(c4.x, c4.y);
-                    v[2 * j + 1] = make_float2(c4.z, c4.w);
-                }
-                tmem_st16(tm_cb + 16u * i, v);
-            }
-            tmem_wait_st();
-            int O = 0;
-            float off = 0.f, cmax = 0.f;
-            cluster_sync();                                      // block start
-            // ================= alpha sweep carrying (L, At)
-            for (int t = 1; t <= n; ++t) {
-                const int ob = ib ^ 1;
-                if (t > 1) {
-                    wait_inputs(ib);
-                    cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
-                    off = rintf(cmax);
-                }
-                const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
-                const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
-                if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
-                const float gt = g_s[t - 1];
-                const float gsh = -gt * sf_s[t - 1];                          // centring: h = g c - g soft
-                const float2 w2 = splat2(w_s[t - 1]), g2 = splat2(gt), off2 = splat2(off);
-                float tmax = NEG_INF;
-                float2 cb[2][8];
-                tmem_ld16(tm_cb, cb[0]);
-#pragma unroll
-                for (int i = 0; i < BPT; ++i) {
-                    tmem_wait_ld(cb[i & 1]);
-                    if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
-                    float2 Lj[K], Aj[K];
+                for (int h = 0; h < K / 2; ++h) {
+                    float2 a[K];
 #pragma unroll
                     for (int j = 0; j < K; ++j) {
-                        Lj[j] = splat2(Lin[(i * K + j) * CT + tid]);
-                        Aj[j] = splat2(Ain[(i * K + j) * CT + tid] + gsh);
+                        const float2 d = sub2(cb[i & 1][2 * j + h], w2);
+                        a[j] = fma2(mul2(d, d), nl2, splat2(Lin[(i * K + j) * CT + tid]));
                     }
-                    float2 outL[K / 2], outA[K / 2];
+                    const float2 m = max_pairs<K>(a);
+                    float2 sum = make_float2(0.f, 0.f), ax = sum;
 #pragma unroll
-                    for (int h = 0; h < K / 2; ++h) {
-                        float2 a[K];
-#pragma unroll
-                        for (int j = 0; j < K; ++j) {
-                            const float2 d = sub2(cb[i & 1][2 * j + h], w2);
-                            a[j] = fma2(mul2(d, d), nl2, Lj[j]);
-                        }
-                        const float2 m = max_pairs<K>(a);
-                        float2 pj = ex2f2(sub2(a[0], m));
-                        float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][h], Aj[0]));
-#pragma unroll
-                        for (int j = 1; j < K; ++j) {
-                            pj = ex2f2(sub2(a[j], m));
-                            sum = add2(sum, pj);
-                            ax = fma2(pj, fma2(g2, cb[i & 1][2 * j + h], Aj[j]), ax);
-                        }
-                        outL[h] = add2(sub2(m, off2), lg2f2(sum));
-                        outA[h] = mul2(ax, rcpf2(sum));
-                        tmax = max3f(tmax, m.x, m.y);
+                    for (int j = 0; j < K; ++j) {
+                        const float2 pj = ex2f2(sub2(a[j], m));
+                        sum = add2(sum, pj);
+                        ax = fma2(pj, fma2(g2, cb[i & 1][2 * j + h], splat2(Ain[(i * K + j) * CT + tid] + gsh)), ax);
                     }
-                    st_async_v4(push_a[i] + ob_off, outL[0].x, outL[0].y, outL[1].x, outL[1].y, push_a_mbar[i] + ob_mbar);
-                    st_async_v4(push_a[i] + ob_off + QC * 4u, outA[0].x, outA[0].y, outA[1].x, outA[1].y, push_a_mbar[i] + ob_mbar);
+                    outL[h] = add2(sub2(m, off2), lg2f2(sum));
+                    outA[h] = mul2(ax, rcpf2(sum));
+                    tmax = max3f(tmax, m.x, m.y);
                 }
-                tmax = warp_max(tmax);
-                if (lane == 0) {
-#pragma unroll
-                    for (int r = 0; r < CL; ++r) {
-                        st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
-                        mbar_arrive_cluster(full_of[r] + ob_mbar);             // this warp has read all its inputs
-                    }
-                }
-                O += (int)off;
-                if (tid == 0) O_s[t + 1] = O;
-                ib = ob;
+                const uint32_t mb = full_of[i % CL] + ob_mbar;
+                st_async_v4(push_a[i] + ob_off, outL[0].x, outL[0].y, outL[1].x, outL[1].y, mb);
+                st_async_v4(push_a[i] + ob_off + QC * 4u, outA[0].x, outA[0].y, outA[1].x, outA[1].y, mb);
             }
-            // ================= log2 Z
-            wait_inputs(ib);
-            cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
-            {
-                const float *Lfin = msg + ib * 2 * QC;
-                float ssum = 0.f;
-                for (int q = tid; q < QC; q += CT) ssum += ex2f(Lfin[q] - cmax);
-                ssum = warp_sum(ssum);
-                if (lane == 0) {
+            tmax = warp_max(tmax);
+            if (lane == 0) {
 #pragma unroll
-                    for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
-                }
-                cluster_sync();                                  // log Z exchange
+                for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
             }
-            const float lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
-            const int Ofin = O;
-            // ================= beta sweep carrying (M, Bt), with the gradient contraction
-            for (int q = tid; q < 2 * QC; q += CT) msg[ib * 2 * QC + q] = 0.f;  // M_n = 0, Bt_n = 0
-            // codebook -> TMEM, beta pairing: column 16 i + 8 jh + 2 b + e = c[2jh+e | x_i | b]
+            O += (int)off;
+            __syncthreads();                                     // every warp of this CTA has read its inputs
+            if (tid == 0) {
+                O_s[t + 1] = O;
+                bulk_wait_read0();                               // ... and so has the spill
 #pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                float2 v[8];
-                const int x = (int)rank * NBC + i * CT + tid;
-#pragma unroll
-                for (int jh = 0; jh < K / 2; ++jh) {
-                    const float4 c0 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh) * C::Q + (size_t)x * K));
-                    const float4 c1 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh + 1) * C::Q + (size_t)x * K));
-                    v[4 * jh] = make_float2(c0.x, c1.x); v[4 * jh + 1] = make_float2(c0.y, c1.y);
-                    v[4 * jh + 2] = make_float2(c0.z, c1.z); v[4 * jh + 3] = make_float2(c0.w, c1.w);
-                }
-                tmem_st16(tm_cb + 16u * i, v);
+                for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
             }
-            tmem_wait_st();
-            int P = 0;
-            float offM = 0.f;
-            cluster_sync();                                      // beta start
-            // rank 0, warp 0: turn the sums of step t (slots of parity b) into grad_W[t]
-            auto finish_step = [&](int t, int b) {
-                if (rank == 0 && warp == 0) {
-                    const float *pp = part + (b * 32 + lane) * 4;
-                    float a0 = lane < SLOTS ? pp[0] : 0.f, a2 = lane < SLOTS ? pp[1] : 0.f, az = lane < SLOTS ? pp[2] : 0.f;
-                    a0 = warp_sum(a0); a2 = warp_sum(a2); az = warp_sum(az);
-                    if (lane == 0) {
-                        const float i0 = 1.f / a0;
-                        p.gW[blk * n + t - 1] = (g_s[t - 1] - az * i0) + (a2 * i0) * (w_s[t - 1] - sf_s[t - 1]) * invT;
-                        defect = fmaxf(defect, fabsf(a0 - 1.f));
-                    }
-                }
-            };
-            for (int t = n; t >= 1; --t) {
-                const int ob = ib ^ 1;
-                if (t < n) {
-                    wait_inputs(ib);
-                    cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF);
-                    P += (int)offM;
-                    offM = rintf(cmax);
-                    finish_step(t + 1, ib);
-                }
-                const float *Min = msg + ib * 2 * QC, *Bin = Min + QC;
-                const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
-                if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
-                const float wt = w_s[t - 1], gt = g_s[t - 1];
-                const float gsh = -gt * sf_s[t - 1];
-                const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT);
-                const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
-                float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
-                float tmax = NEG_INF;
-                float2 cb[2][8];
-                tmem_ld16(tm_cb, cb[0]);
-#pragma unroll
-                for (int i = 0; i < BPT; ++i, ++chunk) {
-                    float2 acc[8];
-                    tmem_wait_ld(cb[i & 1]);
-                    tmem_ld16(tm_acc + 16u * i, acc);
-                    if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
-                    const uint32_t s = chunk % RD;
-                    mbar_wait_bounded(ring_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
-                    const float *Lh = ring + s * 2 * CH, *Ah = Lh + CH;
-                    float2 Mb[K], Yb[K];
-                    {
-                        const float4 v = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K);
-                        Mb[0] = splat2(v.x - offM); Mb[1] = splat2(v.y - offM);
-                        Mb[2] = splat2(v.z - offM); Mb[3] = splat2(v.w - offM);
-                        const float4 y = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K);
-                        Yb[0] = splat2(y.x + gsh); Yb[1] = splat2(y.y + gsh);
-                        Yb[2] = splat2(y.z + gsh); Yb[3] = splat2(y.w + gsh);
-                    }
-                    float2 u[K / 2][K], d[K / 2][K], m[K / 2], f[K / 2], Ahj[K / 2];
-#pragma unroll
-                    for (int jh = 0; jh < K / 2; ++jh) {
-#pragma unroll
-                        for (int b = 0; b < K; ++b) {
-                            d[jh][b] = sub2(w2, cb[i & 1][4 * jh + b]);
-                            u[jh][b] = fma2(mul2(d[jh][b], d[jh][b]), nl2, Mb[b]);
-                        }
-                        m[jh] = max_pairs<K>(u[jh]);
-                        Ahj[jh] = make_float2(Ah[(2 * jh) * CT + tid], Ah[(2 * jh + 1) * CT + tid]);
-                        const float2 LhD = make_float2(Lh[(2 * jh) * CT + tid] - Dm, Lh[(2 * jh + 1) * CT + tid] - Dm);
-                        f[jh] = ex2f2(add2(m[jh], LhD));
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(ring_empty + 8u * s);           // history chunk consumed
-                    tmem_wait_ld(acc);
-#pragma unroll
-                    for (int jh = 0; jh < K / 2; ++jh) {
-                        const float2 fg = mul2(f[jh], g2), fi = mul2(f[jh], gi2);
-                        float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
-#pragma unroll
-                        for (int b = 0; b < K; ++b) {
-                            const float2 pb = ex2f2(sub2(u[jh][b], m[jh]));
-                            const float2 y = fma2(g2, cb[i & 1][4 * jh + b], Yb[b]);              // h + Bt
-                            const float2 z = fma2(mul2(fi, d[jh][b]), add2(y, Ahj[jh]), fg);      // f (g + (w - c) r / T)
-                            sum = add2(sum, pb);
-                            ya = fma2(pb, y, ya);
-                            zs = fma2(pb, z, zs);
-                            acc[4 * jh + b] = fma2(pb, z, acc[4 * jh + b]);
-                        }
-                        const float2 outM = add2(m[jh], lg2f2(sum));
-                        const float2 outB = mul2(ya, rcpf2(sum));
-                        tmax = max3f(tmax, m[jh].x, m[jh].y);
-                        const uint32_t mb0 = full_of[(2 * jh) * CL / K] + ob_mbar, mb1 = full_of[(2 * jh + 1) * CL / K] + ob_mbar;
-                        st_async_f32(push_b[i][2 * jh] + ob_off, outM.x, mb0);
-                        st_async_f32(push_b[i][2 * jh + 1] + ob_off, outM.y, mb1);
-                        st_async_f32(push_b[i][2 * jh] + ob_off + QC * 4u, outB.x, mb0);
-                        st_async_f32(push_b[i][2 * jh + 1] + ob_off + QC * 4u, outB.y, mb1);
-                        S0 = fma2(f[jh], sum, S0);
-                        S2 = fma2(f[jh], fma2(Ahj[jh], sum, ya), S2);
-                        ZS = add2(ZS, zs);
-                    }
-                    tmem_st16(tm_acc + 16u * i, acc);
-                }
-                tmem_wait_st();
-                const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), zz = warp_sum(ZS.x + ZS.y);
-                tmax = warp_max(tmax);
-                if (lane == 0) {
-#pragma unroll
-                    for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
-                    st_async_v4(part_dst + (uint32_t)(ob * 128) * 4u, s0, s2, zz, 0.f, full_of[0] + ob_mbar);
-#pragma unroll
-                    for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
-                }
-                ib = ob;
-            }
-            wait_inputs(ib);                                     // the sums of step 1
-            finish_step(1, ib);
-            cluster_sync();                                      // block end
+            ib = ob;
         }
-        // this cluster's partial of grad_codebook: state [j|x|b] = j*Q + x*K + b
-        float *gc = p.gc_part + (size_t)cid * C::S;
+        // ================= log2 Z
+        wait_inputs(ib);
+        cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
+        {
+            const float *Lfin = msg + ib * 2 * QC;
+            float ssum = 0.f;
+            for (int q = tid; q < QC; q += CT) ssum += ex2f(Lfin[q] - cmax);
+            ssum = warp_sum(ssum);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
+            }
+            if (tid == 0) bulk_wait_all0();                      // history written before it is read back
+            cluster_sync();                                      // log Z exchange
+        }
+        const float lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
+        const int Ofin = O;
+        // ================= beta sweep carrying (M, Bt), with the gradient contraction
+        for (int q = tid; q < 2 * QC; q += CT) msg[ib * 2 * QC + q] = 0.f;      // M_n = 0, Bt_n = 0
+        // codebook -> TMEM, beta pairing: column 16 i + 8 jh + 2 b + e = c[2jh+e | x_i | b]
 #pragma unroll
         for (int i = 0; i < BPT; ++i) {
-            float2 acc[8];
-            tmem_ld16(tm_acc + 16u * i, acc);
-            tmem_wait_ld(acc);
+            float2 v[8];
             const int x = (int)rank * NBC + i * CT + tid;
 #pragma unroll
-            for (int jh = 0; jh < K / 2; ++jh)
-#pragma unroll
-                for (int b = 0; b < K; ++b) {
-                    gc[(size_t)(2 * jh) * C::Q + (size_t)x * K + b] = acc[4 * jh + b].x;
-                    gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[4 * jh + b].y;
-                }
+            for (int jh = 0; jh < K / 2; ++jh) {
+                const float4 c0 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh) * C::Q + (size_t)x * K));
+                const float4 c1 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh + 1) * C::Q + (size_t)x * K));
+                v[4 * jh] = make_float2(c0.x, c1.x); v[4 * jh + 1] = make_float2(c0.y, c1.y);
+                v[4 * jh + 2] = make_float2(c0.z, c1.z); v[4 * jh + 3] = make_float2(c0.w, c1.w);
+            }
+            tmem_st16(tm_cb + 16u * i, v);
         }
-        if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
+        tmem_wait_st();
+        int P = 0;
+        float offM = 0.f;
+        const uint32_t chunk_end = chunk + (uint32_t)n * BPT;    // chunks of this block: (t = n..1) x (i = 0..BPT-1)
+        // thread 0 streams the history back: request every chunk whose ring slot has been
+        // released by all warps, without ever blocking (called between butterflies)
+        auto feed_ring = [&]() {
+            while (issued != chunk_end) {
+                const uint32_t s = issued % RD;
+                if (!mbar_test(ring_empty + 8u * s, ((issued / RD) & 1u) ^ 1u)) break;
+                const uint32_t rel = issued - (chunk_end - (uint32_t)n * BPT);
+                const int t = n - (int)(rel / BPT), i = (int)(rel % BPT);
+                mbar_expect_tx(ring_full + 8u * s, 2u * CH * 4u);
+                const float *src = hist + ((size_t)(t - 1) * CL + rank) * 2 * QC + (size_t)i * CH;
+                bulk_load(ring_u32 + s * 2u * CH * 4u, src, CH * 4u, ring_full + 8u * s);
+                bulk_load(ring_u32 + s * 2u * CH * 4u + CH * 4u, src + QC, CH * 4u, ring_full + 8u * s);
+                ++issued;
+            }
+        };
+        if (tid == 0) { fence_proxy_async(); feed_ring(); }
+        cluster_sync();                                          // beta start
+        // rank 0, warp 0: turn the sums of step t (slots of parity b) into grad_W[t]
+        auto finish_step = [&](int t, int b) {
+            if (rank == 0 && warp == 0) {
+                const float *pp = part + (b * 32 + lane) * 4;
+                float a0 = lane < SLOTS ? pp[0] : 0.f, a2 = lane < SLOTS ? pp[1] : 0.f, az = lane < SLOTS ? pp[2] : 0.f;
+                a0 = warp_sum(a0); a2 = warp_sum(a2); az = warp_sum(az);
+                if (lane == 0) {
+                    const float i0 = 1.f / a0;
+                    p.gW[blk * n + t - 1] = (g_s[t - 1] - az * i0) + (a2 * i0) * (w_s[t - 1] - sf_s[t - 1]) * invT;
+                    defect = fmaxf(defect, fabsf(a0 - 1.f));
+                }
+            }
+        };
+        for (int t = n; t >= 1; --t) {
+            const int ob = ib ^ 1;
+            if (t < n) {
+                wait_inputs(ib);
+                cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF);
+                P += (int)offM;
+                offM = rintf(cmax);
+                finish_step(t + 1, ib);
+            }
+            const float *Min = msg + ib * 2 * QC, *Bin = Min + QC;
+            const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
+            if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
+            const float wt = w_s[t - 1], gt = g_s[t - 1];
+            const float gsh = -gt * sf_s[t - 1];
+            const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT);
+            const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
+            float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
+            float tmax = NEG_INF;
+            float2 cb[2][8];
+            tmem_ld16(tm_cb, cb[0]);
+#pragma unroll
+            for (int i = 0; i < BPT; ++i, ++chunk) {
+                float2 acc[8];
+                if (tid == 0) feed_ring();
+                tmem_wait_ld(cb[i & 1]);
+                tmem_ld16(tm_acc + 16u * i, acc);
+                if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
+                const uint32_t s = chunk % RD;
+                mbar_wait_bounded(ring_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
+                const float *Lh = ring + s * 2 * CH, *Ah = Lh + CH;
+                const float4 mv = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K);
+                const float4 bv = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K);
+                const float Mb[K] = {mv.x - offM, mv.y - offM, mv.z - offM, mv.w - offM};
+                const float Yb[K] = {bv.x + gsh, bv.y + gsh, bv.z + gsh, bv.w + gsh};
+                tmem_wait_ld(acc);
+#pragma unroll
+                for (int jh = 0; jh < K / 2; ++jh) {
+                    float2 u[K], d[K];
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        d[b] = sub2(w2, cb[i & 1][4 * jh + b]);
+                        u[b] = fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
+                    }
+                    const float2 m = max_pairs<K>(u);
+                    const float2 Ahj = make_float2(Ah[(2 * jh) * CT + tid], Ah[(2 * jh + 1) * CT + tid]);
+                    const float2 LhD = make_float2(Lh[(2 * jh) * CT + tid] - Dm, Lh[(2 * jh + 1) * CT + tid] - Dm);
+                    const float2 f = ex2f2(add2(m, LhD));
+                    const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
+                    float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        const float2 pb = ex2f2(sub2(u[b], m));
+                        const float2 y = fma2(g2, cb[i & 1][4 * jh + b], splat2(Yb[b]));      // h + Bt
+                        const float2 z = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);               // f (g + (w - c) r / T)
+                        sum = add2(sum, pb);
+                        ya = fma2(pb, y, ya);
+                        zs = fma2(pb, z, zs);
+                        acc[4 * jh + b] = fma2(pb, z, acc[4 * jh + b]);
+                    }
+                    const float2 outM = add2(m, lg2f2(sum));
+                    const float2 outB = mul2(ya, rcpf2(sum));
+                    tmax = max3f(tmax, m.x, m.y);
+                    const uint32_t mb0 = full_of[(2 * jh) * CL / K] + ob_mbar, mb1 = full_of[(2 * jh + 1) * CL / K] + ob_mbar;
+                    st_async_f32(push_b[i][2 * jh] + ob_off, outM.x, mb0);
+                    st_async_f32(push_b[i][2 * jh + 1] + ob_off, outM.y, mb1);
+                    st_async_f32(push_b[i][2 * jh] + ob_off + QC * 4u, outB.x, mb0);
+                    st_async_f32(push_b[i][2 * jh + 1] + ob_off + QC * 4u, outB.y, mb1);
+                    S0 = fma2(f, sum, S0);
+                    S2 = fma2(f, fma2(Ahj, sum, ya), S2);
+                    ZS = add2(ZS, zs);
+                }
+                tmem_st16(tm_acc + 16u * i, acc);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ring_empty + 8u * s);               // history chunk consumed by this warp
+            }
+            tmem_wait_st();
+            const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), zz = warp_sum(ZS.x + ZS.y);
+            tmax = warp_max(tmax);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
+                st_async_v4(part_dst + (uint32_t)(ob * 128) * 4u, s0, s2, zz, 0.f, full_of[0] + ob_mbar);
+            }
+            __syncthreads();                                     // every warp of this CTA has read its inputs
+            if (tid == 0) {
+#pragma unroll
+                for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
+            }
+            ib = ob;
+        }
+        wait_inputs(ib);                                         // the sums of step 1
+        finish_step(1, ib);
+        cluster_sync();                                          // block end
     }
+    // this cluster's partial of grad_codebook: state [j|x|b] = j*Q + x*K + b
+    float *gc = p.gc_part + (size_t)cid * C::S;
+#pragma unroll
+    for (int i = 0; i < BPT; ++i) {
+        float2 acc[8];
+        tmem_ld16(tm_acc + 16u * i, acc);
+        tmem_wait_ld(acc);
+        const int x = (int)rank * NBC + i * CT + tid;
+#pragma unroll
+        for (int jh = 0; jh < K / 2; ++jh)
+#pragma unroll
+            for (int b = 0; b < K; ++b) {
+                gc[(size_t)(2 * jh) * C::Q + (size_t)x * K + b] = acc[4 * jh + b].x;
+                gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[4 * jh + b].y;
+            }
+    }
+    if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     cluster_sync();             // no CTA leaves while a peer may still address its shared memory
