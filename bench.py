@@ -32,6 +32,8 @@ METRIC = "bcjr_fwd_bwd_trellis_edge_updates_per_s"
 UNIT = "edges/s"
 WORKLOADS = {"tiny": synth.tiny, "mid": synth.mid, "q_proj": synth.q_proj, "layer": synth.decoder_layer,
              "gate_k3": synth.gate_k3}
+# (Lb, k, kernel) -> measured DRAM bytes per weight block (n = 256), see profiles/*.md
+NCU_DRAM_BYTES_PER_BLOCK = {(16, 2, "bwd"): 66.3e6, (16, 2, "fwd"): 33.1e6}
 MUFU_PER_CLK_PER_SM = 16          # special-function results per clock per SM (CUDA throughput table, cc 10.0)
 NUM_SMS = 148
 
@@ -313,12 +315,11 @@ def main():
     achieved = ops / (dom_ms * 1e-3) / 1e9
     sm_max = clocks.get("sm_max_mhz") or 1965.0
     peak = NUM_SMS * MUFU_PER_CLK_PER_SM * sm_max * 1e6 / 1e9
-    traffic = None
-    tfile = ROOT / "profiles" / "traffic.json"
-    if tfile.exists():
-        tj = json.loads(tfile.read_text()).get(f"{wl.name}:{dom}")
-        if tj:
-            traffic = tj["dram_bytes_per_block"] * nblocks / len(mats)
+    # DRAM bytes per block of the dominant kernel, from the ncu captures summarised under profiles/
+    # (dram__bytes_read.sum + dram__bytes_write.sum of one launch / blocks of that launch, small
+    # case of the same kernel; traffic grows in proportion to the number of blocks)
+    per_block = NCU_DRAM_BYTES_PER_BLOCK.get((wl.Lb, wl.k, dom)) if diag.last_path else None
+    traffic = per_block * nblocks / len(mats) if per_block else None
     roofline = {"bound": "alu", "kernel": f"bcjr_{dom}", "achieved": achieved, "peak": peak, "unit": "Gop/s (MUFU)",
                 "frac": achieved / peak, "traffic": traffic,
                 "peak_source": f"{NUM_SMS} SMs x {MUFU_PER_CLK_PER_SM} MUFU/clk x {sm_max:.0f} MHz (derived)",

@@ -59,9 +59,14 @@ bcjr_status bcjr_create(bcjr_ctx **out, int device_ordinal);
 /* Frees the context and its scratch memory (synchronises the device first). */
 bcjr_status bcjr_destroy(bcjr_ctx *ctx);
 
-/* Tuning / test hooks.  name = "path": 0 auto, 1 force generic kernels, 2 force cluster
- * kernels (EUNSUPPORTED at call time when they do not cover the shape);
- * name = "max_ctas": cap on resident thread blocks (0 = fill the GPU). */
+/* Tuning / test hooks.
+ *   "path"        0 auto, 1 force the generic kernels, 2 force the large-trellis kernels
+ *                 (BCJR_EUNSUPPORTED at call time when they do not cover the shape)
+ *   "fwd_variant" large-trellis forward kernel: 0 = one CTA per block with the codebook in tensor
+ *                 memory (Lb = 16, k = 2), 1 = two-CTA cluster kernel with the codebook in registers
+ *   "bwd_variant" large-trellis backward kernel: 0 = two-CTA clusters with codebook and gradient
+ *                 accumulators in tensor memory (Lb = 16, k = 2), 1 = four-CTA clusters, registers
+ *   "max_ctas"    cap on resident thread blocks (0 = fill the GPU) */
 bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value);
 
 /*

@@ -167,11 +167,48 @@ def test_mid_trellis_cold_limit_matches_viterbi(ctx):
 
 
 # ------------------------------------------------------------------ S = 2^16
-def test_q_proj_shape_sampled_blocks(ctx):
+@pytest.mark.parametrize("variant", ["tmem", "cluster_registers", "generic"])
+def test_q_proj_shape_sampled_blocks(ctx, variant):
+    # the same sampled blocks through every implementation of the 2^16-state path
     wl = synth.q_proj()
-    idx = synth.sample_blocks(wl.num_blocks(), 6)
+    idx = synth.sample_blocks(wl.num_blocks(), 6 if variant != "generic" else 3)
     W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
-    _check_all(ctx, W, c, g, wl.Lb, wl.k, wl.T, "q_proj sample")
+    opts = {"tmem": dict(path=0, fwd_variant=0, bwd_variant=0),
+            "cluster_registers": dict(path=2, fwd_variant=1, bwd_variant=1),
+            "generic": dict(path=1, fwd_variant=0, bwd_variant=0)}[variant]
+    try:
+        for k_, v_ in opts.items():
+            ctx.set_option(k_, v_)
+        got = _check_all(ctx, W, c, g, wl.Lb, wl.k, wl.T, f"q_proj sample [{variant}]", viterbi=(variant == "tmem"))
+        assert got["diag"].last_path == (0 if variant == "generic" else 1)
+    finally:
+        for k_ in opts:
+            ctx.set_option(k_, 0)
+
+
+def test_q_proj_full_size_sampled_outputs_and_invariants(ctx):
+    """The full 2048 x 2048 matrix (16384 blocks) in the launch configuration the benchmark times.
+    soft and grad_W of a block depend on that block alone, so sampled blocks are compared with
+    the oracle one by one; grad_codebook sums over all blocks and is checked through the shift
+    identity  sum grad_W + sum grad_codebook = sum g  (soft(w + a, c + a) = soft(w, c) + a)."""
+    import torch
+    wl = synth.q_proj()
+    W, c, g = wl.weights(), wl.codebook(), wl.upstream()
+    got = parity.gpu_forward_backward(ctx, W, c, g, wl.Lb, wl.k, wl.T)
+    assert got["diag"].last_path == 1 and got["diag"].device_status == 0
+    assert got["diag"].max_posterior_defect < 1e-3
+    assert np.all(np.isfinite(got["soft"])) and np.all(np.isfinite(got["grad_W"]))
+    idx = synth.sample_blocks(wl.num_blocks(), 8, seed=123)
+    ref_f = oracle.soft_quantize(W[idx], c, wl.Lb, wl.k, wl.T)
+    ref_b = oracle.backward(W[idx], c, g[idx], wl.Lb, wl.k, wl.T)
+    assert parity.rel_inf(got["soft"][idx], ref_f["soft"]) <= parity.SOFT_TOL
+    assert parity.rel_inf(got["grad_W"][idx], ref_b["grad_W"]) <= parity.GRAD_TOL
+    np.testing.assert_allclose(got["logZ"][idx], ref_f["logZ"], rtol=1e-5, atol=1e-3)
+    total = got["grad_W"].astype(np.float64).sum() + got["grad_codebook"].astype(np.float64).sum()
+    gsum = g.astype(np.float64).sum()
+    assert abs(total - gsum) <= 1e-3 * np.abs(g).astype(np.float64).sum() ** 0.5 * 10
+    # the soft codeword is a convex combination of table entries
+    assert got["soft"].min() >= c.min() - 1e-4 and got["soft"].max() <= c.max() + 1e-4
 
 
 @pytest.mark.parametrize("T", [0.01, 0.001])
