@@ -329,6 +329,11 @@ struct DeviceGuard {
 
 extern "C" {
 
+#ifdef BCJR_TIMING
+// development aid, not part of the ABI: cycle counters of the beta sweep of the backward kernel
+void bcjr_debug_duo_timing(unsigned long long *out8) { cudaMemcpyFromSymbol(out8, g_duo_timing, 64); }
+#endif
+
 bcjr_status bcjr_create(bcjr_ctx **out, int device_ordinal)
 {
     if (!out) return BCJR_EINVAL;
@@ -424,7 +429,10 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
 #ifndef BCJR_NO_CLUSTER
     use_cluster = ctx->opt_path != 1 && cluster_supported(Lb, k);
     if (ctx->opt_path == 2 && !use_cluster) return BCJR_EUNSUPPORTED;
-    if (use_cluster) rc = launch_fwd_cluster(ctx, p, k, st);
+    if (use_cluster) {
+        rc = launch_fwd_cluster(ctx, p, k, st);
+        if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { use_cluster = false; rc = BCJR_OK; }   // e.g. n too long
+    }
 #else
     if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
 #endif
@@ -467,7 +475,10 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
 #ifndef BCJR_NO_CLUSTER
     use_cluster = ctx->opt_path != 1 && cluster_supported(ctx->Lb, ctx->k);
     if (ctx->opt_path == 2 && !use_cluster) return BCJR_EUNSUPPORTED;
-    if (use_cluster) rc = launch_bwd_cluster(ctx, p, ctx->k, grad_codebook, st);
+    if (use_cluster) {
+        rc = launch_bwd_cluster(ctx, p, ctx->k, grad_codebook, st);
+        if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { use_cluster = false; rc = BCJR_OK; }
+    }
 #else
     if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
 #endif

@@ -26,6 +26,15 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_mbar)
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_mbar) : "memory");
 }
 
+#ifdef BCJR_TIMING
+__device__ unsigned long long g_duo_timing[8];   // beta sweep, warp 1 of CTA 0: compute, cta barrier, input wait, ring wait
+#define TICK(var) const long long var = clock64()
+#define TACC(slot, a, b) do { if (blockIdx.x == 0 && warp == 1 && lane == 0) tacc[slot] += (unsigned long long)((b) - (a)); } while (0)
+#else
+#define TICK(var)
+#define TACC(slot, a, b)
+#endif
+
 struct DuoCfg {
     static constexpr int LB = 16, KB = 2, K = 4, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
     static constexpr int CL = 2;
@@ -147,6 +156,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
         for (int i = 0; i < BPT; ++i) tmem_st16(tm_acc + 16u * i, z);
         tmem_wait_st();
     }
+#ifdef BCJR_TIMING
+    unsigned long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
     uint32_t chunk = 0;            // history chunks consumed so far (all threads count alike)
     uint32_t issued = 0;           // history chunks requested so far (thread 0)
     float defect = 0.f;
@@ -312,8 +324,10 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
         };
         for (int t = n; t >= 1; --t) {
             const int ob = ib ^ 1;
+            TICK(tk0);
             if (t < n) {
                 wait_inputs(ib);
+                TICK(tk1); TACC(2, tk0, tk1);
                 cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF);
                 P += (int)offM;
                 offM = rintf(cmax);
@@ -338,7 +352,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 tmem_ld16(tm_acc + 16u * i, acc);
                 if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
                 const uint32_t s = chunk % RD;
+                TICK(tr0);
                 mbar_wait_bounded(ring_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
+                TICK(tr1); TACC(3, tr0, tr1);
                 const float *Lh = ring + s * 2 * CH, *Ah = Lh + CH;
                 const float4 mv = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K);
                 const float4 bv = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K);
@@ -393,7 +409,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
                 st_async_v4(part_dst + (uint32_t)(ob * 128) * 4u, s0, s2, zz, 0.f, full_of[0] + ob_mbar);
             }
+            TICK(tb0);
             __syncthreads();                                     // every warp of this CTA has read its inputs
+            TICK(tb1); TACC(1, tb0, tb1); TACC(0, tk0, tb1);
             if (tid == 0) {
 #pragma unroll
                 for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
@@ -420,6 +438,10 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[4 * jh + b].y;
             }
     }
+#ifdef BCJR_TIMING
+    if (blockIdx.x == 0 && warp == 1 && lane == 0)
+        for (int e = 0; e < 8; ++e) g_duo_timing[e] = tacc[e];
+#endif
     if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();

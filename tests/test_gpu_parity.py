@@ -186,6 +186,47 @@ def test_q_proj_shape_sampled_blocks(ctx, variant):
             ctx.set_option(k_, 0)
 
 
+@pytest.mark.parametrize("n,B", [(1, 3), (2, 2), (3, 1), (7, 5), (64, 2), (255, 1)])
+@pytest.mark.parametrize("variant", ["tmem", "cluster_registers"])
+def test_large_trellis_ragged_lengths_and_block_counts(ctx, variant, n, B):
+    # odd and tiny n exercise the buffer-parity and history-ring bookkeeping of the 2^16-state
+    # kernels; B below the number of resident clusters leaves most of the grid without work
+    Lb, k, T = 16, 2, 0.2
+    W, c, g = _rand(n, Lb, B, seed=4000 + n)
+    opts = dict(path=2, fwd_variant=int(variant != "tmem"), bwd_variant=int(variant != "tmem"))
+    try:
+        for k_, v_ in opts.items():
+            ctx.set_option(k_, v_)
+        got = _check_all(ctx, W, c, g, Lb, k, T, f"Lb=16 n={n} B={B} [{variant}]", viterbi=False)
+        assert got["diag"].last_path == 1 and got["diag"].device_status == 0
+    finally:
+        for k_ in opts:
+            ctx.set_option(k_, 0)
+
+
+def test_large_trellis_long_blocks_fall_back_cleanly(ctx):
+    # n = 1100 exceeds the backward TMEM kernel's step table (1024): it must take the next kernel
+    # that covers the shape and still match; n = 2100 exceeds every large-trellis kernel
+    Lb, k, T = 16, 2, 0.3
+    for n in (1100, 2100):
+        W, c, g = _rand(n, Lb, 1, seed=4100 + n)
+        got = _check_all(ctx, W, c, g, Lb, k, T, f"Lb=16 n={n}", viterbi=False)
+        assert got["diag"].device_status == 0
+
+
+def test_results_do_not_depend_on_what_ran_before(ctx):
+    # scratch (history, partial sums, tensor memory) is reused between calls and between
+    # blocks: the same input must give bit-identical output regardless of the previous call
+    wl = synth.q_proj()
+    W, c, g = wl.weights()[:5], wl.codebook(), wl.upstream()[:5]
+    first = parity.gpu_forward_backward(ctx, W, c, g, wl.Lb, wl.k, wl.T)
+    other = _rand(33, 16, 3, seed=9)
+    parity.gpu_forward_backward(ctx, other[0], other[1], other[2], 16, 2, 0.7)
+    again = parity.gpu_forward_backward(ctx, W, c, g, wl.Lb, wl.k, wl.T)
+    for key in ("soft", "logZ", "grad_W", "grad_codebook"):
+        np.testing.assert_array_equal(first[key], again[key], err_msg=key)
+
+
 def test_q_proj_full_size_sampled_outputs_and_invariants(ctx):
     """The full 2048 x 2048 matrix (16384 blocks) in the launch configuration the benchmark times.
     soft and grad_W of a block depend on that block alone, so sampled blocks are compared with
