@@ -12,10 +12,14 @@
 //
 // Step protocol.  Messages are double-buffered.  Every output is pushed with st.async into the
 // consumer CTA's buffer `ob` and credits that CTA's mbarrier full[ob] with its bytes; a phase of
-// full[ob] completes when (a) all bytes have landed and (b) every CTA of the cluster has
-// arrived on it, which a CTA does once all its warps have finished the step and the bulk copy
-// that spills its input buffer to the history has finished reading it -- so nobody still
-// reads the other buffer when the next step starts overwriting it.
+// full[ob] completes when (a) all bytes have landed and (b) every warp of the cluster has
+// arrived on it after its last butterfly of the step (thread 0 of each CTA only after the bulk
+// copy that spills the input buffer to the history has finished reading it) -- so nobody still
+// reads the other buffer when the next step starts overwriting it.  The arrival is relaxed:
+// it has nothing to publish (the data travels with st.async and is accounted in bytes), and the
+// reads it has to follow are complete when it issues, because every value a warp reads from
+// its input buffer feeds, through register dependences, an st.async that precedes the arrival
+// in program order.  (A release arrival per warp costs a cluster-scope fence: 8 % of the kernel.)
 #pragma once
 #include "bcjr_solo.cuh"
 
@@ -23,7 +27,11 @@ namespace bcjr {
 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_mbar)
 {
+#ifdef BCJR_RELEASE_ARRIVE
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_mbar) : "memory");
+#else
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_mbar) : "memory");
+#endif
 }
 
 #ifdef BCJR_TIMING
@@ -43,13 +51,12 @@ struct DuoCfg {
     static constexpr int BPT = NBC / THREADS;                  // 4 butterflies per thread
     static constexpr int SLOTS = CL * NWARP;                   // 32 per-warp partial slots
     static constexpr int CH = K * THREADS;                     // floats per array per history chunk
-    static constexpr int RD = BPT;                             // ring depth: one step of chunks
+    static constexpr int RD = BPT + 1;                         // ring depth: a step and a quarter of chunks
     static constexpr int MAX_N = 1024;
-    static constexpr int ARRIVALS = 1 + CL;                    // armer + one arrival per CTA of the cluster
+    static constexpr int ARRIVALS = 1 + SLOTS;                 // armer + one arrival per warp of the cluster
     static constexpr int OFF_MSG = 0;                          // [2 parity][2 arrays][QC]
     static constexpr int OFF_RING = OFF_MSG + 4 * QC;          // [RD][2 arrays][CH]
-    static constexpr int OFF_W = OFF_RING + RD * 2 * CH;       // w, g, soft: [3][MAX_N]
-    static constexpr int OFF_O = OFF_W + 3 * MAX_N;            // int [MAX_N + 2]
+    static constexpr int OFF_O = OFF_RING + RD * 2 * CH;       // int [MAX_N + 2]
     static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;     // [2][32]
     static constexpr int OFF_PART = OFF_WMAX + 64;             // [2][32][4]
     static constexpr int OFF_LZ = OFF_PART + 256;              // [32]
@@ -83,7 +90,6 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
 
     float *msg = smem + C::OFF_MSG;
     float *ring = smem + C::OFF_RING;
-    float *w_s = smem + C::OFF_W, *g_s = w_s + C::MAX_N, *sf_s = g_s + C::MAX_N;
     int *O_s = reinterpret_cast<int *>(smem + C::OFF_O);
     float *wmax = smem + C::OFF_WMAX;
     float *part = smem + C::OFF_PART;
@@ -165,11 +171,8 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
 
     for (int64_t blk = cid; blk < p.B; blk += ncl) {
         int ib = 0;
-        for (int t = tid; t < n; t += CT) {
-            w_s[t] = __ldg(p.W + blk * n + t);
-            g_s[t] = __ldg(p.g + blk * n + t);
-            sf_s[t] = __ldg(p.soft + blk * n + t);
-        }
+        // per-step scalars of this block (read through the read-only cache, one line per warp)
+        const float *w_s = p.W + blk * n, *g_s = p.g + blk * n, *sf_s = p.soft + blk * n;
         for (int q = tid; q < 2 * QC; q += CT) msg[q] = 0.f;                   // L_1 = 0, At_1 = 0 (parity 0)
         if (tid == 0) O_s[1] = 0;
         // codebook -> TMEM, alpha pairing: column 16 i + 4 j + l = c[j | x_i | l]
@@ -205,9 +208,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)ib * BUF_BYTES, BUF_BYTES);
                 bulk_commit();
             }
-            const float gt = g_s[t - 1];
-            const float gsh = -gt * sf_s[t - 1];                              // centring: h = g c - g soft
-            const float2 w2 = splat2(w_s[t - 1]), g2 = splat2(gt), off2 = splat2(off);
+            const float gt = __ldg(g_s + t - 1);
+            const float gsh = -gt * __ldg(sf_s + t - 1);                      // centring: h = g c - g soft
+            const float2 w2 = splat2(__ldg(w_s + t - 1)), g2 = splat2(gt), off2 = splat2(off);
             float tmax = NEG_INF;
             float2 cb[2][8];
             tmem_ld16(tm_cb, cb[0]);
@@ -246,10 +249,12 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
             }
             O += (int)off;
-            __syncthreads();                                     // every warp of this CTA has read its inputs
             if (tid == 0) {
                 O_s[t + 1] = O;
-                bulk_wait_read0();                               // ... and so has the spill
+                bulk_wait_read0();                               // the spill has left the input buffer
+            }
+            __syncwarp();
+            if (lane == 0) {                                     // this warp has read all its inputs
 #pragma unroll
                 for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
             }
@@ -317,7 +322,7 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 a0 = warp_sum(a0); a2 = warp_sum(a2); az = warp_sum(az);
                 if (lane == 0) {
                     const float i0 = 1.f / a0;
-                    p.gW[blk * n + t - 1] = (g_s[t - 1] - az * i0) + (a2 * i0) * (w_s[t - 1] - sf_s[t - 1]) * invT;
+                    p.gW[blk * n + t - 1] = (__ldg(g_s + t - 1) - az * i0) + (a2 * i0) * (__ldg(w_s + t - 1) - __ldg(sf_s + t - 1)) * invT;
                     defect = fmaxf(defect, fabsf(a0 - 1.f));
                 }
             }
@@ -336,8 +341,8 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             const float *Min = msg + ib * 2 * QC, *Bin = Min + QC;
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
-            const float wt = w_s[t - 1], gt = g_s[t - 1];
-            const float gsh = -gt * sf_s[t - 1];
+            const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1);
+            const float gsh = -gt * __ldg(sf_s + t - 1);
             const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT);
             const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
             float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
@@ -350,7 +355,6 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 if (tid == 0) feed_ring();
                 tmem_wait_ld(cb[i & 1]);
                 tmem_ld16(tm_acc + 16u * i, acc);
-                if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
                 const uint32_t s = chunk % RD;
                 TICK(tr0);
                 mbar_wait_bounded(ring_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
@@ -360,7 +364,6 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 const float4 bv = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K);
                 const float Mb[K] = {mv.x - offM, mv.y - offM, mv.z - offM, mv.w - offM};
                 const float Yb[K] = {bv.x + gsh, bv.y + gsh, bv.z + gsh, bv.w + gsh};
-                tmem_wait_ld(acc);
 #pragma unroll
                 for (int jh = 0; jh < K / 2; ++jh) {
                     float2 u[K], d[K];
@@ -375,6 +378,7 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                     const float2 f = ex2f2(add2(m, LhD));
                     const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
                     float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
+                    float2 pz[K];
 #pragma unroll
                     for (int b = 0; b < K; ++b) {
                         const float2 pb = ex2f2(sub2(u[b], m));
@@ -382,9 +386,17 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                         const float2 z = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);               // f (g + (w - c) r / T)
                         sum = add2(sum, pb);
                         ya = fma2(pb, y, ya);
-                        zs = fma2(pb, z, zs);
-                        acc[4 * jh + b] = fma2(pb, z, acc[4 * jh + b]);
+                        pz[b] = mul2(pb, z);
+                        zs = add2(zs, pz[b]);
                     }
+                    if (jh == 0) {
+                        // accumulators (requested at the top of the butterfly) are needed only now;
+                        // the next butterfly's codebook slice is requested behind them
+                        tmem_wait_ld(acc);
+                        if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
+                    }
+#pragma unroll
+                    for (int b = 0; b < K; ++b) acc[4 * jh + b] = add2(acc[4 * jh + b], pz[b]);
                     const float2 outM = add2(m, lg2f2(sum));
                     const float2 outB = mul2(ya, rcpf2(sum));
                     tmax = max3f(tmax, m.x, m.y);
@@ -410,9 +422,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 st_async_v4(part_dst + (uint32_t)(ob * 128) * 4u, s0, s2, zz, 0.f, full_of[0] + ob_mbar);
             }
             TICK(tb0);
-            __syncthreads();                                     // every warp of this CTA has read its inputs
+            __syncwarp();
             TICK(tb1); TACC(1, tb0, tb1); TACC(0, tk0, tb1);
-            if (tid == 0) {
+            if (lane == 0) {                                     // this warp has read all its inputs
 #pragma unroll
                 for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
             }
