@@ -14,6 +14,7 @@
 #include "bcjr_cluster.cuh"
 #include "bcjr_solo.cuh"
 #include "bcjr_duo.cuh"
+#include "bcjr_viterbi.cuh"
 #endif
 
 using namespace bcjr;
@@ -287,6 +288,25 @@ bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_co
     return BCJR_EUNSUPPORTED;
 }
 
+// Viterbi, one CTA per block with the codebook in tensor memory (Lb = 16, k = 2).
+bcjr_status launch_vit_solo(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
+{
+    using C = VitSoloCfg;
+    if (p.n > C::MAX_N) return BCJR_EUNSUPPORTED;
+    CU(cudaFuncSetAttribute(viterbi_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    int64_t grid = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    if (grid > p.B) grid = p.B;
+    bcjr_status rc = ensure(ctx, ctx->bp, (size_t)grid * 2 * p.n * C::NB);
+    if (rc) return rc;
+    p.bp = (uint8_t *)ctx->bp.ptr;
+    p.diag = ctx->diag;
+    viterbi_solo_kernel<<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
 // Forward call, one CTA per block with the codebook in tensor memory (Lb = 16, k = 2).
 bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
@@ -512,14 +532,27 @@ bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook, i
     VitParams p{};
     p.W = W; p.cb = codebook; p.path_bits = path_bits; p.path_stride = path_stride_bytes;
     p.states = states; p.hard = hard; p.B = num_blocks; p.Lb = Lb; p.n = n;
-    switch (k) {
-        case 1: rc = launch_vit_generic<1>(ctx, p, st); break;
-        case 2: rc = launch_vit_generic<2>(ctx, p, st); break;
-        case 3: rc = launch_vit_generic<3>(ctx, p, st); break;
-        default: rc = launch_vit_generic<4>(ctx, p, st); break;
+    bool use_large = false;
+#ifndef BCJR_NO_CLUSTER
+    use_large = ctx->opt_path != 1 && Lb == 16 && k == 2;
+    if (ctx->opt_path == 2 && !use_large) return BCJR_EUNSUPPORTED;
+    if (use_large) {
+        rc = launch_vit_solo(ctx, p, st);
+        if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { use_large = false; rc = BCJR_OK; }
+    }
+#else
+    if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
+#endif
+    if (!use_large) {
+        switch (k) {
+            case 1: rc = launch_vit_generic<1>(ctx, p, st); break;
+            case 2: rc = launch_vit_generic<2>(ctx, p, st); break;
+            case 3: rc = launch_vit_generic<3>(ctx, p, st); break;
+            default: rc = launch_vit_generic<4>(ctx, p, st); break;
+        }
     }
     if (rc) return rc;
-    ctx->last_path = 0;
+    ctx->last_path = use_large ? 1 : 0;
     return BCJR_OK;
 }
 

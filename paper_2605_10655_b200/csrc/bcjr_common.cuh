@@ -99,6 +99,7 @@ struct VitParams {
     uint8_t *bp;             // [grid][n*Q] best branch per group per step
     double *msg;             // [grid][2*Q] or null (shared)
     int *path_ws;            // [grid][n] state sequence scratch
+    DeviceDiag *diag;
     int64_t B;
     int Lb, n;
 };

@@ -197,11 +197,31 @@ def test_large_trellis_ragged_lengths_and_block_counts(ctx, variant, n, B):
     try:
         for k_, v_ in opts.items():
             ctx.set_option(k_, v_)
-        got = _check_all(ctx, W, c, g, Lb, k, T, f"Lb=16 n={n} B={B} [{variant}]", viterbi=False)
+        got = _check_all(ctx, W, c, g, Lb, k, T, f"Lb=16 n={n} B={B} [{variant}]", viterbi=(variant == "tmem"))
         assert got["diag"].last_path == 1 and got["diag"].device_status == 0
     finally:
         for k_ in opts:
             ctx.set_option(k_, 0)
+
+
+def test_large_trellis_viterbi_many_blocks_per_cta(ctx):
+    # more blocks than thread blocks: every CTA runs several blocks, alternating its two
+    # backpointer buffers while the trace warp lags one block behind the dynamic programme
+    Lb, k, n = 16, 2, 12
+    W, c, _ = _rand(n, Lb, 450, seed=4200)
+    ref = oracle.viterbi(W, c, Lb, k)
+    got = parity.gpu_viterbi(ctx, W, c, Lb, k)
+    parity.assert_viterbi(got, ref, "viterbi 450 blocks")
+    ctx.set_option("max_ctas", 3)
+    try:
+        parity.assert_viterbi(parity.gpu_viterbi(ctx, W[:40], c, Lb, k), oracle.viterbi(W[:40], c, Lb, k), "3 CTAs")
+    finally:
+        ctx.set_option("max_ctas", 0)
+    ctx.set_option("path", GENERIC)
+    try:
+        parity.assert_viterbi(parity.gpu_viterbi(ctx, W[:6], c, Lb, k), oracle.viterbi(W[:6], c, Lb, k), "generic")
+    finally:
+        ctx.set_option("path", 0)
 
 
 def test_large_trellis_long_blocks_fall_back_cleanly(ctx):
