@@ -149,6 +149,8 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--blocks", type=int, default=0, help="cap on blocks per matrix (0 = all); for profiling")
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 generic kernels, 2 cluster kernels")
+    ap.add_argument("--fwd-variant", type=int, default=0)
+    ap.add_argument("--bwd-variant", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-viterbi", action="store_true")
@@ -180,6 +182,10 @@ def main():
     ctx = Context(local)
     if args.path:
         ctx.set_option("path", args.path)
+    if args.fwd_variant:
+        ctx.set_option("fwd_variant", args.fwd_variant)
+    if args.bwd_variant:
+        ctx.set_option("bwd_variant", args.bwd_variant)
     cb = torch.from_numpy(wl.codebook()).to(dev)
     mats = []
     for i, (name, _) in enumerate(wl.matrices):
