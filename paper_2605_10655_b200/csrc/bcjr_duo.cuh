@@ -173,7 +173,11 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
         int ib = 0;
         // per-step scalars of this block (read through the read-only cache, one line per warp)
         const float *w_s = p.W + blk * n, *g_s = p.g + blk * n, *sf_s = p.soft + blk * n;
-        for (int q = tid; q < 2 * QC; q += CT) msg[q] = 0.f;                   // L_1 = 0, At_1 = 0 (parity 0)
+        // L_1 = 0; the At array carries At + gsh (gsh_t = -g_t soft_t centres h_t = g_t c - g_t soft_t)
+        {
+            const float gsh1 = -__ldg(g_s) * __ldg(sf_s);
+            for (int q = tid; q < QC; q += CT) { msg[q] = 0.f; msg[QC + q] = gsh1; }
+        }
         if (tid == 0) O_s[1] = 0;
         // codebook -> TMEM, alpha pairing: column 16 i + 4 j + l = c[j | x_i | l]
 #pragma unroll
@@ -209,7 +213,8 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 bulk_commit();
             }
             const float gt = __ldg(g_s + t - 1);
-            const float gsh = -gt * __ldg(sf_s + t - 1);                      // centring: h = g c - g soft
+            // shift for the consumers of this step's At (step t+1); unused at t = n
+            const float2 gshn2 = splat2(t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f);
             const float2 w2 = splat2(__ldg(w_s + t - 1)), g2 = splat2(gt), off2 = splat2(off);
             float tmax = NEG_INF;
             float2 cb[2][8];
@@ -218,25 +223,31 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             for (int i = 0; i < BPT; ++i) {
                 tmem_wait_ld(cb[i & 1]);
                 if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
-                float2 outL[K / 2], outA[K / 2];
+                float2 outL[K / 2], outA[K / 2], Lj[K], Aj[K];
+#pragma unroll
+                for (int j = 0; j < K; ++j) {
+                    Lj[j] = splat2(Lin[(i * K + j) * CT + tid]);
+                    Aj[j] = splat2(Ain[(i * K + j) * CT + tid]);
+                }
 #pragma unroll
                 for (int h = 0; h < K / 2; ++h) {
                     float2 a[K];
 #pragma unroll
                     for (int j = 0; j < K; ++j) {
                         const float2 d = sub2(cb[i & 1][2 * j + h], w2);
-                        a[j] = fma2(mul2(d, d), nl2, splat2(Lin[(i * K + j) * CT + tid]));
+                        a[j] = fma2(mul2(d, d), nl2, Lj[j]);
                     }
                     const float2 m = max_pairs<K>(a);
-                    float2 sum = make_float2(0.f, 0.f), ax = sum;
+                    float2 pj = ex2f2(sub2(a[0], m));
+                    float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][h], Aj[0]));
 #pragma unroll
-                    for (int j = 0; j < K; ++j) {
-                        const float2 pj = ex2f2(sub2(a[j], m));
+                    for (int j = 1; j < K; ++j) {
+                        pj = ex2f2(sub2(a[j], m));
                         sum = add2(sum, pj);
-                        ax = fma2(pj, fma2(g2, cb[i & 1][2 * j + h], splat2(Ain[(i * K + j) * CT + tid] + gsh)), ax);
+                        ax = fma2(pj, fma2(g2, cb[i & 1][2 * j + h], Aj[j]), ax);
                     }
                     outL[h] = add2(sub2(m, off2), lg2f2(sum));
-                    outA[h] = mul2(ax, rcpf2(sum));
+                    outA[h] = fma2(ax, rcpf2(sum), gshn2);
                     tmax = max3f(tmax, m.x, m.y);
                 }
                 const uint32_t mb = full_of[i % CL] + ob_mbar;
@@ -278,7 +289,10 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
         const float lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
         const int Ofin = O;
         // ================= beta sweep carrying (M, Bt), with the gradient contraction
-        for (int q = tid; q < 2 * QC; q += CT) msg[ib * 2 * QC + q] = 0.f;      // M_n = 0, Bt_n = 0
+        {
+            const float gshn = -__ldg(g_s + n - 1) * __ldg(sf_s + n - 1);     // M_n = 0, Bt_n = 0 (+ centring shift)
+            for (int q = tid; q < QC; q += CT) { msg[ib * 2 * QC + q] = 0.f; msg[ib * 2 * QC + QC + q] = gshn; }
+        }
         // codebook -> TMEM, beta pairing: column 16 i + 8 jh + 2 b + e = c[2jh+e | x_i | b]
 #pragma unroll
         for (int i = 0; i < BPT; ++i) {
@@ -342,9 +356,10 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
             const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1);
-            const float gsh = -gt * __ldg(sf_s + t - 1);
-            const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT);
-            const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
+            const float2 gsh2 = splat2(-gt * __ldg(sf_s + t - 1));            // shift carried by the stored At
+            const float2 gshp2 = splat2(t > 1 ? -__ldg(g_s + t - 2) * __ldg(sf_s + t - 2) : 0.f);   // for step t-1
+            const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT), offM2 = splat2(offM);
+            const float2 Dm2 = splat2((float)(Ofin - O_s[t] - P) + lsefin);
             float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
             float tmax = NEG_INF;
             float2 cb[2][8];
@@ -353,7 +368,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             for (int i = 0; i < BPT; ++i, ++chunk) {
                 float2 acc[8];
                 if (tid == 0) feed_ring();
+                TICK(tc0);
                 tmem_wait_ld(cb[i & 1]);
+                TICK(tc1); TACC(5, tc0, tc1);
                 tmem_ld16(tm_acc + 16u * i, acc);
                 const uint32_t s = chunk % RD;
                 TICK(tr0);
@@ -362,43 +379,44 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
                 const float *Lh = ring + s * 2 * CH, *Ah = Lh + CH;
                 const float4 mv = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K);
                 const float4 bv = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K);
-                const float Mb[K] = {mv.x - offM, mv.y - offM, mv.z - offM, mv.w - offM};
-                const float Yb[K] = {bv.x + gsh, bv.y + gsh, bv.z + gsh, bv.w + gsh};
+                const float2 Mb[K] = {splat2(mv.x), splat2(mv.y), splat2(mv.z), splat2(mv.w)};
+                const float2 Yb[K] = {splat2(bv.x), splat2(bv.y), splat2(bv.z), splat2(bv.w)};
 #pragma unroll
                 for (int jh = 0; jh < K / 2; ++jh) {
                     float2 u[K], d[K];
 #pragma unroll
                     for (int b = 0; b < K; ++b) {
                         d[b] = sub2(w2, cb[i & 1][4 * jh + b]);
-                        u[b] = fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
+                        u[b] = fma2(mul2(d[b], d[b]), nl2, Mb[b]);
                     }
                     const float2 m = max_pairs<K>(u);
-                    const float2 Ahj = make_float2(Ah[(2 * jh) * CT + tid], Ah[(2 * jh + 1) * CT + tid]);
-                    const float2 LhD = make_float2(Lh[(2 * jh) * CT + tid] - Dm, Lh[(2 * jh + 1) * CT + tid] - Dm);
-                    const float2 f = ex2f2(add2(m, LhD));
+                    const float2 Ahj = sub2(make_float2(Ah[(2 * jh) * CT + tid], Ah[(2 * jh + 1) * CT + tid]), gsh2);
+                    const float2 Lhj = make_float2(Lh[(2 * jh) * CT + tid], Lh[(2 * jh + 1) * CT + tid]);
+                    const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
                     const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
                     float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
-                    float2 pz[K];
+                    float2 pbs[K], zz[K];
 #pragma unroll
                     for (int b = 0; b < K; ++b) {
-                        const float2 pb = ex2f2(sub2(u[b], m));
-                        const float2 y = fma2(g2, cb[i & 1][4 * jh + b], splat2(Yb[b]));      // h + Bt
-                        const float2 z = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);               // f (g + (w - c) r / T)
-                        sum = add2(sum, pb);
-                        ya = fma2(pb, y, ya);
-                        pz[b] = mul2(pb, z);
-                        zs = add2(zs, pz[b]);
+                        pbs[b] = ex2f2(sub2(u[b], m));
+                        const float2 y = fma2(g2, cb[i & 1][4 * jh + b], Yb[b]);               // h + Bt
+                        zz[b] = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);                        // f (g + (w - c) r / T)
+                        sum = add2(sum, pbs[b]);
+                        ya = fma2(pbs[b], y, ya);
+                        zs = fma2(pbs[b], zz[b], zs);
                     }
                     if (jh == 0) {
                         // accumulators (requested at the top of the butterfly) are needed only now;
                         // the next butterfly's codebook slice is requested behind them
+                        TICK(ta0);
                         tmem_wait_ld(acc);
+                        TICK(ta1); TACC(4, ta0, ta1);
                         if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
                     }
 #pragma unroll
-                    for (int b = 0; b < K; ++b) acc[4 * jh + b] = add2(acc[4 * jh + b], pz[b]);
-                    const float2 outM = add2(m, lg2f2(sum));
-                    const float2 outB = mul2(ya, rcpf2(sum));
+                    for (int b = 0; b < K; ++b) acc[4 * jh + b] = fma2(pbs[b], zz[b], acc[4 * jh + b]);
+                    const float2 outM = add2(sub2(m, offM2), lg2f2(sum));
+                    const float2 outB = fma2(ya, rcpf2(sum), gshp2);
                     tmax = max3f(tmax, m.x, m.y);
                     const uint32_t mb0 = full_of[(2 * jh) * CL / K] + ob_mbar, mb1 = full_of[(2 * jh + 1) * CL / K] + ob_mbar;
                     st_async_f32(push_b[i][2 * jh] + ob_off, outM.x, mb0);
@@ -415,7 +433,7 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             }
             tmem_wait_st();
             const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), zz = warp_sum(ZS.x + ZS.y);
-            tmax = warp_max(tmax);
+            tmax = warp_max(tmax) - offM;
             if (lane == 0) {
 #pragma unroll
                 for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
