@@ -456,6 +456,7 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
             float v = (lane < SLOTS ? lz[lane] : 0.f) + (lane + 32 < SLOTS ? lz[lane + 32] : 0.f);
             v = warp_sum(v);
             lsefin = cmax + lg2f(v);
+            if (tid == 0) diag_check_finite(p.diag, lsefin);
         }
         const int Ofin = O;
         if (tid == 0 && rank == 0 && p.logZ)
@@ -795,6 +796,7 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
             float v = (lane < CL * NWARP ? lz[lane] : 0.f) + (lane + 32 < CL * NWARP ? lz[lane + 32] : 0.f);
             v = warp_sum(v);
             lsefin = cmax + lg2f(v);
+            if (tid == 0) diag_check_finite(p.diag, lsefin);
         }
         const int Ofin = O;
         // ================= beta sweep carrying (M, Bt), with the gradient contraction

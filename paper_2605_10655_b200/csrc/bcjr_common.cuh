@@ -57,6 +57,13 @@ __device__ __forceinline__ void diag_max(unsigned int *slot, float v) {
     atomicMax(slot, __float_as_uint(v));
 }
 
+// A non-finite log Z means non-finite inputs (or a table / temperature far outside fp32 range):
+// recorded once as BCJR_ENUMERIC (-7); the outputs of that block are then meaningless.
+__device__ __forceinline__ void diag_check_finite(DeviceDiag *diag, float v)
+{
+    if (!(fabsf(v) <= 3.0e38f)) atomicCAS(&diag->status, 0, -7);
+}
+
 struct FwdParams {
     const float *W;          // [B*n]
     const float *cb;         // [S]

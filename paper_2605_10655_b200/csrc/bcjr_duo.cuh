@@ -287,6 +287,7 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             cluster_sync();                                      // log Z exchange
         }
         const float lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
+        if (tid == 0) diag_check_finite(p.diag, lsefin);
         const int Ofin = O;
         // ================= beta sweep carrying (M, Bt), with the gradient contraction
         {

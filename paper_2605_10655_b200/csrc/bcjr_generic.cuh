@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
         float tot = 0.f;
         for (int i = 0; i < nwarp; ++i) tot += lzpart[i];
         const float lsefin = cmax + lg2f(tot);
+        if (tid == 0) diag_check_finite(p.diag, lsefin);
         const int Ofin = O;
         if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
         // ---- beta sweep fused with the posterior and the expectation
@@ -248,6 +249,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams 
         float tot = 0.f;
         for (int i = 0; i < nwarp; ++i) tot += lzpart[i];
         const float lsefin = cmax + lg2f(tot);
+        if (tid == 0) diag_check_finite(p.diag, lsefin);
         const int Ofin = O;
         float *Min = msgbuf, *Mout = msgbuf + Q, *Bin = msgbuf + 2 * Q, *Bout = msgbuf + 3 * Q;
         for (int q = tid; q < Q; q += nthr) { Min[q] = 0.f; Bin[q] = 0.f; }

@@ -256,6 +256,7 @@ __global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams
                 compute_barrier(CT);
             }
             const float lsefin = cmax + lg2f(warp_sum(lane < NWARP ? lz[lane] : 0.f));
+            if (tid == 0) diag_check_finite(p.diag, lsefin);
             const int Ofin = O;
             if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
             // the last spill (L_n, buffer (n-1)&1) must have left its buffer before it is reused

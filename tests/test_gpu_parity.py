@@ -234,6 +234,26 @@ def test_large_trellis_long_blocks_fall_back_cleanly(ctx):
         assert got["diag"].device_status == 0
 
 
+def test_non_finite_input_is_reported_not_fatal(ctx):
+    # a NaN weight poisons its own block only; the call completes, the status says so, and the
+    # context keeps working
+    import torch
+    from paper_2605_10655_b200 import BcjrError
+    for Lb, n in ((8, 16), (16, 8)):
+        W, c, g = _rand(n, Lb, 3, seed=77)
+        W[1, n // 2] = np.nan
+        dev = torch.device("cuda", 0)
+        Wd, cd = torch.from_numpy(W).to(dev), torch.from_numpy(c).to(dev)
+        soft, _ = ctx.bcjr_soft_quantize(Wd, cd, Lb, 2, n, 0.5)
+        with pytest.raises(BcjrError) as ei:
+            ctx.sync_status()
+        assert ei.value.code == -7
+        soft = soft.cpu().numpy()
+        ref = oracle.soft_quantize(W[[0, 2]], c, Lb, 2, 0.5)["soft"]
+        assert parity.rel_inf(soft[[0, 2]], ref) <= parity.SOFT_TOL       # the other blocks are intact
+        assert ctx.sync_status().device_status == 0                          # cleared by the query
+
+
 def test_results_do_not_depend_on_what_ran_before(ctx):
     # scratch (history, partial sums, tensor memory) is reused between calls and between
     # blocks: the same input must give bit-identical output regardless of the previous call
