@@ -326,10 +326,21 @@ def main():
     # case of the same kernel; traffic grows in proportion to the number of blocks)
     per_block = NCU_DRAM_BYTES_PER_BLOCK.get((wl.Lb, wl.k, dom)) if diag.last_path else None
     traffic = per_block * nblocks / len(mats) if per_block else None
+    hbm_peak = None
+    try:
+        hbm_peak = json.loads((ROOT / "MEASURED_PEAKS.json").read_text()).get("hbm_gbs")
+    except (OSError, ValueError):
+        pass
+    hbm = None
+    if traffic:
+        gbs = traffic / (dom_ms * 1e-3) / 1e9
+        hbm = {"achieved_gbs": gbs, "peak_gbs": hbm_peak or 6650.0,
+               "peak_source": "MEASURED_PEAKS.json (measured copy bandwidth)" if hbm_peak else "fallback 6.65 TB/s",
+               "frac": gbs / (hbm_peak or 6650.0)}
     roofline = {"bound": "alu", "kernel": f"bcjr_{dom}", "achieved": achieved, "peak": peak, "unit": "Gop/s (MUFU)",
                 "frac": achieved / peak, "traffic": traffic,
                 "peak_source": f"{NUM_SMS} SMs x {MUFU_PER_CLK_PER_SM} MUFU/clk x {sm_max:.0f} MHz (derived)",
-                "avg_launch_ms": dom_ms,
+                "avg_launch_ms": dom_ms, "hbm": hbm,
                 "whole_step_frac": mufu_ops_per_state_step(wl.k, "both") * state_steps / (ms_per_step * 1e-3) / 1e9 / peak}
 
     if rank == 0:
