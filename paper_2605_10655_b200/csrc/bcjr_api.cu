@@ -307,19 +307,20 @@ bcjr_status launch_vit_solo(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
     return BCJR_OK;
 }
 
-// Forward call, one CTA per block with the codebook in tensor memory (Lb = 16, k = 2).
+// Forward call, one CTA per block with the codebook in tensor memory (Lb = 16; k = 2, 3).
+template <int KB>
 bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
-    using C = SoloCfg;
+    using C = SoloCfg<KB>;
     if (p.n > C::MAX_N) return BCJR_EUNSUPPORTED;
-    CU(cudaFuncSetAttribute(fwd_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    CU(cudaFuncSetAttribute(fwd_solo_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
     int64_t grid = ctx->num_sms;
     if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
     if (grid > p.B) grid = p.B;
     bcjr_status rc = ensure(ctx, ctx->hist, (size_t)grid * p.n * C::Q * 4);
     if (rc) return rc;
     p.hist = (float *)ctx->hist.ptr;
-    fwd_solo_kernel<<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    fwd_solo_kernel<KB><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
     ctx->launches += 1;
     CU(cudaGetLastError());
     return BCJR_OK;
@@ -328,7 +329,8 @@ bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
-    if (k == 2 && ctx->opt_fwd_variant != 1) return launch_fwd_solo(ctx, p, st);
+    if (k == 2 && ctx->opt_fwd_variant != 1) return launch_fwd_solo<2>(ctx, p, st);
+    if (k == 3 && ctx->opt_fwd_variant != 1) return launch_fwd_solo<3>(ctx, p, st);
     if (k == 2) return launch_fwd_cluster_t<16, 2, FWD_CL_K2, FWD_THREADS_K2>(ctx, p, st);
     if (k == 3) return launch_fwd_cluster_t<16, 3, 2, 512>(ctx, p, st);
     return BCJR_EUNSUPPORTED;

@@ -68,14 +68,21 @@ __device__ __forceinline__ void compute_barrier(int nthreads)
     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }
 
+// KB = 2: 8 butterflies of 16 states per thread; KB = 3: 2 butterflies of 64 states per thread.
+// A butterfly's K*K codebook entries are fetched in units of sixteen TMEM columns (eight packed
+// pairs): with K = 4 one unit is the whole butterfly, with K = 8 a unit is one output pair h of
+// the alpha sweep (pairs over j) or one input pair jh of the beta sweep (pairs over b).
+template <int KB_>
 struct SoloCfg {
-    static constexpr int LB = 16, KB = 2, K = 4, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
+    static constexpr int LB = 16, KB = KB_, K = 1 << KB, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
     static constexpr int CTHREADS = 512;                       // compute threads
     static constexpr int THREADS = CTHREADS + 32;              // + the copy warp
     static constexpr int NWARP = CTHREADS / 32;
-    static constexpr int BPT = NB / CTHREADS;                  // 8 butterflies per thread
+    static constexpr int BPT = NB / CTHREADS;                  // butterflies per thread
+    static constexpr int UNITS = K * K / 16;                   // 16-column units per butterfly
+    static constexpr int HPU = (K / 2) / UNITS;                // pairs h (alpha) or jh (beta) covered by one unit
     static constexpr int CH = K * CTHREADS;                    // floats per history chunk (one slot of all threads)
-    static constexpr int RD = BPT;                             // ring depth: one step of chunks
+    static constexpr int RD = KB == 2 ? BPT : 4;               // ring depth in chunks
     static constexpr int MAX_N = 2048;
     static constexpr int OFF_MSG = 0;                          // [2][Q]
     static constexpr int OFF_RING = OFF_MSG + 2 * Q;           // [RD][CH]
@@ -92,12 +99,43 @@ struct SoloCfg {
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
     static_assert(BPT * K * K == 128, "a thread's codebook slice fills its 128 TMEM columns");
+    static_assert(UNITS * HPU == K / 2 && (K == 4 || K == 8), "unit decomposition");
+    // pair index inside a unit: alpha pair (j, h), beta pair (jh, b)
+    __host__ __device__ static constexpr int a_idx(int j, int h) { return K == 4 ? 2 * j + h : j; }
+    __host__ __device__ static constexpr int b_idx(int jh, int b) { return K == 4 ? 4 * jh + b : b; }
 };
 
-__global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams p)
+// stage one butterfly's codebook entries into TMEM in the pairing of a sweep
+template <typename C>
+__device__ __forceinline__ void stage_codebook(const float *cbk, int x, uint32_t tm_butterfly, bool beta)
 {
-    using C = SoloCfg;
+    constexpr int K = C::K;
+#pragma unroll
+    for (int u = 0; u < C::UNITS; ++u) {
+        float2 v[8];
+#pragma unroll
+        for (int hh = 0; hh < C::HPU; ++hh) {
+            const int h = u * C::HPU + hh;                     // alpha: output pair (2h, 2h+1); beta: input pair (2h, 2h+1)
+#pragma unroll
+            for (int o = 0; o < K; ++o) {
+                // alpha: pair (j = o, h) = (c[o | x | 2h], c[o | x | 2h+1]);  beta: pair (jh = h, b = o) = (c[2h | x | o], c[2h+1 | x | o])
+                const float lo = beta ? __ldg(cbk + (size_t)(2 * h) * C::Q + (size_t)x * K + o)
+                                      : __ldg(cbk + (size_t)o * C::Q + (size_t)x * K + 2 * h);
+                const float hi = beta ? __ldg(cbk + (size_t)(2 * h + 1) * C::Q + (size_t)x * K + o)
+                                      : __ldg(cbk + (size_t)o * C::Q + (size_t)x * K + 2 * h + 1);
+                v[beta ? C::b_idx(hh, o) : C::a_idx(o, hh)] = make_float2(lo, hi);
+            }
+        }
+        tmem_st16(tm_butterfly + 16u * u, v);
+    }
+}
+
+template <int KB>
+__global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdParams p)
+{
+    using C = SoloCfg<KB>;
     constexpr int K = C::K, NB = C::NB, Q = C::Q, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, CH = C::CH, RD = C::RD;
+    constexpr int UNITS = C::UNITS, HPU = C::HPU, NU = BPT * UNITS;
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = p.n;
@@ -163,7 +201,7 @@ __global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams
         const uint32_t tm = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
         // destinations of the outputs (floats from the start of a message buffer)
         //   alpha: L([x|l]) -> butterfly x2 = (x*K) mod NB, input j2 = (x*K) / NB: [(i2*K + j2)*CT + tid2 .. +K)
-        //   beta : M([j|x]) -> butterfly x1 = (j*NB + x) / K, input b1 = x mod K:  [(x1*K + b1)]
+        //   beta : M([j|x]) -> butterfly x1 = (j*NB + x) / K, input b1 = x mod K:  [x1*K + b1]
         int push_a[BPT];
 #pragma unroll
         for (int i = 0; i < BPT; ++i) {
@@ -171,7 +209,6 @@ __global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams
             const int q2 = x * K, j2 = q2 / NB, x2 = q2 % NB;
             push_a[i] = ((x2 / CT) * K + j2) * CT + (x2 % CT);
         }
-        const int push_b0 = (tid / K) * K + (tid % K);         // + (j*(NB/K) + i*CT/K) * K per (i, j)
         uint32_t use_freed[2] = {0u, 0u}, chunk = 0;          // completed phases per mbarrier
         float defect = 0.f, zgap = 0.f;
 
@@ -180,18 +217,8 @@ __global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams
             for (int t = tid; t < n; t += CT) w_s[t] = __ldg(w + t);
             for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // L_1 = 0 in buffer 0
             if (tid == 0) O_s[1] = 0;
-            // codebook -> TMEM in the alpha pairing: column 16 i + 4 j + l = c[j | x_i | l]
 #pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                float2 v[8];
-#pragma unroll
-                for (int j = 0; j < K; ++j) {
-                    const float4 c4 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)j * Q + (size_t)(i * CT + tid) * K));
-                    v[2 * j] = make_float2(c4.x, c4.y);
-                    v[2 * j + 1] = make_float2(c4.z, c4.w);
-                }
-                tmem_st16(tm + 16u * i, v);
-            }
+            for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), false);
             tmem_wait_st();
             int O = 0;
             float off = 0.f, cmax = 0.f;
@@ -216,28 +243,35 @@ __global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams
                 tmem_ld16(tm, cb[0]);
 #pragma unroll
                 for (int i = 0; i < BPT; ++i) {
-                    tmem_wait_ld(cb[i & 1]);
-                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
-                    float2 Lj[K];
+                    float Lj[K];
 #pragma unroll
-                    for (int j = 0; j < K; ++j) Lj[j] = splat2(Lin[(i * K + j) * CT + tid]);
+                    for (int j = 0; j < K; ++j) Lj[j] = Lin[(i * K + j) * CT + tid];
                     float2 out[K / 2];
 #pragma unroll
-                    for (int h = 0; h < K / 2; ++h) {
-                        float2 a[K];
+                    for (int u = 0; u < UNITS; ++u) {
+                        const int g = i * UNITS + u;                             // unit counter (compile time after unrolling)
+                        tmem_wait_ld(cb[g & 1]);
+                        if (g + 1 < NU) tmem_ld16(tm + 16u * (g + 1), cb[(g + 1) & 1]);
 #pragma unroll
-                        for (int j = 0; j < K; ++j) {
-                            const float2 d = sub2(cb[i & 1][2 * j + h], w2);
-                            a[j] = fma2(mul2(d, d), nl2, Lj[j]);
+                        for (int hh = 0; hh < HPU; ++hh) {
+                            const int h = u * HPU + hh;
+                            float2 a[K];
+#pragma unroll
+                            for (int j = 0; j < K; ++j) {
+                                const float2 d = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
+                                a[j] = fma2(mul2(d, d), nl2, splat2(Lj[j]));
+                            }
+                            const float2 m = max_pairs<K>(a);
+                            float2 sum = ex2f2(sub2(a[0], m));
+#pragma unroll
+                            for (int j = 1; j < K; ++j) sum = add2(sum, ex2f2(sub2(a[j], m)));
+                            out[h] = add2(sub2(m, off2), lg2f2(sum));
+                            tmax = max3f(tmax, m.x, m.y);
                         }
-                        const float2 m = max_pairs<K>(a);
-                        float2 sum = ex2f2(sub2(a[0], m));
-#pragma unroll
-                        for (int j = 1; j < K; ++j) sum = add2(sum, ex2f2(sub2(a[j], m)));
-                        out[h] = add2(sub2(m, off2), lg2f2(sum));
-                        tmax = max3f(tmax, m.x, m.y);
                     }
-                    *reinterpret_cast<float4 *>(Lout + push_a[i]) = make_float4(out[0].x, out[0].y, out[1].x, out[1].y);
+#pragma unroll
+                    for (int h = 0; h < K / 2; h += 2)
+                        *reinterpret_cast<float4 *>(Lout + push_a[i] + 2 * h) = make_float4(out[h].x, out[h].y, out[h + 1].x, out[h + 1].y);
                 }
                 tmax = warp_max(tmax);
                 if (lane == 0) wmax[(cur ^ 1) * 32 + warp] = tmax;
@@ -264,19 +298,8 @@ __global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams
             ++use_freed[(n - 1) & 1];
             // ================= beta sweep
             for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // M_n = 0 in buffer 0
-            // codebook -> TMEM in the beta pairing: column 16 i + 8 jh + 2 b + e = c[2jh+e | x_i | b]
 #pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                float2 v[8];
-#pragma unroll
-                for (int jh = 0; jh < K / 2; ++jh) {
-                    const float4 c0 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh) * Q + (size_t)(i * CT + tid) * K));
-                    const float4 c1 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh + 1) * Q + (size_t)(i * CT + tid) * K));
-                    v[4 * jh] = make_float2(c0.x, c1.x); v[4 * jh + 1] = make_float2(c0.y, c1.y);
-                    v[4 * jh + 2] = make_float2(c0.z, c1.z); v[4 * jh + 3] = make_float2(c0.w, c1.w);
-                }
-                tmem_st16(tm + 16u * i, v);
-            }
+            for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), true);
             tmem_wait_st();
             int P = 0;
             float offM = 0.f;
@@ -302,55 +325,62 @@ __global__ void __launch_bounds__(SoloCfg::THREADS, 1) fwd_solo_kernel(FwdParams
                     }
                 }
                 const float2 w2 = splat2(w_s[t - 1]);
-                const float Dm = ((float)(Ofin - O_s[t] - P) + lsefin) - offM;
+                const float2 offM2 = splat2(offM);
+                const float2 Dm2 = splat2((float)(Ofin - O_s[t] - P) + lsefin);
                 float2 num2 = make_float2(0.f, 0.f), den2 = make_float2(0.f, 0.f);
                 float tmax = NEG_INF;
                 float2 cb[2][8];
                 tmem_ld16(tm, cb[0]);
 #pragma unroll
                 for (int i = 0; i < BPT; ++i, ++chunk) {
-                    tmem_wait_ld(cb[i & 1]);
-                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
                     const uint32_t s = chunk % RD;
                     mbar_wait_bounded(mbar_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
                     const float *Lh = ring + s * CH;
-                    float2 Mb[K];
-                    {
-                        const float4 v = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K);
-                        Mb[0] = splat2(v.x - offM); Mb[1] = splat2(v.y - offM);
-                        Mb[2] = splat2(v.z - offM); Mb[3] = splat2(v.w - offM);
+                    float Mb[K];
+#pragma unroll
+                    for (int b = 0; b < K; b += 4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K + b);
+                        Mb[b] = v.x; Mb[b + 1] = v.y; Mb[b + 2] = v.z; Mb[b + 3] = v.w;
                     }
 #pragma unroll
-                    for (int jh = 0; jh < K / 2; ++jh) {
-                        float2 u[K];
+                    for (int u = 0; u < UNITS; ++u) {
+                        const int g = i * UNITS + u;
+                        tmem_wait_ld(cb[g & 1]);
+                        if (g + 1 < NU) tmem_ld16(tm + 16u * (g + 1), cb[(g + 1) & 1]);
 #pragma unroll
-                        for (int b = 0; b < K; ++b) {
-                            const float2 d = sub2(cb[i & 1][4 * jh + b], w2);
-                            u[b] = fma2(mul2(d, d), nl2, Mb[b]);
-                        }
-                        const float2 m = max_pairs<K>(u);
-                        const float2 LhD = make_float2(Lh[(2 * jh) * CT + tid] - Dm, Lh[(2 * jh + 1) * CT + tid] - Dm);
-                        const float2 f = ex2f2(add2(m, LhD));
-                        float2 pb = ex2f2(sub2(u[0], m));
-                        float2 sum = pb, craw = mul2(pb, cb[i & 1][4 * jh]);
+                        for (int hh = 0; hh < HPU; ++hh) {
+                            const int jh = u * HPU + hh;
+                            float2 uu[K];
 #pragma unroll
-                        for (int b = 1; b < K; ++b) {
-                            pb = ex2f2(sub2(u[b], m));
-                            sum = add2(sum, pb);
-                            craw = fma2(pb, cb[i & 1][4 * jh + b], craw);
+                            for (int b = 0; b < K; ++b) {
+                                const float2 d = sub2(cb[g & 1][C::b_idx(hh, b)], w2);
+                                uu[b] = fma2(mul2(d, d), nl2, splat2(Mb[b]));
+                            }
+                            const float2 m = max_pairs<K>(uu);
+                            const float2 Lhj = make_float2(Lh[(2 * jh) * CT + tid], Lh[(2 * jh + 1) * CT + tid]);
+                            const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
+                            float2 pb = ex2f2(sub2(uu[0], m));
+                            float2 sum = pb, craw = mul2(pb, cb[g & 1][C::b_idx(hh, 0)]);
+#pragma unroll
+                            for (int b = 1; b < K; ++b) {
+                                pb = ex2f2(sub2(uu[b], m));
+                                sum = add2(sum, pb);
+                                craw = fma2(pb, cb[g & 1][C::b_idx(hh, b)], craw);
+                            }
+                            const float2 out = add2(sub2(m, offM2), lg2f2(sum));
+                            tmax = max3f(tmax, m.x, m.y);
+                            // M([j|x]) with x = i*CT + tid goes to [x1*K + b1], x1 = j*(NB/K) + x/K, b1 = x%K
+                            Mout[((2 * jh) * (NB / K) + (i * CT + tid) / K) * K + (tid % K)] = out.x;
+                            Mout[((2 * jh + 1) * (NB / K) + (i * CT + tid) / K) * K + (tid % K)] = out.y;
+                            num2 = fma2(f, craw, num2);
+                            den2 = fma2(f, sum, den2);
                         }
-                        const float2 out = add2(m, lg2f2(sum));
-                        tmax = max3f(tmax, m.x, m.y);
-                        Mout[push_b0 + ((2 * jh) * (NB / K) + i * (CT / K)) * K] = out.x;
-                        Mout[push_b0 + ((2 * jh + 1) * (NB / K) + i * (CT / K)) * K] = out.y;
-                        num2 = fma2(f, craw, num2);
-                        den2 = fma2(f, sum, den2);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(mbar_empty + 8u * s);             // this warp is done with the chunk
                 }
                 const float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
-                tmax = warp_max(tmax);
+                tmax = warp_max(tmax) - offM;
                 if (lane == 0) {
                     wmax[(cur ^ 1) * 32 + warp] = tmax;
                     part[((cur ^ 1) * 32 + warp) * 2] = num;
