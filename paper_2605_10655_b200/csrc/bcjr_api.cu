@@ -256,20 +256,21 @@ bcjr_status launch_bwd_cluster_t(bcjr_ctx *ctx, BwdParams p, float *grad_codeboo
     return BCJR_OK;
 }
 
-// Backward call, clusters of two with codebook and accumulators in tensor memory (Lb = 16, k = 2).
+// Backward call, clusters of two with codebook and accumulators in tensor memory (Lb = 16; k = 2, 3).
+template <int KB>
 bcjr_status launch_bwd_duo(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
 {
-    using C = DuoCfg;
+    using C = DuoCfg<KB>;
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1];
-    bcjr_status rc = plan_cluster(ctx, bwd_duo_kernel, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    bcjr_status rc = plan_cluster(ctx, bwd_duo_kernel<KB>, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
     if (rc) return rc;
     const int ncl = cfg.gridDim.x / C::CL;
     if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * p.n * 2 * C::Q * 4))) return rc;
     if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * C::S * 4))) return rc;
     p.hist = (float *)ctx->hist.ptr;
     p.gc_part = (float *)ctx->gc_part.ptr;
-    CU(cudaLaunchKernelEx(&cfg, bwd_duo_kernel, p));
+    CU(cudaLaunchKernelEx(&cfg, bwd_duo_kernel<KB>, p));
     ctx->launches += 1;
     if (grad_codebook) {
         reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, C::S, grad_codebook);
@@ -282,7 +283,8 @@ bcjr_status launch_bwd_duo(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cud
 bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_codebook, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
-    if (k == 2 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg::MAX_N) return launch_bwd_duo(ctx, p, grad_codebook, st);
+    if (k == 2 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<2>::MAX_N) return launch_bwd_duo<2>(ctx, p, grad_codebook, st);
+    if (k == 3 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<3>::MAX_N) return launch_bwd_duo<3>(ctx, p, grad_codebook, st);
     if (k == 2) return launch_bwd_cluster_t<16, 2, 4, 512>(ctx, p, grad_codebook, st);
     if (k == 3) return launch_bwd_cluster_t<16, 3, 4, 256>(ctx, p, grad_codebook, st);
     return BCJR_EUNSUPPORTED;

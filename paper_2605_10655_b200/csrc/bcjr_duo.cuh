@@ -43,15 +43,18 @@ __device__ unsigned long long g_duo_timing[8];   // beta sweep, warp 1 of CTA 0:
 #define TACC(slot, a, b)
 #endif
 
+template <int KB_>
 struct DuoCfg {
-    static constexpr int LB = 16, KB = 2, K = 4, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
+    static constexpr int LB = 16, KB = KB_, K = 1 << KB, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
     static constexpr int CL = 2;
     static constexpr int NBC = NB / CL, QC = Q / CL;
     static constexpr int THREADS = 512, NWARP = THREADS / 32;
-    static constexpr int BPT = NBC / THREADS;                  // 4 butterflies per thread
+    static constexpr int BPT = NBC / THREADS;                  // butterflies per thread: 4 (k = 2), 1 (k = 3)
+    static constexpr int UNITS = K * K / 16;                   // 16-column TMEM units per butterfly
+    static constexpr int HPU = (K / 2) / UNITS;                // pairs h (alpha) / jh (beta) per unit
     static constexpr int SLOTS = CL * NWARP;                   // 32 per-warp partial slots
     static constexpr int CH = K * THREADS;                     // floats per array per history chunk
-    static constexpr int RD = BPT + 1;                         // ring depth: a step and a quarter of chunks
+    static constexpr int RD = KB == 2 ? BPT + 1 : 3;           // ring depth in chunks
     static constexpr int MAX_N = 1024;
     static constexpr int ARRIVALS = 1 + SLOTS;                 // armer + one arrival per warp of the cluster
     static constexpr int OFF_MSG = 0;                          // [2 parity][2 arrays][QC]
@@ -69,13 +72,18 @@ struct DuoCfg {
     static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
     static_assert(2 * BPT * K * K == 128, "codebook + accumulators fill the thread's 128 TMEM columns");
     static_assert(K % CL == 0, "beta destinations: CTA of output j is j*CL/K");
+    static_assert(UNITS * HPU == K / 2 && (K == 4 || K == 8), "unit decomposition");
+    __host__ __device__ static constexpr int a_idx(int j, int h) { return K == 4 ? 2 * j + h : j; }
+    __host__ __device__ static constexpr int b_idx(int jh, int b) { return K == 4 ? 4 * jh + b : b; }
 };
 
-__global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p)
+template <int KB>
+__global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdParams p)
 {
-    using C = DuoCfg;
+    using C = DuoCfg<KB>;
     constexpr int K = C::K, NB = C::NB, NBC = C::NBC, QC = C::QC, BPT = C::BPT, NWARP = C::NWARP, CT = C::THREADS;
-    constexpr int CL = C::CL, SLOTS = C::SLOTS, CH = C::CH, RD = C::RD;
+    constexpr int CL = C::CL, SLOTS = C::SLOTS, CH = C::CH, RD = C::RD, UNITS = C::UNITS, HPU = C::HPU, NU = BPT * UNITS;
+    constexpr int KK = K * K;
     constexpr uint32_t BUF_BYTES = 2u * QC * 4u;                 // (L, At) of one parity
     constexpr uint32_t TX_MSG = BUF_BYTES + SLOTS * 4u;          // messages + gauge slots
     constexpr uint32_t TX_PART = SLOTS * 16u;                    // posterior sums (rank 0 only)
@@ -126,16 +134,16 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
 
     const uint32_t tm_cb = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
     const uint32_t tm_acc = tm_cb + 64u;
-    uint32_t push_a[BPT], push_b[BPT][K];
+    uint32_t push_a[BPT], push_a_mbar[BPT], push_b[BPT][K];
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
         const int x = (int)rank * NBC + i * CT + tid;
         {
-            // L([x|l]) -> butterfly x2 = (x*K) mod NB, input j2 = (x*K) / NB, at [(i2*K + j2)*CT + tid2 .. +K);
-            // with 512 threads and clusters of two the destination CTA is i & 1
+            // L([x|l]) -> butterfly x2 = (x*K) mod NB, input j2 = (x*K) / NB, at [(i2*K + j2)*CT + tid2 .. +K)
             const int q2 = x * K, j2 = q2 / NB, x2 = q2 % NB;
             const int r2 = x2 / NBC, xl2 = x2 % NBC;
             push_a[i] = mapa_u32(msg_u32 + (uint32_t)(((xl2 / CT) * K + j2) * CT + xl2 % CT) * 4u, (uint32_t)r2);
+            push_a_mbar[i] = full_of[r2];
         }
 #pragma unroll
         for (int j = 0; j < K; ++j) {
@@ -145,7 +153,6 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(xl1 * K + b1) * 4u, (uint32_t)r1);
         }
     }
-    static_assert(NBC / K == CT, "alpha destination CTA of butterfly slot i is i mod CL");
     uint32_t wmax_dst[CL], lz_dst[CL];
 #pragma unroll
     for (int r = 0; r < CL; ++r) {
@@ -153,13 +160,13 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
         lz_dst[r] = mapa_u32(lz_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
     }
     const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 16u, 0u);
-    // zero the accumulators (beta pairing: column 64 + 16 i + 8 jh + 2 b + e <-> state [2jh+e | x_i | b])
+    // zero the accumulators (laid out like the beta-paired codebook, 64 columns further)
     {
         float2 z[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) z[e] = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int i = 0; i < BPT; ++i) tmem_st16(tm_acc + 16u * i, z);
+        for (int g = 0; g < NU; ++g) tmem_st16(tm_acc + 16u * g, z);
         tmem_wait_st();
     }
 #ifdef BCJR_TIMING
@@ -179,19 +186,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             for (int q = tid; q < QC; q += CT) { msg[q] = 0.f; msg[QC + q] = gsh1; }
         }
         if (tid == 0) O_s[1] = 0;
-        // codebook -> TMEM, alpha pairing: column 16 i + 4 j + l = c[j | x_i | l]
 #pragma unroll
-        for (int i = 0; i < BPT; ++i) {
-            float2 v[8];
-            const int x = (int)rank * NBC + i * CT + tid;
-#pragma unroll
-            for (int j = 0; j < K; ++j) {
-                const float4 c4 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)j * C::Q + (size_t)x * K));
-                v[2 * j] = make_float2(c4.x, c4.y);
-                v[2 * j + 1] = make_float2(c4.z, c4.w);
-            }
-            tmem_st16(tm_cb + 16u * i, v);
-        }
+        for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, alpha pairing
+            stage_codebook<C>(p.cb, (int)rank * NBC + i * CT + tid, tm_cb + (uint32_t)(KK * i), false);
         tmem_wait_st();
         int O = 0;
         float off = 0.f, cmax = 0.f;
@@ -221,38 +218,47 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             tmem_ld16(tm_cb, cb[0]);
 #pragma unroll
             for (int i = 0; i < BPT; ++i) {
-                tmem_wait_ld(cb[i & 1]);
-                if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
-                float2 outL[K / 2], outA[K / 2], Lj[K], Aj[K];
+                float2 outL[K / 2], outA[K / 2];
+                float Lj[K], Aj[K];
 #pragma unroll
                 for (int j = 0; j < K; ++j) {
-                    Lj[j] = splat2(Lin[(i * K + j) * CT + tid]);
-                    Aj[j] = splat2(Ain[(i * K + j) * CT + tid]);
+                    Lj[j] = Lin[(i * K + j) * CT + tid];
+                    Aj[j] = Ain[(i * K + j) * CT + tid];
                 }
 #pragma unroll
-                for (int h = 0; h < K / 2; ++h) {
-                    float2 a[K];
+                for (int u = 0; u < UNITS; ++u) {
+                    const int g = i * UNITS + u;
+                    tmem_wait_ld(cb[g & 1]);
+                    if (g + 1 < NU) tmem_ld16(tm_cb + 16u * (g + 1), cb[(g + 1) & 1]);
 #pragma unroll
-                    for (int j = 0; j < K; ++j) {
-                        const float2 d = sub2(cb[i & 1][2 * j + h], w2);
-                        a[j] = fma2(mul2(d, d), nl2, Lj[j]);
-                    }
-                    const float2 m = max_pairs<K>(a);
-                    float2 pj = ex2f2(sub2(a[0], m));
-                    float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][h], Aj[0]));
+                    for (int hh = 0; hh < HPU; ++hh) {
+                        const int h = u * HPU + hh;
+                        float2 a[K];
 #pragma unroll
-                    for (int j = 1; j < K; ++j) {
-                        pj = ex2f2(sub2(a[j], m));
-                        sum = add2(sum, pj);
-                        ax = fma2(pj, fma2(g2, cb[i & 1][2 * j + h], Aj[j]), ax);
+                        for (int j = 0; j < K; ++j) {
+                            const float2 d = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
+                            a[j] = fma2(mul2(d, d), nl2, splat2(Lj[j]));
+                        }
+                        const float2 m = max_pairs<K>(a);
+                        float2 pj = ex2f2(sub2(a[0], m));
+                        float2 sum = pj, ax = mul2(pj, fma2(g2, cb[g & 1][C::a_idx(0, hh)], splat2(Aj[0])));
+#pragma unroll
+                        for (int j = 1; j < K; ++j) {
+                            pj = ex2f2(sub2(a[j], m));
+                            sum = add2(sum, pj);
+                            ax = fma2(pj, fma2(g2, cb[g & 1][C::a_idx(j, hh)], splat2(Aj[j])), ax);
+                        }
+                        outL[h] = add2(sub2(m, off2), lg2f2(sum));
+                        outA[h] = fma2(ax, rcpf2(sum), gshn2);
+                        tmax = max3f(tmax, m.x, m.y);
                     }
-                    outL[h] = add2(sub2(m, off2), lg2f2(sum));
-                    outA[h] = fma2(ax, rcpf2(sum), gshn2);
-                    tmax = max3f(tmax, m.x, m.y);
                 }
-                const uint32_t mb = full_of[i % CL] + ob_mbar;
-                st_async_v4(push_a[i] + ob_off, outL[0].x, outL[0].y, outL[1].x, outL[1].y, mb);
-                st_async_v4(push_a[i] + ob_off + QC * 4u, outA[0].x, outA[0].y, outA[1].x, outA[1].y, mb);
+                const uint32_t mb = push_a_mbar[i] + ob_mbar;
+#pragma unroll
+                for (int h = 0; h < K / 2; h += 2) {
+                    st_async_v4(push_a[i] + ob_off + 8u * h, outL[h].x, outL[h].y, outL[h + 1].x, outL[h + 1].y, mb);
+                    st_async_v4(push_a[i] + ob_off + QC * 4u + 8u * h, outA[h].x, outA[h].y, outA[h + 1].x, outA[h + 1].y, mb);
+                }
             }
             tmax = warp_max(tmax);
             if (lane == 0) {
@@ -294,20 +300,9 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             const float gshn = -__ldg(g_s + n - 1) * __ldg(sf_s + n - 1);     // M_n = 0, Bt_n = 0 (+ centring shift)
             for (int q = tid; q < QC; q += CT) { msg[ib * 2 * QC + q] = 0.f; msg[ib * 2 * QC + QC + q] = gshn; }
         }
-        // codebook -> TMEM, beta pairing: column 16 i + 8 jh + 2 b + e = c[2jh+e | x_i | b]
 #pragma unroll
-        for (int i = 0; i < BPT; ++i) {
-            float2 v[8];
-            const int x = (int)rank * NBC + i * CT + tid;
-#pragma unroll
-            for (int jh = 0; jh < K / 2; ++jh) {
-                const float4 c0 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh) * C::Q + (size_t)x * K));
-                const float4 c1 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)(2 * jh + 1) * C::Q + (size_t)x * K));
-                v[4 * jh] = make_float2(c0.x, c1.x); v[4 * jh + 1] = make_float2(c0.y, c1.y);
-                v[4 * jh + 2] = make_float2(c0.z, c1.z); v[4 * jh + 3] = make_float2(c0.w, c1.w);
-            }
-            tmem_st16(tm_cb + 16u * i, v);
-        }
+        for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, beta pairing
+            stage_codebook<C>(p.cb, (int)rank * NBC + i * CT + tid, tm_cb + (uint32_t)(KK * i), true);
         tmem_wait_st();
         int P = 0;
         float offM = 0.f;
@@ -367,68 +362,68 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
             tmem_ld16(tm_cb, cb[0]);
 #pragma unroll
             for (int i = 0; i < BPT; ++i, ++chunk) {
-                float2 acc[8];
                 if (tid == 0) feed_ring();
-                TICK(tc0);
-                tmem_wait_ld(cb[i & 1]);
-                TICK(tc1); TACC(5, tc0, tc1);
-                tmem_ld16(tm_acc + 16u * i, acc);
                 const uint32_t s = chunk % RD;
                 TICK(tr0);
                 mbar_wait_bounded(ring_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
                 TICK(tr1); TACC(3, tr0, tr1);
                 const float *Lh = ring + s * 2 * CH, *Ah = Lh + CH;
-                const float4 mv = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K);
-                const float4 bv = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K);
-                const float2 Mb[K] = {splat2(mv.x), splat2(mv.y), splat2(mv.z), splat2(mv.w)};
-                const float2 Yb[K] = {splat2(bv.x), splat2(bv.y), splat2(bv.z), splat2(bv.w)};
+                float Mb[K], Yb[K];
 #pragma unroll
-                for (int jh = 0; jh < K / 2; ++jh) {
-                    float2 u[K], d[K];
-#pragma unroll
-                    for (int b = 0; b < K; ++b) {
-                        d[b] = sub2(w2, cb[i & 1][4 * jh + b]);
-                        u[b] = fma2(mul2(d[b], d[b]), nl2, Mb[b]);
-                    }
-                    const float2 m = max_pairs<K>(u);
-                    const float2 Ahj = sub2(make_float2(Ah[(2 * jh) * CT + tid], Ah[(2 * jh + 1) * CT + tid]), gsh2);
-                    const float2 Lhj = make_float2(Lh[(2 * jh) * CT + tid], Lh[(2 * jh + 1) * CT + tid]);
-                    const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
-                    const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
-                    float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
-                    float2 pbs[K], zz[K];
-#pragma unroll
-                    for (int b = 0; b < K; ++b) {
-                        pbs[b] = ex2f2(sub2(u[b], m));
-                        const float2 y = fma2(g2, cb[i & 1][4 * jh + b], Yb[b]);               // h + Bt
-                        zz[b] = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);                        // f (g + (w - c) r / T)
-                        sum = add2(sum, pbs[b]);
-                        ya = fma2(pbs[b], y, ya);
-                        zs = fma2(pbs[b], zz[b], zs);
-                    }
-                    if (jh == 0) {
-                        // accumulators (requested at the top of the butterfly) are needed only now;
-                        // the next butterfly's codebook slice is requested behind them
-                        TICK(ta0);
-                        tmem_wait_ld(acc);
-                        TICK(ta1); TACC(4, ta0, ta1);
-                        if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
-                    }
-#pragma unroll
-                    for (int b = 0; b < K; ++b) acc[4 * jh + b] = fma2(pbs[b], zz[b], acc[4 * jh + b]);
-                    const float2 outM = add2(sub2(m, offM2), lg2f2(sum));
-                    const float2 outB = fma2(ya, rcpf2(sum), gshp2);
-                    tmax = max3f(tmax, m.x, m.y);
-                    const uint32_t mb0 = full_of[(2 * jh) * CL / K] + ob_mbar, mb1 = full_of[(2 * jh + 1) * CL / K] + ob_mbar;
-                    st_async_f32(push_b[i][2 * jh] + ob_off, outM.x, mb0);
-                    st_async_f32(push_b[i][2 * jh + 1] + ob_off, outM.y, mb1);
-                    st_async_f32(push_b[i][2 * jh] + ob_off + QC * 4u, outB.x, mb0);
-                    st_async_f32(push_b[i][2 * jh + 1] + ob_off + QC * 4u, outB.y, mb1);
-                    S0 = fma2(f, sum, S0);
-                    S2 = fma2(f, fma2(Ahj, sum, ya), S2);
-                    ZS = add2(ZS, zs);
+                for (int b = 0; b < K; b += 4) {
+                    const float4 mv = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K + b);
+                    const float4 bv = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K + b);
+                    Mb[b] = mv.x; Mb[b + 1] = mv.y; Mb[b + 2] = mv.z; Mb[b + 3] = mv.w;
+                    Yb[b] = bv.x; Yb[b + 1] = bv.y; Yb[b + 2] = bv.z; Yb[b + 3] = bv.w;
                 }
-                tmem_st16(tm_acc + 16u * i, acc);
+#pragma unroll
+                for (int u = 0; u < UNITS; ++u) {
+                    const int g = i * UNITS + u;
+                    float2 acc[8];
+                    tmem_wait_ld(cb[g & 1]);
+                    tmem_ld16(tm_acc + 16u * g, acc);
+                    if (g + 1 < NU) tmem_ld16(tm_cb + 16u * (g + 1), cb[(g + 1) & 1]);
+                    bool acc_ready = false;
+#pragma unroll
+                    for (int hh = 0; hh < HPU; ++hh) {
+                        const int jh = u * HPU + hh;
+                        float2 uu[K], d[K];
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+                            d[b] = sub2(w2, cb[g & 1][C::b_idx(hh, b)]);
+                            uu[b] = fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
+                        }
+                        const float2 m = max_pairs<K>(uu);
+                        const float2 Ahj = sub2(make_float2(Ah[(2 * jh) * CT + tid], Ah[(2 * jh + 1) * CT + tid]), gsh2);
+                        const float2 Lhj = make_float2(Lh[(2 * jh) * CT + tid], Lh[(2 * jh + 1) * CT + tid]);
+                        const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
+                        const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
+                        if (!acc_ready) { tmem_wait_ld(acc); acc_ready = true; }
+                        float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
+#pragma unroll
+                        for (int b = 0; b < K; ++b) {
+                            const float2 pb = ex2f2(sub2(uu[b], m));
+                            const float2 y = fma2(g2, cb[g & 1][C::b_idx(hh, b)], splat2(Yb[b]));   // h + Bt
+                            const float2 z = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);                  // f (g + (w - c) r / T)
+                            sum = add2(sum, pb);
+                            ya = fma2(pb, y, ya);
+                            zs = fma2(pb, z, zs);
+                            acc[C::b_idx(hh, b)] = fma2(pb, z, acc[C::b_idx(hh, b)]);
+                        }
+                        const float2 outM = add2(sub2(m, offM2), lg2f2(sum));
+                        const float2 outB = fma2(ya, rcpf2(sum), gshp2);
+                        tmax = max3f(tmax, m.x, m.y);
+                        const uint32_t mb0 = full_of[(2 * jh) * CL / K] + ob_mbar, mb1 = full_of[(2 * jh + 1) * CL / K] + ob_mbar;
+                        st_async_f32(push_b[i][2 * jh] + ob_off, outM.x, mb0);
+                        st_async_f32(push_b[i][2 * jh + 1] + ob_off, outM.y, mb1);
+                        st_async_f32(push_b[i][2 * jh] + ob_off + QC * 4u, outB.x, mb0);
+                        st_async_f32(push_b[i][2 * jh + 1] + ob_off + QC * 4u, outB.y, mb1);
+                        S0 = fma2(f, sum, S0);
+                        S2 = fma2(f, fma2(Ahj, sum, ya), S2);
+                        ZS = add2(ZS, zs);
+                    }
+                    tmem_st16(tm_acc + 16u * g, acc);
+                }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(ring_empty + 8u * s);               // history chunk consumed by this warp
             }
@@ -453,21 +448,26 @@ __global__ void __launch_bounds__(DuoCfg::THREADS, 1) bwd_duo_kernel(BwdParams p
         finish_step(1, ib);
         cluster_sync();                                          // block end
     }
-    // this cluster's partial of grad_codebook: state [j|x|b] = j*Q + x*K + b
+    // this cluster's partial of grad_codebook: beta pair (jh, b) of butterfly x holds states [2jh | x | b], [2jh+1 | x | b]
     float *gc = p.gc_part + (size_t)cid * C::S;
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
-        float2 acc[8];
-        tmem_ld16(tm_acc + 16u * i, acc);
-        tmem_wait_ld(acc);
         const int x = (int)rank * NBC + i * CT + tid;
 #pragma unroll
-        for (int jh = 0; jh < K / 2; ++jh)
+        for (int u = 0; u < UNITS; ++u) {
+            float2 acc[8];
+            tmem_ld16(tm_acc + 16u * (i * UNITS + u), acc);
+            tmem_wait_ld(acc);
 #pragma unroll
-            for (int b = 0; b < K; ++b) {
-                gc[(size_t)(2 * jh) * C::Q + (size_t)x * K + b] = acc[4 * jh + b].x;
-                gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[4 * jh + b].y;
+            for (int hh = 0; hh < HPU; ++hh) {
+                const int jh = u * HPU + hh;
+#pragma unroll
+                for (int b = 0; b < K; ++b) {
+                    gc[(size_t)(2 * jh) * C::Q + (size_t)x * K + b] = acc[C::b_idx(hh, b)].x;
+                    gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[C::b_idx(hh, b)].y;
+                }
             }
+        }
     }
 #ifdef BCJR_TIMING
     if (blockIdx.x == 0 && warp == 1 && lane == 0)

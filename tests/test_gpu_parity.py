@@ -292,12 +292,25 @@ def test_q_proj_full_size_sampled_outputs_and_invariants(ctx):
     assert got["soft"].min() >= c.min() - 1e-4 and got["soft"].max() <= c.max() + 1e-4
 
 
-@pytest.mark.parametrize("T", [0.01, 0.001])
-def test_three_bit_student_t_low_temperature(ctx, T):
+@pytest.mark.parametrize("T,variant", [(0.01, "tmem"), (0.001, "tmem"), (0.01, "cluster_registers")])
+def test_three_bit_student_t_low_temperature(ctx, T, variant):
     wl = synth.gate_k3()
     idx = synth.sample_blocks(wl.num_blocks(), 4)
     W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
-    got = _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"k=3 student-t T={T}", viterbi=(T == 0.01))
+    v = int(variant != "tmem")
+    try:
+        ctx.set_option("fwd_variant", v); ctx.set_option("bwd_variant", v)
+        got = _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"k=3 student-t T={T} [{variant}]", viterbi=(T == 0.01 and v == 0))
+    finally:
+        ctx.set_option("fwd_variant", 0); ctx.set_option("bwd_variant", 0)
+    assert got["diag"].last_path == 1
     assert np.all(np.isfinite(got["soft"])) and np.all(np.isfinite(got["grad_W"]))
     tot = got["grad_W"].astype(np.float64).sum() + got["grad_codebook"].astype(np.float64).sum()
     assert abs(tot - g.astype(np.float64).sum()) < 1e-2 * np.abs(g).sum()
+
+
+@pytest.mark.parametrize("n,B", [(1, 2), (5, 3), (33, 1)])
+def test_three_bit_ragged_lengths(ctx, n, B):
+    Lb, k, T = 16, 3, 0.2
+    W, c, g = _rand(n, Lb, B, seed=4300 + n)
+    _check_all(ctx, W, c, g, Lb, k, T, f"Lb=16 k=3 n={n} B={B}", viterbi=(n == 5))
