@@ -66,7 +66,13 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *                 memory (Lb = 16, k = 2), 1 = two-CTA cluster kernel with the codebook in registers
  *   "bwd_variant" large-trellis backward kernel: 0 = two-CTA clusters with codebook and gradient
  *                 accumulators in tensor memory (Lb = 16, k = 2), 1 = four-CTA clusters, registers
- *   "max_ctas"    cap on resident thread blocks (0 = fill the GPU) */
+ *   "max_ctas"    cap on resident thread blocks (0 = fill the GPU)
+ *   "wait_limit_ms"  wall-time budget of one device-side wait (default 2000).  A wait that outlasts it
+ *                 gives up: the kernel still runs to its end, the outputs of the call are
+ *                 meaningless and bcjr_sync_status returns BCJR_ETIMEOUT; the context stays usable.
+ *   "debug_drop_history_load"  test hook for that path: while non-zero, thread block 0 never requests
+ *                 the first history chunk of a large-trellis call, so one of its waits must run out.
+ * The last two synchronise the device before they take effect. */
 bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value);
 
 /*

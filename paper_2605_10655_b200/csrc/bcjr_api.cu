@@ -21,6 +21,8 @@ using namespace bcjr;
 
 namespace {
 
+const unsigned long long kDefaultWaitLimitNs = 2000000000ull;   // 2 s per device-side wait
+
 struct Buffer {
     void *ptr = nullptr;
     size_t bytes = 0;
@@ -374,7 +376,8 @@ bcjr_status bcjr_create(bcjr_ctx **out, int device_ordinal)
     cudaDeviceProp prop;
     if (!guard.ok || cudaGetDeviceProperties(&prop, device_ordinal) != cudaSuccess ||
         cudaMalloc((void **)&ctx->diag, sizeof(DeviceDiag)) != cudaSuccess ||
-        cudaMemset(ctx->diag, 0, sizeof(DeviceDiag)) != cudaSuccess) {
+        cudaMemset(ctx->diag, 0, sizeof(DeviceDiag)) != cudaSuccess ||
+        cudaMemcpy(&ctx->diag->wait_limit_ns, &kDefaultWaitLimitNs, sizeof(kDefaultWaitLimitNs), cudaMemcpyHostToDevice) != cudaSuccess) {
         cudaGetLastError();
         delete ctx;
         return BCJR_ECUDA;
@@ -417,6 +420,20 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
     if (!strcmp(name, "fwd_variant")) {
         if (value < 0 || value > 1) return BCJR_EINVAL;
         ctx->opt_fwd_variant = (int)value;
+        return BCJR_OK;
+    }
+    if (!strcmp(name, "wait_limit_ms") || !strcmp(name, "debug_drop_history_load")) {
+        // device-side configuration: written behind everything already queued on the device
+        DeviceGuard guard(ctx->device);
+        if (!guard.ok || value < 0 || value > 600000) return BCJR_EINVAL;
+        CU(cudaDeviceSynchronize());
+        if (name[0] == 'w') {
+            const unsigned long long ns = (unsigned long long)(value > 0 ? value : 1) * 1000000ull;
+            CU(cudaMemcpy(&ctx->diag->wait_limit_ns, &ns, sizeof(ns), cudaMemcpyHostToDevice));
+        } else {
+            const int flag = value != 0;
+            CU(cudaMemcpy(&ctx->diag->drop_history_load, &flag, sizeof(flag), cudaMemcpyHostToDevice));
+        }
         return BCJR_OK;
     }
     if (!strcmp(name, "max_ctas")) {
@@ -597,8 +614,8 @@ bcjr_status bcjr_sync_status(bcjr_ctx *ctx, void *cuda_stream, bcjr_diag *out)
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CU(cudaStreamSynchronize(st));
     DeviceDiag h;
-    CU(cudaMemcpy(&h, ctx->diag, sizeof(h), cudaMemcpyDeviceToHost));
-    CU(cudaMemset(ctx->diag, 0, sizeof(DeviceDiag)));
+    CU(cudaMemcpy(&h, ctx->diag, DIAG_STATUS_BYTES, cudaMemcpyDeviceToHost));
+    CU(cudaMemset(ctx->diag, 0, DIAG_STATUS_BYTES));
     if (out) {
         out->device_status = h.status;
         float f;

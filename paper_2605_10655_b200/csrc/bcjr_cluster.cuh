@@ -111,18 +111,106 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity)
         : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after ~2^20 polls, raises BCJR_ETIMEOUT (-6) in the diagnostics and
-// sets the CTA-wide abort flag so that later waits return at once; the kernel then runs to its
-// end (with meaningless numbers) instead of hanging.
-__device__ __forceinline__ void mbar_wait_bounded(uint32_t mbar, uint32_t parity, volatile int *abort_flag, DeviceDiag *diag)
+// Device-side waits are bounded by wall time (the context's wait budget, default 2 s): a wait that
+// runs out raises BCJR_ETIMEOUT (-6) in the diagnostics and sets the CTA-wide abort flag; the kernel
+// then runs to its end on meaningless numbers instead of hanging (see Proto below).
+__device__ __forceinline__ unsigned long long global_timer_ns()
 {
-    if (mbar_try_wait(mbar, parity)) return;                     // fast path: one probe
-    if (*abort_flag) return;
-    for (int i = 0; i < (1 << 20); ++i)
-        if (mbar_try_wait(mbar, parity)) return;
-    *abort_flag = 1;
-    atomicCAS(&diag->status, 0, -6);
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
+// After a wait has run out the threads no longer wait for their inputs, so asynchronous copies may
+// still be on their way into this CTA's shared memory when the kernel reaches its end.  Leaving
+// with copies in flight is not allowed: the thread that requested bulk loads waits for each of the
+// last `depth` of them (time-bounded, ignoring the abort flag), and every thread lets the
+// st.async traffic addressed to this CTA land (a fixed, short delay) before the CTA exits.
+__device__ __forceinline__ void drain_bulk_loads(uint32_t mbar_base, uint32_t issued, uint32_t depth, DeviceDiag *diag)
+{
+    const unsigned long long limit = diag->wait_limit_ns;
+    for (uint32_t c = issued > depth ? issued - depth : 0u; c < issued; ++c) {
+        const uint32_t mbar = mbar_base + 8u * (c % depth), parity = (c / depth) & 1u;
+        const unsigned long long t0 = global_timer_ns();
+        for (int outer = 0; outer < (1 << 22); ++outer) {
+            if (mbar_try_wait(mbar, parity)) break;
+            if (global_timer_ns() - t0 > limit) break;
+        }
+    }
+}
+__device__ __forceinline__ void settle_after_abort()
+{
+    const unsigned long long t0 = global_timer_ns();
+    for (int i = 0; i < (1 << 16) && global_timer_ns() - t0 < 200000ull; ++i) __nanosleep(1000);
+}
+__device__ __forceinline__ void mbar_arrive_local(uint32_t mbar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+}
+// Relaxed arrival on a (possibly remote) mbarrier of the cluster: it publishes nothing by itself.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_mbar)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_mbar) : "memory");
+}
+// Protocol operations of one thread.  `live` turns false when one of this thread's waits runs out
+// (or finds that another thread of the CTA has given up).  A thread that is not live issues no
+// further mbarrier arrivals, transaction announcements, asynchronous stores or bulk copies, but
+// still reaches every CTA and cluster barrier, on meaningless numbers.  Two forms are used:
+//   * per operation: the guarded members below (arrive, expect_tx, load, store, async_*);
+//   * per step: the hot kernels take a warp-uniform vote (warp_live) right after the step's first
+//     wait and skip the step's work when a lane is dead; inside an admitted step the operations
+//     are issued unguarded, so a wait that runs out in mid-step lets the thread finish that one
+//     step.  Either way a thread is at most one step ahead of the last completed phase when it
+//     stops, so no transaction count runs away and nothing is issued after the last barrier.
+struct Proto {
+    uint32_t live;
+    volatile int *abort_flag;
+    DeviceDiag *diag;
+    __device__ __forceinline__ void wait(uint32_t mbar, uint32_t parity)
+    {
+        if (mbar_try_wait(mbar, parity)) return;                 // fast path: one probe
+        if (!live) return;
+        if (*abort_flag) { live = 0u; return; }
+        unsigned long long t0 = 0;
+        for (int i = 0; i < (1 << 24); ++i) {                    // hard cap besides the time budget
+            if (mbar_try_wait(mbar, parity)) return;
+            if ((i & 1023) == 1023) {
+                const unsigned long long now = global_timer_ns();
+                if (t0 == 0) t0 = now;
+                if (*abort_flag || now - t0 > diag->wait_limit_ns) break;
+            }
+        }
+        live = 0u;
+        *abort_flag = 1;
+        atomicCAS(&diag->status, 0, -6);
+    }
+    // warp-uniform liveness, taken once per step: a warp with a dead lane stops as a whole
+    __device__ __forceinline__ bool warp_live()
+    {
+        live = __all_sync(0xffffffffu, live != 0u) ? 1u : 0u;
+        return live != 0u;
+    }
+    __device__ __forceinline__ void arrive(uint32_t mbar) const
+    {
+        if (live) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+    }
+    __device__ __forceinline__ void arrive_cluster(uint32_t remote_mbar) const
+    {
+        if (live) asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_mbar) : "memory");
+    }
+    __device__ __forceinline__ void expect_tx(uint32_t mbar, uint32_t bytes) const { if (live) mbar_expect_tx(mbar, bytes); }
+    __device__ __forceinline__ void load(uint32_t sdst, const void *gsrc, uint32_t bytes, uint32_t mbar) const
+    {
+        if (live) bulk_load(sdst, gsrc, bytes, mbar);
+    }
+    __device__ __forceinline__ void store(void *gdst, uint32_t ssrc, uint32_t bytes) const { if (live) bulk_store(gdst, ssrc, bytes); }
+    __device__ __forceinline__ void async_f32(uint32_t addr, float v, uint32_t mbar) const { if (live) st_async_f32(addr, v, mbar); }
+    __device__ __forceinline__ void async_v2(uint32_t addr, float a, float b, uint32_t mbar) const { if (live) st_async_v2(addr, a, b, mbar); }
+    __device__ __forceinline__ void async_v4(uint32_t addr, float a, float b, float c, float d, uint32_t mbar) const
+    {
+        if (live) st_async_v4(addr, a, b, c, d, mbar);
+    }
+};
+
 // non-blocking probe of a phase
 __device__ __forceinline__ bool mbar_test(uint32_t mbar, uint32_t parity)
 {
@@ -306,6 +394,7 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
     float *part = smem + C::OFF_PART;
     float *lz = smem + C::OFF_LZ;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
+    Proto pr{1u, abort_flag, p.diag};
     const uint32_t mbar_stage = smem_u32(smem + C::OFF_MBAR);
     const uint32_t mbar_full = mbar_stage + 8u * C::NSTAGE;
     const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage);
@@ -362,7 +451,7 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
 
     // wait until every input of this CTA for the coming step has landed in buffer b
     auto wait_inputs = [&](int b) {
-        mbar_wait_bounded(mbar_full + 8u * b, (full_phase >> b) & 1u, abort_flag, p.diag);
+        pr.wait(mbar_full + 8u * b, (full_phase >> b) & 1u);
         full_phase ^= 1u << b;
     };
 
@@ -390,10 +479,10 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
                 const float *Lin = msg + ib * QC;
                 const uint32_t ob_off = (uint32_t)(ob * QC) * 4u, ob_mbar = 8u * ob;
                 if (tid == 0) {
-                    mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
+                    pr.expect_tx(mbar_full + ob_mbar, TX_MSG);
                     bulk_wait_read0();                                   // previous spill has left its buffer
                     fence_proxy_async();
-                    bulk_store(hist + ((size_t)(t - 1) * CL + rank) * QC, msg_u32 + (uint32_t)(ib * QC) * 4u, QC * 4u);
+                    pr.store(hist + ((size_t)(t - 1) * CL + rank) * QC, msg_u32 + (uint32_t)(ib * QC) * 4u, QC * 4u);
                     bulk_commit();
                 }
                 const float2 w2 = splat2(w_s[t - 1]);
@@ -423,13 +512,13 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
                     }
 #pragma unroll
                     for (int h = 0; h < K / 2; h += 2)
-                        st_async_v4(push_a[i] + ob_off + 8u * h, out[h].x, out[h].y, out[h + 1].x, out[h + 1].y,
+                        pr.async_v4(push_a[i] + ob_off + 8u * h, out[h].x, out[h].y, out[h + 1].x, out[h + 1].y,
                                     push_a_mbar[i] + ob_mbar);
                 }
                 tmax = warp_max(tmax);
                 if (lane == 0) {
 #pragma unroll
-                    for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 64) * 4u, tmax, full_of[r] + ob_mbar);
+                    for (int r = 0; r < CL; ++r) pr.async_f32(wmax_dst[r] + (uint32_t)(ob * 64) * 4u, tmax, full_of[r] + ob_mbar);
                 }
                 O += (int)off;
                 if (tid == 0) O_s[t + 1] = O;
@@ -467,9 +556,9 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
             fence_proxy_async();
             for (int d = 0; d < 2 && n - d >= 1; ++d) {
                 const uint32_t s = loads_issued % C::NSTAGE;
-                mbar_expect_tx(mbar_stage + 8u * s, QC * 4u);
-                bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(n - d - 1) * CL + rank) * QC, QC * 4u, mbar_stage + 8u * s);
-                ++loads_issued;
+                pr.expect_tx(mbar_stage + 8u * s, QC * 4u);
+                pr.load(stage_u32 + s * QC * 4u, hist + ((size_t)(n - d - 1) * CL + rank) * QC, QC * 4u, mbar_stage + 8u * s);
+                loads_issued += pr.live ? 1u : 0u;
             }
         }
         int P = 0;
@@ -505,17 +594,17 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
                 const float *Min = msg + ib * QC;
                 const uint32_t ob_off = (uint32_t)(ob * QC) * 4u, ob_mbar = 8u * ob;
                 if (tid == 0) {
-                    mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
+                    pr.expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
                     if (t - 2 >= 1) {                                    // prefetch L_{t-2}
                         fence_proxy_async();
                         const uint32_t s = loads_issued % C::NSTAGE;
-                        mbar_expect_tx(mbar_stage + 8u * s, QC * 4u);
-                        bulk_load(stage_u32 + s * QC * 4u, hist + ((size_t)(t - 3) * CL + rank) * QC, QC * 4u, mbar_stage + 8u * s);
-                        ++loads_issued;
+                        pr.expect_tx(mbar_stage + 8u * s, QC * 4u);
+                        pr.load(stage_u32 + s * QC * 4u, hist + ((size_t)(t - 3) * CL + rank) * QC, QC * 4u, mbar_stage + 8u * s);
+                        loads_issued += pr.live ? 1u : 0u;
                     }
                 }
                 const uint32_t st = loads_done % C::NSTAGE;
-                mbar_wait_bounded(mbar_stage + 8u * st, (loads_done / C::NSTAGE) & 1u, abort_flag, p.diag);
+                pr.wait(mbar_stage + 8u * st, (loads_done / C::NSTAGE) & 1u);
                 ++loads_done;
                 const float *Lh = stage + st * QC;
                 const float2 w2 = splat2(w_s[t - 1]);
@@ -554,8 +643,8 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
                         }
                         const float2 out = add2(m, lg2f2(sum));
                         tmax = max3f(tmax, m.x, m.y);
-                        st_async_f32(push_b[i][2 * jh] + ob_off, out.x, full_of[(2 * jh) * CL / K] + ob_mbar);
-                        st_async_f32(push_b[i][2 * jh + 1] + ob_off, out.y, full_of[(2 * jh + 1) * CL / K] + ob_mbar);
+                        pr.async_f32(push_b[i][2 * jh] + ob_off, out.x, full_of[(2 * jh) * CL / K] + ob_mbar);
+                        pr.async_f32(push_b[i][2 * jh + 1] + ob_off, out.y, full_of[(2 * jh + 1) * CL / K] + ob_mbar);
                         num2 = fma2(f, craw, num2);
                         den2 = fma2(f, sum, den2);
                     }
@@ -564,8 +653,8 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
                 tmax = warp_max(tmax);
                 if (lane == 0) {
 #pragma unroll
-                    for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 64) * 4u, tmax, full_of[r] + ob_mbar);
-                    st_async_v2(part_dst + (uint32_t)(ob * 128) * 4u, num, den, full_of[0] + ob_mbar);
+                    for (int r = 0; r < CL; ++r) pr.async_f32(wmax_dst[r] + (uint32_t)(ob * 64) * 4u, tmax, full_of[r] + ob_mbar);
+                    pr.async_v2(part_dst + (uint32_t)(ob * 128) * 4u, num, den, full_of[0] + ob_mbar);
                 }
                 ib = ob;
             }
@@ -596,7 +685,10 @@ __global__ void __launch_bounds__(THREADS, 1) fwd_cluster_kernel(FwdParams p)
         diag_max(&p.diag->max_defect, defect);
         diag_max(&p.diag->max_logz_gap, zgap);
     }
+    if (*abort_flag && tid == 0) drain_bulk_loads(mbar_stage, loads_issued, C::NSTAGE, p.diag);
+    __syncthreads();
     cluster_sync();             // no CTA leaves while a peer may still address its shared memory
+    if (*abort_flag) settle_after_abort();
 }
 
 // --------------------------------------------------------------------------------------
@@ -654,6 +746,7 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
     float *part = smem + BC::OFF_PART;
     float *lz = smem + BC::OFF_LZ;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + BC::OFF_FLAG);
+    Proto pr{1u, abort_flag, p.diag};
     const uint32_t mbar0 = smem_u32(smem + BC::OFF_MBAR);
     const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage);
     const uint32_t wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
@@ -722,7 +815,7 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
                 const uint32_t nxt_off = (uint32_t)((t & 1) * 2 * QC) * 4u;
                 if (tid == 0) {
                     fence_proxy_async();
-                    bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)(cur * 2 * QC) * 4u, STEP_BYTES);
+                    pr.store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)(cur * 2 * QC) * 4u, STEP_BYTES);
                     bulk_commit();
                 }
                 const float gt = g_s[t - 1];
@@ -805,9 +898,9 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
             fence_proxy_async();
             for (int d = 0; d < 2 && n - d >= 1; ++d) {
                 const uint32_t s = loads_issued % BC::NSTAGE;
-                mbar_expect_tx(mbar0 + 8u * s, STEP_BYTES);
-                bulk_load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(n - d - 1) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
-                ++loads_issued;
+                pr.expect_tx(mbar0 + 8u * s, STEP_BYTES);
+                pr.load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(n - d - 1) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
+                loads_issued += pr.live ? 1u : 0u;
             }
         }
         int P = 0;
@@ -823,12 +916,12 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
                 if (tid == 0 && t - 2 >= 1) {
                     fence_proxy_async();
                     const uint32_t s = loads_issued % BC::NSTAGE;
-                    mbar_expect_tx(mbar0 + 8u * s, STEP_BYTES);
-                    bulk_load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(t - 3) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
-                    ++loads_issued;
+                    pr.expect_tx(mbar0 + 8u * s, STEP_BYTES);
+                    pr.load(stage_u32 + s * STEP_BYTES, hist + ((size_t)(t - 3) * CL + rank) * 2 * QC, STEP_BYTES, mbar0 + 8u * s);
+                    loads_issued += pr.live ? 1u : 0u;
                 }
                 const uint32_t st = loads_done % BC::NSTAGE;
-                mbar_wait_bounded(mbar0 + 8u * st, (loads_done / BC::NSTAGE) & 1u, abort_flag, p.diag);
+                pr.wait(mbar0 + 8u * st, (loads_done / BC::NSTAGE) & 1u);
                 ++loads_done;
                 const float *Lh = stage + st * 2 * QC, *Ah = Lh + QC;
                 const float wt = w_s[t - 1], gt = g_s[t - 1], sft = sf_s[t - 1];
@@ -928,7 +1021,10 @@ __global__ void __launch_bounds__(THREADS, 1) bwd_cluster_kernel(BwdParams p)
             }
     }
     if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
-    cluster_sync();
+    if (*abort_flag && tid == 0) drain_bulk_loads(mbar0, loads_issued, BC::NSTAGE, p.diag);
+    __syncthreads();
+    cluster_sync();             // no CTA leaves while a peer may still address its shared memory
+    if (*abort_flag) settle_after_abort();
 }
 
 // ---------------------------------------------------------------------------- host side

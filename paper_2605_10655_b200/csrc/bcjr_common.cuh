@@ -49,7 +49,12 @@ struct DeviceDiag {
     unsigned int max_defect;     // float bits of max |sum gamma - 1|
     unsigned int max_logz_gap;   // float bits of max |log2 Z(alpha) - log2 Z(beta)|
     int pad;
+    // configuration, written by the host when an option changes (not cleared by status queries)
+    unsigned long long wait_limit_ns;   // budget of one device-side wait before it gives up
+    int drop_history_load;              // test hook: CTA 0 never requests its first history chunk
+    int pad2;
 };
+constexpr size_t DIAG_STATUS_BYTES = 16;   // the part bcjr_sync_status reads and clears
 
 __device__ __forceinline__ void diag_max(unsigned int *slot, float v) {
     // v >= 0: float ordering equals unsigned ordering of the bit patterns

@@ -25,14 +25,6 @@
 
 namespace bcjr {
 
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t remote_mbar)
-{
-#ifdef BCJR_RELEASE_ARRIVE
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_mbar) : "memory");
-#else
-    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_mbar) : "memory");
-#endif
-}
 
 #ifdef BCJR_TIMING
 __device__ unsigned long long g_duo_timing[8];   // beta sweep, warp 1 of CTA 0: compute, cta barrier, input wait, ring wait
@@ -104,6 +96,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     float *lz = smem + C::OFF_LZ;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
+    Proto pr{1u, abort_flag, p.diag};
     const uint32_t ring_full = smem_u32(smem + C::OFF_MBAR);
     const uint32_t ring_empty = ring_full + 8u * RD;
     const uint32_t mbar_full = ring_empty + 8u * RD;             // [2], one per message parity
@@ -128,7 +121,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     const uint32_t tmem_base = *tmem_slot;
     uint32_t full_phase = 0;       // bit b = parity to wait for on full[b]
     auto wait_inputs = [&](int b) {
-        mbar_wait_bounded(mbar_full + 8u * b, (full_phase >> b) & 1u, abort_flag, p.diag);
+        pr.wait(mbar_full + 8u * b, (full_phase >> b) & 1u);
         full_phase ^= 1u << b;
     };
 
@@ -201,6 +194,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
                 off = rintf(cmax);
             }
+            if (!pr.warp_live()) break;                          // a wait ran out: this warp issues nothing more
             const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) {
@@ -273,7 +267,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             __syncwarp();
             if (lane == 0) {                                     // this warp has read all its inputs
 #pragma unroll
-                for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
+                for (int r = 0; r < CL; ++r) mbar_arrive_remote(full_of[r] + ob_mbar);
             }
             ib = ob;
         }
@@ -310,15 +304,17 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         // thread 0 streams the history back: request every chunk whose ring slot has been
         // released by all warps, without ever blocking (called between butterflies)
         auto feed_ring = [&]() {
-            while (issued != chunk_end) {
+            while (pr.live && issued != chunk_end) {
                 const uint32_t s = issued % RD;
                 if (!mbar_test(ring_empty + 8u * s, ((issued / RD) & 1u) ^ 1u)) break;
                 const uint32_t rel = issued - (chunk_end - (uint32_t)n * BPT);
                 const int t = n - (int)(rel / BPT), i = (int)(rel % BPT);
-                mbar_expect_tx(ring_full + 8u * s, 2u * CH * 4u);
+                pr.expect_tx(ring_full + 8u * s, 2u * CH * 4u);
                 const float *src = hist + ((size_t)(t - 1) * CL + rank) * 2 * QC + (size_t)i * CH;
-                bulk_load(ring_u32 + s * 2u * CH * 4u, src, CH * 4u, ring_full + 8u * s);
-                bulk_load(ring_u32 + s * 2u * CH * 4u + CH * 4u, src + QC, CH * 4u, ring_full + 8u * s);
+                if (!(issued == 0 && blockIdx.x == 0 && p.diag->drop_history_load)) {   // test hook: a wait that runs out
+                    pr.load(ring_u32 + s * 2u * CH * 4u, src, CH * 4u, ring_full + 8u * s);
+                    pr.load(ring_u32 + s * 2u * CH * 4u + CH * 4u, src + QC, CH * 4u, ring_full + 8u * s);
+                }
                 ++issued;
             }
         };
@@ -348,6 +344,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 offM = rintf(cmax);
                 finish_step(t + 1, ib);
             }
+            if (!pr.warp_live()) break;                          // a wait ran out: this warp issues nothing more
             const float *Min = msg + ib * 2 * QC, *Bin = Min + QC;
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
@@ -365,7 +362,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 if (tid == 0) feed_ring();
                 const uint32_t s = chunk % RD;
                 TICK(tr0);
-                mbar_wait_bounded(ring_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
+                pr.wait(ring_full + 8u * s, (chunk / RD) & 1u);
                 TICK(tr1); TACC(3, tr0, tr1);
                 const float *Lh = ring + s * 2 * CH, *Ah = Lh + CH;
                 float Mb[K], Yb[K];
@@ -425,7 +422,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                     tmem_st16(tm_acc + 16u * g, acc);
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(ring_empty + 8u * s);               // history chunk consumed by this warp
+                if (lane == 0) mbar_arrive_local(ring_empty + 8u * s);               // history chunk consumed by this warp
             }
             tmem_wait_st();
             const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), zz = warp_sum(ZS.x + ZS.y);
@@ -440,7 +437,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             TICK(tb1); TACC(1, tb0, tb1); TACC(0, tk0, tb1);
             if (lane == 0) {                                     // this warp has read all its inputs
 #pragma unroll
-                for (int r = 0; r < CL; ++r) mbar_arrive_cluster(full_of[r] + ob_mbar);
+                for (int r = 0; r < CL; ++r) mbar_arrive_remote(full_of[r] + ob_mbar);
             }
             ib = ob;
         }
@@ -474,9 +471,11 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         for (int e = 0; e < 8; ++e) g_duo_timing[e] = tacc[e];
 #endif
     if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
+    if (*abort_flag && tid == 0) drain_bulk_loads(ring_full, issued, RD, p.diag);   // no copy may be in flight at exit
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     cluster_sync();             // no CTA leaves while a peer may still address its shared memory
+    if (*abort_flag) settle_after_abort();
     if (warp == 0) tmem_dealloc_512(tmem_base);
 }
 

@@ -59,10 +59,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float2 (&v)[8])
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t mbar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
-}
 __device__ __forceinline__ void compute_barrier(int nthreads)
 {
     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
@@ -151,6 +147,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
     float *lz = smem + C::OFF_LZ;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
+    Proto pr{1u, abort_flag, p.diag};
     const uint32_t mbar_full = smem_u32(smem + C::OFF_MBAR);
     const uint32_t mbar_empty = mbar_full + 8u * RD;
     const uint32_t mbar_ready = mbar_empty + 8u * RD;          // [2] compute -> copy warp: buffer holds L_t
@@ -174,26 +171,30 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
         // ============================ copy warp (one elected lane) ============================
         if (lane == 0) {
             uint32_t use_ready[2] = {0u, 0u}, chunk = 0;      // completed phases per mbarrier
+            uint32_t requested = 0;                            // chunks up to the last one actually requested
             for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
                 for (int t = 1; t <= n; ++t) {                 // alpha: spill L_t once the buffer is complete
                     const uint32_t b = (uint32_t)(t - 1) & 1u;
-                    mbar_wait_bounded(mbar_ready + 8u * b, use_ready[b] & 1u, abort_flag, p.diag);
+                    pr.wait(mbar_ready + 8u * b, use_ready[b] & 1u);
                     ++use_ready[b];
                     fence_proxy_async();
-                    bulk_store(hist + (size_t)(t - 1) * Q, msg_u32 + b * Q * 4u, Q * 4u);
+                    pr.store(hist + (size_t)(t - 1) * Q, msg_u32 + b * Q * 4u, Q * 4u);
                     bulk_commit();
                     bulk_wait_read0();
-                    mbar_arrive(mbar_freed + 8u * b);
+                    pr.arrive(mbar_freed + 8u * b);
                 }
                 bulk_wait_all0();                              // history written before it is read back
                 for (int t = n; t >= 1; --t)                   // beta: stream L_t back, one slot chunk at a time
                     for (int i = 0; i < BPT; ++i, ++chunk) {
                         const uint32_t s = chunk % RD;
-                        mbar_wait_bounded(mbar_empty + 8u * s, ((chunk / RD) & 1u) ^ 1u, abort_flag, p.diag);
-                        mbar_expect_tx(mbar_full + 8u * s, CH * 4u);
-                        bulk_load(ring_u32 + s * CH * 4u, hist + (size_t)(t - 1) * Q + (size_t)i * CH, CH * 4u, mbar_full + 8u * s);
+                        pr.wait(mbar_empty + 8u * s, ((chunk / RD) & 1u) ^ 1u);
+                        pr.expect_tx(mbar_full + 8u * s, CH * 4u);
+                        if (chunk == 0 && blockIdx.x == 0 && p.diag->drop_history_load) continue;   // test hook: a wait that runs out
+                        if (pr.live) requested = chunk + 1;
+                        pr.load(ring_u32 + s * CH * 4u, hist + (size_t)(t - 1) * Q + (size_t)i * CH, CH * 4u, mbar_full + 8u * s);
                     }
             }
+            if (!pr.live || *abort_flag) drain_bulk_loads(mbar_full, requested, RD, p.diag);   // no copy may be in flight at exit
         }
     } else {
         // ============================ compute warps ============================
@@ -228,14 +229,15 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                 const int cur = (t - 1) & 1;
                 const float *Lin = msg + cur * Q;
                 float *Lout = msg + (cur ^ 1) * Q;
-                if (tid == 0) mbar_arrive(mbar_ready + 8u * cur);                // L_t complete: spill it
+                if (tid == 0) pr.arrive(mbar_ready + 8u * cur);                // L_t complete: spill it
                 if (t > 1) {
                     cmax = warp_max(lane < NWARP ? wmax[cur * 32 + lane] : NEG_INF) - off;
                     off = rintf(cmax);
                     // the buffer written now was spilled during the previous step: wait until read
-                    mbar_wait_bounded(mbar_freed + 8u * (cur ^ 1), use_freed[cur ^ 1] & 1u, abort_flag, p.diag);
+                    pr.wait(mbar_freed + 8u * (cur ^ 1), use_freed[cur ^ 1] & 1u);
                     ++use_freed[cur ^ 1];
                 }
+                if (!pr.warp_live()) { compute_barrier(CT); continue; }          // a wait ran out: only keep the barriers
                 const float2 w2 = splat2(w_s[t - 1]);
                 const float2 off2 = splat2(off);
                 float tmax = NEG_INF;
@@ -294,7 +296,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             const int Ofin = O;
             if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
             // the last spill (L_n, buffer (n-1)&1) must have left its buffer before it is reused
-            mbar_wait_bounded(mbar_freed + 8u * ((n - 1) & 1), use_freed[(n - 1) & 1] & 1u, abort_flag, p.diag);
+            pr.wait(mbar_freed + 8u * ((n - 1) & 1), use_freed[(n - 1) & 1] & 1u);
             ++use_freed[(n - 1) & 1];
             // ================= beta sweep
             for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // M_n = 0 in buffer 0
@@ -324,6 +326,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                         }
                     }
                 }
+                if (!pr.warp_live()) { compute_barrier(CT); continue; }          // a wait ran out: only keep the barriers
                 const float2 w2 = splat2(w_s[t - 1]);
                 const float2 offM2 = splat2(offM);
                 const float2 Dm2 = splat2((float)(Ofin - O_s[t] - P) + lsefin);
@@ -334,7 +337,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
 #pragma unroll
                 for (int i = 0; i < BPT; ++i, ++chunk) {
                     const uint32_t s = chunk % RD;
-                    mbar_wait_bounded(mbar_full + 8u * s, (chunk / RD) & 1u, abort_flag, p.diag);
+                    pr.wait(mbar_full + 8u * s, (chunk / RD) & 1u);
                     const float *Lh = ring + s * CH;
                     float Mb[K];
 #pragma unroll
@@ -377,7 +380,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                         }
                     }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(mbar_empty + 8u * s);             // this warp is done with the chunk
+                    if (lane == 0) mbar_arrive_local(mbar_empty + 8u * s);             // this warp is done with the chunk
                 }
                 const float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
                 tmax = warp_max(tmax) - offM;

@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
     volatile int *best = reinterpret_cast<volatile int *>(smem + C::OFF_BEST);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
+    Proto pr{1u, abort_flag, p.diag};
     const uint32_t tb_ready = smem_u32(smem + C::OFF_MBAR);      // [2] compute -> trace warp
     const uint32_t tb_done = tb_ready + 16u;                     // [2] trace warp -> compute
     // backpointers of this CTA: [2 parities][n][NB] bytes
@@ -80,11 +81,12 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
         uint32_t it = 0;
         for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x, ++it) {
             const uint32_t par = it & 1u;
-            mbar_wait_bounded(tb_ready + 8u * par, (it >> 1) & 1u, abort_flag, p.diag);
+            pr.wait(tb_ready + 8u * par, (it >> 1) & 1u);
+            if (!__all_sync(0xffffffffu, pr.live)) continue;     // a wait ran out: nothing valid to trace
             const uint8_t *bp = bp_base + (size_t)par * n * NB;
             if (lane == 0) {
                 // predecessor of s at step t+1 is j*Q + (s >> k), j = branch stored for group s >> k
-                int s = best[par];
+                int s = best[par] & (C::S - 1);
                 path[n - 1] = s;
                 for (int t = n - 1; t >= 1; --t) {
                     const int q = s >> KB;
@@ -117,7 +119,7 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(tb_done + 8u * par);      // this backpointer buffer may be reused
+            if (lane == 0) pr.arrive(tb_done + 8u * par);      // this backpointer buffer may be reused
         }
     } else {
         // ============================ compute warps ============================
@@ -140,7 +142,7 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
             const uint32_t par = it & 1u;
             const float *w = p.W + blk * n;
             // the backpointer buffer of this parity was last used two blocks ago: wait until traced
-            if (it >= 2) mbar_wait_bounded(tb_done + 8u * par, ((it >> 1) - 1u) & 1u, abort_flag, p.diag);
+            if (it >= 2) pr.wait(tb_done + 8u * par, ((it >> 1) - 1u) & 1u);
             uint8_t *bp = bp_base + (size_t)par * n * NB;
             for (int q = tid; q < Q; q += CT) mv[q] = 0.0;           // mv_1 = 0: free first state
             compute_barrier(CT);
@@ -223,7 +225,7 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(tb_ready + 8u * par);         // hand the block to the trace warp
+            if (lane == 0) pr.arrive(tb_ready + 8u * par);         // hand the block to the trace warp
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

@@ -254,6 +254,28 @@ def test_non_finite_input_is_reported_not_fatal(ctx):
         assert ctx.sync_status().device_status == 0                          # cleared by the query
 
 
+def test_device_wait_that_runs_out_is_reported_and_survivable(ctx):
+    # No GPU fault is provoked: a history chunk is simply never requested, the consumer's bounded
+    # wait gives up after its (shortened) budget, the kernel runs to its end and the host reads
+    # BCJR_ETIMEOUT.  Afterwards the same context computes correct results again.
+    from paper_2605_10655_b200 import BcjrError
+    Lb, k, n, T = 16, 2, 6, 0.3
+    W, c, g = _rand(n, Lb, 2, seed=4400)
+    ref = oracle.soft_quantize(W, c, Lb, k, T)
+    try:
+        ctx.set_option("wait_limit_ms", 20)
+        ctx.set_option("debug_drop_history_load", 1)
+        with pytest.raises(BcjrError) as ei:
+            parity.gpu_forward_backward(ctx, W, c, g, Lb, k, T)
+        assert ei.value.code == -6
+    finally:
+        ctx.set_option("debug_drop_history_load", 0)
+        ctx.set_option("wait_limit_ms", 2000)
+    got = parity.gpu_forward_backward(ctx, W, c, g, Lb, k, T)
+    assert got["diag"].device_status == 0
+    assert parity.rel_inf(got["soft"], ref["soft"]) <= parity.SOFT_TOL
+
+
 def test_results_do_not_depend_on_what_ran_before(ctx):
     # scratch (history, partial sums, tensor memory) is reused between calls and between
     # blocks: the same input must give bit-identical output regardless of the previous call
