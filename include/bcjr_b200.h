@@ -121,6 +121,21 @@ bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook,
                          uint16_t *states, float *hard, void *cuda_stream);
 
 /*
+ * BCJR-STE forward (Section 3.7, "BCJR-STE variant"): the value that goes forward is the hard
+ * Viterbi codeword, while the state saved on the context is that of the temperature-T relaxation,
+ * so that a following bcjr_backward returns the gradient of the finite-temperature soft codeword
+ * (the straight-through gradient replaced by the true gradient of the relaxation).  Equivalent
+ * to bcjr_soft_quantize followed by viterbi_hard on the same inputs.
+ *   hard    device out  [num_blocks * n] exact copies of codebook entries (required)
+ *   states  device out  [num_blocks * n] uint16, may be NULL
+ *   soft    device out  [num_blocks * n] soft codeword at T, may be NULL (kept internally only)
+ * Same argument checks, borrowing rules and error behaviour as the two calls it is made of.
+ */
+bcjr_status bcjr_ste_forward(bcjr_ctx *ctx, const float *W, const float *codebook,
+                             int Lb, int k, int n, int64_t num_blocks, float T,
+                             float *hard, uint16_t *states, float *soft, void *cuda_stream);
+
+/*
  * One training-style step with HOST buffers (pinned or pageable): copies W, codebook and
  * grad_soft to the device, runs bcjr_soft_quantize and bcjr_backward, and copies soft,
  * grad_W and grad_codebook back, all on `cuda_stream`; returns after the stream has been

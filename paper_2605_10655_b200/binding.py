@@ -13,7 +13,7 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libbcjr_b200.so"
 
 EXPORTS = ["bcjr_create", "bcjr_destroy", "bcjr_set_option", "bcjr_soft_quantize", "bcjr_backward",
-           "viterbi_hard", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
+           "viterbi_hard", "bcjr_ste_forward", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
            "bcjr_last_cuda_error", "bcjr_status_string", "bcjr_soft_quantize_static",
            "bcjr_static_scratch_bytes"]
 
@@ -50,6 +50,8 @@ def load_library() -> ctypes.CDLL:
     lib.bcjr_soft_quantize.argtypes = [vp, vp, vp, i, i, i, i64, f, vp, vp, vp]
     lib.bcjr_backward.restype = i; lib.bcjr_backward.argtypes = [vp, vp, vp, vp, vp]
     lib.viterbi_hard.restype = i; lib.viterbi_hard.argtypes = [vp, vp, vp, i, i, i, i64, vp, i64, vp, vp, vp]
+    lib.bcjr_ste_forward.restype = i
+    lib.bcjr_ste_forward.argtypes = [vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
     lib.bcjr_step_host.restype = i
     lib.bcjr_step_host.argtypes = [vp, vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
     lib.bcjr_sync_status.restype = i; lib.bcjr_sync_status.argtypes = [vp, vp, ctypes.POINTER(Diag)]
@@ -191,6 +193,24 @@ class Context:
                                     ctypes.c_void_p(hard.data_ptr()) if want_hard else None, _stream_ptr(stream))
         self._check(rc, "viterbi_hard")
         return bits, states, hard
+
+    def bcjr_ste_forward(self, W, codebook, Lb, k, n, T, want_states=False, want_soft=False, stream=None):
+        """Hard Viterbi codeword forward, finite-T state saved for bcjr_backward.  Returns (hard, states, soft)."""
+        import torch
+        B = W.numel() // n
+        if B * n != W.numel():
+            raise ValueError("W.numel() must be a multiple of n")
+        hard = torch.empty((B, n), dtype=torch.float32, device=W.device)
+        states = torch.empty((B, n), dtype=torch.int16, device=W.device) if want_states else None
+        soft = torch.empty((B, n), dtype=torch.float32, device=W.device) if want_soft else None
+        rc = self._lib.bcjr_ste_forward(self._h, _dev(W, torch.float32, name="W"),
+                                        _dev(codebook, torch.float32, 1 << Lb, "codebook"), Lb, k, n, B, float(T),
+                                        ctypes.c_void_p(hard.data_ptr()),
+                                        ctypes.c_void_p(states.data_ptr()) if want_states else None,
+                                        ctypes.c_void_p(soft.data_ptr()) if want_soft else None, _stream_ptr(stream))
+        self._check(rc, "bcjr_ste_forward")
+        self._saved = (W, codebook, Lb, B * n)
+        return hard, states, soft
 
     def bcjr_step_host(self, W, codebook, grad_soft, Lb, k, n, T, soft=None, grad_W=None, grad_codebook=None,
                        stream=None):

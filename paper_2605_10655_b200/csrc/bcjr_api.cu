@@ -577,6 +577,29 @@ bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook, i
     return BCJR_OK;
 }
 
+bcjr_status bcjr_ste_forward(bcjr_ctx *ctx, const float *W, const float *codebook, int Lb, int k, int n,
+                             int64_t num_blocks, float T, float *hard, uint16_t *states, float *soft,
+                             void *cuda_stream)
+{
+    if (!ctx) return BCJR_EINVAL;
+    if (!(T > 0.f) || !std::isfinite(T)) return BCJR_EINVAL;
+    bcjr_status rc = check_dims(Lb, k, n, num_blocks);
+    if (rc) return rc;
+    if (num_blocks > 0 && (!W || !codebook || !hard)) return BCJR_EINVAL;
+    float *soft_out = soft;
+    if (!soft_out && num_blocks > 0) {
+        // the relaxation's output is only needed as saved state: let it land in the context's own copy
+        DeviceGuard guard(ctx->device);
+        if (!guard.ok) return BCJR_ECUDA;
+        if ((rc = ensure(ctx, ctx->soft_copy, (size_t)num_blocks * n * 4))) return rc;
+        soft_out = (float *)ctx->soft_copy.ptr;
+    }
+    if ((rc = bcjr_soft_quantize(ctx, W, codebook, Lb, k, n, num_blocks, T, soft_out, nullptr, cuda_stream))) return rc;
+    rc = viterbi_hard(ctx, W, codebook, Lb, k, n, num_blocks, nullptr, 0, states, hard, cuda_stream);
+    if (rc) ctx->have_fwd = false;
+    return rc;
+}
+
 bcjr_status bcjr_step_host(bcjr_ctx *ctx, const float *W_host, const float *codebook_host,
                            const float *grad_soft_host, int Lb, int k, int n, int64_t num_blocks, float T,
                            float *soft_host, float *grad_W_host, float *grad_codebook_host, void *cuda_stream)

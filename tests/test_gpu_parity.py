@@ -276,6 +276,30 @@ def test_device_wait_that_runs_out_is_reported_and_survivable(ctx):
     assert parity.rel_inf(got["soft"], ref["soft"]) <= parity.SOFT_TOL
 
 
+@pytest.mark.parametrize("Lb,k,n,B,T", [(8, 2, 64, 16, 0.5), (16, 2, 48, 3, 0.1), (16, 3, 40, 2, 0.05)])
+def test_ste_forward_emits_hard_codeword_and_keeps_the_soft_gradient(ctx, Lb, k, n, B, T):
+    # BCJR-STE: hard Viterbi codeword forward, gradient of the temperature-T relaxation backward
+    import torch
+    W, c, g = _rand(n, Lb, B, seed=5100 + Lb + k)
+    dev = torch.device("cuda", ctx.device)
+    Wd, cd, gd = (torch.from_numpy(a).to(dev) for a in (W, c, g))
+    hard, states, soft = ctx.bcjr_ste_forward(Wd, cd, Lb, k, n, T, want_states=True, want_soft=True)
+    gW, gc = ctx.bcjr_backward(gd)
+    assert ctx.sync_status().device_status == 0
+    ref_v = oracle.viterbi(W, c, Lb, k)
+    np.testing.assert_array_equal(hard.cpu().numpy().view(np.uint32), ref_v["hard"].view(np.uint32))
+    np.testing.assert_array_equal(states.cpu().numpy().view(np.uint16), ref_v["states"])
+    ref_f, ref_b = oracle.soft_quantize(W, c, Lb, k, T), oracle.backward(W, c, g, Lb, k, T)
+    assert parity.rel_inf(soft.cpu().numpy(), ref_f["soft"]) <= parity.SOFT_TOL
+    assert parity.rel_inf(gW.cpu().numpy(), ref_b["grad_W"]) <= parity.GRAD_TOL
+    assert parity.rel_inf(gc.cpu().numpy(), ref_b["grad_codebook"]) <= parity.GRAD_TOL
+    # without the optional outputs the saved state is the same
+    hard2, _, _ = ctx.bcjr_ste_forward(Wd, cd, Lb, k, n, T)
+    gW2, gc2 = ctx.bcjr_backward(gd)
+    ctx.sync_status()
+    assert torch.equal(hard, hard2) and torch.equal(gW, gW2) and torch.equal(gc, gc2)
+
+
 def test_results_do_not_depend_on_what_ran_before(ctx):
     # scratch (history, partial sums, tensor memory) is reused between calls and between
     # blocks: the same input must give bit-identical output regardless of the previous call
