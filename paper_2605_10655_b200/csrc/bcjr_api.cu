@@ -292,20 +292,21 @@ bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_co
     return BCJR_EUNSUPPORTED;
 }
 
-// Viterbi, one CTA per block with the codebook in tensor memory (Lb = 16, k = 2).
+// Viterbi, one CTA per block with the codebook in tensor memory (Lb = 16; k = 2, 3).
+template <int KB>
 bcjr_status launch_vit_solo(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
 {
-    using C = VitSoloCfg;
+    using C = VitSoloCfg<KB>;
     if (p.n > C::MAX_N) return BCJR_EUNSUPPORTED;
-    CU(cudaFuncSetAttribute(viterbi_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    CU(cudaFuncSetAttribute(viterbi_solo_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
     int64_t grid = ctx->num_sms;
     if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
     if (grid > p.B) grid = p.B;
-    bcjr_status rc = ensure(ctx, ctx->bp, (size_t)grid * 2 * p.n * C::NB);
+    bcjr_status rc = ensure(ctx, ctx->bp, (size_t)grid * 2 * p.n * C::ROW_BYTES);
     if (rc) return rc;
     p.bp = (uint8_t *)ctx->bp.ptr;
     p.diag = ctx->diag;
-    viterbi_solo_kernel<<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    viterbi_solo_kernel<KB><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
     ctx->launches += 1;
     CU(cudaGetLastError());
     return BCJR_OK;
@@ -555,10 +556,10 @@ bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook, i
     p.states = states; p.hard = hard; p.B = num_blocks; p.Lb = Lb; p.n = n;
     bool use_large = false;
 #ifndef BCJR_NO_CLUSTER
-    use_large = ctx->opt_path != 1 && Lb == 16 && k == 2;
+    use_large = ctx->opt_path != 1 && Lb == 16 && (k == 2 || k == 3);
     if (ctx->opt_path == 2 && !use_large) return BCJR_EUNSUPPORTED;
     if (use_large) {
-        rc = launch_vit_solo(ctx, p, st);
+        rc = k == 2 ? launch_vit_solo<2>(ctx, p, st) : launch_vit_solo<3>(ctx, p, st);
         if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { use_large = false; rc = BCJR_OK; }
     }
 #else

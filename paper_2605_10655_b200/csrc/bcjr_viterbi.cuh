@@ -1,4 +1,4 @@
-// Viterbi hard code for the 2^16-state trellis (k = 2): one CTA per weight block.
+// Viterbi hard code for the 2^16-state trellis (k = 2 or 3): one CTA per weight block.
 //
 // Same butterfly ownership as the sum-product kernels, in the (min, +) semiring and in IEEE
 // double (bit-identical with a sequential double implementation: d = (double)w - (double)c,
@@ -10,19 +10,24 @@
 //     index q lives at a step-dependent address, rotr(q, k*step) on the Lb-k index bits (the
 //     perfect shuffle undone one step at a time), XOR-swizzled so that whichever five index bits
 //     vary across a warp land on different banks.  One CTA barrier per step;
-//   - backpointers: one byte per butterfly and step (four 2-bit branches), 1 MB per block,
-//     streamed to global memory; an extra warp backtracks block b, and writes its outputs,
+//   - backpointers: one word per butterfly and step (K branches of k bits: a byte for k = 2, 32
+//     bits for k = 3), 4 KB per step and 1 MB per 256-step block, streamed to global memory; an extra warp backtracks block b, and writes its outputs,
 //     while the compute warps already run block b+1 (two backpointer buffers per CTA).
 #pragma once
 #include "bcjr_solo.cuh"
 
 namespace bcjr {
 
+template <int KB_>
 struct VitSoloCfg {
-    static constexpr int LB = 16, KB = 2, K = 4, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
+    static constexpr int LB = 16, KB = KB_, K = 1 << KB, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
     static constexpr int QB = LB - KB;                          // index bits of a group
     static constexpr int CTHREADS = 512, THREADS = CTHREADS + 32, NWARP = CTHREADS / 32;
-    static constexpr int BPT = NB / CTHREADS;                   // 8 butterflies per thread: x = tid*BPT + i
+    static constexpr int BPT = NB / CTHREADS;                   // butterflies per thread (8 / 2): x = tid*BPT + i
+    static constexpr int UNITS = K * K / 16;                    // 16-column TMEM units per butterfly
+    static constexpr int JPU = K / UNITS;                       // predecessors j covered by one unit
+    static constexpr int WORD_BITS = 64 / BPT;                  // backpointer word of one butterfly (8 / 32 bits)
+    static constexpr int ROW_BYTES = NB * WORD_BITS / 8;        // backpointers of one step
     static constexpr int MAX_N = 4096;
     static constexpr int OFF_MV = 0;                            // double [Q]  (2 floats each)
     static constexpr int OFF_PATH = OFF_MV + 2 * Q;             // int [MAX_N] state sequence of the block being traced
@@ -34,21 +39,26 @@ struct VitSoloCfg {
     static constexpr int SMEM_FLOATS = OFF_FLAG + 2;
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static_assert(OFF_MBAR % 2 == 0 && OFF_RED % 2 == 0, "8-byte alignment");
+    static_assert(BPT * K * K == 128, "a thread's codebook slice fills its 128 TMEM columns");
+    static_assert(K * KB <= WORD_BITS && (WORD_BITS == 8 || WORD_BITS == 32), "backpointer word");
 };
 
-// step-dependent physical slot of a 14-bit group index: rotate right, then fold the upper bits
+// step-dependent physical slot of a QB-bit group index: rotate right, then fold the upper bits
 // into the bank bits (XOR-linear, so it distributes over disjoint bit fields)
+template <int QB>
 __device__ __forceinline__ uint32_t vit_rotr(uint32_t v, int r)
 {
-    constexpr uint32_t M = (1u << VitSoloCfg::QB) - 1u;
-    return ((v >> r) | (v << (VitSoloCfg::QB - r))) & M;
+    constexpr uint32_t M = (1u << QB) - 1u;
+    return ((v >> r) | (v << (QB - r))) & M;
 }
 __device__ __forceinline__ uint32_t vit_swz(uint32_t v) { return v ^ ((v >> 5) & 31u) ^ ((v >> 10) & 15u); }
 
-__global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(VitParams p)
+template <int KB>
+__global__ void __launch_bounds__(VitSoloCfg<KB>::THREADS, 1) viterbi_solo_kernel(VitParams p)
 {
-    using C = VitSoloCfg;
-    constexpr int K = C::K, KB = C::KB, Q = C::Q, NB = C::NB, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, QB = C::QB;
+    using C = VitSoloCfg<KB>;
+    constexpr int K = C::K, Q = C::Q, NB = C::NB, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, QB = C::QB;
+    constexpr int UNITS = C::UNITS, JPU = C::JPU, WB = C::WORD_BITS, ROWB = C::ROW_BYTES;
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = p.n;
@@ -62,8 +72,8 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
     Proto pr{1u, abort_flag, p.diag};
     const uint32_t tb_ready = smem_u32(smem + C::OFF_MBAR);      // [2] compute -> trace warp
     const uint32_t tb_done = tb_ready + 16u;                     // [2] trace warp -> compute
-    // backpointers of this CTA: [2 parities][n][NB] bytes
-    uint8_t *bp_base = p.bp + (size_t)blockIdx.x * 2 * (size_t)n * NB;
+    // backpointers of this CTA: [2 parities][n][ROWB] bytes
+    uint8_t *bp_base = p.bp + (size_t)blockIdx.x * 2 * (size_t)n * ROWB;
     const int nbits = C::LB + KB * (n - 1);
 
     if (tid == 0) {
@@ -83,14 +93,17 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
             const uint32_t par = it & 1u;
             pr.wait(tb_ready + 8u * par, (it >> 1) & 1u);
             if (!__all_sync(0xffffffffu, pr.live)) continue;     // a wait ran out: nothing valid to trace
-            const uint8_t *bp = bp_base + (size_t)par * n * NB;
+            const uint8_t *bp = bp_base + (size_t)par * n * ROWB;
             if (lane == 0) {
                 // predecessor of s at step t+1 is j*Q + (s >> k), j = branch stored for group s >> k
                 int s = best[par] & (C::S - 1);
                 path[n - 1] = s;
                 for (int t = n - 1; t >= 1; --t) {
                     const int q = s >> KB;
-                    const int j = (__ldcg(bp + (size_t)t * NB + (q >> KB)) >> (2 * (q & (K - 1)))) & (K - 1);
+                    unsigned word;
+                    if (WB == 8) word = __ldcg(bp + (size_t)t * ROWB + (q >> KB));
+                    else word = __ldcg(reinterpret_cast<const unsigned *>(bp + (size_t)t * ROWB) + (q >> KB));
+                    const int j = (int)(word >> (KB * (q & (K - 1)))) & (K - 1);
                     s = j * Q + q;
                     path[t - 1] = s;
                 }
@@ -124,18 +137,23 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
     } else {
         // ============================ compute warps ============================
         const uint32_t tm = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
-        // codebook -> TMEM: column 16 i + 4 j + l = c[j | x_i | l], x_i = tid*BPT + i
+        // codebook -> TMEM: column K*K*i + K*j + l = c[j | x_i | l], x_i = tid*BPT + i
 #pragma unroll
-        for (int i = 0; i < BPT; ++i) {
-            float2 v[8];
+        for (int i = 0; i < BPT; ++i)
 #pragma unroll
-            for (int j = 0; j < K; ++j) {
-                const float4 c4 = __ldg(reinterpret_cast<const float4 *>(p.cb + (size_t)j * Q + (size_t)(tid * BPT + i) * K));
-                v[2 * j] = make_float2(c4.x, c4.y);
-                v[2 * j + 1] = make_float2(c4.z, c4.w);
+            for (int u = 0; u < UNITS; ++u) {
+                float2 v[8];
+#pragma unroll
+                for (int jj = 0; jj < JPU; ++jj)
+#pragma unroll
+                    for (int l4 = 0; l4 < K; l4 += 4) {
+                        const float4 c4 = __ldg(reinterpret_cast<const float4 *>(
+                            p.cb + (size_t)(u * JPU + jj) * Q + (size_t)(tid * BPT + i) * K + l4));
+                        v[jj * (K / 2) + l4 / 2] = make_float2(c4.x, c4.y);
+                        v[jj * (K / 2) + l4 / 2 + 1] = make_float2(c4.z, c4.w);
+                    }
+                tmem_st16(tm + 16u * (i * UNITS + u), v);
             }
-            tmem_st16(tm + 16u * i, v);
-        }
         tmem_wait_st();
         uint32_t it = 0;
         for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x, ++it) {
@@ -143,7 +161,7 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
             const float *w = p.W + blk * n;
             // the backpointer buffer of this parity was last used two blocks ago: wait until traced
             if (it >= 2) pr.wait(tb_done + 8u * par, ((it >> 1) - 1u) & 1u);
-            uint8_t *bp = bp_base + (size_t)par * n * NB;
+            uint8_t *bp = bp_base + (size_t)par * n * ROWB;
             for (int q = tid; q < Q; q += CT) mv[q] = 0.0;           // mv_1 = 0: free first state
             compute_barrier(CT);
             for (int t = 1; t <= n; ++t) {
@@ -152,7 +170,7 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
                 const double wt = (double)__ldg(w + t - 1);
                 uint32_t SJ[K];
 #pragma unroll
-                for (int j = 0; j < K; ++j) SJ[j] = vit_swz(vit_rotr((uint32_t)j << (QB - KB), r));
+                for (int j = 0; j < K; ++j) SJ[j] = vit_swz(vit_rotr<QB>((uint32_t)j << (QB - KB), r));
                 unsigned long long bytes = 0ull;
                 double bv = 0.0;
                 int bi = 0x7fffffff;
@@ -160,50 +178,48 @@ __global__ void __launch_bounds__(VitSoloCfg::THREADS, 1) viterbi_solo_kernel(Vi
                 tmem_ld16(tm, cb[0]);
 #pragma unroll
                 for (int i = 0; i < BPT; ++i) {
-                    tmem_wait_ld(cb[i & 1]);
-                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
                     const uint32_t x = (uint32_t)(tid * BPT + i);
-                    const uint32_t sx = vit_swz(vit_rotr(x, r));
-                    double in[K];
+                    const uint32_t sx = vit_swz(vit_rotr<QB>(x, r));
+                    double in[K], bm[K];
+                    unsigned word = 0;                               // branch of output l in bits [KB*l, KB*l + KB)
 #pragma unroll
                     for (int j = 0; j < K; ++j) in[j] = mv[sx ^ SJ[j]];
-                    if (t < n) {
-                        double out[K];
-                        unsigned byte = 0;
 #pragma unroll
-                        for (int l = 0; l < K; ++l) {
-                            double bm = 0.0;
-                            int bj = 0;
+                    for (int u = 0; u < UNITS; ++u) {
+                        const int g = i * UNITS + u;
+                        tmem_wait_ld(cb[g & 1]);
+                        if (g + 1 < BPT * UNITS) tmem_ld16(tm + 16u * (g + 1), cb[(g + 1) & 1]);
 #pragma unroll
-                            for (int j = 0; j < K; ++j) {
-                                const float c = (l & 1) ? cb[i & 1][2 * j + (l >> 1)].y : cb[i & 1][2 * j + (l >> 1)].x;
-                                const double d = __dsub_rn(wt, (double)c);
-                                const double mm = __dadd_rn(in[j], __dmul_rn(d, d));
-                                if (j == 0 || mm < bm) { bm = mm; bj = j; }
-                            }
-                            out[l] = bm;
-                            byte |= (unsigned)bj << (2 * l);
-                        }
-                        // output [x|l] takes the slot of input [l|x]
-#pragma unroll
-                        for (int l = 0; l < K; ++l) mv[sx ^ SJ[l]] = out[l];
-                        bytes |= (unsigned long long)byte << (8 * i);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < K; ++j)
+                        for (int jj = 0; jj < JPU; ++jj) {
+                            const int j = u * JPU + jj;              // ascending: the lowest branch wins ties
 #pragma unroll
                             for (int l = 0; l < K; ++l) {
-                                const float c = (l & 1) ? cb[i & 1][2 * j + (l >> 1)].y : cb[i & 1][2 * j + (l >> 1)].x;
+                                const float2 cp = cb[g & 1][jj * (K / 2) + (l >> 1)];
+                                const float c = (l & 1) ? cp.y : cp.x;
                                 const double d = __dsub_rn(wt, (double)c);
                                 const double mm = __dadd_rn(in[j], __dmul_rn(d, d));
-                                const int s = (int)((uint32_t)j * Q + x * K + l);
-                                if (bi == 0x7fffffff || mm < bv || (mm == bv && s < bi)) { bv = mm; bi = s; }
+                                if (t < n) {
+                                    if (j == 0 || mm < bm[l]) {
+                                        bm[l] = mm;
+                                        word = (word & ~((unsigned)(K - 1) << (KB * l))) | ((unsigned)j << (KB * l));
+                                    }
+                                } else {
+                                    const int s = (int)((uint32_t)j * Q + x * K + l);
+                                    if (bi == 0x7fffffff || mm < bv || (mm == bv && s < bi)) { bv = mm; bi = s; }
+                                }
                             }
+                        }
+                    }
+                    if (t < n) {
+                        // output [x|l] takes the slot of input [l|x]
+#pragma unroll
+                        for (int l = 0; l < K; ++l) mv[sx ^ SJ[l]] = bm[l];
+                        bytes |= (unsigned long long)word << (WB * i);
                     }
                 }
                 if (t < n) {
                     // backpointers of step t+1 (row t): 8 contiguous bytes per thread
-                    *reinterpret_cast<unsigned long long *>(bp + (size_t)t * NB + (size_t)tid * BPT) = bytes;
+                    *reinterpret_cast<unsigned long long *>(bp + (size_t)t * ROWB + (size_t)tid * 8) = bytes;
                     compute_barrier(CT);
                 } else {
 #pragma unroll

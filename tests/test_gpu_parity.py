@@ -204,11 +204,13 @@ def test_large_trellis_ragged_lengths_and_block_counts(ctx, variant, n, B):
             ctx.set_option(k_, 0)
 
 
-def test_large_trellis_viterbi_many_blocks_per_cta(ctx):
+@pytest.mark.parametrize("k,n", [(2, 12), (3, 17)])
+def test_large_trellis_viterbi_many_blocks_per_cta(ctx, k, n):
     # more blocks than thread blocks: every CTA runs several blocks, alternating its two
     # backpointer buffers while the trace warp lags one block behind the dynamic programme
-    Lb, k, n = 16, 2, 12
-    W, c, _ = _rand(n, Lb, 450, seed=4200)
+    # (n = 17 at k = 3 takes the metric addresses once round their 13-step rotation period)
+    Lb = 16
+    W, c, _ = _rand(n, Lb, 450, seed=4200 + k)
     ref = oracle.viterbi(W, c, Lb, k)
     got = parity.gpu_viterbi(ctx, W, c, Lb, k)
     parity.assert_viterbi(got, ref, "viterbi 450 blocks")
