@@ -1,4 +1,4 @@
-"""ctypes front end of the float64 CPU oracle (``bcjr_oracle.c``).
+"""ctypes front end of the float64 CPU oracle (``bcjr_oracle.c``, ``bcjr_oracle_vec.c``).
 
 TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by ``__graft_entry__.smoke()`` and by
 ``bench.py``'s CPU-baseline leg.  The CUDA package never imports this module and this
@@ -17,16 +17,16 @@ from pathlib import Path
 import numpy as np
 
 _HERE = Path(__file__).resolve().parent
-_SRC = _HERE / "bcjr_oracle.c"
+_SRCS = [_HERE / "bcjr_oracle.c", _HERE / "bcjr_oracle_vec.c"]
 _LIB = _HERE / "libbcjr_oracle.so"
 _lib = None
 
 
 def build(force: bool = False) -> Path:
     """Compile the oracle with gcc (no fused multiply-add contraction, OpenMP over blocks)."""
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < max(f.stat().st_mtime for f in _SRCS):
         cmd = ["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
-               "-fPIC", "-shared", str(_SRC), "-o", str(_LIB), "-lm"]
+               "-fPIC", "-shared", *map(str, _SRCS), "-o", str(_LIB), "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 
@@ -49,6 +49,15 @@ def _load():
                                        ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
                                        ctypes.POINTER(ctypes.c_uint16), ctypes.POINTER(ctypes.c_float),
                                        ctypes.POINTER(ctypes.c_uint8), ctypes.c_int64, dp]
+        ci, c64, cd = ctypes.c_int, ctypes.c_int64, ctypes.c_double
+        lib.oracle_vec_soft_quantize.restype = ci
+        lib.oracle_vec_soft_quantize.argtypes = [dp, dp, ci, ci, ci, ci, c64, cd, dp, dp]
+        lib.oracle_vec_backward.restype = ci
+        lib.oracle_vec_backward.argtypes = [dp, dp, dp, ci, ci, ci, ci, c64, cd, dp, dp]
+        lib.oracle_vec_viterbi.restype = ci
+        lib.oracle_vec_viterbi.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                           ci, ci, ci, ci, c64, ctypes.POINTER(ctypes.c_uint16),
+                                           ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_uint8), c64, dp]
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
         _lib = lib
@@ -137,6 +146,50 @@ def viterbi(W, c, Lb, k):
                               states.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16)),
                               hard.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
                               bits.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)), nb, _dptr(cost)))
+    return {"states": states, "hard": hard, "path_bits": bits, "cost": cost}
+
+
+# ---- vector emissions: state s emits the V numbers c[s, :], a step consumes V weights and kb bits
+def soft_quantize_vec(W, c, Lb, kb, V, T):
+    """W: [B, n] (n a multiple of V), c: [S, V].  Returns dict(soft [B,n], logZ [B])."""
+    lib = _load()
+    W = _f64(W); c = _f64(c)
+    B, n = W.shape
+    assert c.shape == (1 << Lb, V)
+    set_threads(Lb, n // V, B, arrays_per_thread=2)
+    soft = np.empty((B, n)); logZ = np.empty(B)
+    _check(lib.oracle_vec_soft_quantize(_dptr(W), _dptr(c), Lb, kb, V, n, B, float(T), _dptr(soft), _dptr(logZ)))
+    return {"soft": soft, "logZ": logZ}
+
+
+def backward_vec(W, c, g, Lb, kb, V, T):
+    """Gradients of sum(g * soft): grad_W [B,n], grad_codebook [S,V] (summed over blocks)."""
+    lib = _load()
+    W = _f64(W); c = _f64(c); g = _f64(g)
+    B, n = W.shape
+    assert g.shape == W.shape and c.shape == (1 << Lb, V)
+    set_threads(Lb, n // V, B, arrays_per_thread=5)
+    gW = np.empty((B, n)); gc = np.empty((1 << Lb, V))
+    _check(lib.oracle_vec_backward(_dptr(W), _dptr(c), _dptr(g), Lb, kb, V, n, B, float(T), _dptr(gW), _dptr(gc)))
+    return {"grad_W": gW, "grad_codebook": gc}
+
+
+def viterbi_vec(W, c, Lb, kb, V):
+    """Hard code.  Returns dict(states [B, n/V] u16, hard [B,n] f32, path_bits [B,nbytes] u8, cost [B])."""
+    lib = _load()
+    W = np.ascontiguousarray(W, dtype=np.float32); c = np.ascontiguousarray(c, dtype=np.float32)
+    B, n = W.shape
+    assert c.shape == (1 << Lb, V) and n % V == 0
+    nt = n // V
+    set_threads(Lb, nt, B, arrays_per_thread=1)
+    nb = path_bytes(Lb, kb, nt)
+    states = np.empty((B, nt), dtype=np.uint16); hard = np.empty((B, n), dtype=np.float32)
+    bits = np.zeros((B, nb), dtype=np.uint8); cost = np.empty(B)
+    _check(lib.oracle_vec_viterbi(W.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+                                  c.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), Lb, kb, V, n, B,
+                                  states.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16)),
+                                  hard.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+                                  bits.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)), nb, _dptr(cost)))
     return {"states": states, "hard": hard, "path_bits": bits, "cost": cost}
 
 

@@ -82,3 +82,43 @@ def pack_path_bits(states, Lb, k):
         if b:
             out[i >> 3] |= 1 << (7 - (i & 7))
     return out
+
+
+# ---------------------------------------------------------------- vector emissions (V numbers per step)
+def vec_soft_codeword(w, c, Lb, kb, V, T, paths=None):
+    """w: [n], c: [S, V]; a step consumes V weights and kb bits.  Returns (soft [n], logZ)."""
+    w = np.asarray(w, dtype=np.float64).reshape(-1, V); c = np.asarray(c, dtype=np.float64)
+    nt = w.shape[0]
+    if paths is None:
+        paths = enumerate_paths(Lb, kb, nt)
+    emitted = c[paths]                                        # [P, nt, V]
+    E = 0.5 * ((w[None] - emitted) ** 2).sum(axis=(1, 2))
+    m = (-E / T).max()
+    p = np.exp(-E / T - m)
+    Z = p.sum()
+    soft = (p[:, None, None] * emitted).sum(axis=0) / Z
+    return soft.reshape(-1), m + np.log(Z)
+
+
+def vec_fd_gradients(w, c, g, Lb, kb, V, T, h=1e-6):
+    w = np.asarray(w, dtype=np.float64).copy(); c = np.asarray(c, dtype=np.float64).copy()
+    g = np.asarray(g, dtype=np.float64)
+    paths = enumerate_paths(Lb, kb, len(w) // V)
+    f = lambda ww, cc: float(np.dot(g, vec_soft_codeword(ww, cc, Lb, kb, V, T, paths)[0]))
+    gw = np.zeros_like(w); gc = np.zeros_like(c)
+    for i in range(len(w)):
+        wp = w.copy(); wp[i] += h; wm = w.copy(); wm[i] -= h
+        gw[i] = (f(wp, c) - f(wm, c)) / (2 * h)
+    for u in range(c.shape[0]):
+        for v in range(V):
+            cp = c.copy(); cp[u, v] += h; cm = c.copy(); cm[u, v] -= h
+            gc[u, v] = (f(w, cp) - f(w, cm)) / (2 * h)
+    return gw, gc
+
+
+def vec_best_path(w, c, Lb, kb, V):
+    w = np.asarray(w, dtype=np.float64).reshape(-1, V); c = np.asarray(c, dtype=np.float64)
+    paths = enumerate_paths(Lb, kb, w.shape[0])
+    cost = ((w[None] - c[paths]) ** 2).sum(axis=(1, 2))
+    order = np.argsort(cost, kind="stable")
+    return paths[order[0]], cost[order[0]], cost[order[1]] - cost[order[0]]
