@@ -31,18 +31,18 @@ from paper_2605_10655_b200 import shard, synth  # noqa: E402
 METRIC = "bcjr_fwd_bwd_trellis_edge_updates_per_s"
 UNIT = "edges/s"
 WORKLOADS = {"tiny": synth.tiny, "mid": synth.mid, "q_proj": synth.q_proj, "layer": synth.decoder_layer,
-             "gate_k3": synth.gate_k3}
+             "gate_k3": synth.gate_k3, "qtip_v2": synth.qtip_v2}
 # (Lb, k, kernel) -> measured DRAM bytes per weight block (n = 256), see profiles/*.md
 NCU_DRAM_BYTES_PER_BLOCK = {(16, 2, "bwd"): 66.3e6, (16, 2, "fwd"): 33.1e6}
 MUFU_PER_CLK_PER_SM = 16          # special-function results per clock per SM (CUDA throughput table, cc 10.0)
 NUM_SMS = 148
 
 
-def mufu_ops_per_state_step(k: int, kernel: str) -> float:
+def mufu_ops_per_state_step(k: int, kernel: str, V: int = 1) -> float:
     """Algorithmic special-function operations per state per step (one ex2 per state, plus per
     group of K states: one lg2; the beta sweeps add one ex2 per group for the posterior; the
     backward-pass sweeps add one rcp per group for the conditional expectation)."""
-    K = 1 << k
+    K = 1 << (k * V)
     fwd = (1 + 1 / K) + (1 + 2 / K)
     bwd = (1 + 2 / K) + (1 + 3 / K)
     return {"fwd": fwd, "bwd": bwd, "both": fwd + bwd}[kernel]
@@ -107,11 +107,15 @@ def cpu_baseline(wl, seconds_hint: float = 20.0):
     nblk = max(1, min(wl.num_blocks(), 4 * cores * min(scale, 64)))
     W, c, g = wl.weights(0)[:nblk], wl.codebook(), wl.upstream(0)[:nblk]
     t0 = time.time()
-    oracle.soft_quantize(W, c, wl.Lb, wl.k, wl.T)
-    oracle.backward(W, c, g, wl.Lb, wl.k, wl.T)
+    if wl.V == 1:
+        oracle.soft_quantize(W, c, wl.Lb, wl.k, wl.T)
+        oracle.backward(W, c, g, wl.Lb, wl.k, wl.T)
+    else:
+        oracle.soft_quantize_vec(W, c, wl.Lb, wl.k * wl.V, wl.V, wl.T)
+        oracle.backward_vec(W, c, g, wl.Lb, wl.k * wl.V, wl.V, wl.T)
     dt = time.time() - t0
     threads = oracle.num_threads()
-    edges = 2 * nblk * wl.n * wl.S * wl.K
+    edges = 2 * nblk * wl.steps * wl.S * wl.K
     return {"value": edges / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"{nblk} blocks of {wl.name} (n={wl.n}, Lb={wl.Lb}, k={wl.k}, T={wl.T}), "
                       f"forward+backward, {dt:.1f} s"}, dt
@@ -199,12 +203,12 @@ def main():
     total_steps = args.warmup + args.steps
     temps = anneal_schedule(0.3, 0.01, total_steps) if wl.name.startswith("llama32_1b_decoder") else [wl.T] * total_steps
     nblocks = sum(m["W"].shape[0] for m in mats)
-    edges_per_step = 2 * nblocks * wl.n * wl.S * wl.K
+    edges_per_step = 2 * nblocks * wl.steps * wl.S * wl.K
     for m in mats:
         m["soft"] = torch.empty_like(m["W"]); m["gW"] = torch.empty_like(m["W"])
         m["g"] = torch.empty_like(m["W"])
-    gc = torch.empty(wl.S, dtype=torch.float32, device=dev)
-    gc_total = torch.zeros(wl.S, dtype=torch.float32, device=dev)
+    gc = torch.empty(wl.S * wl.V, dtype=torch.float32, device=dev)
+    gc_total = torch.zeros(wl.S * wl.V, dtype=torch.float32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # > L2 (126 MB)
     gen = torch.Generator(device=dev)
 
@@ -218,7 +222,10 @@ def main():
         for m in mats:
             if ev is not None:
                 ev["f0"].append(torch.cuda.Event(enable_timing=True)); ev["f0"][-1].record()
-            ctx.bcjr_soft_quantize(m["W"], cb, wl.Lb, wl.k, wl.n, T, soft=m["soft"])
+            if wl.V == 1:
+                ctx.bcjr_soft_quantize(m["W"], cb, wl.Lb, wl.k, wl.n, T, soft=m["soft"])
+            else:
+                ctx.bcjr_soft_quantize_vec(m["W"], cb, wl.Lb, wl.k, wl.V, wl.n, T, soft=m["soft"])
             if ev is not None:
                 ev["f1"].append(torch.cuda.Event(enable_timing=True)); ev["f1"][-1].record()
             ctx.bcjr_backward(m["g"], grad_W=m["gW"], grad_codebook=gc)
@@ -267,21 +274,26 @@ def main():
     # ---- Viterbi leg (same workload, same run)
     vit = None
     if not args.no_viterbi:
-        ctx.viterbi_hard(mats[0]["W"], cb, wl.Lb, wl.k, wl.n)      # warm-up
+        def vit_call(Wd):
+            if wl.V == 1:
+                ctx.viterbi_hard(Wd, cb, wl.Lb, wl.k, wl.n)
+            else:
+                ctx.viterbi_hard_vec(Wd, cb, wl.Lb, wl.k, wl.V, wl.n)
+        vit_call(mats[0]["W"])                                      # warm-up
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         flush.zero_()
         e0.record()
         for m in mats:
-            ctx.viterbi_hard(m["W"], cb, wl.Lb, wl.k, wl.n)
+            vit_call(m["W"])
         e1.record()
         torch.cuda.synchronize()
         vms = e0.elapsed_time(e1)
-        vit = {"ms": vms, "edges_per_s": nblocks * wl.n * wl.S * wl.K / (vms * 1e-3)}
+        vit = {"ms": vms, "edges_per_s": nblocks * wl.steps * wl.S * wl.K / (vms * 1e-3)}
 
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and wl.V == 1:          # the host-buffer entry point covers the scalar trellis
         host = []
         for m in mats:
             host.append({"W": m["W_host"], "g": m["g"].cpu().pin_memory(),
@@ -314,17 +326,17 @@ def main():
                "d2h_bytes_per_step": 2 * wbytes + len(host) * wl.S * 4}
 
     # ---- roofline of the dominant kernel (the backward-pass kernel): special-function pipe
-    state_steps = nblocks * wl.n * wl.S
+    state_steps = nblocks * wl.steps * wl.S
     dom = "bwd" if bwd_ms >= fwd_ms else "fwd"
     dom_ms = (bwd_ms if dom == "bwd" else fwd_ms) / (args.steps * len(mats))
-    ops = mufu_ops_per_state_step(wl.k, dom) * state_steps / len(mats)
+    ops = mufu_ops_per_state_step(wl.k, dom, wl.V) * state_steps / len(mats)
     achieved = ops / (dom_ms * 1e-3) / 1e9
     sm_max = clocks.get("sm_max_mhz") or 1965.0
     peak = NUM_SMS * MUFU_PER_CLK_PER_SM * sm_max * 1e6 / 1e9
     # DRAM bytes per block of the dominant kernel, from the ncu captures summarised under profiles/
     # (dram__bytes_read.sum + dram__bytes_write.sum of one launch / blocks of that launch, small
     # case of the same kernel; traffic grows in proportion to the number of blocks)
-    per_block = NCU_DRAM_BYTES_PER_BLOCK.get((wl.Lb, wl.k, dom)) if diag.last_path else None
+    per_block = NCU_DRAM_BYTES_PER_BLOCK.get((wl.Lb, wl.k, dom)) if diag.last_path and wl.V == 1 else None
     traffic = per_block * nblocks / len(mats) if per_block else None
     hbm_peak = None
     try:
@@ -341,7 +353,7 @@ def main():
                 "frac": achieved / peak, "traffic": traffic,
                 "peak_source": f"{NUM_SMS} SMs x {MUFU_PER_CLK_PER_SM} MUFU/clk x {sm_max:.0f} MHz (derived)",
                 "avg_launch_ms": dom_ms, "hbm": hbm,
-                "whole_step_frac": mufu_ops_per_state_step(wl.k, "both") * state_steps / (ms_per_step * 1e-3) / 1e9 / peak}
+                "whole_step_frac": mufu_ops_per_state_step(wl.k, "both", wl.V) * state_steps / (ms_per_step * 1e-3) / 1e9 / peak}
 
     if rank == 0:
         base = None
@@ -351,7 +363,7 @@ def main():
                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                "config": {"workload": wl.name, "matrices": [m["name"] for m in mats], "blocks": nblocks, "n": wl.n,
-                          "Lb": wl.Lb, "k": wl.k, "T": [temps[args.warmup], temps[-1]],
+                          "Lb": wl.Lb, "k": wl.k, "V": wl.V, "T": [temps[args.warmup], temps[-1]],
                           "l2": "256 MB flush write between timed steps; per-step working set >> L2",
                           "path": "cluster" if diag.last_path else "generic"},
                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": base,

@@ -121,6 +121,31 @@ bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook,
                          uint16_t *states, float *hard, void *cuda_stream);
 
 /*
+ * Vector emissions (the paper's "L=16, k=2, V=2" configuration, Section 3.1 and Section 4
+ * "Quantization configuration"; its kernel section's 128-step, 16-predecessor recursion): every
+ * state emits V numbers, a trellis step consumes V weights and k*V input bits,
+ *     s' = ((s << kV) | b) mod 2^Lb,   e_t(s) = -(1/(2T)) sum_v (w[V t + v] - codebook[s*V + v])^2,
+ *     soft[V t + v] = sum_s codebook[s*V + v] gamma_t(s).
+ * The paper writes only the scalar emission; this vector form is the reading taken here.
+ *   codebook   device in  [2^Lb * V], row s = the V numbers state s emits
+ *   n          weights per block, a multiple of V (n / V trellis steps)
+ *   k, V       V = 1 forwards to the scalar call; V = 2 with k = 1 or 2 is supported, anything else
+ *              returns BCJR_EUNSUPPORTED.  With V = 2 every array must be 8-byte aligned (BCJR_EINVAL).
+ * A following bcjr_backward then expects/returns grad_codebook as [2^Lb * V].
+ * viterbi_hard_vec: states [num_blocks * n/V] uint16, hard [num_blocks * n] (the emitted numbers),
+ * path bits Lb + kV (n/V - 1) per block in the layout of viterbi_hard; squared error summed over
+ * the V components in IEEE double, components added in order, no fused multiply-add.
+ * Otherwise as bcjr_soft_quantize / viterbi_hard.
+ */
+bcjr_status bcjr_soft_quantize_vec(bcjr_ctx *ctx, const float *W, const float *codebook,
+                                   int Lb, int k, int V, int n, int64_t num_blocks, float T,
+                                   float *soft, float *logZ, void *cuda_stream);
+bcjr_status viterbi_hard_vec(bcjr_ctx *ctx, const float *W, const float *codebook,
+                             int Lb, int k, int V, int n, int64_t num_blocks,
+                             uint8_t *path_bits, int64_t path_stride_bytes,
+                             uint16_t *states, float *hard, void *cuda_stream);
+
+/*
  * BCJR-STE forward (Section 3.7, "BCJR-STE variant"): the value that goes forward is the hard
  * Viterbi codeword, while the state saved on the context is that of the temperature-T relaxation,
  * so that a following bcjr_backward returns the gradient of the finite-temperature soft codeword

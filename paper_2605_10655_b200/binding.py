@@ -13,7 +13,7 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libbcjr_b200.so"
 
 EXPORTS = ["bcjr_create", "bcjr_destroy", "bcjr_set_option", "bcjr_soft_quantize", "bcjr_backward",
-           "viterbi_hard", "bcjr_ste_forward", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
+           "viterbi_hard", "bcjr_soft_quantize_vec", "viterbi_hard_vec", "bcjr_ste_forward", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
            "bcjr_last_cuda_error", "bcjr_status_string", "bcjr_soft_quantize_static",
            "bcjr_static_scratch_bytes"]
 
@@ -50,6 +50,10 @@ def load_library() -> ctypes.CDLL:
     lib.bcjr_soft_quantize.argtypes = [vp, vp, vp, i, i, i, i64, f, vp, vp, vp]
     lib.bcjr_backward.restype = i; lib.bcjr_backward.argtypes = [vp, vp, vp, vp, vp]
     lib.viterbi_hard.restype = i; lib.viterbi_hard.argtypes = [vp, vp, vp, i, i, i, i64, vp, i64, vp, vp, vp]
+    lib.bcjr_soft_quantize_vec.restype = i
+    lib.bcjr_soft_quantize_vec.argtypes = [vp, vp, vp, i, i, i, i, i64, f, vp, vp, vp]
+    lib.viterbi_hard_vec.restype = i
+    lib.viterbi_hard_vec.argtypes = [vp, vp, vp, i, i, i, i, i64, vp, i64, vp, vp, vp]
     lib.bcjr_ste_forward.restype = i
     lib.bcjr_ste_forward.argtypes = [vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
     lib.bcjr_step_host.restype = i
@@ -170,10 +174,10 @@ class Context:
         if grad_W is None:
             grad_W = torch.empty_like(W)
         if grad_codebook is None:
-            grad_codebook = torch.empty(1 << Lb, dtype=torch.float32, device=W.device)
+            grad_codebook = torch.empty(codebook.numel(), dtype=torch.float32, device=W.device)
         rc = self._lib.bcjr_backward(self._h, _dev(grad_soft, torch.float32, numel, "grad_soft"),
                                      _dev(grad_W, torch.float32, numel, "grad_W"),
-                                     _dev(grad_codebook, torch.float32, 1 << Lb, "grad_codebook"),
+                                     _dev(grad_codebook, torch.float32, codebook.numel(), "grad_codebook"),
                                      _stream_ptr(stream))
         self._check(rc, "bcjr_backward")
         return grad_W, grad_codebook
@@ -192,6 +196,40 @@ class Context:
                                     ctypes.c_void_p(states.data_ptr()) if want_states else None,
                                     ctypes.c_void_p(hard.data_ptr()) if want_hard else None, _stream_ptr(stream))
         self._check(rc, "viterbi_hard")
+        return bits, states, hard
+
+    def bcjr_soft_quantize_vec(self, W, codebook, Lb, k, V, n, T, soft=None, logZ=None, stream=None):
+        """Vector emissions: codebook [2^Lb, V], a step consumes V weights.  Returns (soft, logZ)."""
+        import torch
+        B = W.numel() // n
+        if B * n != W.numel():
+            raise ValueError("W.numel() must be a multiple of n")
+        if soft is None:
+            soft = torch.empty_like(W)
+        if logZ is None:
+            logZ = torch.empty(B, dtype=torch.float32, device=W.device)
+        rc = self._lib.bcjr_soft_quantize_vec(self._h, _dev(W, torch.float32, name="W"),
+                                              _dev(codebook, torch.float32, (1 << Lb) * V, "codebook"), Lb, k, V, n, B,
+                                              float(T), _dev(soft, torch.float32, B * n, "soft"),
+                                              _dev(logZ, torch.float32, B, "logZ"), _stream_ptr(stream))
+        self._check(rc, "bcjr_soft_quantize_vec")
+        self._saved = (W, codebook, Lb, B * n)
+        return soft, logZ
+
+    def viterbi_hard_vec(self, W, codebook, Lb, k, V, n, want_states=True, want_hard=True, stream=None):
+        """Returns (path_bits [B, nbytes], states [B, n/V] or None, hard [B, n] or None)."""
+        import torch
+        B = W.numel() // n
+        nb = path_bytes(Lb, k * V, n // V)
+        bits = torch.empty((B, nb), dtype=torch.uint8, device=W.device)
+        states = torch.empty((B, n // V), dtype=torch.int16, device=W.device) if want_states else None
+        hard = torch.empty((B, n), dtype=torch.float32, device=W.device) if want_hard else None
+        rc = self._lib.viterbi_hard_vec(self._h, _dev(W, torch.float32, name="W"),
+                                        _dev(codebook, torch.float32, (1 << Lb) * V, "codebook"), Lb, k, V, n, B,
+                                        ctypes.c_void_p(bits.data_ptr()), nb,
+                                        ctypes.c_void_p(states.data_ptr()) if want_states else None,
+                                        ctypes.c_void_p(hard.data_ptr()) if want_hard else None, _stream_ptr(stream))
+        self._check(rc, "viterbi_hard_vec")
         return bits, states, hard
 
     def bcjr_ste_forward(self, W, codebook, Lb, k, n, T, want_states=False, want_soft=False, stream=None):

@@ -12,6 +12,7 @@
 #include "bcjr_generic.cuh"
 #ifndef BCJR_NO_CLUSTER
 #include "bcjr_cluster.cuh"
+#include "bcjr_vec.cuh"
 #include "bcjr_solo.cuh"
 #include "bcjr_duo.cuh"
 #include "bcjr_viterbi.cuh"
@@ -40,6 +41,7 @@ struct bcjr_ctx {
     bool have_fwd = false;
     const float *W = nullptr, *cb = nullptr;
     int Lb = 0, k = 0, n = 0;
+    int V = 1;                 // numbers emitted per state and step by the saved forward call
     int64_t B = 0;
     float T = 0.f;
     // options
@@ -98,10 +100,11 @@ struct GenericLaunch {
 };
 
 template <typename Kern>
-bcjr_status plan_generic(bcjr_ctx *ctx, Kern kern, int Q, size_t msg_bytes, int64_t B, GenericLaunch *out)
+bcjr_status plan_generic(bcjr_ctx *ctx, Kern kern, int Q, size_t msg_bytes, int64_t B, GenericLaunch *out,
+                         int header_floats = GEN_SMEM_HEADER)
 {
     out->threads = generic_threads(Q);
-    const size_t header = GEN_SMEM_HEADER * sizeof(float);
+    const size_t header = (size_t)header_floats * sizeof(float);
     const size_t budget = (size_t)ctx->max_smem_optin - 1024;
     out->msg_global = header + msg_bytes > budget;
     out->smem = out->msg_global ? header : header + msg_bytes;
@@ -180,6 +183,80 @@ bcjr_status launch_vit_generic(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
     CU(cudaGetLastError());
     return BCJR_OK;
 }
+
+// ---- vector emissions (V weights per step, KB = k V bits per step): one CTA per block
+template <int KB, int V>
+bcjr_status launch_fwd_vec(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    const int Q = 1 << (p.Lb - KB), nt = p.n / V;
+    GenericLaunch gl;
+    bcjr_status rc = plan_generic(ctx, fwd_vec_kernel<KB, V>, Q, (size_t)2 * Q * 4, p.B, &gl, VEC_SMEM_HEADER);
+    if (rc) return rc;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)gl.grid * nt * Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, (size_t)gl.grid * (nt + 2) * 4))) return rc;
+    if (gl.msg_global && (rc = ensure(ctx, ctx->msg, (size_t)gl.grid * 2 * Q * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    p.msg = gl.msg_global ? (float *)ctx->msg.ptr : nullptr;
+    fwd_vec_kernel<KB, V><<<gl.grid, gl.threads, gl.smem, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+template <int KB, int V>
+bcjr_status launch_bwd_vec(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    const int S = 1 << p.Lb, Q = S >> KB, nt = p.n / V;
+    GenericLaunch gl;
+    bcjr_status rc = plan_generic(ctx, bwd_vec_kernel<KB, V>, Q, (size_t)4 * Q * 4, p.B, &gl, VEC_SMEM_HEADER);
+    if (rc) return rc;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)gl.grid * 2 * nt * Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, (size_t)gl.grid * (nt + 2) * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->gc_part, (size_t)gl.grid * S * V * 4))) return rc;
+    if (gl.msg_global && (rc = ensure(ctx, ctx->msg, (size_t)gl.grid * 4 * Q * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    p.gc_part = (float *)ctx->gc_part.ptr;
+    p.msg = gl.msg_global ? (float *)ctx->msg.ptr : nullptr;
+    bwd_vec_kernel<KB, V><<<gl.grid, gl.threads, gl.smem, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    if (grad_codebook) {
+        reduce_gc_kernel<<<(S * V + 255) / 256, 256, 0, st>>>(p.gc_part, gl.grid, S * V, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
+template <int KB, int V>
+bcjr_status launch_vit_vec(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
+{
+    const int Q = 1 << (p.Lb - KB), nt = p.n / V;
+    GenericLaunch gl;
+    bcjr_status rc = plan_generic(ctx, viterbi_vec_kernel<KB, V>, Q, (size_t)2 * Q * 8, p.B, &gl, VEC_SMEM_HEADER);
+    if (rc) return rc;
+    if ((rc = ensure(ctx, ctx->bp, (size_t)gl.grid * nt * Q))) return rc;
+    if ((rc = ensure(ctx, ctx->path_ws, (size_t)gl.grid * nt * 4))) return rc;
+    if (gl.msg_global && (rc = ensure(ctx, ctx->msg, (size_t)gl.grid * 2 * Q * 8))) return rc;
+    p.bp = (uint8_t *)ctx->bp.ptr;
+    p.path_ws = (int *)ctx->path_ws.ptr;
+    p.msg = gl.msg_global ? (double *)ctx->msg.ptr : nullptr;
+    viterbi_vec_kernel<KB, V><<<gl.grid, gl.threads, gl.smem, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+// V = 2 only: (k, V) = (1, 2) and (2, 2); every array that is read two floats at a time must be 8-byte aligned
+bcjr_status check_vec(int Lb, int k, int V, int n, int64_t B)
+{
+    if (V < 1 || k < 1 || n < 1 || B < 0 || n % V) return BCJR_EINVAL;
+    if (V != 2 || k > 2) return BCJR_EUNSUPPORTED;
+    return check_dims(Lb, k * V, n / V, B);
+}
+bool aligned8(const void *p) { return ((uintptr_t)p & 7u) == 0; }
 
 #ifndef BCJR_NO_CLUSTER
 #ifndef FWD_THREADS_K2
@@ -459,6 +536,7 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
     ctx->have_fwd = false;
     if (num_blocks == 0) {
         ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = 0; ctx->T = T;
+        ctx->V = 1;
         ctx->have_fwd = true;
         return BCJR_OK;
     }
@@ -489,6 +567,7 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
     if (rc) return rc;
     ctx->last_path = use_cluster ? 1 : 0;
     ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = num_blocks; ctx->T = T;
+    ctx->V = 1;
     ctx->have_fwd = true;
     return BCJR_OK;
 }
@@ -504,7 +583,7 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int S = 1 << ctx->Lb;
     if (ctx->B == 0) {
-        if (grad_codebook) CU(cudaMemsetAsync(grad_codebook, 0, (size_t)S * 4, st));
+        if (grad_codebook) CU(cudaMemsetAsync(grad_codebook, 0, (size_t)S * ctx->V * 4, st));
         return BCJR_OK;
     }
     BwdParams p{};
@@ -513,6 +592,13 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
     p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)ctx->T));
     p.invT = (float)(1.0 / (double)ctx->T);
     bcjr_status rc = BCJR_OK;
+    if (ctx->V == 2) {                                   // saved by bcjr_soft_quantize_vec: k bits per weight
+        if (!aligned8(grad_soft) || !aligned8(grad_W)) return BCJR_EINVAL;
+        rc = ctx->k == 1 ? launch_bwd_vec<2, 2>(ctx, p, grad_codebook, st) : launch_bwd_vec<4, 2>(ctx, p, grad_codebook, st);
+        if (rc) return rc;
+        ctx->last_path = 0;
+        return BCJR_OK;
+    }
     bool use_cluster = false;
 #ifndef BCJR_NO_CLUSTER
     use_cluster = ctx->opt_path != 1 && cluster_supported(ctx->Lb, ctx->k);
@@ -575,6 +661,62 @@ bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook, i
     }
     if (rc) return rc;
     ctx->last_path = use_large ? 1 : 0;
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_soft_quantize_vec(bcjr_ctx *ctx, const float *W, const float *codebook, int Lb, int k, int V,
+                                   int n, int64_t num_blocks, float T, float *soft, float *logZ, void *cuda_stream)
+{
+    if (!ctx) return BCJR_EINVAL;
+    if (V == 1) return bcjr_soft_quantize(ctx, W, codebook, Lb, k, n, num_blocks, T, soft, logZ, cuda_stream);
+    if (!(T > 0.f) || !std::isfinite(T)) return BCJR_EINVAL;
+    bcjr_status rc = check_vec(Lb, k, V, n, num_blocks);
+    if (rc) return rc;
+    if (num_blocks > 0 && (!W || !codebook || !soft)) return BCJR_EINVAL;
+    if (!aligned8(W) || !aligned8(codebook) || !aligned8(soft)) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    ctx->have_fwd = false;
+    if (num_blocks > 0) {
+        if ((rc = ensure(ctx, ctx->soft_copy, (size_t)num_blocks * n * 4))) return rc;
+        FwdParams p{};
+        p.W = W; p.cb = codebook; p.soft = soft; p.soft_copy = (float *)ctx->soft_copy.ptr; p.logZ = logZ;
+        p.diag = ctx->diag; p.B = num_blocks; p.Lb = Lb; p.n = n;
+        p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)T));
+        rc = k == 1 ? launch_fwd_vec<2, 2>(ctx, p, st) : launch_fwd_vec<4, 2>(ctx, p, st);
+        if (rc) return rc;
+        ctx->last_path = 0;
+    }
+    ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = num_blocks; ctx->T = T;
+    ctx->V = V;
+    ctx->have_fwd = true;
+    return BCJR_OK;
+}
+
+bcjr_status viterbi_hard_vec(bcjr_ctx *ctx, const float *W, const float *codebook, int Lb, int k, int V, int n,
+                             int64_t num_blocks, uint8_t *path_bits, int64_t path_stride_bytes, uint16_t *states,
+                             float *hard, void *cuda_stream)
+{
+    if (!ctx) return BCJR_EINVAL;
+    if (V == 1)
+        return viterbi_hard(ctx, W, codebook, Lb, k, n, num_blocks, path_bits, path_stride_bytes, states, hard, cuda_stream);
+    bcjr_status rc = check_vec(Lb, k, V, n, num_blocks);
+    if (rc) return rc;
+    if (num_blocks > 0 && (!W || !codebook)) return BCJR_EINVAL;
+    if (!aligned8(W) || !aligned8(codebook)) return BCJR_EINVAL;
+    const int64_t nbits = Lb + (int64_t)k * V * (n / V - 1);
+    if (path_bits && path_stride_bytes < (nbits + 7) / 8) return BCJR_EINVAL;
+    if (num_blocks == 0) return BCJR_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    VitParams p{};
+    p.W = W; p.cb = codebook; p.path_bits = path_bits; p.path_stride = path_stride_bytes;
+    p.states = states; p.hard = hard; p.B = num_blocks; p.Lb = Lb; p.n = n;
+    rc = k == 1 ? launch_vit_vec<2, 2>(ctx, p, st) : launch_vit_vec<4, 2>(ctx, p, st);
+    if (rc) return rc;
+    ctx->last_path = 0;
     return BCJR_OK;
 }
 

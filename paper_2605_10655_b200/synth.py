@@ -20,9 +20,10 @@ import numpy as np
 BLOCK_N = 256  # weights per trellis block in the Llama-shaped workloads
 
 
-def codebook(Lb: int, seed: int = 0) -> np.ndarray:
-    """Emission table c[s], s in [0, 2^Lb): iid N(0,1), float32."""
-    return np.random.default_rng(seed).standard_normal(1 << Lb).astype(np.float32)
+def codebook(Lb: int, seed: int = 0, V: int = 1) -> np.ndarray:
+    """Emission table c[s], s in [0, 2^Lb): iid N(0,1), float32; [2^Lb, V] when a state emits V numbers."""
+    shape = (1 << Lb,) if V == 1 else (1 << Lb, V)
+    return np.random.default_rng(seed).standard_normal(shape).astype(np.float32)
 
 
 def gaussian(shape, seed: int) -> np.ndarray:
@@ -49,6 +50,7 @@ class Workload:
     c_seed: int = 0
     dist: str = "normal"
     extra_T: Tuple[float, ...] = field(default_factory=tuple)
+    V: int = 1                 # numbers emitted per state and step (a step consumes V weights, k*V bits)
 
     @property
     def S(self) -> int:
@@ -56,17 +58,21 @@ class Workload:
 
     @property
     def K(self) -> int:
-        return 1 << self.k
+        return 1 << (self.k * self.V)
+
+    @property
+    def steps(self) -> int:
+        return self.n // self.V
 
     def num_blocks(self) -> int:
         return sum(r * c // self.n for _, (r, c) in self.matrices)
 
     def edges_per_sweep(self) -> int:
         """Trellis-edge updates of one sweep: blocks * steps * states * branches."""
-        return self.num_blocks() * self.n * self.S * self.K
+        return self.num_blocks() * self.steps * self.S * self.K
 
     def codebook(self) -> np.ndarray:
-        return codebook(self.Lb, self.c_seed)
+        return codebook(self.Lb, self.c_seed, self.V)
 
     def weights(self, idx: int = 0) -> np.ndarray:
         """Matrix `idx` as [num_blocks, n] (row-major split of each row into blocks of n)."""
@@ -114,6 +120,13 @@ def gate_k3() -> Workload:
     return Workload("gate_student_t_3bpw", Lb=16, k=3, n=BLOCK_N, T=0.01,
                     matrices=[("gate_proj", (8192, 2048))], w_seed=5001, g_seed=5501,
                     dist="student_t", extra_T=(0.01, 0.001))
+
+
+def qtip_v2() -> Workload:
+    # the paper's own trellis configuration (16 state bits, 2 bits per weight, 2 weights per step:
+    # 128 steps per 256-weight block, 16 predecessors per state) on the q_proj shape
+    return Workload("llama32_1b_q_proj_v2", Lb=16, k=2, n=BLOCK_N, T=0.1,
+                    matrices=[("q_proj", (2048, 2048))], w_seed=6001, g_seed=6501, V=2)
 
 
 def sample_blocks(num_blocks: int, count: int, seed: int = 99) -> np.ndarray:

@@ -35,6 +35,8 @@ def test_status_strings_and_host_side_argument_checks():
     assert lib.bcjr_soft_quantize(None, None, None, 8, 2, 64, 1, 0.5, None, None, None) == -1
     assert lib.bcjr_backward(None, None, None, None, None) == -1
     assert lib.viterbi_hard(None, None, None, 8, 2, 64, 1, None, 0, None, None, None) == -1
+    assert lib.bcjr_soft_quantize_vec(None, None, None, 8, 2, 2, 64, 1, 0.5, None, None, None) == -1
+    assert lib.viterbi_hard_vec(None, None, None, 8, 2, 2, 64, 1, None, 0, None, None, None) == -1
     assert lib.bcjr_ste_forward(None, None, None, 8, 2, 64, 1, 0.5, None, None, None, None) == -1
     assert lib.bcjr_destroy(None) == -1
     assert binding.path_bytes(16, 2, 256) == 66 and binding.path_bytes(16, 3, 256) == 98
