@@ -35,7 +35,7 @@ struct bcjr_ctx {
     int device = 0;
     int num_sms = 0;
     int max_smem_optin = 0;
-    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, staging[6];
+    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, cb_beta, staging[6];
     DeviceDiag *diag = nullptr;
     // saved by bcjr_soft_quantize for bcjr_backward
     bool have_fwd = false;
@@ -198,8 +198,12 @@ bcjr_status launch_fwd_vec(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
     p.hist = (float *)ctx->hist.ptr;
     p.stepO = (int *)ctx->stepO.ptr;
     p.msg = gl.msg_global ? (float *)ctx->msg.ptr : nullptr;
+    const int SV = (1 << p.Lb) * V;
+    if ((rc = ensure(ctx, ctx->cb_beta, (size_t)SV * 4))) return rc;
+    regroup_table_kernel<<<(SV + 255) / 256, 256, 0, st>>>(p.cb, (float *)ctx->cb_beta.ptr, 1 << p.Lb, KB, V);
+    p.cb_beta = (const float *)ctx->cb_beta.ptr;
     fwd_vec_kernel<KB, V><<<gl.grid, gl.threads, gl.smem, st>>>(p);
-    ctx->launches += 1;
+    ctx->launches += 2;
     CU(cudaGetLastError());
     return BCJR_OK;
 }
@@ -219,11 +223,15 @@ bcjr_status launch_bwd_vec(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cud
     p.stepO = (int *)ctx->stepO.ptr;
     p.gc_part = (float *)ctx->gc_part.ptr;
     p.msg = gl.msg_global ? (float *)ctx->msg.ptr : nullptr;
+    // the regrouped table of the forward call may be stale (another call in between): rebuild it
+    if ((rc = ensure(ctx, ctx->cb_beta, (size_t)S * V * 4))) return rc;
+    regroup_table_kernel<<<(S * V + 255) / 256, 256, 0, st>>>(p.cb, (float *)ctx->cb_beta.ptr, S, KB, V);
+    p.cb_beta = (const float *)ctx->cb_beta.ptr;
     bwd_vec_kernel<KB, V><<<gl.grid, gl.threads, gl.smem, st>>>(p);
-    ctx->launches += 1;
+    ctx->launches += 2;
     CU(cudaGetLastError());
     if (grad_codebook) {
-        reduce_gc_kernel<<<(S * V + 255) / 256, 256, 0, st>>>(p.gc_part, gl.grid, S * V, grad_codebook);
+        reduce_gc_vec_kernel<<<(S * V + 255) / 256, 256, 0, st>>>(p.gc_part, gl.grid, S, KB, V, grad_codebook);
         ctx->launches += 1;
         CU(cudaGetLastError());
     }
@@ -472,7 +480,7 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx)
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
     Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp, &ctx->path_ws,
-                     &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
+                     &ctx->cb_beta, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
                      &ctx->staging[5]};
     for (Buffer *b : all)
         if (b->ptr) cudaFree(b->ptr);
@@ -799,7 +807,7 @@ int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx)
 {
     if (!ctx) return 0;
     const Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp,
-                           &ctx->path_ws, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
+                           &ctx->path_ws, &ctx->cb_beta, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
                            &ctx->staging[4], &ctx->staging[5]};
     int64_t tot = 0;
     for (const Buffer *b : all) tot += (int64_t)b->bytes;

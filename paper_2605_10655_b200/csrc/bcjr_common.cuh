@@ -72,6 +72,7 @@ __device__ __forceinline__ void diag_check_finite(DeviceDiag *diag, float v)
 struct FwdParams {
     const float *W;          // [B*n]
     const float *cb;         // [S]
+    const float *cb_beta;    // vector-emission kernels only: the table regrouped [K][Q][V] for the beta sweep
     float *soft;             // [B*n]
     float *soft_copy;        // [B*n] context-owned copy, read again by the backward pass
     float *logZ;             // [B] or null (natural log)
@@ -87,6 +88,7 @@ struct FwdParams {
 struct BwdParams {
     const float *W;
     const float *cb;
+    const float *cb_beta;    // vector-emission kernels only: the table regrouped [K][Q][V]
     const float *g;          // upstream gradient [B*n]
     const float *soft;       // saved soft codeword [B*n]
     float *gW;               // [B*n]

@@ -9,7 +9,10 @@
 // groups q = tid, tid + blockDim, ..., compressed messages L_t / M_t of Q = S / 2^KB entries in
 // shared memory, gauge-fixed history of L_t in a per-CTA global buffer), with the per-step scalars
 // (weight, upstream gradient, soft value, posterior sums) widened to V components.  The table is
-// laid out [S][V] and read through the read-only cache.
+// laid out [S][V] and read through the read-only cache.  The alpha sweep reads entry q + jQ for
+// consecutive q (coalesced); the beta sweep reads entry qK + b, which for consecutive q is a
+// 128-byte stride, so it reads a copy regrouped as [b][q][V] (made once per call by
+// regroup_table_kernel) and keeps the per-CTA gradient accumulators in the same layout.
 #pragma once
 #include "bcjr_generic.cuh"
 
@@ -41,6 +44,25 @@ __device__ __forceinline__ float dist2(const VecOf<V> &w, const VecOf<V> &c)
 #pragma unroll
     for (int i = 0; i < V; ++i) { const float d = w.v[i] - c.v[i]; e = fmaf(d, d, e); }
     return e;
+}
+
+// dst[(b*Q + q)*V + v] = src[((q << KB) + b)*V + v]
+__global__ void regroup_table_kernel(const float *src, float *dst, int S, int KB, int V)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= S * V) return;
+    const int v = i % V, u = i / V, Q = S >> KB, b = u / Q, q = u % Q;
+    dst[i] = src[(size_t)((q << KB) + b) * V + v];
+}
+// Deterministic sum of the per-CTA gradient partials ([K][Q][V] each) into the table's own layout.
+__global__ void reduce_gc_vec_kernel(const float *part, int nparts, int S, int KB, int V, float *out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;       // index in the regrouped layout
+    if (i >= S * V) return;
+    const int v = i % V, u = i / V, Q = S >> KB, b = u / Q, q = u % Q;
+    float acc = 0.f;
+    for (int r = 0; r < nparts; ++r) acc += part[(size_t)r * S * V + i];
+    out[(size_t)((q << KB) + b) * V + v] = acc;
 }
 
 constexpr int VEC_PART = 8;            // floats per per-warp slot of posterior sums (>= 2 + 2 V)
@@ -132,7 +154,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_vec_kernel(FwdParams p)
 #pragma unroll
                 for (int b = 0; b < K; ++b) {
                     const int s = q * K + b;
-                    c[b] = load_vec<V>(p.cb + (size_t)s * V);
+                    c[b] = load_vec<V>(p.cb_beta + ((size_t)b * Q + q) * V);
                     u[b] = fmaf(dist2<V>(wt, c[b]), -lam2, Min[s & (Q - 1)]);
                     m = fmaxf(m, u[b]);
                 }
@@ -224,7 +246,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_vec_kernel(BwdParams p)
     float *histL = p.hist + (size_t)blockIdx.x * 2 * nt * Q;
     float *histA = histL + (size_t)nt * Q;
     int *stepO = p.stepO + (size_t)blockIdx.x * (nt + 2);
-    float *gc = p.gc_part + (size_t)blockIdx.x * S * V;
+    float *gc = p.gc_part + (size_t)blockIdx.x * S * V;           // [K][Q][V], like cb_beta
     const float lam2 = p.lam2, invT = p.invT;
     float defect = 0.f;
     static_assert(2 + 2 * V <= VEC_PART, "posterior sums per warp slot");
@@ -309,7 +331,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_vec_kernel(BwdParams p)
 #pragma unroll
                 for (int b = 0; b < K; ++b) {
                     const int s = q * K + b;
-                    c[b] = load_vec<V>(p.cb + (size_t)s * V);
+                    c[b] = load_vec<V>(p.cb_beta + ((size_t)b * Q + q) * V);
                     u[b] = fmaf(dist2<V>(wt, c[b]), -lam2, Min[s & (Q - 1)]);
                     float h = Bin[s & (Q - 1)];
 #pragma unroll
@@ -341,7 +363,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_vec_kernel(BwdParams p)
                         const float cm = c[b].v[v] - st.v[v];
                         S1[v] = fmaf(gam, cm, S1[v]);
                         S3[v] = fmaf(gr, cm, S3[v]);
-                        gc[(size_t)(q * K + b) * V + v] += gam * fmaf(invT * (wt.v[v] - c[b].v[v]), r, gt.v[v]);
+                        gc[((size_t)b * Q + q) * V + v] += gam * fmaf(invT * (wt.v[v] - c[b].v[v]), r, gt.v[v]);
                     }
                 }
             }
