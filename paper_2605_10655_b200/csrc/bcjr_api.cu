@@ -13,6 +13,7 @@
 #ifndef BCJR_NO_CLUSTER
 #include "bcjr_cluster.cuh"
 #include "bcjr_vec.cuh"
+#include "bcjr_vec4.cuh"
 #include "bcjr_solo.cuh"
 #include "bcjr_duo.cuh"
 #include "bcjr_viterbi.cuh"
@@ -296,6 +297,26 @@ bcjr_status plan_cluster(bcjr_ctx *ctx, Kern kern, int CL, int threads, size_t s
     if (ctx->opt_max_ctas > 0 && ncl > ctx->opt_max_ctas / CL) ncl = ctx->opt_max_ctas / CL > 0 ? ctx->opt_max_ctas / CL : 1;
     if (ncl > B) ncl = (int)B;
     cfg->gridDim = dim3(CL * ncl, 1, 1);
+    return BCJR_OK;
+}
+
+// Lb = 16, 4 bits and 2 weights per step: one block per cluster of four CTAs, table slice in shared memory
+bcjr_status launch_fwd_vec4(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    using C = Vec4Cfg;
+    if (p.n > C::MAX_N || ((uintptr_t)p.cb & 15u)) return BCJR_EUNSUPPORTED;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    bcjr_status rc = plan_cluster(ctx, fwd_vec4_kernel, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    if (rc) return rc;
+    const int ncl = cfg.gridDim.x / C::CL, nt = p.n / C::V;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * nt * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->cb_beta, (size_t)C::S * C::V * 4))) return rc;
+    regroup_table_kernel<<<(C::S * C::V + 255) / 256, 256, 0, st>>>(p.cb, (float *)ctx->cb_beta.ptr, C::S, C::KB, C::V);
+    p.hist = (float *)ctx->hist.ptr;
+    p.cb_beta = (const float *)ctx->cb_beta.ptr;
+    CU(cudaLaunchKernelEx(&cfg, fwd_vec4_kernel, p));
+    ctx->launches += 2;
     return BCJR_OK;
 }
 
@@ -692,9 +713,20 @@ bcjr_status bcjr_soft_quantize_vec(bcjr_ctx *ctx, const float *W, const float *c
         p.W = W; p.cb = codebook; p.soft = soft; p.soft_copy = (float *)ctx->soft_copy.ptr; p.logZ = logZ;
         p.diag = ctx->diag; p.B = num_blocks; p.Lb = Lb; p.n = n;
         p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)T));
-        rc = k == 1 ? launch_fwd_vec<2, 2>(ctx, p, st) : launch_fwd_vec<4, 2>(ctx, p, st);
+        bool large = false;
+#ifndef BCJR_NO_CLUSTER
+        large = ctx->opt_path != 1 && Lb == 16 && k == 2;
+        if (ctx->opt_path == 2 && !large) return BCJR_EUNSUPPORTED;
+        if (large) {
+            rc = launch_fwd_vec4(ctx, p, st);
+            if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { large = false; rc = BCJR_OK; }   // e.g. n too long
+        }
+#else
+        if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
+#endif
+        if (!large) rc = k == 1 ? launch_fwd_vec<2, 2>(ctx, p, st) : launch_fwd_vec<4, 2>(ctx, p, st);
         if (rc) return rc;
-        ctx->last_path = 0;
+        ctx->last_path = large ? 1 : 0;
     }
     ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = num_blocks; ctx->T = T;
     ctx->V = V;

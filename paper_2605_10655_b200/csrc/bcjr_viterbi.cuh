@@ -57,7 +57,7 @@ template <int KB>
 __global__ void __launch_bounds__(VitSoloCfg<KB>::THREADS, 1) viterbi_solo_kernel(VitParams p)
 {
     using C = VitSoloCfg<KB>;
-    constexpr int K = C::K, Q = C::Q, NB = C::NB, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, QB = C::QB;
+    constexpr int K = C::K, Q = C::Q, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, QB = C::QB;
     constexpr int UNITS = C::UNITS, JPU = C::JPU, WB = C::WORD_BITS, ROWB = C::ROW_BYTES;
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

@@ -30,10 +30,11 @@ def _run(ctx, W, c, g, Lb, k, V, T, viterbi=True):
     n = W.shape[1]
     Wd, cd, gd = (torch.from_numpy(np.ascontiguousarray(a)).to(dev) for a in (W, c, g))
     soft, logZ = ctx.bcjr_soft_quantize_vec(Wd, cd, Lb, k, V, n, T)
+    fwd_path = ctx.sync_status().last_path
     gW, gc = ctx.bcjr_backward(gd)
     diag = ctx.sync_status()
     out = {"soft": soft.cpu().numpy(), "logZ": logZ.cpu().numpy(), "grad_W": gW.cpu().numpy(),
-           "grad_codebook": gc.cpu().numpy().reshape(1 << Lb, V), "diag": diag}
+           "grad_codebook": gc.cpu().numpy().reshape(1 << Lb, V), "diag": diag, "fwd_path": fwd_path}
     if viterbi:
         bits, states, hard = ctx.viterbi_hard_vec(Wd, cd, Lb, k, V, n)
         ctx.sync_status()
@@ -66,10 +67,22 @@ def test_two_weights_per_step_small_and_mid_trellises(ctx, Lb, k, nt, B, T):
     _check(ctx, Lb, k, 2, nt, B, T, seed=8000 + Lb * 10 + k, what=f"V=2 Lb={Lb} k={k} nt={nt} B={B} T={T}")
 
 
+@pytest.mark.parametrize("path", [0, 1], ids=["cluster", "generic"])
 @pytest.mark.parametrize("T", [0.3, 0.05])
-def test_sixteen_bit_state_sixteen_predecessors(ctx, T):
-    # the paper's own configuration: Lb = 16, 2 bits per weight, 2 weights per step
-    _check(ctx, 16, 2, 2, 24, 3, T, seed=8100, what=f"V=2 Lb=16 k=2 T={T}")
+def test_sixteen_bit_state_sixteen_predecessors(ctx, T, path):
+    # the paper's own configuration: Lb = 16, 2 bits per weight, 2 weights per step; on the
+    # four-CTA cluster kernels (default) and on the one-CTA-per-block kernels
+    ctx.set_option("path", path)
+    try:
+        got = _check(ctx, 16, 2, 2, 24, 3, T, seed=8100, what=f"V=2 Lb=16 k=2 T={T} path={path}")
+        assert got["fwd_path"] == (1 if path == 0 else 0)
+    finally:
+        ctx.set_option("path", 0)
+
+
+@pytest.mark.parametrize("nt,B", [(1, 2), (2, 5), (3, 1), (37, 70)])
+def test_cluster_kernels_ragged_step_counts_and_more_blocks_than_clusters(ctx, nt, B):
+    _check(ctx, 16, 2, 2, nt, B, 0.2, seed=8500 + nt, what=f"V=2 Lb=16 nt={nt} B={B}")
 
 
 def test_sixteen_bit_state_one_bit_per_weight(ctx):
