@@ -301,21 +301,25 @@ bcjr_status plan_cluster(bcjr_ctx *ctx, Kern kern, int CL, int threads, size_t s
 }
 
 // Lb = 16, 4 bits and 2 weights per step: one block per cluster of four CTAs, table slice in shared memory
+#ifndef VEC4_NBLK
+#define VEC4_NBLK 2
+#endif
 bcjr_status launch_fwd_vec4(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
-    using C = Vec4Cfg;
+    using C = Vec4Cfg<VEC4_NBLK>;
     if (p.n > C::MAX_N || ((uintptr_t)p.cb & 15u)) return BCJR_EUNSUPPORTED;
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1];
-    bcjr_status rc = plan_cluster(ctx, fwd_vec4_kernel, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    auto kern = fwd_vec4_kernel<VEC4_NBLK>;
+    bcjr_status rc = plan_cluster(ctx, kern, C::CL, C::THREADS, C::SMEM_BYTES, (p.B + C::NBLK - 1) / C::NBLK, &cfg, attr, st);
     if (rc) return rc;
     const int ncl = cfg.gridDim.x / C::CL, nt = p.n / C::V;
-    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * nt * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * C::NBLK * nt * C::Q * 4))) return rc;
     if ((rc = ensure(ctx, ctx->cb_beta, (size_t)C::S * C::V * 4))) return rc;
     regroup_table_kernel<<<(C::S * C::V + 255) / 256, 256, 0, st>>>(p.cb, (float *)ctx->cb_beta.ptr, C::S, C::KB, C::V);
     p.hist = (float *)ctx->hist.ptr;
     p.cb_beta = (const float *)ctx->cb_beta.ptr;
-    CU(cudaLaunchKernelEx(&cfg, fwd_vec4_kernel, p));
+    CU(cudaLaunchKernelEx(&cfg, kern, p));
     ctx->launches += 2;
     return BCJR_OK;
 }
