@@ -324,6 +324,34 @@ bcjr_status launch_fwd_vec4(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
     return BCJR_OK;
 }
 
+bcjr_status launch_bwd_vec4(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    using C = Vec4BwdCfg<VEC4_NBLK>;
+    constexpr int S = C::F::S, V = 2, KB = 4;
+    if (p.n > C::MAX_N || ((uintptr_t)p.cb & 15u)) return BCJR_EUNSUPPORTED;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    auto kern = bwd_vec4_kernel<VEC4_NBLK>;
+    bcjr_status rc = plan_cluster(ctx, kern, C::CL, C::THREADS, C::SMEM_BYTES, (p.B + C::NBLK - 1) / C::NBLK, &cfg, attr, st);
+    if (rc) return rc;
+    const int ncl = cfg.gridDim.x / C::CL, nt = p.n / V;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * C::NBLK * 2 * nt * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * S * V * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->cb_beta, (size_t)S * V * 4))) return rc;
+    regroup_table_kernel<<<(S * V + 255) / 256, 256, 0, st>>>(p.cb, (float *)ctx->cb_beta.ptr, S, KB, V);
+    p.hist = (float *)ctx->hist.ptr;
+    p.gc_part = (float *)ctx->gc_part.ptr;
+    p.cb_beta = (const float *)ctx->cb_beta.ptr;
+    CU(cudaLaunchKernelEx(&cfg, kern, p));
+    ctx->launches += 2;
+    if (grad_codebook) {
+        reduce_gc_vec_kernel<<<(S * V + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, S, KB, V, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
 template <int LB, int KB, int CL, int THREADS>
 bcjr_status launch_fwd_cluster_t(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
@@ -627,9 +655,21 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
     bcjr_status rc = BCJR_OK;
     if (ctx->V == 2) {                                   // saved by bcjr_soft_quantize_vec: k bits per weight
         if (!aligned8(grad_soft) || !aligned8(grad_W)) return BCJR_EINVAL;
-        rc = ctx->k == 1 ? launch_bwd_vec<2, 2>(ctx, p, grad_codebook, st) : launch_bwd_vec<4, 2>(ctx, p, grad_codebook, st);
+        bool large = false;
+#ifndef BCJR_NO_CLUSTER
+        large = ctx->opt_path != 1 && ctx->Lb == 16 && ctx->k == 2;
+        if (ctx->opt_path == 2 && !large) return BCJR_EUNSUPPORTED;
+        if (large) {
+            rc = launch_bwd_vec4(ctx, p, grad_codebook, st);
+            if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { large = false; rc = BCJR_OK; }
+        }
+#else
+        if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
+#endif
+        if (!large)
+            rc = ctx->k == 1 ? launch_bwd_vec<2, 2>(ctx, p, grad_codebook, st) : launch_bwd_vec<4, 2>(ctx, p, grad_codebook, st);
         if (rc) return rc;
-        ctx->last_path = 0;
+        ctx->last_path = large ? 1 : 0;
         return BCJR_OK;
     }
     bool use_cluster = false;

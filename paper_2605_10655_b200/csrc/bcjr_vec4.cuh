@@ -383,4 +383,401 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
     if (warp == 0) tmem_dealloc_512(tmem_base);
 }
 
+// --------------------------------------------------------------------------------------
+// Backward call on the same clusters.  Every message carries a second value, the conditional
+// expectation of the centred emitted sum (first-order expectation semiring; the recursions are
+// those of bwd_vec_kernel).  Per thread the tensor memory holds the table slice (64 columns) and,
+// next to it, the gradient accumulators of the thread's beta-sweep states (64 columns, same
+// layout), kept over all steps and all blocks and written once to this cluster's partial sum.
+//   h_t(s) = sum_v g[V t + v] (c[s][v] - soft[V t + v]); the constant -g.soft of the consumer's
+//   step is added by the producer of At / Bt, so a consumer forms g.c + (carried value) only.
+//   z_v(s) = gamma_t(s) (g_v + (w_v - c[s][v]) r_t(s) / T)  is the accumulator increment;
+//   grad_W[V t + v] = g_v - (sum_s z_v) / S0 + (S2 / S0) (w_v - soft_v) / T,  S0 = sum gamma, S2 = sum gamma r.
+// --------------------------------------------------------------------------------------
+template <int NBLK_>
+struct Vec4BwdCfg {
+    using F = Vec4Cfg<NBLK_>;
+    static constexpr int Q = F::Q, QC = F::QC, CL = F::CL, THREADS = F::THREADS, NWARP = F::NWARP, SLOTS = F::SLOTS, K = F::K;
+    static constexpr int NBUF = 3, NBLK = NBLK_, UNITS = 4;
+    static constexpr int MAX_N = 1024, MAX_NT = MAX_N / 2;
+    static constexpr int OFF_MSG = 0;                                  // [NBUF][NBLK][2][QC]: (L, At) or (M, Bt)
+    static constexpr int OFF_W = OFF_MSG + NBUF * NBLK * 2 * QC;       // [NBLK][3][MAX_N]: w, g, soft
+    static constexpr int OFF_O = OFF_W + NBLK * 3 * MAX_N;             // int [NBLK][MAX_NT + 4]
+    static constexpr int OFF_WMAX = OFF_O + NBLK * (MAX_NT + 4);       // [NBUF][NBLK][64]
+    static constexpr int OFF_PART = OFF_WMAX + NBUF * NBLK * 64;       // [NBUF][NBLK][64][4]: S0, S2, ZS_0, ZS_1
+    static constexpr int OFF_LZ = OFF_PART + NBUF * NBLK * 64 * 4;     // [NBLK][64]
+    static constexpr int OFF_MBAR = OFF_LZ + NBLK * 64;                // uint64 [NBUF][NBLK]
+    static constexpr int OFF_TMEM = OFF_MBAR + 2 * NBUF * NBLK + 2;
+    static constexpr int OFF_FLAG = OFF_TMEM + 2;
+    static constexpr int SMEM_FLOATS = OFF_FLAG + 4;
+    static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
+    static_assert(OFF_MBAR % 2 == 0 && OFF_MSG % 4 == 0 && OFF_PART % 4 == 0, "alignment");
+    static_assert(SMEM_BYTES <= 232448, "shared memory of one CTA");
+    static_assert(NBLK <= NWARP && NBUF * NBLK <= 32, "one finishing warp per block in flight; phase bits");
+};
+
+template <int NBLK_>
+__global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel(BwdParams p)
+{
+    using C = Vec4BwdCfg<NBLK_>;
+    constexpr int K = C::K, Q = C::Q, QC = C::QC, CL = C::CL, NWARP = C::NWARP, NBUF = C::NBUF, SLOTS = C::SLOTS, CT = C::THREADS;
+    constexpr int NBLK = C::NBLK, OSTR = C::MAX_NT + 4, UNITS = C::UNITS, MAXN = C::MAX_N;
+    constexpr uint32_t TX_MSG = 2u * QC * 4u + SLOTS * 4u;       // a quarter of both message arrays + gauge slots
+    constexpr uint32_t TX_PART = SLOTS * 16u;                    // posterior sums (rank 0 only)
+    extern __shared__ __align__(16) float smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t cid = cluster_id_x(), ncl = cluster_count_x();
+    const int n = p.n, nt = n / 2;
+    const float2 nl2 = splat2(-p.lam2);
+    const float invT = p.invT;
+
+    float *msg = smem + C::OFF_MSG;
+    float *w_s = smem + C::OFF_W;
+    int *O_s = reinterpret_cast<int *>(smem + C::OFF_O);
+    float *wmax = smem + C::OFF_WMAX;
+    float *part = smem + C::OFF_PART;
+    float *lz = smem + C::OFF_LZ;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
+    Proto pr{1u, abort_flag, p.diag};
+    const uint32_t mbar_full = smem_u32(smem + C::OFF_MBAR);
+    const uint32_t msg_u32 = smem_u32(msg), wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
+
+    const int q0 = (int)rank * QC + 2 * tid;                     // alpha sweep: groups q0, q0 + 1
+    const int q0b = warp * 256 + (int)rank * 64 + 2 * lane;      // beta sweep: groups q0b, q0b + 1
+    float *histL = p.hist + (size_t)cid * NBLK * 2 * nt * Q;     // [NBLK][nt][Q]: row t = L_{t+1}
+    float *histA = histL + (size_t)NBLK * nt * Q;                // same shape: At_{t+1} (with the consumer's shift)
+
+    uint32_t full_of[CL], msg_of[CL], wmax_dst[CL], lz_dst[CL];
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+        full_of[r] = mapa_u32(mbar_full, (uint32_t)r);
+        msg_of[r] = mapa_u32(msg_u32, (uint32_t)r);
+        wmax_dst[r] = mapa_u32(wmax_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+        lz_dst[r] = mapa_u32(lz_u32 + (uint32_t)((int)rank * NWARP + warp) * 4u, (uint32_t)r);
+    }
+    const uint32_t part_dst = mapa_u32(part_u32 + (uint32_t)((int)rank * NWARP + warp) * 16u, 0u);
+    const int ra = (q0 & 255) >> 6;
+    const uint32_t push_a = (ra == 0 ? msg_of[0] : ra == 1 ? msg_of[1] : ra == 2 ? msg_of[2] : msg_of[3])
+                            + (uint32_t)((q0 >> 8) * 64 + (q0 & 63)) * 4u;
+    const uint32_t push_a_mbar = ra == 0 ? full_of[0] : ra == 1 ? full_of[1] : ra == 2 ? full_of[2] : full_of[3];
+    const int rb = warp >> 2;
+    const uint32_t push_b = (rb == 0 ? msg_of[0] : rb == 1 ? msg_of[1] : rb == 2 ? msg_of[2] : msg_of[3])
+                            + (uint32_t)(((q0b & 15) >> 1) * 128 + 2 * ((q0b >> 4) & 63)) * 4u;
+    const uint32_t push_b_mbar = rb == 0 ? full_of[0] : rb == 1 ? full_of[1] : rb == 2 ? full_of[2] : full_of[3];
+
+    if (tid == 0) {
+        for (int s = 0; s < NBUF * NBLK; ++s) mbar_init(mbar_full + 8u * s, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc_512(smem_u32(const_cast<uint32_t *>(tmem_slot)));
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tm = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
+    const uint32_t tm_acc = tm + 64u;
+    {
+        float2 z[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z[e] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < UNITS; ++u) tmem_st16(tm_acc + 16u * u, z);
+        tmem_wait_st();
+    }
+    uint32_t full_phase = 0;
+    int ib = 0;
+    float defect = 0.f;
+    auto wait_inputs = [&](int b, int k) {
+        const int s = b * NBLK + k;
+        pr.wait(mbar_full + 8u * s, (full_phase >> s) & 1u);
+        full_phase ^= 1u << s;
+    };
+
+    for (int64_t base = (int64_t)cid * NBLK; base < p.B; base += (int64_t)ncl * NBLK) {
+        const int nact = (int)(p.B - base < NBLK ? p.B - base : NBLK);
+        for (int k = 0; k < nact; ++k) {
+            const float *w = p.W + (base + k) * n, *g = p.g + (base + k) * n, *sf = p.soft + (base + k) * n;
+            float *wk = w_s + k * 3 * MAXN;
+            for (int t = tid; t < n; t += CT) { wk[t] = __ldg(w + t); wk[MAXN + t] = __ldg(g + t); wk[2 * MAXN + t] = __ldg(sf + t); }
+            if (tid == 0) O_s[k * OSTR + 1] = 0;
+        }
+        __syncthreads();
+        for (int k = 0; k < nact; ++k) {
+            // L_1 = 0; the At array carries At + (shift of the consumer's step): At_1 = 0, shift -g_1.soft_1
+            const float *wk = w_s + k * 3 * MAXN;
+            const float gs1 = -(wk[MAXN] * wk[2 * MAXN] + wk[MAXN + 1] * wk[2 * MAXN + 1]);
+            float *m0 = msg + (size_t)(ib * NBLK + k) * 2 * QC;
+            for (int q = tid; q < QC; q += CT) { m0[q] = 0.f; m0[QC + q] = gs1; }
+        }
+        vec4_stage_table(tm, p.cb, q0);
+        int O[NBLK];
+        float off[NBLK], cmax[NBLK];
+#pragma unroll
+        for (int k = 0; k < NBLK; ++k) { O[k] = 0; off[k] = 0.f; cmax[k] = 0.f; }
+        cluster_sync();
+        // ================= alpha sweep carrying (L, At)
+        for (int t = 1; t <= nt; ++t) {
+            const int ob = ib == NBUF - 1 ? 0 : ib + 1;
+#pragma unroll
+            for (int k = 0; k < NBLK; ++k) {
+                if (k < nact) {
+                    const int si = ib * NBLK + k, so = ob * NBLK + k;
+                    if (t > 1) {
+                        wait_inputs(ib, k);
+                        cmax[k] = warp_max(slot_max(wmax + si * 64, lane, SLOTS)) - off[k];
+                        off[k] = rintf(cmax[k]);
+                    }
+                    const float *Lin = msg + (size_t)si * 2 * QC + (tid >> 3), *Ain = Lin + QC;
+                    if (tid == 0) pr.expect_tx(mbar_full + 8u * so, TX_MSG);
+                    const float *wk = w_s + k * 3 * MAXN + 2 * (t - 1);
+                    const float2 wx = splat2(wk[0]), wy = splat2(wk[1]);
+                    const float2 gx = splat2(wk[MAXN]), gy = splat2(wk[MAXN + 1]);
+                    // shift for the consumers of this step's At (step t + 1); unused at t = nt
+                    const float gsn = t < nt ? -(wk[MAXN + 2] * wk[2 * MAXN + 2] + wk[MAXN + 3] * wk[2 * MAXN + 3]) : 0.f;
+                    float2 a[K], x[K], cb[2][8];
+                    tmem_ld16(tm, cb[0]);
+#pragma unroll
+                    for (int u = 0; u < UNITS; ++u) {
+                        tmem_wait_ld(cb[u & 1]);
+                        if (u + 1 < UNITS) tmem_ld16(tm + 16u * (u + 1), cb[(u + 1) & 1]);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int j = 4 * u + e;
+                            const float2 cx = cb[u & 1][2 * e], cy = cb[u & 1][2 * e + 1];
+                            const float2 dx = sub2(cx, wx), dy = sub2(cy, wy);
+                            a[j] = fma2(fma2(dy, dy, mul2(dx, dx)), nl2, splat2(Lin[64 * j]));
+                            x[j] = fma2(gx, cx, fma2(gy, cy, splat2(Ain[64 * j])));      // g.c + (At - g.soft)
+                        }
+                    }
+                    const float2 m = max_pairs<K>(a);
+                    float2 sum = make_float2(0.f, 0.f), ax = sum;
+#pragma unroll
+                    for (int j = 0; j < K; ++j) {
+                        const float2 pj = ex2f2(sub2(a[j], m));
+                        sum = add2(sum, pj);
+                        ax = fma2(pj, x[j], ax);
+                    }
+                    const float2 outL = add2(sub2(m, splat2(off[k])), lg2f2(sum));
+                    const float2 outA = fma2(ax, rcpf2(sum), splat2(gsn));
+                    pr.async_v2(push_a + (uint32_t)(so * 2 * QC) * 4u, outL.x, outL.y, push_a_mbar + 8u * so);
+                    pr.async_v2(push_a + (uint32_t)(so * 2 * QC + QC) * 4u, outA.x, outA.y, push_a_mbar + 8u * so);
+                    if (t < nt) {
+                        *reinterpret_cast<float2 *>(histL + ((size_t)k * nt + t) * Q + q0) = outL;
+                        *reinterpret_cast<float2 *>(histA + ((size_t)k * nt + t) * Q + q0) = outA;
+                    }
+                    const float tmax = warp_max(fmaxf(m.x, m.y));
+                    if (lane == 0) {
+#pragma unroll
+                        for (int r = 0; r < CL; ++r) pr.async_f32(wmax_dst[r] + (uint32_t)(so * 64) * 4u, tmax, full_of[r] + 8u * so);
+                    }
+                    O[k] += (int)off[k];
+                    if (tid == 0) O_s[k * OSTR + t + 1] = O[k];
+                }
+            }
+            ib = ob;
+        }
+        // ================= log2 Z
+#pragma unroll
+        for (int k = 0; k < NBLK; ++k) {
+            if (k < nact) {
+                const int si = ib * NBLK + k;
+                wait_inputs(ib, k);
+                cmax[k] = warp_max(slot_max(wmax + si * 64, lane, SLOTS)) - off[k];
+                const float *Lfin = msg + (size_t)si * 2 * QC;
+                float ssum = 0.f;
+                for (int e = tid; e < QC; e += CT) ssum += ex2f(Lfin[e] - cmax[k]);
+                ssum = warp_sum(ssum);
+                if (lane == 0) {
+#pragma unroll
+                    for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r] + (uint32_t)(k * 64) * 4u, ssum);
+                }
+            }
+        }
+        cluster_sync();
+        float lsefin[NBLK];
+        int Ofin[NBLK];
+#pragma unroll
+        for (int k = 0; k < NBLK; ++k) {
+            lsefin[k] = 0.f; Ofin[k] = O[k];
+            if (k < nact) {
+                float v = (lane < SLOTS ? lz[k * 64 + lane] : 0.f) + (lane + 32 < SLOTS ? lz[k * 64 + lane + 32] : 0.f);
+                v = warp_sum(v);
+                lsefin[k] = cmax[k] + lg2f(v);
+                if (tid == 0) diag_check_finite(p.diag, lsefin[k]);
+            }
+        }
+        // ================= beta sweep carrying (M, Bt), with the gradient contraction
+        for (int k = 0; k < nact; ++k) {
+            // M_nt = 0, Bt_nt = 0 (+ the shift of step nt)
+            const float *wk = w_s + k * 3 * MAXN;
+            const float gsl = -(wk[MAXN + n - 2] * wk[2 * MAXN + n - 2] + wk[MAXN + n - 1] * wk[2 * MAXN + n - 1]);
+            float *m0 = msg + (size_t)(ib * NBLK + k) * 2 * QC;
+            for (int q = tid; q < QC; q += CT) { m0[q] = 0.f; m0[QC + q] = gsl; }
+        }
+        vec4_stage_table(tm, p.cb_beta, q0b);
+        int P[NBLK];
+        float offM[NBLK];
+        float2 Ls[NBLK], As[NBLK];
+#pragma unroll
+        for (int k = 0; k < NBLK; ++k) {
+            P[k] = 0; offM[k] = 0.f;
+            const bool have = k < nact && nt > 1;
+            Ls[k] = have ? __ldcg(reinterpret_cast<const float2 *>(histL + ((size_t)k * nt + nt - 1) * Q + q0b)) : make_float2(0.f, 0.f);
+            // At_1 = 0 carries the shift of step 1 like every other row
+            As[k] = have ? __ldcg(reinterpret_cast<const float2 *>(histA + ((size_t)k * nt + nt - 1) * Q + q0b))
+                         : splat2(k < nact ? -(w_s[k * 3 * MAXN + MAXN] * w_s[k * 3 * MAXN + 2 * MAXN] + w_s[k * 3 * MAXN + MAXN + 1] * w_s[k * 3 * MAXN + 2 * MAXN + 1]) : 0.f);
+        }
+        cluster_sync();
+        // rank 0, warp k: turn the sums of step t of block k (slots of buffer b) into grad_W of that step
+        auto finish_step = [&](int t, int b, int k) {
+            if (rank == 0 && warp == k) {
+                const float *pp = part + (size_t)((b * NBLK + k) * 64) * 4;
+                const float4 s4 = *reinterpret_cast<const float4 *>(pp + lane * 4);
+                const float4 o = *reinterpret_cast<const float4 *>(pp + (lane + 32) * 4);
+                const float a0 = warp_sum(s4.x + o.x), a2 = warp_sum(s4.y + o.y), z0 = warp_sum(s4.z + o.z), z1 = warp_sum(s4.w + o.w);
+                if (lane == 0) {
+                    const float *wk = w_s + k * 3 * MAXN + 2 * (t - 1);
+                    const float i0 = 1.f / a0;
+                    const float gw0 = (wk[MAXN] - z0 * i0) + (a2 * i0) * (wk[0] - wk[2 * MAXN]) * invT;
+                    const float gw1 = (wk[MAXN + 1] - z1 * i0) + (a2 * i0) * (wk[1] - wk[2 * MAXN + 1]) * invT;
+                    *reinterpret_cast<float2 *>(p.gW + (base + k) * n + 2 * (t - 1)) = make_float2(gw0, gw1);
+                    defect = fmaxf(defect, fabsf(a0 - 1.f));
+                }
+            }
+        };
+        for (int t = nt; t >= 1; --t) {
+            const int ob = ib == NBUF - 1 ? 0 : ib + 1;
+#pragma unroll
+            for (int k = 0; k < NBLK; ++k) {
+                if (k < nact) {
+                    const int si = ib * NBLK + k, so = ob * NBLK + k;
+                    if (t < nt) {
+                        wait_inputs(ib, k);
+                        cmax[k] = warp_max(slot_max(wmax + si * 64, lane, SLOTS));
+                        P[k] += (int)offM[k];
+                        offM[k] = rintf(cmax[k]);
+                        finish_step(t + 1, ib, k);
+                    }
+                    const float *Min = msg + (size_t)si * 2 * QC + 4 * lane, *Bin = Min + QC;
+                    if (tid == 0) pr.expect_tx(mbar_full + 8u * so, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
+                    const float *wk = w_s + k * 3 * MAXN + 2 * (t - 1);
+                    const float2 wx = splat2(wk[0]), wy = splat2(wk[1]);
+                    const float2 gx = splat2(wk[MAXN]), gy = splat2(wk[MAXN + 1]);
+                    const float gs = -(wk[MAXN] * wk[2 * MAXN] + wk[MAXN + 1] * wk[2 * MAXN + 1]);              // shift carried by the stored At
+                    const float gsp = t > 1 ? -(wk[MAXN - 2] * wk[2 * MAXN - 2] + wk[MAXN - 1] * wk[2 * MAXN - 1]) : 0.f;   // for step t - 1
+                    float2 Ls_next = make_float2(0.f, 0.f), As_next = Ls_next;
+                    if (t > 2) {
+                        Ls_next = __ldcg(reinterpret_cast<const float2 *>(histL + ((size_t)k * nt + t - 2) * Q + q0b));
+                        As_next = __ldcg(reinterpret_cast<const float2 *>(histA + ((size_t)k * nt + t - 2) * Q + q0b));
+                    } else if (t == 2) {
+                        As_next = splat2(-(wk[MAXN - 2] * wk[2 * MAXN - 2] + wk[MAXN - 1] * wk[2 * MAXN - 1]));          // At_1 = 0 + shift of step 1
+                    }
+                    const float Dm = ((float)(Ofin[k] - O_s[k * OSTR + t] - P[k]) + lsefin[k]) - offM[k];
+                    const float2 offM2 = splat2(offM[k]);
+                    float2 u[K], cb[8];
+#pragma unroll
+                    for (int un = 0; un < UNITS; ++un) {
+                        tmem_ld16(tm + 16u * un, cb);
+                        tmem_wait_ld(cb);
+#pragma unroll
+                        for (int e = 0; e < 4; e += 2) {
+                            const int b = 4 * un + e;
+                            const float4 Mv = *reinterpret_cast<const float4 *>(Min + 128 * (b >> 1));
+#pragma unroll
+                            for (int bb = 0; bb < 2; ++bb) {
+                                const float2 dx = sub2(cb[2 * (e + bb)], wx), dy = sub2(cb[2 * (e + bb) + 1], wy);
+                                const float2 Mb = bb == 0 ? make_float2(Mv.x, Mv.z) : make_float2(Mv.y, Mv.w);
+                                u[b + bb] = fma2(fma2(dy, dy, mul2(dx, dx)), nl2, sub2(Mb, offM2));
+                            }
+                        }
+                    }
+                    const float2 m = max_pairs<K>(u);
+                    const float2 f = ex2f2(add2(m, sub2(Ls[k], splat2(Dm))));
+                    const float2 fi = mul2(f, splat2(invT));
+                    const float2 Ahj = sub2(As[k], splat2(gs));                        // At_t without the shift
+                    float2 sum = make_float2(0.f, 0.f), ya = sum, S0 = sum, S2 = sum, Z0 = sum, Z1 = sum;
+#pragma unroll
+                    for (int un = 0; un < UNITS; ++un) {                                   // second pass, with the accumulators
+                        float2 acc[8];
+                        tmem_ld16(tm + 16u * un, cb);
+                        tmem_ld16(tm_acc + 16u * un, acc);
+                        tmem_wait_ld(cb);
+                        tmem_wait_ld(acc);
+#pragma unroll
+                        for (int e = 0; e < 4; e += 2) {
+                            const int b = 4 * un + e;
+                            const float4 Bv = *reinterpret_cast<const float4 *>(Bin + 128 * (b >> 1));
+#pragma unroll
+                            for (int bb = 0; bb < 2; ++bb) {
+                                const float2 cx = cb[2 * (e + bb)], cy = cb[2 * (e + bb) + 1];
+                                const float2 Bb = bb == 0 ? make_float2(Bv.x, Bv.z) : make_float2(Bv.y, Bv.w);
+                                const float2 y = fma2(gx, cx, fma2(gy, cy, Bb));             // g.c + (Bt - g.soft) = h + Bt
+                                const float2 pb = ex2f2(sub2(u[b + bb], m));
+                                sum = add2(sum, pb);
+                                ya = fma2(pb, y, ya);
+                                const float2 r = add2(y, Ahj);
+                                const float2 gam = mul2(pb, f), q = mul2(mul2(pb, fi), r);     // gamma, gamma r / T
+                                S0 = add2(S0, gam);
+                                S2 = fma2(gam, r, S2);
+                                const float2 zx = fma2(q, sub2(wx, cx), mul2(gam, gx));
+                                const float2 zy = fma2(q, sub2(wy, cy), mul2(gam, gy));
+                                Z0 = add2(Z0, zx); Z1 = add2(Z1, zy);
+                                acc[2 * (e + bb)] = add2(acc[2 * (e + bb)], zx);
+                                acc[2 * (e + bb) + 1] = add2(acc[2 * (e + bb) + 1], zy);
+                            }
+                        }
+                        tmem_st16(tm_acc + 16u * un, acc);
+                    }
+                    tmem_wait_st();
+                    const float2 outM = add2(m, lg2f2(sum));
+                    const float2 outB = fma2(ya, rcpf2(sum), splat2(gsp));
+                    pr.async_v2(push_b + (uint32_t)(so * 2 * QC) * 4u, outM.x, outM.y, push_b_mbar + 8u * so);
+                    pr.async_v2(push_b + (uint32_t)(so * 2 * QC + QC) * 4u, outB.x, outB.y, push_b_mbar + 8u * so);
+                    const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), z0 = warp_sum(Z0.x + Z0.y), z1 = warp_sum(Z1.x + Z1.y);
+                    const float tmax = warp_max(fmaxf(m.x, m.y));
+                    if (lane == 0) {
+#pragma unroll
+                        for (int r = 0; r < CL; ++r) pr.async_f32(wmax_dst[r] + (uint32_t)(so * 64) * 4u, tmax, full_of[r] + 8u * so);
+                        pr.async_v4(part_dst + (uint32_t)(so * 256) * 4u, s0, s2, z0, z1, full_of[0] + 8u * so);
+                    }
+                    Ls[k] = Ls_next; As[k] = As_next;
+                }
+            }
+            ib = ob;
+        }
+#pragma unroll
+        for (int k = 0; k < NBLK; ++k) {
+            if (k < nact) {
+                wait_inputs(ib, k);                                          // the sums of step 1
+                finish_step(1, ib, k);
+            }
+        }
+        cluster_sync();         // nobody still reads this round's buffers when the next round starts
+    }
+    // this cluster's partial of the table gradient, in the regrouped layout [b][q][V]
+    {
+        float *gc = p.gc_part + (size_t)cid * C::F::S * 2;
+#pragma unroll
+        for (int un = 0; un < UNITS; ++un) {
+            float2 acc[8];
+            tmem_ld16(tm_acc + 16u * un, acc);
+            tmem_wait_ld(acc);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int b = 4 * un + e;
+                *reinterpret_cast<float4 *>(gc + ((size_t)b * Q + q0b) * 2) =
+                    make_float4(acc[2 * e].x, acc[2 * e + 1].x, acc[2 * e].y, acc[2 * e + 1].y);   // (z0.x, z0.y, z1.x, z1.y)
+            }
+        }
+    }
+    if (rank == 0 && lane == 0 && warp < NBLK) diag_max(&p.diag->max_defect, defect);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync();             // no CTA leaves while a peer may still address its shared memory
+    if (*abort_flag) settle_after_abort();
+    if (warp == 0) tmem_dealloc_512(tmem_base);
+}
+
 }  // namespace bcjr
