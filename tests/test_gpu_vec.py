@@ -110,6 +110,14 @@ def test_full_block_length_sampled_blocks(ctx):
     assert got["diag"].max_posterior_defect < 1e-3
 
 
+def test_long_blocks_fall_back_to_the_one_cta_kernels(ctx):
+    # 1030 weights per block: the cluster forward kernel still takes it (<= 2048), the cluster
+    # backward kernel does not (<= 1024) and hands over to the one-CTA kernel; 2100 exceeds both
+    for nt in (515, 1050):
+        got = _check(ctx, 16, 2, 2, nt, 1, 0.3, seed=8600 + nt, what=f"V=2 Lb=16 nt={nt}")
+        assert got["diag"].device_status == 0
+
+
 def test_single_emission_forwards_to_the_scalar_call_and_bad_arguments(ctx):
     import torch
     from paper_2605_10655_b200 import BcjrError
