@@ -1,0 +1,46 @@
+"""Pins of the QAT-loop oracle (schedule, computed Gaussian table, Adam) against closed forms."""
+import numpy as np
+from scipy.stats import norm
+
+from oracle import qat_oracle as qo
+
+
+def test_schedule_end_points_and_constant_ratio():
+    T0, Te, N = 1.0, 0.02, 10
+    T = [qo.temperature(T0, Te, t, N) for t in range(N + 1)]
+    assert T[0] == T0 and abs(T[-1] - Te) < 1e-15
+    r = np.array(T[1:]) / np.array(T[:-1])
+    np.testing.assert_allclose(r, (Te / T0) ** (1.0 / N), rtol=1e-13)
+
+
+def test_gaussian_table_inverts_the_normal_cdf_at_cell_centres():
+    for Lb in (4, 8, 16):
+        S = 1 << Lb
+        c = qo.gaussian_codebook(Lb)
+        np.testing.assert_allclose(norm.cdf(c), (np.arange(S) + 0.5) / S, rtol=0, atol=1e-13)   # independent routine
+        np.testing.assert_allclose(c, -c[::-1], atol=1e-12)                                      # antisymmetric
+        assert np.all(np.diff(c) > 0)
+    assert abs(qo.gaussian_codebook(16).var() - 1.0) < 1e-3
+
+
+def test_adam_first_step_and_constant_gradient_closed_forms():
+    rng = np.random.default_rng(3)
+    p0 = rng.standard_normal(50); g = rng.standard_normal(50) * 10.0 ** rng.integers(-6, 3, 50)
+    lr, eps = 1e-3, 1e-8
+    p, m, v = qo.adam_update(p0, g, 0.0, 0.0, 1, lr, eps=eps)
+    np.testing.assert_allclose(p, p0 - lr * g / (np.abs(g) + eps), rtol=1e-12, atol=0)
+    # constant gradient: the bias-corrected moments equal g and g^2 at every step
+    m = np.zeros(50); v = np.zeros(50); p = p0.copy()
+    for t in range(1, 8):
+        p, m, v = qo.adam_update(p, g, m, v, t, lr, eps=eps)
+    np.testing.assert_allclose(p, p0 - 7 * lr * g / (np.abs(g) + eps), rtol=1e-10, atol=0)
+
+
+def test_adam_zero_gradient_and_moment_decay():
+    p0 = np.array([1.0, -2.0]); m0 = np.array([0.5, -0.25]); v0 = np.array([4.0, 1.0])
+    p, m, v = qo.adam_update(p0, np.zeros(2), m0, v0, 3, 0.1, 0.9, 0.999, 1e-8)
+    np.testing.assert_allclose(m, 0.9 * m0); np.testing.assert_allclose(v, 0.999 * v0)
+    expect = p0 - 0.1 * (0.9 * m0 / (1 - 0.9 ** 3)) / (np.sqrt(0.999 * v0 / (1 - 0.999 ** 3)) + 1e-8)
+    np.testing.assert_allclose(p, expect, rtol=1e-14)
+    p, _, _ = qo.adam_update(p0, np.zeros(2), 0.0, 0.0, 1, 0.1)
+    np.testing.assert_array_equal(p, p0)
