@@ -291,6 +291,23 @@ def main():
         vms = e0.elapsed_time(e1)
         vit = {"ms": vms, "edges_per_s": nblocks * wl.steps * wl.S * wl.K / (vms * 1e-3)}
 
+    # ---- the Adam update that follows the backward pass in the QAT loop (HBM-bound: 28 bytes per weight)
+    upd = None
+    if not args.no_viterbi:
+        big = max(mats, key=lambda m: m["W"].numel())
+        numel = big["W"].numel()
+        mW = torch.zeros_like(big["W"]); vW = torch.zeros_like(big["W"]); Wc = big["W"].clone()
+        ctx.bcjr_adam_update(Wc, big["gW"], mW, vW, 1, 1e-4)       # warm-up
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.bcjr_adam_update(Wc, big["gW"], mW, vW, 2, 1e-4)
+        e1.record()
+        torch.cuda.synchronize()
+        ums = e0.elapsed_time(e1)
+        upd = {"kernel": "adam_kernel", "weights": numel, "ms": ums, "gbs": 28.0 * numel / (ums * 1e-3) / 1e9}
+        del mW, vW, Wc
+
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
     e2e = None
     if not args.no_e2e and wl.V == 1:          # the host-buffer entry point covers the scalar trellis
@@ -368,7 +385,7 @@ def main():
                           "path": "cluster" if diag.last_path else "generic"},
                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": base,
                "breakdown": {"fwd_ms_per_step": fwd_ms / args.steps, "bwd_ms_per_step": bwd_ms / args.steps,
-                             "viterbi": vit, "max_posterior_defect": diag.max_posterior_defect}}
+                             "viterbi": vit, "qat_update": upd, "max_posterior_defect": diag.max_posterior_defect}}
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

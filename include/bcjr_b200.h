@@ -146,6 +146,33 @@ bcjr_status viterbi_hard_vec(bcjr_ctx *ctx, const float *W, const float *codeboo
                              uint16_t *states, float *hard, void *cuda_stream);
 
 /*
+ * The steps on either side of the trellis pass in the per-layer QAT loop (Algorithm 1).
+ *
+ * bcjr_temperature: the annealing schedule of Section 3.6, T_t = T_0 (T_end / T_0)^(t / N_steps)
+ *   (host arithmetic; t = 0 gives T_0, t = N_steps gives T_end; 0.0 on invalid arguments).
+ * bcjr_gaussian_codebook: the computed Gaussian emission of Section 3.1 written out as a table,
+ *   codebook[s] = Phi^-1((s + 1/2) / 2^Lb), s = 0 .. 2^Lb - 1 (device out).  The paper's "incoherent
+ *   permutation" of this table is not specified and is not applied.
+ * bcjr_adam_update: one Adam step (the update Algorithm 1 applies to the continuous pre-image) on a
+ *   device array, in place: m, v are the moment buffers (device, same size, zero before step 1),
+ *   t >= 1 the step number; bias-corrected.  All four arrays 16-byte aligned (BCJR_EINVAL otherwise).
+ * bcjr_backward_adam: bcjr_backward into context-owned gradient buffers followed by the Adam step
+ *   on W_latent (which must be the W given to the last forward call on this context) and, when
+ *   `codebook` is not NULL (then it must be that call's codebook), on the table with step size lr_c.
+ *   The saved forward state is consumed: the next bcjr_backward needs a new forward call.
+ * The paper has the loss of Algorithm 1 (layer output against the teacher's) outside these calls:
+ * the caller turns the soft codeword into grad_soft.
+ */
+double bcjr_temperature(double T0, double T_end, int t, int n_steps);
+bcjr_status bcjr_gaussian_codebook(bcjr_ctx *ctx, int Lb, float *codebook, void *cuda_stream);
+bcjr_status bcjr_adam_update(bcjr_ctx *ctx, float *param, const float *grad, float *m, float *v,
+                             int64_t numel, int t, float lr, float beta1, float beta2, float eps,
+                             void *cuda_stream);
+bcjr_status bcjr_backward_adam(bcjr_ctx *ctx, const float *grad_soft, float *W_latent, float *m_W, float *v_W,
+                               float *codebook, float *m_c, float *v_c, int t, float lr_W, float lr_c,
+                               float beta1, float beta2, float eps, void *cuda_stream);
+
+/*
  * BCJR-STE forward (Section 3.7, "BCJR-STE variant"): the value that goes forward is the hard
  * Viterbi codeword, while the state saved on the context is that of the temperature-T relaxation,
  * so that a following bcjr_backward returns the gradient of the finite-temperature soft codeword

@@ -13,7 +13,8 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libbcjr_b200.so"
 
 EXPORTS = ["bcjr_create", "bcjr_destroy", "bcjr_set_option", "bcjr_soft_quantize", "bcjr_backward",
-           "viterbi_hard", "bcjr_soft_quantize_vec", "viterbi_hard_vec", "bcjr_ste_forward", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
+           "viterbi_hard", "bcjr_soft_quantize_vec", "viterbi_hard_vec", "bcjr_ste_forward", "bcjr_temperature", "bcjr_gaussian_codebook", "bcjr_adam_update",
+           "bcjr_backward_adam", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
            "bcjr_last_cuda_error", "bcjr_status_string", "bcjr_soft_quantize_static",
            "bcjr_static_scratch_bytes"]
 
@@ -56,6 +57,13 @@ def load_library() -> ctypes.CDLL:
     lib.viterbi_hard_vec.argtypes = [vp, vp, vp, i, i, i, i, i64, vp, i64, vp, vp, vp]
     lib.bcjr_ste_forward.restype = i
     lib.bcjr_ste_forward.argtypes = [vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
+    lib.bcjr_temperature.restype = ctypes.c_double
+    lib.bcjr_temperature.argtypes = [ctypes.c_double, ctypes.c_double, i, i]
+    lib.bcjr_gaussian_codebook.restype = i; lib.bcjr_gaussian_codebook.argtypes = [vp, i, vp, vp]
+    lib.bcjr_adam_update.restype = i
+    lib.bcjr_adam_update.argtypes = [vp, vp, vp, vp, vp, i64, i, f, f, f, f, vp]
+    lib.bcjr_backward_adam.restype = i
+    lib.bcjr_backward_adam.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, f, f, f, f, f, vp]
     lib.bcjr_step_host.restype = i
     lib.bcjr_step_host.argtypes = [vp, vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
     lib.bcjr_sync_status.restype = i; lib.bcjr_sync_status.argtypes = [vp, vp, ctypes.POINTER(Diag)]
@@ -67,6 +75,11 @@ def load_library() -> ctypes.CDLL:
     lib.bcjr_static_scratch_bytes.restype = i64; lib.bcjr_static_scratch_bytes.argtypes = []
     _lib = lib
     return lib
+
+
+def temperature(T0: float, T_end: float, t: int, n_steps: int) -> float:
+    """Annealing schedule of Section 3.6 (library routine)."""
+    return float(load_library().bcjr_temperature(T0, T_end, t, n_steps))
 
 
 def status_string(code: int) -> str:
@@ -249,6 +262,41 @@ class Context:
         self._check(rc, "bcjr_ste_forward")
         self._saved = (W, codebook, Lb, B * n)
         return hard, states, soft
+
+    def bcjr_gaussian_codebook(self, Lb, device=None, stream=None):
+        """Table of the computed Gaussian emission c(s) = Phi^-1((s + 1/2) / 2^Lb)."""
+        import torch
+        out = torch.empty(1 << Lb, dtype=torch.float32, device=torch.device("cuda", self.device) if device is None else device)
+        self._check(self._lib.bcjr_gaussian_codebook(self._h, Lb, ctypes.c_void_p(out.data_ptr()), _stream_ptr(stream)),
+                    "bcjr_gaussian_codebook")
+        return out
+
+    def bcjr_adam_update(self, param, grad, m, v, t, lr, beta1=0.9, beta2=0.999, eps=1e-8, stream=None):
+        """One Adam step on `param` in place (m, v: moment buffers of the same size)."""
+        import torch
+        n = param.numel()
+        rc = self._lib.bcjr_adam_update(self._h, _dev(param, torch.float32, n, "param"), _dev(grad, torch.float32, n, "grad"),
+                                        _dev(m, torch.float32, n, "m"), _dev(v, torch.float32, n, "v"), n, int(t),
+                                        float(lr), float(beta1), float(beta2), float(eps), _stream_ptr(stream))
+        self._check(rc, "bcjr_adam_update")
+
+    def bcjr_backward_adam(self, grad_soft, m_W, v_W, t, lr_W, m_c=None, v_c=None, lr_c=0.0,
+                           beta1=0.9, beta2=0.999, eps=1e-8, stream=None):
+        """Backward pass + Adam on the W (and, with m_c/v_c, the codebook) of the last forward call, in place."""
+        import torch
+        if self._saved is None:
+            raise BcjrError(-4, "bcjr_backward_adam")
+        W, codebook, Lb, numel = self._saved
+        upd_c = m_c is not None
+        rc = self._lib.bcjr_backward_adam(
+            self._h, _dev(grad_soft, torch.float32, numel, "grad_soft"), _dev(W, torch.float32, numel, "W"),
+            _dev(m_W, torch.float32, numel, "m_W"), _dev(v_W, torch.float32, numel, "v_W"),
+            _dev(codebook, torch.float32, codebook.numel(), "codebook") if upd_c else None,
+            _dev(m_c, torch.float32, codebook.numel(), "m_c") if upd_c else None,
+            _dev(v_c, torch.float32, codebook.numel(), "v_c") if upd_c else None,
+            int(t), float(lr_W), float(lr_c), float(beta1), float(beta2), float(eps), _stream_ptr(stream))
+        self._check(rc, "bcjr_backward_adam")
+        self._saved = None
 
     def bcjr_step_host(self, W, codebook, grad_soft, Lb, k, n, T, soft=None, grad_W=None, grad_codebook=None,
                        stream=None):

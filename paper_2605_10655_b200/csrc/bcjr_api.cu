@@ -14,6 +14,7 @@
 #include "bcjr_cluster.cuh"
 #include "bcjr_vec.cuh"
 #include "bcjr_vec4.cuh"
+#include "bcjr_qat.cuh"
 #include "bcjr_solo.cuh"
 #include "bcjr_duo.cuh"
 #include "bcjr_viterbi.cuh"
@@ -36,7 +37,7 @@ struct bcjr_ctx {
     int device = 0;
     int num_sms = 0;
     int max_smem_optin = 0;
-    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, cb_beta, staging[6];
+    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, cb_beta, grad_w, grad_c, staging[6];
     DeviceDiag *diag = nullptr;
     // saved by bcjr_soft_quantize for bcjr_backward
     bool have_fwd = false;
@@ -533,7 +534,7 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx)
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
     Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp, &ctx->path_ws,
-                     &ctx->cb_beta, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
+                     &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
                      &ctx->staging[5]};
     for (Buffer *b : all)
         if (b->ptr) cudaFree(b->ptr);
@@ -827,6 +828,70 @@ bcjr_status bcjr_ste_forward(bcjr_ctx *ctx, const float *W, const float *codeboo
     return rc;
 }
 
+double bcjr_temperature(double T0, double T_end, int t, int n_steps)
+{
+    if (!(T0 > 0.0) || !(T_end > 0.0) || n_steps < 1) return 0.0;
+    return T0 * std::pow(T_end / T0, (double)t / (double)n_steps);
+}
+
+bcjr_status bcjr_gaussian_codebook(bcjr_ctx *ctx, int Lb, float *codebook, void *cuda_stream)
+{
+    if (!ctx || !codebook || Lb < 1 || Lb > 16) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    const int S = 1 << Lb;
+    gaussian_table_kernel<<<(S + 255) / 256, 256, 0, (cudaStream_t)cuda_stream>>>(codebook, S);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_adam_update(bcjr_ctx *ctx, float *param, const float *grad, float *m, float *v, int64_t numel,
+                             int t, float lr, float beta1, float beta2, float eps, void *cuda_stream)
+{
+    if (!ctx || numel < 0 || t < 1) return BCJR_EINVAL;
+    if (!(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps > 0.f) || !std::isfinite(lr)) return BCJR_EINVAL;
+    if (numel == 0) return BCJR_OK;
+    if (!param || !grad || !m || !v) return BCJR_EINVAL;
+    if (((uintptr_t)param | (uintptr_t)grad | (uintptr_t)m | (uintptr_t)v) & 15u) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    AdamParams a{};
+    a.p = param; a.g = grad; a.m = m; a.v = v; a.numel = numel;
+    a.lr_c1 = (float)((double)lr / (1.0 - std::pow((double)beta1, (double)t)));
+    a.inv_c2 = (float)(1.0 / (1.0 - std::pow((double)beta2, (double)t)));
+    a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
+    int64_t blocks = (numel / 4 + 255) / 256;
+    const int64_t cap = (int64_t)ctx->num_sms * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    adam_kernel<<<(int)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(a);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_backward_adam(bcjr_ctx *ctx, const float *grad_soft, float *W_latent, float *m_W, float *v_W,
+                               float *codebook, float *m_c, float *v_c, int t, float lr_W, float lr_c,
+                               float beta1, float beta2, float eps, void *cuda_stream)
+{
+    if (!ctx) return BCJR_EINVAL;
+    if (!ctx->have_fwd) return BCJR_ESTATE;
+    if (W_latent != ctx->W || (codebook && codebook != ctx->cb)) return BCJR_EINVAL;   // must be the saved tensors
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    const int64_t numel = ctx->B * ctx->n, csize = ((int64_t)1 << ctx->Lb) * ctx->V;
+    bcjr_status rc;
+    if ((rc = ensure(ctx, ctx->grad_w, (size_t)(numel > 0 ? numel : 1) * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->grad_c, (size_t)csize * 4))) return rc;
+    float *gW = (float *)ctx->grad_w.ptr, *gc = (float *)ctx->grad_c.ptr;
+    if ((rc = bcjr_backward(ctx, grad_soft, gW, codebook ? gc : nullptr, cuda_stream))) return rc;
+    if ((rc = bcjr_adam_update(ctx, W_latent, gW, m_W, v_W, numel, t, lr_W, beta1, beta2, eps, cuda_stream))) return rc;
+    if (codebook && (rc = bcjr_adam_update(ctx, codebook, gc, m_c, v_c, csize, t, lr_c, beta1, beta2, eps, cuda_stream))) return rc;
+    ctx->have_fwd = false;      // the saved inputs have changed: a new forward call is needed
+    return BCJR_OK;
+}
+
 bcjr_status bcjr_step_host(bcjr_ctx *ctx, const float *W_host, const float *codebook_host,
                            const float *grad_soft_host, int Lb, int k, int n, int64_t num_blocks, float T,
                            float *soft_host, float *grad_W_host, float *grad_codebook_host, void *cuda_stream)
@@ -883,7 +948,7 @@ int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx)
 {
     if (!ctx) return 0;
     const Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp,
-                           &ctx->path_ws, &ctx->cb_beta, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
+                           &ctx->path_ws, &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
                            &ctx->staging[4], &ctx->staging[5]};
     int64_t tot = 0;
     for (const Buffer *b : all) tot += (int64_t)b->bytes;

@@ -39,6 +39,11 @@ def test_status_strings_and_host_side_argument_checks():
     assert lib.viterbi_hard_vec(None, None, None, 8, 2, 2, 64, 1, None, 0, None, None, None) == -1
     assert lib.bcjr_ste_forward(None, None, None, 8, 2, 64, 1, 0.5, None, None, None, None) == -1
     assert lib.bcjr_destroy(None) == -1
+    assert lib.bcjr_adam_update(None, None, None, None, None, 4, 1, 1e-3, 0.9, 0.999, 1e-8, None) == -1
+    assert lib.bcjr_gaussian_codebook(None, 8, None, None) == -1
+    # the schedule is host arithmetic: end points and the constant ratio of Section 3.6
+    assert binding.temperature(1.0, 0.02, 0, 10) == 1.0 and abs(binding.temperature(1.0, 0.02, 10, 10) - 0.02) < 1e-15
+    assert abs(binding.temperature(1.0, 0.02, 3, 10) - 0.02 ** 0.3) < 1e-15 and binding.temperature(-1.0, 0.02, 1, 10) == 0.0
     assert binding.path_bytes(16, 2, 256) == 66 and binding.path_bytes(16, 3, 256) == 98
 
 
