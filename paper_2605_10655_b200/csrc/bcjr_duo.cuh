@@ -6,20 +6,25 @@
 // tensor memory is used: each CTA keeps its half of the codebook (64 columns per thread) and its
 // half of the accumulators (64 columns per thread) in TMEM, lane-private, exactly the access
 // pattern of a thread that owns the same butterflies for the whole kernel.  Registers are then
-// free for the arithmetic, shared memory for the messages and the history ring, and clusters
+// free for the arithmetic, shared memory for the messages and the history staging, and clusters
 // of two fill all 148 SMs (clusters of four, needed when the accumulators live in registers,
 // fill only 132).
 //
 // Step protocol.  Messages are double-buffered.  Every output is pushed with st.async into the
 // consumer CTA's buffer `ob` and credits that CTA's mbarrier full[ob] with its bytes; a phase of
 // full[ob] completes when (a) all bytes have landed and (b) every warp of the cluster has
-// arrived on it after its last butterfly of the step (thread 0 of each CTA only after the bulk
-// copy that spills the input buffer to the history has finished reading it) -- so nobody still
-// reads the other buffer when the next step starts overwriting it.  The arrival is relaxed:
+// arrived on it after its last butterfly of the step -- so nobody still reads the other buffer
+// when the next step starts overwriting it.  The arrival is relaxed:
 // it has nothing to publish (the data travels with st.async and is accounted in bytes), and the
 // reads it has to follow are complete when it issues, because every value a warp reads from
 // its input buffer feeds, through register dependences, an st.async that precedes the arrival
 // in program order.  (A release arrival per warp costs a cluster-scope fence: 8 % of the kernel.)
+//
+// History.  The inputs (L, At) of a butterfly in the alpha sweep are exactly what the same thread
+// needs for that butterfly in the beta sweep, so the history is thread-private: the thread stores
+// its inputs with 16-byte global stores ([step][CTA][butterfly slot][16-byte chunk][thread]) and
+// streams them back with cp.async into its own staging slots, RD - 1 butterflies ahead
+// (cp.async.wait_group; no mbarrier, no producer thread, no branch in the butterfly loop).
 #pragma once
 #include "bcjr_solo.cuh"
 
@@ -45,18 +50,18 @@ struct DuoCfg {
     static constexpr int UNITS = K * K / 16;                   // 16-column TMEM units per butterfly
     static constexpr int HPU = (K / 2) / UNITS;                // pairs h (alpha) / jh (beta) per unit
     static constexpr int SLOTS = CL * NWARP;                   // 32 per-warp partial slots
-    static constexpr int CH = K * THREADS;                     // floats per array per history chunk
-    static constexpr int RD = KB == 2 ? BPT + 1 : 3;           // ring depth in chunks
+    static constexpr int NCH = 2 * K / 4;                      // 16-byte chunks per butterfly and thread: K values of L, K of At
+    static constexpr int RD = KB == 2 ? BPT + 1 : 3;           // staging depth in butterflies
     static constexpr int MAX_N = 1024;
     static constexpr int ARRIVALS = 1 + SLOTS;                 // armer + one arrival per warp of the cluster
     static constexpr int OFF_MSG = 0;                          // [2 parity][2 arrays][QC]
-    static constexpr int OFF_RING = OFF_MSG + 4 * QC;          // [RD][2 arrays][CH]
-    static constexpr int OFF_O = OFF_RING + RD * 2 * CH;       // int [MAX_N + 2]
+    static constexpr int OFF_RING = OFF_MSG + 4 * QC;          // float4 [RD][NCH][THREADS]
+    static constexpr int OFF_O = OFF_RING + RD * NCH * THREADS * 4;   // int [MAX_N + 2]
     static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;     // [2][32]
     static constexpr int OFF_PART = OFF_WMAX + 64;             // [2][32][4]
     static constexpr int OFF_LZ = OFF_PART + 256;              // [32]
-    static constexpr int OFF_MBAR = OFF_LZ + 32;               // uint64: ring_full[RD], ring_empty[RD], full[2]
-    static constexpr int NMBAR = 2 * RD + 2;
+    static constexpr int OFF_MBAR = OFF_LZ + 32;               // uint64: full[2]
+    static constexpr int NMBAR = 2;
     static constexpr int OFF_TMEM = OFF_MBAR + 2 * NMBAR;
     static constexpr int OFF_FLAG = OFF_TMEM + 2;
     static constexpr int SMEM_FLOATS = OFF_FLAG + 2;
@@ -74,7 +79,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
 {
     using C = DuoCfg<KB>;
     constexpr int K = C::K, NB = C::NB, NBC = C::NBC, QC = C::QC, BPT = C::BPT, NWARP = C::NWARP, CT = C::THREADS;
-    constexpr int CL = C::CL, SLOTS = C::SLOTS, CH = C::CH, RD = C::RD, UNITS = C::UNITS, HPU = C::HPU, NU = BPT * UNITS;
+    constexpr int CL = C::CL, SLOTS = C::SLOTS, NCH = C::NCH, RD = C::RD, UNITS = C::UNITS, HPU = C::HPU, NU = BPT * UNITS;
     constexpr int KK = K * K;
     constexpr uint32_t BUF_BYTES = 2u * QC * 4u;                 // (L, At) of one parity
     constexpr uint32_t TX_MSG = BUF_BYTES + SLOTS * 4u;          // messages + gauge slots
@@ -89,7 +94,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     const float2 nl2 = splat2(-p.lam2);
 
     float *msg = smem + C::OFF_MSG;
-    float *ring = smem + C::OFF_RING;
+    float4 *stage4 = reinterpret_cast<float4 *>(smem + C::OFF_RING);      // [RD][NCH][CT], thread-private entries
     int *O_s = reinterpret_cast<int *>(smem + C::OFF_O);
     float *wmax = smem + C::OFF_WMAX;
     float *part = smem + C::OFF_PART;
@@ -97,20 +102,18 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
     Proto pr{1u, abort_flag, p.diag};
-    const uint32_t ring_full = smem_u32(smem + C::OFF_MBAR);
-    const uint32_t ring_empty = ring_full + 8u * RD;
-    const uint32_t mbar_full = ring_empty + 8u * RD;             // [2], one per message parity
-    const uint32_t msg_u32 = smem_u32(msg), ring_u32 = smem_u32(ring);
+    const uint32_t mbar_full = smem_u32(smem + C::OFF_MBAR);     // [2], one per message parity
+    const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage4) + (uint32_t)tid * 16u;
     const uint32_t wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
 
-    float *hist = p.hist + (size_t)cid * n * 2 * C::Q;           // [n][CL][2][QC]
+    // history of this cluster: float4 [n][CL][BPT][NCH][CT]; this thread's entries
+    float4 *hist4 = reinterpret_cast<float4 *>(p.hist + (size_t)cid * n * 2 * C::Q) + tid;
 
     uint32_t full_of[CL];
 #pragma unroll
     for (int r = 0; r < CL; ++r) full_of[r] = mapa_u32(mbar_full, (uint32_t)r);
 
     if (tid == 0) {
-        for (int s = 0; s < RD; ++s) { mbar_init(ring_full + 8u * s, 1); mbar_init(ring_empty + 8u * s, NWARP); }
         for (int s = 0; s < 2; ++s) mbar_init(mbar_full + 8u * s, C::ARRIVALS);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -165,8 +168,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
 #ifdef BCJR_TIMING
     unsigned long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #endif
-    uint32_t chunk = 0;            // history chunks consumed so far (all threads count alike)
-    uint32_t issued = 0;           // history chunks requested so far (thread 0)
+    // test hook for the waits' abort path: one warp of CTA 0 withholds an arrival of its first block
+    const bool drop_hook = blockIdx.x == 0 && warp == 1 && p.diag->drop_history_load != 0;
     float defect = 0.f;
 
     for (int64_t blk = cid; blk < p.B; blk += ncl) {
@@ -197,12 +200,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             if (!pr.warp_live()) break;                          // a wait ran out: this warp issues nothing more
             const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
-            if (tid == 0) {
-                mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
-                fence_proxy_async();                                           // spill (L_t, At_t)
-                bulk_store(hist + ((size_t)(t - 1) * CL + rank) * 2 * QC, msg_u32 + (uint32_t)ib * BUF_BYTES, BUF_BYTES);
-                bulk_commit();
-            }
+            if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
+            float4 *hrow = hist4 + ((size_t)(t - 1) * CL + rank) * (BPT * NCH * CT);      // (L_t, At_t) of this thread's butterflies
             const float gt = __ldg(g_s + t - 1);
             // shift for the consumers of this step's At (step t+1); unused at t = n
             const float2 gshn2 = splat2(t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f);
@@ -218,6 +217,11 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 for (int j = 0; j < K; ++j) {
                     Lj[j] = Lin[(i * K + j) * CT + tid];
                     Aj[j] = Ain[(i * K + j) * CT + tid];
+                }
+#pragma unroll
+                for (int q = 0; q < K / 4; ++q) {
+                    hrow[(i * NCH + q) * CT] = make_float4(Lj[4 * q], Lj[4 * q + 1], Lj[4 * q + 2], Lj[4 * q + 3]);
+                    hrow[(i * NCH + K / 4 + q) * CT] = make_float4(Aj[4 * q], Aj[4 * q + 1], Aj[4 * q + 2], Aj[4 * q + 3]);
                 }
 #pragma unroll
                 for (int u = 0; u < UNITS; ++u) {
@@ -260,10 +264,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
             }
             O += (int)off;
-            if (tid == 0) {
-                O_s[t + 1] = O;
-                bulk_wait_read0();                               // the spill has left the input buffer
-            }
+            if (tid == 0) O_s[t + 1] = O;
             __syncwarp();
             if (lane == 0) {                                     // this warp has read all its inputs
 #pragma unroll
@@ -283,7 +284,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
 #pragma unroll
                 for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
             }
-            if (tid == 0) bulk_wait_all0();                      // history written before it is read back
             cluster_sync();                                      // log Z exchange
         }
         const float lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
@@ -300,25 +300,22 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         tmem_wait_st();
         int P = 0;
         float offM = 0.f;
-        const uint32_t chunk_end = chunk + (uint32_t)n * BPT;    // chunks of this block: (t = n..1) x (i = 0..BPT-1)
-        // thread 0 streams the history back: request every chunk whose ring slot has been
-        // released by all warps, without ever blocking (called between butterflies)
-        auto feed_ring = [&]() {
-            while (pr.live && issued != chunk_end) {
-                const uint32_t s = issued % RD;
-                if (!mbar_test(ring_empty + 8u * s, ((issued / RD) & 1u) ^ 1u)) break;
-                const uint32_t rel = issued - (chunk_end - (uint32_t)n * BPT);
-                const int t = n - (int)(rel / BPT), i = (int)(rel % BPT);
-                pr.expect_tx(ring_full + 8u * s, 2u * CH * 4u);
-                const float *src = hist + ((size_t)(t - 1) * CL + rank) * 2 * QC + (size_t)i * CH;
-                if (!(issued == 0 && blockIdx.x == 0 && p.diag->drop_history_load)) {   // test hook: a wait that runs out
-                    pr.load(ring_u32 + s * 2u * CH * 4u, src, CH * 4u, ring_full + 8u * s);
-                    pr.load(ring_u32 + s * 2u * CH * 4u + CH * 4u, src + QC, CH * 4u, ring_full + 8u * s);
-                }
-                ++issued;
+        // history stream: chunk c of this block = butterfly (t = n - c / BPT, i = c % BPT), staged RD - 1 ahead
+        const uint32_t nchunks = (uint32_t)n * BPT;
+        auto issue_chunk = [&](uint32_t c, uint32_t slot) {
+            if (c < nchunks) {
+                const int t = n - (int)(c / BPT), i = (int)(c % BPT);
+                const float4 *src = hist4 + (((size_t)(t - 1) * CL + rank) * BPT + i) * (NCH * CT);
+                const uint32_t dst = stage_u32 + slot * (uint32_t)(NCH * CT * 16);
+#pragma unroll
+                for (int q = 0; q < NCH; ++q)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(src + q * CT) : "memory");
             }
+            asm volatile("cp.async.commit_group;" ::: "memory");
         };
-        if (tid == 0) { fence_proxy_async(); feed_ring(); }
+#pragma unroll
+        for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c, c);
+        uint32_t chunk = 0, slot = 0;                            // next chunk to consume and its staging slot
         cluster_sync();                                          // beta start
         // rank 0, warp 0: turn the sums of step t (slots of parity b) into grad_W[t]
         auto finish_step = [&](int t, int b) {
@@ -359,12 +356,18 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             tmem_ld16(tm_cb, cb[0]);
 #pragma unroll
             for (int i = 0; i < BPT; ++i, ++chunk) {
-                if (tid == 0) feed_ring();
-                const uint32_t s = chunk % RD;
                 TICK(tr0);
-                pr.wait(ring_full + 8u * s, (chunk / RD) & 1u);
+                issue_chunk(chunk + RD - 1, slot == 0 ? RD - 1 : slot - 1);          // refill the slot consumed last
+                asm volatile("cp.async.wait_group %0;" ::"n"(RD - 1) : "memory");     // chunk `chunk` has landed
                 TICK(tr1); TACC(3, tr0, tr1);
-                const float *Lh = ring + s * 2 * CH, *Ah = Lh + CH;
+                float Lh[K], Ah[K];
+#pragma unroll
+                for (int q = 0; q < K / 4; ++q) {
+                    const float4 l4 = stage4[(slot * NCH + q) * CT + tid], a4 = stage4[(slot * NCH + K / 4 + q) * CT + tid];
+                    Lh[4 * q] = l4.x; Lh[4 * q + 1] = l4.y; Lh[4 * q + 2] = l4.z; Lh[4 * q + 3] = l4.w;
+                    Ah[4 * q] = a4.x; Ah[4 * q + 1] = a4.y; Ah[4 * q + 2] = a4.z; Ah[4 * q + 3] = a4.w;
+                }
+                slot = slot + 1 == RD ? 0 : slot + 1;
                 float Mb[K], Yb[K];
 #pragma unroll
                 for (int b = 0; b < K; b += 4) {
@@ -391,8 +394,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                             uu[b] = fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
                         }
                         const float2 m = max_pairs<K>(uu);
-                        const float2 Ahj = sub2(make_float2(Ah[(2 * jh) * CT + tid], Ah[(2 * jh + 1) * CT + tid]), gsh2);
-                        const float2 Lhj = make_float2(Lh[(2 * jh) * CT + tid], Lh[(2 * jh + 1) * CT + tid]);
+                        const float2 Ahj = sub2(make_float2(Ah[2 * jh], Ah[2 * jh + 1]), gsh2);
+                        const float2 Lhj = make_float2(Lh[2 * jh], Lh[2 * jh + 1]);
                         const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
                         const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
                         if (!acc_ready) { tmem_wait_ld(acc); acc_ready = true; }
@@ -421,8 +424,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                     }
                     tmem_st16(tm_acc + 16u * g, acc);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive_local(ring_empty + 8u * s);               // history chunk consumed by this warp
             }
             tmem_wait_st();
             const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), zz = warp_sum(ZS.x + ZS.y);
@@ -435,12 +436,13 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             TICK(tb0);
             __syncwarp();
             TICK(tb1); TACC(1, tb0, tb1); TACC(0, tk0, tb1);
-            if (lane == 0) {                                     // this warp has read all its inputs
+            if (lane == 0 && !(drop_hook && t == n && blk == cid)) {   // this warp has read all its inputs
 #pragma unroll
                 for (int r = 0; r < CL; ++r) mbar_arrive_remote(full_of[r] + ob_mbar);
             }
             ib = ob;
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         wait_inputs(ib);                                         // the sums of step 1
         finish_step(1, ib);
         cluster_sync();                                          // block end
@@ -471,7 +473,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         for (int e = 0; e < 8; ++e) g_duo_timing[e] = tacc[e];
 #endif
     if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
-    if (*abort_flag && tid == 0) drain_bulk_loads(ring_full, issued, RD, p.diag);   // no copy may be in flight at exit
+    asm volatile("cp.async.wait_all;" ::: "memory");           // no copy may be in flight at exit (a warp may have left the loop early)
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     cluster_sync();             // no CTA leaves while a peer may still address its shared memory
