@@ -11,10 +11,12 @@
 // the compressed message vector (64 KB) double-buffered in shared memory, one SM handles a
 // block alone: the per-step exchange is a CTA barrier instead of a cluster-wide handshake.
 //
-// Warp roles: 16 compute warps (512 threads, 8 butterflies each) and one copy warp that moves
-// the history with bulk copies -- alpha: shared -> global, one 64 KB message buffer per step;
-// beta: global -> shared in 8 KB chunks (one butterfly slot of all threads), through a ring of
-// 8 chunks with full/empty mbarriers.
+// 16 warps (512 threads, 8 butterflies each at k = 2), all computing.  The history is
+// thread-private: the alpha inputs L_t of a butterfly are what the same thread needs for that
+// butterfly in the beta sweep, so it stores them with 16-byte global stores
+// ([step][butterfly slot][16-byte chunk][thread]) and streams them back with cp.async into its own
+// staging slots, RD - 1 butterflies ahead (cp.async.wait_group: no mbarrier, no copy warp, no
+// branch in the butterfly loop).  No thread of this kernel spins on anything.
 #pragma once
 #include "bcjr_cluster.cuh"
 
@@ -71,25 +73,24 @@ __device__ __forceinline__ void compute_barrier(int nthreads)
 template <int KB_>
 struct SoloCfg {
     static constexpr int LB = 16, KB = KB_, K = 1 << KB, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB);
-    static constexpr int CTHREADS = 512;                       // compute threads
-    static constexpr int THREADS = CTHREADS + 32;              // + the copy warp
+    static constexpr int CTHREADS = 512;                       // every thread computes
+    static constexpr int THREADS = CTHREADS;
     static constexpr int NWARP = CTHREADS / 32;
     static constexpr int BPT = NB / CTHREADS;                  // butterflies per thread
     static constexpr int UNITS = K * K / 16;                   // 16-column units per butterfly
     static constexpr int HPU = (K / 2) / UNITS;                // pairs h (alpha) or jh (beta) covered by one unit
-    static constexpr int CH = K * CTHREADS;                    // floats per history chunk (one slot of all threads)
-    static constexpr int RD = KB == 2 ? BPT : 4;               // ring depth in chunks
+    static constexpr int NCH = K / 4;                          // 16-byte chunks per butterfly and thread (K values of L)
+    static constexpr int RD = KB == 2 ? BPT : 4;               // staging depth in butterflies
     static constexpr int MAX_N = 2048;
     static constexpr int OFF_MSG = 0;                          // [2][Q]
-    static constexpr int OFF_RING = OFF_MSG + 2 * Q;           // [RD][CH]
-    static constexpr int OFF_W = OFF_RING + RD * CH;           // [MAX_N]
+    static constexpr int OFF_RING = OFF_MSG + 2 * Q;           // float4 [RD][NCH][CTHREADS], thread-private entries
+    static constexpr int OFF_W = OFF_RING + RD * NCH * CTHREADS * 4;   // [MAX_N]
     static constexpr int OFF_O = OFF_W + MAX_N;                // int [MAX_N + 2]
     static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;     // [2][32]
     static constexpr int OFF_PART = OFF_WMAX + 64;             // [2][32][2]
     static constexpr int OFF_LZ = OFF_PART + 128;              // [32]
-    static constexpr int OFF_MBAR = OFF_LZ + 32;               // uint64: full[RD], empty[RD], ready[2], freed[2]
-    static constexpr int NMBAR = 2 * RD + 4;
-    static constexpr int OFF_TMEM = OFF_MBAR + 2 * NMBAR;      // uint32 TMEM base
+    static constexpr int OFF_MBAR = OFF_LZ + 32;               // (no mbarrier left in this kernel; kept 8-byte aligned)
+    static constexpr int OFF_TMEM = OFF_MBAR + 2;              // uint32 TMEM base
     static constexpr int OFF_FLAG = OFF_TMEM + 2;
     static constexpr int SMEM_FLOATS = OFF_FLAG + 2;
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
@@ -130,7 +131,7 @@ template <int KB>
 __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdParams p)
 {
     using C = SoloCfg<KB>;
-    constexpr int K = C::K, NB = C::NB, Q = C::Q, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, CH = C::CH, RD = C::RD;
+    constexpr int K = C::K, NB = C::NB, Q = C::Q, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, NCH = C::NCH, RD = C::RD;
     constexpr int UNITS = C::UNITS, HPU = C::HPU, NU = BPT * UNITS;
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -139,64 +140,25 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
     const float2 nl2 = splat2(-p.lam2);
 
     float *msg = smem + C::OFF_MSG;
-    float *ring = smem + C::OFF_RING;
+    float4 *stage4 = reinterpret_cast<float4 *>(smem + C::OFF_RING);
     float *w_s = smem + C::OFF_W;
     int *O_s = reinterpret_cast<int *>(smem + C::OFF_O);
     float *wmax = smem + C::OFF_WMAX;
     float *part = smem + C::OFF_PART;
     float *lz = smem + C::OFF_LZ;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAG);
-    Proto pr{1u, abort_flag, p.diag};
-    const uint32_t mbar_full = smem_u32(smem + C::OFF_MBAR);
-    const uint32_t mbar_empty = mbar_full + 8u * RD;
-    const uint32_t mbar_ready = mbar_empty + 8u * RD;          // [2] compute -> copy warp: buffer holds L_t
-    const uint32_t mbar_freed = mbar_ready + 16u;              // [2] copy warp -> compute: buffer has been read
-    const uint32_t msg_u32 = smem_u32(msg), ring_u32 = smem_u32(ring);
+    const uint32_t stage_u32 = smem_u32(stage4) + (uint32_t)tid * 16u;
 
-    float *hist = p.hist + (size_t)blockIdx.x * n * Q;         // [n][Q], layout of the alpha input buffer
+    // history of this CTA: float4 [n][BPT][NCH][CT], row t = the alpha inputs L_t of every butterfly;
+    // a thread writes and reads back only its own entries
+    float4 *hist4 = reinterpret_cast<float4 *>(p.hist + (size_t)blockIdx.x * n * Q) + tid;
 
-    if (tid == 0) {
-        for (int s = 0; s < RD; ++s) { mbar_init(mbar_full + 8u * s, 1); mbar_init(mbar_empty + 8u * s, NWARP); }
-        for (int s = 0; s < 2; ++s) { mbar_init(mbar_ready + 8u * s, 1); mbar_init(mbar_freed + 8u * s, 1); }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     if (warp == 0) tmem_alloc_512(smem_u32(const_cast<uint32_t *>(tmem_slot)));
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == NWARP) {
-        // ============================ copy warp (one elected lane) ============================
-        if (lane == 0) {
-            uint32_t use_ready[2] = {0u, 0u}, chunk = 0;      // completed phases per mbarrier
-            uint32_t requested = 0;                            // chunks up to the last one actually requested
-            for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
-                for (int t = 1; t <= n; ++t) {                 // alpha: spill L_t once the buffer is complete
-                    const uint32_t b = (uint32_t)(t - 1) & 1u;
-                    pr.wait(mbar_ready + 8u * b, use_ready[b] & 1u);
-                    ++use_ready[b];
-                    fence_proxy_async();
-                    pr.store(hist + (size_t)(t - 1) * Q, msg_u32 + b * Q * 4u, Q * 4u);
-                    bulk_commit();
-                    bulk_wait_read0();
-                    pr.arrive(mbar_freed + 8u * b);
-                }
-                bulk_wait_all0();                              // history written before it is read back
-                for (int t = n; t >= 1; --t)                   // beta: stream L_t back, one slot chunk at a time
-                    for (int i = 0; i < BPT; ++i, ++chunk) {
-                        const uint32_t s = chunk % RD;
-                        pr.wait(mbar_empty + 8u * s, ((chunk / RD) & 1u) ^ 1u);
-                        pr.expect_tx(mbar_full + 8u * s, CH * 4u);
-                        if (chunk == 0 && blockIdx.x == 0 && p.diag->drop_history_load) continue;   // test hook: a wait that runs out
-                        if (pr.live) requested = chunk + 1;
-                        pr.load(ring_u32 + s * CH * 4u, hist + (size_t)(t - 1) * Q + (size_t)i * CH, CH * 4u, mbar_full + 8u * s);
-                    }
-            }
-            if (!pr.live || *abort_flag) drain_bulk_loads(mbar_full, requested, RD, p.diag);   // no copy may be in flight at exit
-        }
-    } else {
+    {
         // ============================ compute warps ============================
         // TMEM: lanes of this warp's sub-partition, 128 columns per thread
         const uint32_t tm = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
@@ -210,7 +172,6 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             const int q2 = x * K, j2 = q2 / NB, x2 = q2 % NB;
             push_a[i] = ((x2 / CT) * K + j2) * CT + (x2 % CT);
         }
-        uint32_t use_freed[2] = {0u, 0u}, chunk = 0;          // completed phases per mbarrier
         float defect = 0.f, zgap = 0.f;
 
         for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
@@ -229,15 +190,11 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                 const int cur = (t - 1) & 1;
                 const float *Lin = msg + cur * Q;
                 float *Lout = msg + (cur ^ 1) * Q;
-                if (tid == 0) pr.arrive(mbar_ready + 8u * cur);                // L_t complete: spill it
                 if (t > 1) {
                     cmax = warp_max(lane < NWARP ? wmax[cur * 32 + lane] : NEG_INF) - off;
                     off = rintf(cmax);
-                    // the buffer written now was spilled during the previous step: wait until read
-                    pr.wait(mbar_freed + 8u * (cur ^ 1), use_freed[cur ^ 1] & 1u);
-                    ++use_freed[cur ^ 1];
                 }
-                if (!pr.warp_live()) { compute_barrier(CT); continue; }          // a wait ran out: only keep the barriers
+                float4 *hrow = hist4 + (size_t)(t - 1) * (BPT * NCH * CT);
                 const float2 w2 = splat2(w_s[t - 1]);
                 const float2 off2 = splat2(off);
                 float tmax = NEG_INF;
@@ -248,6 +205,9 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                     float Lj[K];
 #pragma unroll
                     for (int j = 0; j < K; ++j) Lj[j] = Lin[(i * K + j) * CT + tid];
+#pragma unroll
+                    for (int q = 0; q < NCH; ++q)
+                        hrow[(i * NCH + q) * CT] = make_float4(Lj[4 * q], Lj[4 * q + 1], Lj[4 * q + 2], Lj[4 * q + 3]);
                     float2 out[K / 2];
 #pragma unroll
                     for (int u = 0; u < UNITS; ++u) {
@@ -295,9 +255,6 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             if (tid == 0) diag_check_finite(p.diag, lsefin);
             const int Ofin = O;
             if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
-            // the last spill (L_n, buffer (n-1)&1) must have left its buffer before it is reused
-            pr.wait(mbar_freed + 8u * ((n - 1) & 1), use_freed[(n - 1) & 1] & 1u);
-            ++use_freed[(n - 1) & 1];
             // ================= beta sweep
             for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // M_n = 0 in buffer 0
 #pragma unroll
@@ -305,6 +262,22 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             tmem_wait_st();
             int P = 0;
             float offM = 0.f;
+            // history stream: chunk c = butterfly (t = n - c / BPT, i = c % BPT), staged RD - 1 ahead with cp.async
+            const uint32_t nchunks = (uint32_t)n * BPT;
+            auto issue_chunk = [&](uint32_t c, uint32_t slot) {
+                if (c < nchunks) {
+                    const int t = n - (int)(c / BPT), i = (int)(c % BPT);
+                    const float4 *src = hist4 + ((size_t)(t - 1) * BPT + i) * (NCH * CT);
+                    const uint32_t dst = stage_u32 + slot * (uint32_t)(NCH * CT * 16);
+#pragma unroll
+                    for (int q = 0; q < NCH; ++q)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(src + q * CT) : "memory");
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            };
+#pragma unroll
+            for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c, c);
+            uint32_t chunk = 0, slot = 0;
             compute_barrier(CT);
             for (int t = n; t >= 1; --t) {
                 const int cur = (n - t) & 1;
@@ -326,7 +299,6 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                         }
                     }
                 }
-                if (!pr.warp_live()) { compute_barrier(CT); continue; }          // a wait ran out: only keep the barriers
                 const float2 w2 = splat2(w_s[t - 1]);
                 const float2 offM2 = splat2(offM);
                 const float2 Dm2 = splat2((float)(Ofin - O_s[t] - P) + lsefin);
@@ -336,9 +308,15 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                 tmem_ld16(tm, cb[0]);
 #pragma unroll
                 for (int i = 0; i < BPT; ++i, ++chunk) {
-                    const uint32_t s = chunk % RD;
-                    pr.wait(mbar_full + 8u * s, (chunk / RD) & 1u);
-                    const float *Lh = ring + s * CH;
+                    issue_chunk(chunk + RD - 1, slot == 0 ? RD - 1 : slot - 1);      // refill the slot consumed last
+                    asm volatile("cp.async.wait_group %0;" ::"n"(RD - 1) : "memory"); // chunk `chunk` has landed
+                    float Lh[K];
+#pragma unroll
+                    for (int q = 0; q < NCH; ++q) {
+                        const float4 l4 = stage4[(slot * NCH + q) * CT + tid];
+                        Lh[4 * q] = l4.x; Lh[4 * q + 1] = l4.y; Lh[4 * q + 2] = l4.z; Lh[4 * q + 3] = l4.w;
+                    }
+                    slot = slot + 1 == RD ? 0 : slot + 1;
                     float Mb[K];
 #pragma unroll
                     for (int b = 0; b < K; b += 4) {
@@ -360,7 +338,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                                 uu[b] = fma2(mul2(d, d), nl2, splat2(Mb[b]));
                             }
                             const float2 m = max_pairs<K>(uu);
-                            const float2 Lhj = make_float2(Lh[(2 * jh) * CT + tid], Lh[(2 * jh + 1) * CT + tid]);
+                            const float2 Lhj = make_float2(Lh[2 * jh], Lh[2 * jh + 1]);
                             const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
                             float2 pb = ex2f2(sub2(uu[0], m));
                             float2 sum = pb, craw = mul2(pb, cb[g & 1][C::b_idx(hh, 0)]);
@@ -379,8 +357,6 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                             den2 = fma2(f, sum, den2);
                         }
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_local(mbar_empty + 8u * s);             // this warp is done with the chunk
                 }
                 const float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
                 tmax = warp_max(tmax) - offM;
@@ -424,6 +400,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             diag_max(&p.diag->max_logz_gap, zgap);
         }
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0) tmem_dealloc_512(tmem_base);
