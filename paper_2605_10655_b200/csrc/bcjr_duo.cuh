@@ -302,19 +302,24 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         float offM = 0.f;
         // history stream: chunk c of this block = butterfly (t = n - c / BPT, i = c % BPT), staged RD - 1 ahead
         const uint32_t nchunks = (uint32_t)n * BPT;
-        auto issue_chunk = [&](uint32_t c, uint32_t slot) {
-            if (c < nchunks) {
-                const int t = n - (int)(c / BPT), i = (int)(c % BPT);
-                const float4 *src = hist4 + (((size_t)(t - 1) * CL + rank) * BPT + i) * (NCH * CT);
+        // running source pointer of the next chunk to request: butterflies i = 0..BPT-1 of step t, then step t - 1
+        const float4 *nsrc = hist4 + ((size_t)(n - 1) * CL + rank) * (BPT * NCH * CT);
+        uint32_t nleft = nchunks;                                // chunks not yet requested
+        int ni = 0;
+        auto issue_chunk = [&](uint32_t slot) {
+            if (nleft != 0) {
                 const uint32_t dst = stage_u32 + slot * (uint32_t)(NCH * CT * 16);
 #pragma unroll
                 for (int q = 0; q < NCH; ++q)
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(src + q * CT) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(nsrc + q * CT) : "memory");
+                --nleft;
+                if (++ni == BPT) { ni = 0; nsrc -= (size_t)(CL * BPT + BPT - 1) * (NCH * CT); }
+                else nsrc += NCH * CT;
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
 #pragma unroll
-        for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c, c);
+        for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c);
         uint32_t chunk = 0, slot = 0;                            // next chunk to consume and its staging slot
         cluster_sync();                                          // beta start
         // rank 0, warp 0: turn the sums of step t (slots of parity b) into grad_W[t]
@@ -357,7 +362,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
 #pragma unroll
             for (int i = 0; i < BPT; ++i, ++chunk) {
                 TICK(tr0);
-                issue_chunk(chunk + RD - 1, slot == 0 ? RD - 1 : slot - 1);          // refill the slot consumed last
+                issue_chunk(slot == 0 ? RD - 1 : slot - 1);          // refill the slot consumed last
                 asm volatile("cp.async.wait_group %0;" ::"n"(RD - 1) : "memory");     // chunk `chunk` has landed
                 TICK(tr1); TACC(3, tr0, tr1);
                 float Lh[K], Ah[K];

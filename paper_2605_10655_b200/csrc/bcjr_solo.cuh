@@ -264,19 +264,24 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             float offM = 0.f;
             // history stream: chunk c = butterfly (t = n - c / BPT, i = c % BPT), staged RD - 1 ahead with cp.async
             const uint32_t nchunks = (uint32_t)n * BPT;
-            auto issue_chunk = [&](uint32_t c, uint32_t slot) {
-                if (c < nchunks) {
-                    const int t = n - (int)(c / BPT), i = (int)(c % BPT);
-                    const float4 *src = hist4 + ((size_t)(t - 1) * BPT + i) * (NCH * CT);
+            // running source pointer of the next chunk to request: butterflies i = 0..BPT-1 of step t, then step t - 1
+            const float4 *nsrc = hist4 + (size_t)(n - 1) * (BPT * NCH * CT);
+            uint32_t nleft = nchunks;                            // chunks not yet requested
+            int ni = 0;
+            auto issue_chunk = [&](uint32_t slot) {
+                if (nleft != 0) {
                     const uint32_t dst = stage_u32 + slot * (uint32_t)(NCH * CT * 16);
 #pragma unroll
                     for (int q = 0; q < NCH; ++q)
-                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(src + q * CT) : "memory");
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(nsrc + q * CT) : "memory");
+                    --nleft;
+                    if (++ni == BPT) { ni = 0; nsrc -= (size_t)(2 * BPT - 1) * (NCH * CT); }
+                    else nsrc += NCH * CT;
                 }
                 asm volatile("cp.async.commit_group;" ::: "memory");
             };
 #pragma unroll
-            for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c, c);
+            for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c);
             uint32_t chunk = 0, slot = 0;
             compute_barrier(CT);
             for (int t = n; t >= 1; --t) {
@@ -308,7 +313,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                 tmem_ld16(tm, cb[0]);
 #pragma unroll
                 for (int i = 0; i < BPT; ++i, ++chunk) {
-                    issue_chunk(chunk + RD - 1, slot == 0 ? RD - 1 : slot - 1);      // refill the slot consumed last
+                    issue_chunk(slot == 0 ? RD - 1 : slot - 1);      // refill the slot consumed last
                     asm volatile("cp.async.wait_group %0;" ::"n"(RD - 1) : "memory"); // chunk `chunk` has landed
                     float Lh[K];
 #pragma unroll
