@@ -70,8 +70,9 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *   "wait_limit_ms"  wall-time budget of one device-side wait (default 2000).  A wait that outlasts it
  *                 gives up: the kernel still runs to its end, the outputs of the call are
  *                 meaningless and bcjr_sync_status returns BCJR_ETIMEOUT; the context stays usable.
- *   "debug_drop_history_load"  test hook for that path: while non-zero, thread block 0 never requests
- *                 the first history chunk of a large-trellis call, so one of its waits must run out.
+ *   "debug_drop_history_load"  test hook for that path: while non-zero, one warp of thread block 0
+ *                 withholds one arrival in a large-trellis backward call, so the waits of its cluster
+ *                 must run out.
  * The last two synchronise the device before they take effect. */
 bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value);
 
