@@ -269,16 +269,19 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             uint32_t nleft = nchunks;                            // chunks not yet requested
             int ni = 0;
             auto issue_chunk = [&](uint32_t slot) {
-                if (nleft != 0) {
-                    const uint32_t dst = stage_u32 + slot * (uint32_t)(NCH * CT * 16);
+                // branch-free: once every chunk has been requested the last one is simply requested again
+                // (into a slot nobody reads any more)
+                const uint32_t dst = stage_u32 + slot * (uint32_t)(NCH * CT * 16);
 #pragma unroll
-                    for (int q = 0; q < NCH; ++q)
-                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(nsrc + q * CT) : "memory");
-                    --nleft;
-                    if (++ni == BPT) { ni = 0; nsrc -= (size_t)(2 * BPT - 1) * (NCH * CT); }
-                    else nsrc += NCH * CT;
-                }
+                for (int q = 0; q < NCH; ++q)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(nsrc + q * CT) : "memory");
                 asm volatile("cp.async.commit_group;" ::: "memory");
+                const bool more = nleft > 1;
+                const bool wrap = ni == BPT - 1;
+                const ptrdiff_t adv = wrap ? -(ptrdiff_t)((size_t)(2 * BPT - 1) * (NCH * CT)) : (ptrdiff_t)(NCH * CT);
+                nsrc += more ? adv : 0;
+                ni = wrap ? 0 : ni + 1;
+                nleft -= more ? 1u : 0u;
             };
 #pragma unroll
             for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c);
