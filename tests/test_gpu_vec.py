@@ -118,6 +118,23 @@ def test_long_blocks_fall_back_to_the_one_cta_kernels(ctx):
         assert got["diag"].device_status == 0
 
 
+def test_stored_vector_emission_values(ctx):
+    import importlib.util
+    import json
+    from pathlib import Path
+    here = Path(__file__).parent
+    spec = importlib.util.spec_from_file_location("make_golden", here / "golden" / "make_golden.py")
+    mg = importlib.util.module_from_spec(spec); spec.loader.exec_module(mg)
+    gold = json.loads((here / "golden" / "vec_expected.json").read_text())
+    Lb, k, V, T, W, c, g = mg.vec_case()
+    got = _run(ctx, W, c, g, Lb, k, V, T)
+    assert parity.rel_inf(got["soft"][0], gold["soft_block0"]) <= parity.SOFT_TOL
+    assert parity.rel_inf(got["grad_W"][0], gold["grad_W_block0"]) <= parity.GRAD_TOL
+    assert parity.rel_inf(got["grad_codebook"].sum(axis=0), gold["grad_codebook_sum"]) <= parity.GRAD_TOL
+    assert got["states"][0].tolist() == gold["viterbi_states_block0"]
+    assert [bytes(r).hex() for r in got["path_bits"]] == gold["viterbi_path_bits_hex"]
+
+
 def test_single_emission_forwards_to_the_scalar_call_and_bad_arguments(ctx):
     import torch
     from paper_2605_10655_b200 import BcjrError
