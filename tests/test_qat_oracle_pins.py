@@ -44,3 +44,37 @@ def test_adam_zero_gradient_and_moment_decay():
     np.testing.assert_allclose(p, expect, rtol=1e-14)
     p, _, _ = qo.adam_update(p0, np.zeros(2), 0.0, 0.0, 1, 0.1)
     np.testing.assert_array_equal(p, p0)
+
+
+def test_hadamard_matches_scipy_and_is_orthogonal_up_to_its_size():
+    from scipy.linalg import hadamard as sp_hadamard
+    for n in (1, 2, 8, 64):
+        H = qo.hadamard(n)
+        np.testing.assert_array_equal(H, sp_hadamard(n))                 # independent construction
+        np.testing.assert_array_equal(H @ H, n * np.eye(n))
+
+
+def test_rotation_is_orthogonal_and_inverts_and_spreads_a_spike():
+    rng = np.random.default_rng(8)
+    m, n = 16, 32
+    W = rng.standard_normal((m, n)); sL = rng.choice([-1.0, 1.0], m); sR = rng.choice([-1.0, 1.0], n)
+    Wt = qo.rht_forward(W, sL, sR)
+    np.testing.assert_allclose(qo.rht_inverse(Wt, sL, sR), W, atol=1e-13)
+    np.testing.assert_allclose(np.linalg.norm(Wt), np.linalg.norm(W), rtol=1e-13)   # Frobenius norm kept
+    E = np.zeros((m, n)); E[3, 5] = 1.0                                  # one spike becomes a flat +-1/sqrt(mn) field
+    np.testing.assert_allclose(np.abs(qo.rht_forward(E, sL, sR)), 1.0 / np.sqrt(m * n), rtol=1e-13)
+    # y = W x  is reproduced from the rotated quantities: (W~ applied to the rotated input)
+    x = rng.standard_normal(n)
+    xr = qo.hadamard(n) @ (sR * x) / np.sqrt(n)
+    back = sL * (qo.hadamard(m) @ (Wt @ xr)) / np.sqrt(m)
+    np.testing.assert_allclose(back, W @ x, atol=1e-12)
+
+
+def test_group_scales_normalise_every_group_of_sixteen():
+    rng = np.random.default_rng(9)
+    W = rng.standard_normal((4, 64)) * np.array([1.0, 10.0, 0.1, 3.0])[:, None]
+    s, Wn = qo.group_scales(W)
+    assert s.shape == (4, 4)
+    np.testing.assert_allclose((Wn.reshape(4, 4, 16) ** 2).mean(axis=2), 1.0, rtol=1e-13)
+    np.testing.assert_allclose(Wn.reshape(4, 4, 16) * s[:, :, None], W.reshape(4, 4, 16), rtol=1e-13)
+    np.testing.assert_allclose(qo.group_scales(np.full((1, 16), -2.5))[0], 2.5)
