@@ -307,6 +307,22 @@ def main():
         ums = e0.elapsed_time(e1)
         upd = {"kernel": "adam_kernel", "weights": numel, "ms": ums, "gbs": 28.0 * numel / (ums * 1e-3) / 1e9}
         del mW, vW, Wc
+        # the incoherence rotation that precedes the trellis pass (both sides; algorithmic bytes: read + write once)
+        rows, cols = dict(wl.matrices)[big["name"]]
+        if not args.blocks and rows & (rows - 1) == 0 and cols & (cols - 1) == 0 and cols <= 8192:
+            W2 = big["W"].reshape(rows, cols).clone()
+            sL = torch.ones(rows, device=dev); sR = torch.ones(cols, device=dev)
+            out2 = torch.empty_like(W2)
+            ctx.bcjr_rht(W2, sL, sR, out=out2)                         # warm-up
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx.bcjr_rht(W2, sL, sR, out=out2)
+            e1.record()
+            torch.cuda.synchronize()
+            rms = e0.elapsed_time(e1)
+            upd["rht"] = {"shape": [rows, cols], "ms": rms, "gbs": 8.0 * rows * cols / (rms * 1e-3) / 1e9}
+            del W2, out2
 
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
     e2e = None

@@ -174,6 +174,27 @@ bcjr_status bcjr_backward_adam(bcjr_ctx *ctx, const float *grad_soft, float *W_l
                                float beta1, float beta2, float eps, void *cuda_stream);
 
 /*
+ * Incoherence processing before / after the trellis pass (Section 3.1: "a random-sign Hadamard
+ * rotation on both sides"; Section 4, "Quantization configuration": scales over groups of 16).
+ * The paper gives no formulas; these calls use
+ *     forward:  out = H_m diag(sign_rows) W diag(sign_cols) H_n / sqrt(m n)
+ *     inverse:  out = diag(sign_rows) H_m W H_n diag(sign_cols) / sqrt(m n)
+ * with Sylvester-ordered Walsh-Hadamard matrices (H H = size * I), so inverse(forward(W)) = W, and
+ *     scales[g] = sqrt(mean of the squares of elements 16g .. 16g+15),  W_scaled = W / scales[g]
+ *     (a group of zeros gets scale 0 and stays zero).
+ *   W, out      device [m * n] row-major; out may be W (in place); 16-byte aligned
+ *   m, n        powers of two, >= 8; n <= 8192 (BCJR_EUNSUPPORTED above)
+ *   sign_rows   device [m], sign_cols device [n]: +1.0f / -1.0f (sign_cols 16-byte aligned)
+ *   numel       multiple of 16; scales has numel / 16 entries
+ */
+bcjr_status bcjr_rht(bcjr_ctx *ctx, const float *W, float *out, int m, int n,
+                     const float *sign_rows, const float *sign_cols, int inverse, void *cuda_stream);
+bcjr_status bcjr_group_scale(bcjr_ctx *ctx, const float *W, float *scales, float *W_scaled,
+                             int64_t numel, void *cuda_stream);
+bcjr_status bcjr_group_unscale(bcjr_ctx *ctx, const float *W_scaled, const float *scales, float *W,
+                               int64_t numel, void *cuda_stream);
+
+/*
  * BCJR-STE forward (Section 3.7, "BCJR-STE variant"): the value that goes forward is the hard
  * Viterbi codeword, while the state saved on the context is that of the temperature-T relaxation,
  * so that a following bcjr_backward returns the gradient of the finite-temperature soft codeword

@@ -75,4 +75,5 @@ def group_scales(W, group=16):
     m, n = W.shape
     g = W.reshape(m, n // group, group)
     s = np.sqrt((g * g).mean(axis=2))
-    return s, (g / s[:, :, None]).reshape(m, n)
+    scaled = np.divide(g, s[:, :, None], out=np.zeros_like(g), where=s[:, :, None] > 0)      # an all-zero group stays zero
+    return s, scaled.reshape(m, n)

@@ -14,7 +14,7 @@ LIB_PATH = _PKG / "libbcjr_b200.so"
 
 EXPORTS = ["bcjr_create", "bcjr_destroy", "bcjr_set_option", "bcjr_soft_quantize", "bcjr_backward",
            "viterbi_hard", "bcjr_soft_quantize_vec", "viterbi_hard_vec", "bcjr_ste_forward", "bcjr_temperature", "bcjr_gaussian_codebook", "bcjr_adam_update",
-           "bcjr_backward_adam", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
+           "bcjr_backward_adam", "bcjr_rht", "bcjr_group_scale", "bcjr_group_unscale", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
            "bcjr_last_cuda_error", "bcjr_status_string", "bcjr_soft_quantize_static",
            "bcjr_static_scratch_bytes"]
 
@@ -64,6 +64,9 @@ def load_library() -> ctypes.CDLL:
     lib.bcjr_adam_update.argtypes = [vp, vp, vp, vp, vp, i64, i, f, f, f, f, vp]
     lib.bcjr_backward_adam.restype = i
     lib.bcjr_backward_adam.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, f, f, f, f, f, vp]
+    lib.bcjr_rht.restype = i; lib.bcjr_rht.argtypes = [vp, vp, vp, i, i, vp, vp, i, vp]
+    lib.bcjr_group_scale.restype = i; lib.bcjr_group_scale.argtypes = [vp, vp, vp, vp, i64, vp]
+    lib.bcjr_group_unscale.restype = i; lib.bcjr_group_unscale.argtypes = [vp, vp, vp, vp, i64, vp]
     lib.bcjr_step_host.restype = i
     lib.bcjr_step_host.argtypes = [vp, vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
     lib.bcjr_sync_status.restype = i; lib.bcjr_sync_status.argtypes = [vp, vp, ctypes.POINTER(Diag)]
@@ -297,6 +300,39 @@ class Context:
             int(t), float(lr_W), float(lr_c), float(beta1), float(beta2), float(eps), _stream_ptr(stream))
         self._check(rc, "bcjr_backward_adam")
         self._saved = None
+
+    def bcjr_rht(self, W, sign_rows, sign_cols, inverse=False, out=None, stream=None):
+        """Random-sign Hadamard rotation on both sides of W [m, n] (or its inverse); returns `out`."""
+        import torch
+        m, n = W.shape
+        if out is None:
+            out = torch.empty_like(W)
+        rc = self._lib.bcjr_rht(self._h, _dev(W, torch.float32, m * n, "W"), _dev(out, torch.float32, m * n, "out"), m, n,
+                                _dev(sign_rows, torch.float32, m, "sign_rows"), _dev(sign_cols, torch.float32, n, "sign_cols"),
+                                1 if inverse else 0, _stream_ptr(stream))
+        self._check(rc, "bcjr_rht")
+        return out
+
+    def bcjr_group_scale(self, W, stream=None):
+        """Per-16 scales (root mean square) of W; returns (scales [numel/16], W / scales)."""
+        import torch
+        numel = W.numel()
+        scales = torch.empty(numel // 16, dtype=torch.float32, device=W.device)
+        out = torch.empty_like(W)
+        rc = self._lib.bcjr_group_scale(self._h, _dev(W, torch.float32, numel, "W"), ctypes.c_void_p(scales.data_ptr()),
+                                        _dev(out, torch.float32, numel, "W_scaled"), numel, _stream_ptr(stream))
+        self._check(rc, "bcjr_group_scale")
+        return scales, out
+
+    def bcjr_group_unscale(self, W_scaled, scales, stream=None):
+        import torch
+        numel = W_scaled.numel()
+        out = torch.empty_like(W_scaled)
+        rc = self._lib.bcjr_group_unscale(self._h, _dev(W_scaled, torch.float32, numel, "W_scaled"),
+                                          _dev(scales, torch.float32, numel // 16, "scales"),
+                                          _dev(out, torch.float32, numel, "W"), numel, _stream_ptr(stream))
+        self._check(rc, "bcjr_group_unscale")
+        return out
 
     def bcjr_step_host(self, W, codebook, grad_soft, Lb, k, n, T, soft=None, grad_W=None, grad_codebook=None,
                        stream=None):

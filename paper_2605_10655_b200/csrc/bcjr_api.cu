@@ -15,6 +15,7 @@
 #include "bcjr_vec.cuh"
 #include "bcjr_vec4.cuh"
 #include "bcjr_qat.cuh"
+#include "bcjr_rht.cuh"
 #include "bcjr_solo.cuh"
 #include "bcjr_duo.cuh"
 #include "bcjr_viterbi.cuh"
@@ -493,6 +494,24 @@ struct DeviceGuard {
 
 }  // namespace
 
+namespace {
+int log2_exact(int64_t v)
+{
+    if (v < 1 || (v & (v - 1))) return -1;
+    int l = 0;
+    while ((((int64_t)1) << l) < v) ++l;
+    return l;
+}
+template <int LOGN>
+void launch_fwht_rows(const float *in, float *out, const float *s, int m, float scale, int pre, int sms, cudaStream_t st)
+{
+    constexpr int N = 1 << LOGN, T = N / 8;
+    int grid = sms * (T >= 1024 ? 1 : 1024 / T);
+    if (grid > m) grid = m;
+    fwht_rows_kernel<LOGN><<<grid, T, (size_t)(N + N / 8) * 4, st>>>(in, out, s, m, scale, pre);
+}
+}  // namespace
+
 extern "C" {
 
 #ifdef BCJR_TIMING
@@ -889,6 +908,83 @@ bcjr_status bcjr_backward_adam(bcjr_ctx *ctx, const float *grad_soft, float *W_l
     if ((rc = bcjr_adam_update(ctx, W_latent, gW, m_W, v_W, numel, t, lr_W, beta1, beta2, eps, cuda_stream))) return rc;
     if (codebook && (rc = bcjr_adam_update(ctx, codebook, gc, m_c, v_c, csize, t, lr_c, beta1, beta2, eps, cuda_stream))) return rc;
     ctx->have_fwd = false;      // the saved inputs have changed: a new forward call is needed
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_rht(bcjr_ctx *ctx, const float *W, float *out, int m, int n, const float *sign_rows,
+                     const float *sign_cols, int inverse, void *cuda_stream)
+{
+    if (!ctx || !W || !out || !sign_rows || !sign_cols) return BCJR_EINVAL;
+    const int lm = log2_exact(m), ln = log2_exact(n);
+    if (lm < 3 || ln < 3) return BCJR_EINVAL;                     // powers of two, at least 8
+    if (ln > 13 || lm > 24) return BCJR_EUNSUPPORTED;            // a row must fit shared memory
+    if (((uintptr_t)W | (uintptr_t)out | (uintptr_t)sign_cols) & 15u) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int pre = inverse ? 0 : 1;
+    const float srow = (float)(1.0 / std::sqrt((double)n)), scol = (float)(1.0 / std::sqrt((double)m));
+    switch (ln) {
+        case 3: launch_fwht_rows<3>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 4: launch_fwht_rows<4>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 5: launch_fwht_rows<5>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 6: launch_fwht_rows<6>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 7: launch_fwht_rows<7>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 8: launch_fwht_rows<8>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 9: launch_fwht_rows<9>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 10: launch_fwht_rows<10>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 11: launch_fwht_rows<11>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        case 12: launch_fwht_rows<12>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+        default: launch_fwht_rows<13>(W, out, sign_cols, m, srow, pre, ctx->num_sms, st); break;
+    }
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    // columns: radix-8 passes over the row-index bits, in place on `out`
+    const int n4 = n / 4;
+    const int64_t total = (int64_t)(m / 8) * n4;
+    int blocks = (int)((total + 255) / 256 < (int64_t)ctx->num_sms * 8 ? (total + 255) / 256 : (int64_t)ctx->num_sms * 8);
+    if (blocks < 1) blocks = 1;
+    for (int o = 0;; o += 3) {
+        const bool last = o + 3 >= lm;
+        const int oo = last ? lm - 3 : o, first = o - oo;
+        const int mode = (!inverse && o == 0) ? 1 : (inverse && last) ? 2 : 0;
+        fwht_cols_pass_kernel<<<blocks, 256, 0, st>>>(out, sign_rows, m, n4, oo, first, last ? scol : 1.f, mode);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+        if (last) break;
+    }
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_group_scale(bcjr_ctx *ctx, const float *W, float *scales, float *W_scaled, int64_t numel, void *cuda_stream)
+{
+    if (!ctx || numel < 0 || numel % 16) return BCJR_EINVAL;
+    if (numel == 0) return BCJR_OK;
+    if (!W || !scales || !W_scaled || (((uintptr_t)W | (uintptr_t)W_scaled) & 15u)) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    const int64_t groups = numel / 16;
+    int64_t blocks = (groups + 255) / 256;
+    if (blocks > (int64_t)ctx->num_sms * 16) blocks = (int64_t)ctx->num_sms * 16;
+    group_scale_kernel<<<(int)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(W, scales, W_scaled, groups);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+bcjr_status bcjr_group_unscale(bcjr_ctx *ctx, const float *W_scaled, const float *scales, float *W, int64_t numel, void *cuda_stream)
+{
+    if (!ctx || numel < 0 || numel % 16) return BCJR_EINVAL;
+    if (numel == 0) return BCJR_OK;
+    if (!W || !scales || !W_scaled || (((uintptr_t)W | (uintptr_t)W_scaled) & 15u)) return BCJR_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    const int64_t groups = numel / 16;
+    int64_t blocks = (groups + 255) / 256;
+    if (blocks > (int64_t)ctx->num_sms * 16) blocks = (int64_t)ctx->num_sms * 16;
+    group_unscale_kernel<<<(int)blocks, 256, 0, (cudaStream_t)cuda_stream>>>(W_scaled, scales, W, groups);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
     return BCJR_OK;
 }
 

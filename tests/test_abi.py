@@ -41,6 +41,9 @@ def test_status_strings_and_host_side_argument_checks():
     assert lib.bcjr_destroy(None) == -1
     assert lib.bcjr_adam_update(None, None, None, None, None, 4, 1, 1e-3, 0.9, 0.999, 1e-8, None) == -1
     assert lib.bcjr_gaussian_codebook(None, 8, None, None) == -1
+    assert lib.bcjr_rht(None, None, None, 8, 8, None, None, 0, None) == -1
+    assert lib.bcjr_group_scale(None, None, None, None, 16, None) == -1
+    assert lib.bcjr_group_unscale(None, None, None, None, 16, None) == -1
     # the schedule is host arithmetic: end points and the constant ratio of Section 3.6
     assert binding.temperature(1.0, 0.02, 0, 10) == 1.0 and abs(binding.temperature(1.0, 0.02, 10, 10) - 0.02) < 1e-15
     assert abs(binding.temperature(1.0, 0.02, 3, 10) - 0.02 ** 0.3) < 1e-15 and binding.temperature(-1.0, 0.02, 1, 10) == 0.0

@@ -105,3 +105,59 @@ def test_annealed_qat_loop_follows_the_oracle_loop(ctx):
     with pytest.raises(BcjrError) as e:
         ctx.bcjr_backward(g)
     assert e.value.code == -4
+
+
+@pytest.mark.parametrize("m,n", [(8, 8), (16, 64), (64, 16), (32, 512), (128, 2048), (8, 8192), (2048, 32)])
+def test_hadamard_rotation_matches_the_matrix_product_and_inverts(ctx, m, n):
+    import torch
+    rng = np.random.default_rng(m * 31 + n)
+    W = rng.standard_normal((m, n)).astype(np.float32)
+    sL = rng.choice([-1.0, 1.0], m).astype(np.float32); sR = rng.choice([-1.0, 1.0], n).astype(np.float32)
+    dev = torch.device("cuda", ctx.device)
+    Wd, sLd, sRd = (torch.from_numpy(a).to(dev) for a in (W, sL, sR))
+    Wt = ctx.bcjr_rht(Wd, sLd, sRd)
+    ref = qo.rht_forward(W, sL, sR)                                  # dense matrix products in float64
+    # log2(m n) butterfly stages of float32 additions on O(1) values
+    assert np.abs(Wt.cpu().numpy() - ref).max() <= 2e-6 * np.abs(ref).max() * np.log2(m * n)
+    back = ctx.bcjr_rht(Wt, sLd, sRd, inverse=True)
+    assert np.abs(back.cpu().numpy() - W).max() <= 4e-6 * np.abs(W).max() * np.log2(m * n)
+    ref_inv = qo.rht_inverse(ref, sL, sR)
+    np.testing.assert_allclose(ref_inv, W, atol=1e-5)
+    # in place
+    Wc = Wd.clone()
+    ctx.bcjr_rht(Wc, sLd, sRd, out=Wc)
+    ctx.sync_status()
+    assert torch.equal(Wc, Wt)
+
+
+def test_rotation_rejects_sizes_that_are_not_powers_of_two(ctx):
+    import torch
+    from paper_2605_10655_b200 import BcjrError
+    dev = torch.device("cuda", ctx.device)
+    W = torch.zeros((24, 16), device=dev); s24 = torch.ones(24, device=dev); s16 = torch.ones(16, device=dev)
+    with pytest.raises(BcjrError) as e:
+        ctx.bcjr_rht(W, s24, s16)
+    assert e.value.code == -1
+    W = torch.zeros((8, 16384), device=dev)
+    with pytest.raises(BcjrError) as e:
+        ctx.bcjr_rht(W, torch.ones(8, device=dev), torch.ones(16384, device=dev))
+    assert e.value.code == -5
+
+
+def test_group_scales_and_their_inverse(ctx):
+    import torch
+    rng = np.random.default_rng(5)
+    W = (rng.standard_normal((37, 64)) * 10.0 ** rng.integers(-3, 3, (37, 1))).astype(np.float32)
+    W[5, 16:32] = 0.0                                                # an all-zero group
+    dev = torch.device("cuda", ctx.device)
+    Wd = torch.from_numpy(W).to(dev)
+    scales, Ws = ctx.bcjr_group_scale(Wd)
+    rs, rWs = qo.group_scales(np.where(W == 0, 0, W))
+    got_s = scales.cpu().numpy().reshape(37, 4)
+    np.testing.assert_allclose(got_s, rs, rtol=2e-6)
+    mask = np.repeat(rs > 0, 16, axis=1)
+    np.testing.assert_allclose(Ws.cpu().numpy()[mask], rWs[mask], rtol=4e-6, atol=1e-7)
+    assert torch.all(Ws[5, 16:32] == 0) and got_s[5, 1] == 0
+    back = ctx.bcjr_group_unscale(Ws, scales)
+    ctx.sync_status()
+    np.testing.assert_allclose(back.cpu().numpy(), W, rtol=3e-7, atol=0)
