@@ -44,7 +44,7 @@ def adam_update(p, g, m, v, t, lr, beta1=0.9, beta2=0.999, eps=1e-8):
 
 # ---- incoherence processing (Section 3.1 / Section 4 "Quantization configuration"): a random-sign
 # Hadamard rotation on both sides of the weight matrix, and a scale per group of 16 elements.
-# The paper names both and gives no formula; the forms fixed here (and in the design doc) are the
+# The paper names both and gives no formula; the forms fixed here are the
 # QuIP#-style ones:  W~ = H_m diag(sL) W diag(sR) H_n / sqrt(m n)  with the Sylvester-ordered
 # Walsh-Hadamard matrices H (entries +-1, H H = size * I), so that the inverse is
 # W = diag(sL) H_m W~ H_n diag(sR) / sqrt(m n);  scale of a group = root mean square of its 16 elements.
