@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
     };
 
     for (int64_t base = (int64_t)cid * NBLK; base < p.B; base += (int64_t)ncl * NBLK) {
-        const int nact = (int)(p.B - base < NBLK ? p.B - base : NBLK);        // blocks in flight this round
+        const int nact = (int)(p.B - base < NBLK ? p.B - base : NBLK);        // blocks in flight in this batch
         for (int k = 0; k < nact; ++k) {
             const float *w = p.W + (base + k) * n;
             for (int t = tid; t < n; t += CT) w_s[k * C::MAX_N + t] = __ldg(w + t);
@@ -371,7 +371,7 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
                 zgap = fmaxf(zgap, fabsf((float)(P[k] - Ofin[k]) + (lz_beta - lsefin[k])));
             }
         }
-        cluster_sync();         // nobody still reads this round's buffers when the next round starts
+        cluster_sync();         // nobody still reads this batch's buffers when the next batch starts
     }
     // defect lives in warps 0..NBLK-1 of rank 0, zgap everywhere
     if (rank == 0 && lane == 0 && warp < NBLK) diag_max(&p.diag->max_defect, defect);
@@ -754,7 +754,7 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                 finish_step(1, ib, k);
             }
         }
-        cluster_sync();         // nobody still reads this round's buffers when the next round starts
+        cluster_sync();         // nobody still reads this batch's buffers when the next batch starts
     }
     // this cluster's partial of the table gradient, in the regrouped layout [b][q][V]
     {
