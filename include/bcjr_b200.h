@@ -195,7 +195,7 @@ bcjr_status bcjr_group_unscale(bcjr_ctx *ctx, const float *W_scaled, const float
                                int64_t numel, void *cuda_stream);
 
 /*
- * BCJR-STE forward (Section 3.7, "BCJR-STE variant"): the value that goes forward is the hard
+ * BCJR-STE forward (Section 3.8, "BCJR-STE variant"): the value that goes forward is the hard
  * Viterbi codeword, while the state saved on the context is that of the temperature-T relaxation,
  * so that a following bcjr_backward returns the gradient of the finite-temperature soft codeword
  * (the straight-through gradient replaced by the true gradient of the relaxation).  Equivalent
