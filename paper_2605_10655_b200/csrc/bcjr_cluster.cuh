@@ -258,6 +258,28 @@ __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
 __device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
 __device__ __forceinline__ float2 lg2f2(float2 a) { return make_float2(lg2f(a.x), lg2f(a.y)); }
 __device__ __forceinline__ float2 rcpf2(float2 a) { return make_float2(rcpf(a.x), rcpf(a.y)); }
+// 2^x for x <= 0 on the FP32 pipe (no special-function instruction): x = n + f with n the nearest
+// integer and |f| <= 1/2, 2^f by the degree-5 interpolant at the Chebyshev nodes of [-1/2, 1/2] (relative
+// error 2.4e-7 evaluated in float32, about that of ex2.approx), the
+// factor 2^n by an add on the exponent field.  Arguments below -125 are clamped (the result there
+// is ~2e-38 against a group maximum of 1, far below anything the sums can see).
+__device__ __forceinline__ float2 ex2_poly2(float2 x)
+{
+    x.x = fmaxf(x.x, -125.f); x.y = fmaxf(x.y, -125.f);
+    const float2 magic = splat2(12582912.f);                     // 1.5 * 2^23: adding it rounds to the nearest integer
+    const float2 t = add2(x, magic);
+    const float2 n = sub2(t, magic);
+    const float2 f = sub2(x, n);
+    float2 p = fma2(splat2(1.3390863e-3f), f, splat2(9.6760318e-3f));
+    p = fma2(p, f, splat2(5.5503570e-2f));
+    p = fma2(p, f, splat2(2.4022107e-1f));
+    p = fma2(p, f, splat2(6.9314718e-1f));
+    p = fma2(p, f, splat2(1.0000001f));
+    // t = 1.5 * 2^23 + n exactly, so its low mantissa bits hold n (two's complement): shift them onto the exponent
+    p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+    p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+    return p;
+}
 __device__ __forceinline__ float max3f(float a, float b, float c)
 {
     float d;

@@ -20,6 +20,7 @@
 #pragma once
 #include "bcjr_cluster.cuh"
 
+
 namespace bcjr {
 
 // ---------------------------------------------------------------------------- TMEM helpers
@@ -226,7 +227,8 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                             const float2 m = max_pairs<K>(a);
                             float2 sum = ex2f2(sub2(a[0], m));
 #pragma unroll
-                            for (int j = 1; j < K; ++j) sum = add2(sum, ex2f2(sub2(a[j], m)));
+                            for (int j = 1; j < K; ++j)      // every fourth exponential on the FP32 pipe: the MUFU is this sweep's bottleneck
+                                sum = add2(sum, (j % 4 == 3) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m)));
                             out[h] = add2(sub2(m, off2), lg2f2(sum));
                             tmax = max3f(tmax, m.x, m.y);
                         }
