@@ -23,8 +23,8 @@
 // History.  The inputs (L, At) of a butterfly in the alpha sweep are exactly what the same thread
 // needs for that butterfly in the beta sweep, so the history is thread-private: the thread stores
 // its inputs with 16-byte global stores ([step][CTA][butterfly slot][16-byte chunk][thread]) and
-// streams them back with cp.async into its own staging slots, RD - 1 butterflies ahead
-// (cp.async.wait_group; no mbarrier, no producer thread, no branch in the butterfly loop).
+// streams them back with cp.async into its own staging slots, a whole step ahead (one
+// cp.async.wait_group per step; no mbarrier, no producer thread, no branch in the butterfly loop).
 #pragma once
 #include "bcjr_solo.cuh"
 
@@ -51,7 +51,7 @@ struct DuoCfg {
     static constexpr int HPU = (K / 2) / UNITS;                // pairs h (alpha) / jh (beta) per unit
     static constexpr int SLOTS = CL * NWARP;                   // 32 per-warp partial slots
     static constexpr int NCH = 2 * K / 4;                      // 16-byte chunks per butterfly and thread: K values of L, K of At
-    static constexpr int RD = KB == 2 ? BPT + 1 : 3;           // staging depth in butterflies
+    static constexpr int RD = BPT;                             // staging slots: one per butterfly of a step
     static constexpr int MAX_N = 1024;
     static constexpr int ARRIVALS = 1 + SLOTS;                 // armer + one arrival per warp of the cluster
     static constexpr int OFF_MSG = 0;                          // [2 parity][2 arrays][QC]
@@ -300,7 +300,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         tmem_wait_st();
         int P = 0;
         float offM = 0.f;
-        // history stream: chunk c of this block = butterfly (t = n - c / BPT, i = c % BPT), staged RD - 1 ahead
+        // history stream: chunk c of this block = butterfly (t = n - c / BPT, i = c % BPT), staged one step ahead
         const uint32_t nchunks = (uint32_t)n * BPT;
         // running source pointer of the next chunk to request: butterflies i = 0..BPT-1 of step t, then step t - 1
         const float4 *nsrc = hist4 + ((size_t)(n - 1) * CL + rank) * (BPT * NCH * CT);
@@ -322,8 +322,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             nleft -= more ? 1u : 0u;
         };
 #pragma unroll
-        for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c);
-        uint32_t chunk = 0, slot = 0;                            // next chunk to consume and its staging slot
+        for (uint32_t c = 0; c < RD; ++c) issue_chunk(c);           // the first step's butterflies
+        uint32_t chunk = 0;
         cluster_sync();                                          // beta start
         // rank 0, warp 0: turn the sums of step t (slots of parity b) into grad_W[t]
         auto finish_step = [&](int t, int b) {
@@ -362,20 +362,19 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             float tmax = NEG_INF;
             float2 cb[2][8];
             tmem_ld16(tm_cb, cb[0]);
+            asm volatile("cp.async.wait_group 0;" ::: "memory");    // this step's history, requested during the previous step
 #pragma unroll
             for (int i = 0; i < BPT; ++i, ++chunk) {
                 TICK(tr0);
-                issue_chunk(slot == 0 ? RD - 1 : slot - 1);          // refill the slot consumed last
-                asm volatile("cp.async.wait_group %0;" ::"n"(RD - 1) : "memory");     // chunk `chunk` has landed
                 TICK(tr1); TACC(3, tr0, tr1);
                 float Lh[K], Ah[K];
 #pragma unroll
                 for (int q = 0; q < K / 4; ++q) {
-                    const float4 l4 = stage4[(slot * NCH + q) * CT + tid], a4 = stage4[(slot * NCH + K / 4 + q) * CT + tid];
+                    const float4 l4 = stage4[(i * NCH + q) * CT + tid], a4 = stage4[(i * NCH + K / 4 + q) * CT + tid];
                     Lh[4 * q] = l4.x; Lh[4 * q + 1] = l4.y; Lh[4 * q + 2] = l4.z; Lh[4 * q + 3] = l4.w;
                     Ah[4 * q] = a4.x; Ah[4 * q + 1] = a4.y; Ah[4 * q + 2] = a4.z; Ah[4 * q + 3] = a4.w;
                 }
-                slot = slot + 1 == RD ? 0 : slot + 1;
+                issue_chunk(i);                                      // this slot's entry for the next step (a whole step ahead)
                 float Mb[K], Yb[K];
 #pragma unroll
                 for (int b = 0; b < K; b += 4) {
