@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                         float2 sum = pj, ax = mul2(pj, fma2(g2, cb[g & 1][C::a_idx(0, hh)], splat2(Aj[0])));
 #pragma unroll
                         for (int j = 1; j < K; ++j) {
-                            pj = (j % 4 == 3) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));
+                            pj = (KB == 2 && j % 4 == 3) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));   // no gain at K = 8
                             sum = add2(sum, pj);
                             ax = fma2(pj, fma2(g2, cb[g & 1][C::a_idx(j, hh)], splat2(Aj[j])), ax);
                         }
