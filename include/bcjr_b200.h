@@ -63,9 +63,9 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *   "path"        0 auto, 1 force the generic kernels, 2 force the large-trellis kernels
  *                 (BCJR_EUNSUPPORTED at call time when they do not cover the shape)
  *   "fwd_variant" large-trellis forward kernel: 0 = one CTA per block with the codebook in tensor
- *                 memory (Lb = 16, k = 2), 1 = two-CTA cluster kernel with the codebook in registers
+ *                 memory (Lb = 16, k = 2 or 3), 1 = two-CTA cluster kernel with the codebook in registers
  *   "bwd_variant" large-trellis backward kernel: 0 = two-CTA clusters with codebook and gradient
- *                 accumulators in tensor memory (Lb = 16, k = 2), 1 = four-CTA clusters, registers
+ *                 accumulators in tensor memory (Lb = 16, k = 2 or 3), 1 = four-CTA clusters, registers
  *   "max_ctas"    cap on resident thread blocks (0 = fill the GPU)
  *   "wait_limit_ms"  wall-time budget of one device-side wait (default 2000).  A wait that outlasts it
  *                 gives up: the kernel still runs to its end, the outputs of the call are
