@@ -695,9 +695,9 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                     }
                     const float2 m = max_pairs<K>(u);
                     const float2 f = ex2f2(add2(m, sub2(Ls[k], splat2(Dm))));
-                    const float2 fi = mul2(f, splat2(invT));
+                    const float2 iT2 = splat2(invT);
                     const float2 Ahj = sub2(As[k], splat2(gs));                        // At_t without the shift
-                    float2 sum = make_float2(0.f, 0.f), ya = sum, S0 = sum, S2 = sum, Z0 = sum, Z1 = sum;
+                    float2 sum = make_float2(0.f, 0.f), ya = sum, Z0 = sum, Z1 = sum;
 #pragma unroll
                     for (int un = 0; un < UNITS; ++un) {                                   // second pass, with the accumulators
                         float2 acc[8];
@@ -717,12 +717,10 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                                 const float2 pb = ex2f2(sub2(u[b + bb], m));
                                 sum = add2(sum, pb);
                                 ya = fma2(pb, y, ya);
-                                const float2 r = add2(y, Ahj);
-                                const float2 gam = mul2(pb, f), q = mul2(mul2(pb, fi), r);     // gamma, gamma r / T
-                                S0 = add2(S0, gam);
-                                S2 = fma2(gam, r, S2);
-                                const float2 zx = fma2(q, sub2(wx, cx), mul2(gam, gx));
-                                const float2 zy = fma2(q, sub2(wy, cy), mul2(gam, gy));
+                                const float2 rT = mul2(add2(y, Ahj), iT2);                 // r / T
+                                const float2 gam = mul2(pb, f);                            // gamma
+                                const float2 zx = mul2(gam, fma2(rT, sub2(wx, cx), gx));   // gamma (g_v + (w_v - c_v) r / T)
+                                const float2 zy = mul2(gam, fma2(rT, sub2(wy, cy), gy));
                                 Z0 = add2(Z0, zx); Z1 = add2(Z1, zy);
                                 acc[2 * (e + bb)] = add2(acc[2 * (e + bb)], zx);
                                 acc[2 * (e + bb) + 1] = add2(acc[2 * (e + bb) + 1], zy);
@@ -731,6 +729,8 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                         tmem_st16(tm_acc + 16u * un, acc);
                     }
                     tmem_wait_st();
+                    // S0 = sum gamma = f sum rho;  S2 = sum gamma r = f (sum rho y + At sum rho)
+                    const float2 S0 = mul2(f, sum), S2 = mul2(f, fma2(Ahj, sum, ya));
                     const float2 outM = add2(m, lg2f2(sum));
                     const float2 outB = fma2(ya, rcpf2(sum), splat2(gsp));
                     pr.async_v2(push_b + (uint32_t)(so * 2 * QC) * 4u, outM.x, outM.y, push_b_mbar + 8u * so);
