@@ -291,8 +291,8 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
                                                  : make_float2(0.f, 0.f);
                     const float *wk = w_s + k * C::MAX_N + 2 * (t - 1);
                     const float2 wx = splat2(wk[0]), wy = splat2(wk[1]);
-                    // the outputs are shifted by offM: fold the shift into the inputs and into D
-                    const float Dm = ((float)(Ofin[k] - O_s[k * OSTR + t] - P[k]) + lsefin[k]) - offM[k];
+                    // the outputs are shifted by offM (once per group, below); D refers to the unshifted inputs
+                    const float Dm = ((float)(Ofin[k] - O_s[k * OSTR + t] - P[k]) + lsefin[k]);
                     const float2 offM2 = splat2(offM[k]);
                     float2 u[K], cb[2][8];
                     tmem_ld16(tm, cb[0]);
@@ -308,7 +308,7 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
                             for (int bb = 0; bb < 2; ++bb) {
                                 const float2 dx = sub2(cb[un & 1][2 * (e + bb)], wx), dy = sub2(cb[un & 1][2 * (e + bb) + 1], wy);
                                 const float2 Mb = bb == 0 ? make_float2(Mv.x, Mv.z) : make_float2(Mv.y, Mv.w);
-                                u[b + bb] = fma2(fma2(dy, dy, mul2(dx, dx)), nl2, sub2(Mb, offM2));
+                                u[b + bb] = fma2(fma2(dy, dy, mul2(dx, dx)), nl2, Mb);
                             }
                         }
                     }
@@ -326,12 +326,12 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
                             cy = fma2(pb, cb[un & 1][2 * e + 1], cy);
                         }
                     }
-                    const float2 out = add2(m, lg2f2(sum));
+                    const float2 out = add2(sub2(m, offM2), lg2f2(sum));
                     const float2 f = ex2f2(add2(m, sub2(Ls[k], splat2(Dm))));
                     pr.async_v2(push_b + (uint32_t)(so * QC) * 4u, out.x, out.y, push_b_mbar + 8u * so);
                     const float2 fd = mul2(f, sum), fx = mul2(f, cx), fy = mul2(f, cy);
                     const float den = warp_sum(fd.x + fd.y), n0 = warp_sum(fx.x + fx.y), n1 = warp_sum(fy.x + fy.y);
-                    const float tmax = warp_max(fmaxf(m.x, m.y));
+                    const float tmax = warp_max(fmaxf(m.x, m.y)) - offM[k];
                     if (lane == 0) {
 #pragma unroll
                         for (int r = 0; r < CL; ++r) pr.async_f32(wmax_dst[r] + (uint32_t)(so * 64) * 4u, tmax, full_of[r] + 8u * so);
@@ -674,7 +674,7 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                     } else if (t == 2) {
                         As_next = splat2(-(wk[MAXN - 2] * wk[2 * MAXN - 2] + wk[MAXN - 1] * wk[2 * MAXN - 1]));          // At_1 = 0 + shift of step 1
                     }
-                    const float Dm = ((float)(Ofin[k] - O_s[k * OSTR + t] - P[k]) + lsefin[k]) - offM[k];
+                    const float Dm = ((float)(Ofin[k] - O_s[k * OSTR + t] - P[k]) + lsefin[k]);
                     const float2 offM2 = splat2(offM[k]);
                     float2 u[K], cb[8];
 #pragma unroll
@@ -689,7 +689,7 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                             for (int bb = 0; bb < 2; ++bb) {
                                 const float2 dx = sub2(cb[2 * (e + bb)], wx), dy = sub2(cb[2 * (e + bb) + 1], wy);
                                 const float2 Mb = bb == 0 ? make_float2(Mv.x, Mv.z) : make_float2(Mv.y, Mv.w);
-                                u[b + bb] = fma2(fma2(dy, dy, mul2(dx, dx)), nl2, sub2(Mb, offM2));
+                                u[b + bb] = fma2(fma2(dy, dy, mul2(dx, dx)), nl2, Mb);
                             }
                         }
                     }
@@ -731,12 +731,12 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                     tmem_wait_st();
                     // S0 = sum gamma = f sum rho;  S2 = sum gamma r = f (sum rho y + At sum rho)
                     const float2 S0 = mul2(f, sum), S2 = mul2(f, fma2(Ahj, sum, ya));
-                    const float2 outM = add2(m, lg2f2(sum));
+                    const float2 outM = add2(sub2(m, offM2), lg2f2(sum));
                     const float2 outB = fma2(ya, rcpf2(sum), splat2(gsp));
                     pr.async_v2(push_b + (uint32_t)(so * 2 * QC) * 4u, outM.x, outM.y, push_b_mbar + 8u * so);
                     pr.async_v2(push_b + (uint32_t)(so * 2 * QC + QC) * 4u, outB.x, outB.y, push_b_mbar + 8u * so);
                     const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), z0 = warp_sum(Z0.x + Z0.y), z1 = warp_sum(Z1.x + Z1.y);
-                    const float tmax = warp_max(fmaxf(m.x, m.y));
+                    const float tmax = warp_max(fmaxf(m.x, m.y)) - offM[k];
                     if (lane == 0) {
 #pragma unroll
                         for (int r = 0; r < CL; ++r) pr.async_f32(wmax_dst[r] + (uint32_t)(so * 64) * 4u, tmax, full_of[r] + 8u * so);
