@@ -38,6 +38,27 @@ __device__ __forceinline__ float warp_max(float v) {
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
     return r;
 }
+// Sums of several values over the warp in one butterfly: the first rounds halve the number of values a
+// lane carries (it keeps one half, sends the other), the rest run on a single value.
+// Two values, 5 shuffles: lanes 0-15 return the sum of a, lanes 16-31 the sum of b.
+__device__ __forceinline__ float warp_sum2_split(float a, float b, int lane) {
+    const bool hi = lane & 16;
+    float v = (hi ? b : a) + __shfl_xor_sync(0xffffffffu, hi ? a : b, 16);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// Three values, 6 shuffles: lanes 0-7 return the sum of a, lanes 8-15 of b, lanes 16-23 of c.
+__device__ __forceinline__ float warp_sum3_split(float a, float b, float c, int lane) {
+    const bool hi = lane & 16, h8 = lane & 8;
+    const float rx = __shfl_xor_sync(0xffffffffu, hi ? a : c, 16);
+    const float ry = __shfl_xor_sync(0xffffffffu, hi ? b : 0.f, 16);
+    const float u = (hi ? c : a) + rx, w = (hi ? 0.f : b) + ry;
+    float v = (h8 ? w : u) + __shfl_xor_sync(0xffffffffu, h8 ? u : w, 8);
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     constexpr int KK = K * K;
     constexpr uint32_t BUF_BYTES = 2u * QC * 4u;                 // (L, At) of one parity
     constexpr uint32_t TX_MSG = BUF_BYTES + SLOTS * 4u;          // messages + gauge slots
-    constexpr uint32_t TX_PART = SLOTS * 16u;                    // posterior sums (rank 0 only)
+    constexpr uint32_t TX_PART = SLOTS * 12u;                    // posterior sums (rank 0 only)
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = cluster_ctarank();
@@ -433,12 +433,10 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 }
             }
             tmem_wait_st();
-            const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), zz = warp_sum(ZS.x + ZS.y);
             tmax = warp_max(tmax) - offM;
             if (lane == 0) {
 #pragma unroll
                 for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
-                st_async_v4(part_dst + (uint32_t)(ob * 128) * 4u, s0, s2, zz, 0.f, full_of[0] + ob_mbar);
             }
             TICK(tb0);
             __syncwarp();
@@ -447,6 +445,11 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
 #pragma unroll
                 for (int r = 0; r < CL; ++r) mbar_arrive_remote(full_of[r] + ob_mbar);
             }
+            // the posterior sums follow the arrival: the phase cannot complete before their bytes have landed
+            // (they are part of rank 0's expected count), and nobody waits for this warp's shuffles
+            const float s3 = warp_sum3_split(S0.x + S0.y, S2.x + S2.y, ZS.x + ZS.y, lane);
+            if ((lane & 7) == 0 && lane < 24)
+                st_async_f32(part_dst + (uint32_t)(ob * 128 + (lane >> 3)) * 4u, s3, full_of[0] + ob_mbar);
             ib = ob;
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");

@@ -368,13 +368,10 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                         }
                     }
                 }
-                const float num = warp_sum(num2.x + num2.y), den = warp_sum(den2.x + den2.y);
+                const float nd = warp_sum2_split(num2.x + num2.y, den2.x + den2.y, lane);   // lane 0: numerator, lane 16: denominator
                 tmax = warp_max(tmax) - offM;
-                if (lane == 0) {
-                    wmax[(cur ^ 1) * 32 + warp] = tmax;
-                    part[((cur ^ 1) * 32 + warp) * 2] = num;
-                    part[((cur ^ 1) * 32 + warp) * 2 + 1] = den;
-                }
+                if (lane == 0) wmax[(cur ^ 1) * 32 + warp] = tmax;
+                if ((lane & 15) == 0) part[((cur ^ 1) * 32 + warp) * 2 + (lane >> 4)] = nd;
                 compute_barrier(CT);
             }
             {
