@@ -143,10 +143,12 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         }
 #pragma unroll
         for (int j = 0; j < K; ++j) {
-            // M([j|x]) -> butterfly x1 = (j*NB + x) / K, input b1 = x mod K, at [xl1*K + b1], CTA j*CL/K
+            // (M, Bt)([j|x]) -> butterfly x1 = (j*NB + x) / K, input b1 = x mod K, CTA j*CL/K.  The pair travels
+            // as one 8-byte store; inputs 2e, 2e+1 of a butterfly share a 16-byte entry of plane e:
+            // float4 [K/2][NBC] = (M_2e, Bt_2e, M_2e+1, Bt_2e+1)
             const int q1 = j * NB + x, x1 = q1 / K, b1 = q1 % K;
             const int r1 = x1 / NBC, xl1 = x1 % NBC;
-            push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(xl1 * K + b1) * 4u, (uint32_t)r1);
+            push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(((b1 >> 1) * NBC + xl1) * 4 + (b1 & 1) * 2) * 4u, (uint32_t)r1);
         }
     }
     uint32_t wmax_dst[CL], lz_dst[CL];
@@ -292,7 +294,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         // ================= beta sweep carrying (M, Bt), with the gradient contraction
         {
             const float gshn = -__ldg(g_s + n - 1) * __ldg(sf_s + n - 1);     // M_n = 0, Bt_n = 0 (+ centring shift)
-            for (int q = tid; q < QC; q += CT) { msg[ib * 2 * QC + q] = 0.f; msg[ib * 2 * QC + QC + q] = gshn; }
+            for (int f = tid; f < 2 * QC; f += CT) msg[ib * 2 * QC + f] = (f & 1) ? gshn : 0.f;
         }
 #pragma unroll
         for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, beta pairing
@@ -350,7 +352,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 finish_step(t + 1, ib);
             }
             if (!pr.warp_live()) break;                          // a wait ran out: this warp issues nothing more
-            const float *Min = msg + ib * 2 * QC, *Bin = Min + QC;
+            const float4 *MBin = reinterpret_cast<const float4 *>(msg + ib * 2 * QC);
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
             const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1);
@@ -377,11 +379,9 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 issue_chunk(i);                                      // this slot's entry for the next step (a whole step ahead)
                 float Mb[K], Yb[K];
 #pragma unroll
-                for (int b = 0; b < K; b += 4) {
-                    const float4 mv = *reinterpret_cast<const float4 *>(Min + (i * CT + tid) * K + b);
-                    const float4 bv = *reinterpret_cast<const float4 *>(Bin + (i * CT + tid) * K + b);
-                    Mb[b] = mv.x; Mb[b + 1] = mv.y; Mb[b + 2] = mv.z; Mb[b + 3] = mv.w;
-                    Yb[b] = bv.x; Yb[b + 1] = bv.y; Yb[b + 2] = bv.z; Yb[b + 3] = bv.w;
+                for (int e = 0; e < K / 2; ++e) {
+                    const float4 v = MBin[e * NBC + i * CT + tid];
+                    Mb[2 * e] = v.x; Yb[2 * e] = v.y; Mb[2 * e + 1] = v.z; Yb[2 * e + 1] = v.w;
                 }
 #pragma unroll
                 for (int u = 0; u < UNITS; ++u) {
@@ -421,10 +421,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                         const float2 outB = fma2(ya, rcpf2(sum), gshp2);
                         tmax = max3f(tmax, m.x, m.y);
                         const uint32_t mb0 = full_of[(2 * jh) * CL / K] + ob_mbar, mb1 = full_of[(2 * jh + 1) * CL / K] + ob_mbar;
-                        st_async_f32(push_b[i][2 * jh] + ob_off, outM.x, mb0);
-                        st_async_f32(push_b[i][2 * jh + 1] + ob_off, outM.y, mb1);
-                        st_async_f32(push_b[i][2 * jh] + ob_off + QC * 4u, outB.x, mb0);
-                        st_async_f32(push_b[i][2 * jh + 1] + ob_off + QC * 4u, outB.y, mb1);
+                        st_async_v2(push_b[i][2 * jh] + ob_off, outM.x, outB.x, mb0);
+                        st_async_v2(push_b[i][2 * jh + 1] + ob_off, outM.y, outB.y, mb1);
                         S0 = fma2(f, sum, S0);
                         S2 = fma2(f, fma2(Ahj, sum, ya), S2);
                         ZS = add2(ZS, zs);
