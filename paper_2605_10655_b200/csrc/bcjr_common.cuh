@@ -48,17 +48,18 @@ __device__ __forceinline__ float warp_sum2_split(float a, float b, int lane) {
     for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
-// Three values, 6 shuffles: lanes 0-7 return the sum of a, lanes 8-15 of b, lanes 16-23 of c.
-__device__ __forceinline__ float warp_sum3_split(float a, float b, float c, int lane) {
+// Four values, 6 shuffles: lanes 0-7 return the sum of a, lanes 8-15 of b, lanes 16-23 of c, lanes 24-31 of d.
+__device__ __forceinline__ float warp_sum4_split(float a, float b, float c, float d, int lane) {
     const bool hi = lane & 16, h8 = lane & 8;
     const float rx = __shfl_xor_sync(0xffffffffu, hi ? a : c, 16);
-    const float ry = __shfl_xor_sync(0xffffffffu, hi ? b : 0.f, 16);
-    const float u = (hi ? c : a) + rx, w = (hi ? 0.f : b) + ry;
+    const float ry = __shfl_xor_sync(0xffffffffu, hi ? b : d, 16);
+    const float u = (hi ? c : a) + rx, w = (hi ? d : b) + ry;
     float v = (h8 ? w : u) + __shfl_xor_sync(0xffffffffu, h8 ? u : w, 8);
 #pragma unroll
     for (int o = 4; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
+__device__ __forceinline__ float warp_sum3_split(float a, float b, float c, int lane) { return warp_sum4_split(a, b, c, 0.f, lane); }
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

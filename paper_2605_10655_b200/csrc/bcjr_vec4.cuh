@@ -636,7 +636,9 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                 const float *pp = part + (size_t)((b * NBLK + k) * 64) * 4;
                 const float4 s4 = *reinterpret_cast<const float4 *>(pp + lane * 4);
                 const float4 o = *reinterpret_cast<const float4 *>(pp + (lane + 32) * 4);
-                const float a0 = warp_sum(s4.x + o.x), a2 = warp_sum(s4.y + o.y), z0 = warp_sum(s4.z + o.z), z1 = warp_sum(s4.w + o.w);
+                const float v4 = warp_sum4_split(s4.x + o.x, s4.y + o.y, s4.z + o.z, s4.w + o.w, lane);
+                const float a0 = __shfl_sync(0xffffffffu, v4, 0), a2 = __shfl_sync(0xffffffffu, v4, 8);
+                const float z0 = __shfl_sync(0xffffffffu, v4, 16), z1 = __shfl_sync(0xffffffffu, v4, 24);
                 if (lane == 0) {
                     const float *wk = w_s + k * 3 * MAXN + 2 * (t - 1);
                     const float i0 = 1.f / a0;
@@ -735,13 +737,14 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                     const float2 outB = fma2(ya, rcpf2(sum), splat2(gsp));
                     pr.async_v2(push_b + (uint32_t)(so * 2 * QC) * 4u, outM.x, outM.y, push_b_mbar + 8u * so);
                     pr.async_v2(push_b + (uint32_t)(so * 2 * QC + QC) * 4u, outB.x, outB.y, push_b_mbar + 8u * so);
-                    const float s0 = warp_sum(S0.x + S0.y), s2 = warp_sum(S2.x + S2.y), z0 = warp_sum(Z0.x + Z0.y), z1 = warp_sum(Z1.x + Z1.y);
+                    const float v4 = warp_sum4_split(S0.x + S0.y, S2.x + S2.y, Z0.x + Z0.y, Z1.x + Z1.y, lane);   // lanes 0, 8, 16, 24
                     const float tmax = warp_max(fmaxf(m.x, m.y)) - offM[k];
                     if (lane == 0) {
 #pragma unroll
                         for (int r = 0; r < CL; ++r) pr.async_f32(wmax_dst[r] + (uint32_t)(so * 64) * 4u, tmax, full_of[r] + 8u * so);
-                        pr.async_v4(part_dst + (uint32_t)(so * 256) * 4u, s0, s2, z0, z1, full_of[0] + 8u * so);
                     }
+                    if ((lane & 7) == 0)
+                        pr.async_f32(part_dst + (uint32_t)(so * 256 + (lane >> 3)) * 4u, v4, full_of[0] + 8u * so);
                     Ls[k] = Ls_next; As[k] = As_next;
                 }
             }
