@@ -515,8 +515,8 @@ void launch_fwht_rows(const float *in, float *out, const float *s, int m, float 
 extern "C" {
 
 #ifdef BCJR_TIMING
-// development aid, not part of the ABI: cycle counters of the beta sweep of the backward kernel
-void bcjr_debug_duo_timing(unsigned long long *out8) { cudaMemcpyFromSymbol(out8, g_duo_timing, 64); }
+// development aid, not part of the ABI: per-warp cycle counters of the backward kernel's sweeps (CTA 0)
+void bcjr_debug_duo_timing(unsigned long long *out128) { cudaMemcpyFromSymbol(out128, g_duo_timing, 1024); }
 #endif
 
 bcjr_status bcjr_create(bcjr_ctx **out, int device_ordinal)

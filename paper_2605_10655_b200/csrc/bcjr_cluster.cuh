@@ -59,6 +59,26 @@ __device__ __forceinline__ void st_async_v4(uint32_t addr, float a, float b, flo
                  "f"(a), "f"(b), "f"(c), "f"(d), "r"(mbar)
                  : "memory");
 }
+// One output either way: a plain store into this CTA's shared memory (own = true, addr in the CTA's
+// window) or st.async into a peer's (addr in the cluster window, bytes credited to mbar).  No branch.
+__device__ __forceinline__ void push_v2(bool own, uint32_t addr, float a, float b, uint32_t mbar)
+{
+    asm volatile(
+        "{ .reg .pred p; setp.ne.u32 p, %0, 0;\n"
+        "@p st.shared.v2.f32 [%1], {%2, %3};\n"
+        "@!p st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%1], {%2, %3}, [%4]; }" ::"r"((uint32_t)own),
+        "r"(addr), "f"(a), "f"(b), "r"(mbar)
+        : "memory");
+}
+__device__ __forceinline__ void push_v4(bool own, uint32_t addr, float a, float b, float c, float d, uint32_t mbar)
+{
+    asm volatile(
+        "{ .reg .pred p; setp.ne.u32 p, %0, 0;\n"
+        "@p st.shared.v4.f32 [%1], {%2, %3, %4, %5};\n"
+        "@!p st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%1], {%2, %3, %4, %5}, [%6]; }" ::"r"((uint32_t)own),
+        "r"(addr), "f"(a), "f"(b), "f"(c), "f"(d), "r"(mbar)
+        : "memory");
+}
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_sync() { cluster_arrive(); cluster_wait(); }

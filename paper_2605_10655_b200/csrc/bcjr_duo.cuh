@@ -10,15 +10,21 @@
 // of two fill all 148 SMs (clusters of four, needed when the accumulators live in registers,
 // fill only 132).
 //
-// Step protocol.  Messages are double-buffered.  Every output is pushed with st.async into the
-// consumer CTA's buffer `ob` and credits that CTA's mbarrier full[ob] with its bytes; a phase of
-// full[ob] completes when (a) all bytes have landed and (b) every warp of the cluster has
-// arrived on it after its last butterfly of the step -- so nobody still reads the other buffer
-// when the next step starts overwriting it.  The arrival is relaxed:
-// it has nothing to publish (the data travels with st.async and is accounted in bytes), and the
-// reads it has to follow are complete when it issues, because every value a warp reads from
-// its input buffer feeds, through register dependences, an st.async that precedes the arrival
-// in program order.  (A release arrival per warp costs a cluster-scope fence: 8 % of the kernel.)
+// Step protocol.  Messages are double-buffered.  Half of a CTA's outputs are consumed by the CTA
+// itself, half by its peer (the perfect shuffle leaves no better split).  The peer's half is
+// pushed with st.async into the peer's buffer `ob` and credits the peer's mbarrier full[ob] with
+// its bytes; the own half is written with plain shared-memory stores, because st.async sustains
+// only ~10 bytes per clock per SM, whatever the destination: with all 64 KB of a step's outputs
+// on it, it alone set the step time (6.9 k clocks per step; 5.3 k with the own half off it).  A
+// phase of full[ob] completes when (a) the peer's bytes have landed and (b) every warp of the
+// cluster has arrived on it after its last butterfly of the step -- so nobody still reads the
+// other buffer when the next step starts overwriting it.  A warp arrives on its own CTA's
+// barrier with release semantics at CTA scope (that publishes its plain stores to the warps that
+// wait on the barrier) and on the peer's barrier relaxed: there it has nothing to publish (the
+// data travels with st.async and is accounted in bytes), and the reads the arrival has to follow
+// are complete when it issues, because every value a warp reads from its input buffer feeds,
+// through register dependences, a store that precedes the arrival in program order.  (A release
+// arrival at cluster scope per warp costs a fence: 8 % of the kernel.)
 //
 // History.  The inputs (L, At) of a butterfly in the alpha sweep are exactly what the same thread
 // needs for that butterfly in the beta sweep, so the history is thread-private: the thread stores
@@ -32,9 +38,9 @@ namespace bcjr {
 
 
 #ifdef BCJR_TIMING
-__device__ unsigned long long g_duo_timing[8];   // beta sweep, warp 1 of CTA 0: compute, cta barrier, input wait, ring wait
+__device__ unsigned long long g_duo_timing[128]; // CTAs 0 and 1, per warp: alpha step, alpha input wait, beta step, beta input wait (cycles, summed)
 #define TICK(var) const long long var = clock64()
-#define TACC(slot, a, b) do { if (blockIdx.x == 0 && warp == 1 && lane == 0) tacc[slot] += (unsigned long long)((b) - (a)); } while (0)
+#define TACC(slot, a, b) do { if (blockIdx.x < 2 && lane == 0) tacc[slot] += (unsigned long long)((b) - (a)); } while (0)
 #else
 #define TICK(var)
 #define TACC(slot, a, b)
@@ -68,7 +74,7 @@ struct DuoCfg {
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
     static_assert(2 * BPT * K * K == 128, "codebook + accumulators fill the thread's 128 TMEM columns");
-    static_assert(K % CL == 0, "beta destinations: CTA of output j is j*CL/K");
+    static_assert(CL == 2 && K % (2 * CL) == 0, "beta destinations: CTA of output j is j*CL/K");
     static_assert(UNITS * HPU == K / 2 && (K == 4 || K == 8), "unit decomposition");
     __host__ __device__ static constexpr int a_idx(int j, int h) { return K == 4 ? 2 * j + h : j; }
     __host__ __device__ static constexpr int b_idx(int jh, int b) { return K == 4 ? 4 * jh + b : b; }
@@ -82,7 +88,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     constexpr int CL = C::CL, SLOTS = C::SLOTS, NCH = C::NCH, RD = C::RD, UNITS = C::UNITS, HPU = C::HPU, NU = BPT * UNITS;
     constexpr int KK = K * K;
     constexpr uint32_t BUF_BYTES = 2u * QC * 4u;                 // (L, At) of one parity
-    constexpr uint32_t TX_MSG = BUF_BYTES + SLOTS * 4u;          // messages + gauge slots
+    constexpr uint32_t TX_MSG = BUF_BYTES / 2 + SLOTS * 4u;      // the peer's half of the messages + gauge slots
     constexpr uint32_t TX_PART = SLOTS * 12u;                    // posterior sums (rank 0 only)
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -131,6 +137,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     const uint32_t tm_cb = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * 128);
     const uint32_t tm_acc = tm_cb + 64u;
     uint32_t push_a[BPT], push_a_mbar[BPT], push_b[BPT][K];
+    uint32_t own_a = 0;                                          // bit i: the alpha outputs of butterfly slot i stay in this CTA
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
         const int x = (int)rank * NBC + i * CT + tid;
@@ -138,8 +145,10 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             // L([x|l]) -> butterfly x2 = (x*K) mod NB, input j2 = (x*K) / NB, at [(i2*K + j2)*CT + tid2 .. +K)
             const int q2 = x * K, j2 = q2 / NB, x2 = q2 % NB;
             const int r2 = x2 / NBC, xl2 = x2 % NBC;
-            push_a[i] = mapa_u32(msg_u32 + (uint32_t)(((xl2 / CT) * K + j2) * CT + xl2 % CT) * 4u, (uint32_t)r2);
+            const uint32_t a2 = msg_u32 + (uint32_t)(((xl2 / CT) * K + j2) * CT + xl2 % CT) * 4u;
+            push_a[i] = r2 == (int)rank ? a2 : mapa_u32(a2, (uint32_t)r2);     // own CTA: plain address, plain stores
             push_a_mbar[i] = full_of[r2];
+            own_a |= (r2 == (int)rank ? 1u : 0u) << i;
         }
 #pragma unroll
         for (int j = 0; j < K; ++j) {
@@ -148,7 +157,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             // float4 [K/2][NBC] = (M_2e, Bt_2e, M_2e+1, Bt_2e+1)
             const int q1 = j * NB + x, x1 = q1 / K, b1 = q1 % K;
             const int r1 = x1 / NBC, xl1 = x1 % NBC;
-            push_b[i][j] = mapa_u32(msg_u32 + (uint32_t)(((b1 >> 1) * NBC + xl1) * 4 + (b1 & 1) * 2) * 4u, (uint32_t)r1);
+            const uint32_t a1 = msg_u32 + (uint32_t)(((b1 >> 1) * NBC + xl1) * 4 + (b1 & 1) * 2) * 4u;
+            push_b[i][j] = r1 == (int)rank ? a1 : mapa_u32(a1, (uint32_t)r1);  // r1 = j*CL/K for every x
         }
     }
     uint32_t wmax_dst[CL], lz_dst[CL];
@@ -194,8 +204,10 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         // ================= alpha sweep carrying (L, At)
         for (int t = 1; t <= n; ++t) {
             const int ob = ib ^ 1;
+            TICK(ta0);
             if (t > 1) {
                 wait_inputs(ib);
+                TICK(ta1); TACC(1, ta0, ta1);
                 cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
                 off = rintf(cmax);
             }
@@ -254,10 +266,11 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                     }
                 }
                 const uint32_t mb = push_a_mbar[i] + ob_mbar;
+                const bool own = (own_a >> i) & 1u;
 #pragma unroll
                 for (int h = 0; h < K / 2; h += 2) {
-                    st_async_v4(push_a[i] + ob_off + 8u * h, outL[h].x, outL[h].y, outL[h + 1].x, outL[h + 1].y, mb);
-                    st_async_v4(push_a[i] + ob_off + QC * 4u + 8u * h, outA[h].x, outA[h].y, outA[h + 1].x, outA[h + 1].y, mb);
+                    push_v4(own, push_a[i] + ob_off + 8u * h, outL[h].x, outL[h].y, outL[h + 1].x, outL[h + 1].y, mb);
+                    push_v4(own, push_a[i] + ob_off + QC * 4u + 8u * h, outA[h].x, outA[h].y, outA[h + 1].x, outA[h + 1].y, mb);
                 }
             }
             tmax = warp_max(tmax);
@@ -268,10 +281,11 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             O += (int)off;
             if (tid == 0) O_s[t + 1] = O;
             __syncwarp();
-            if (lane == 0) {                                     // this warp has read all its inputs
-#pragma unroll
-                for (int r = 0; r < CL; ++r) mbar_arrive_remote(full_of[r] + ob_mbar);
+            if (lane == 0) {                                     // this warp has read all its inputs and written its outputs
+                mbar_arrive_local(mbar_full + ob_mbar);
+                mbar_arrive_remote(full_of[rank ^ 1u] + ob_mbar);
             }
+            TICK(ta2); TACC(0, ta0, ta2);
             ib = ob;
         }
         // ================= log2 Z
@@ -345,7 +359,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             TICK(tk0);
             if (t < n) {
                 wait_inputs(ib);
-                TICK(tk1); TACC(2, tk0, tk1);
+                TICK(tk1); TACC(3, tk0, tk1);
                 cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF);
                 P += (int)offM;
                 offM = rintf(cmax);
@@ -367,8 +381,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             asm volatile("cp.async.wait_group 0;" ::: "memory");    // this step's history, requested during the previous step
 #pragma unroll
             for (int i = 0; i < BPT; ++i, ++chunk) {
-                TICK(tr0);
-                TICK(tr1); TACC(3, tr0, tr1);
                 float Lh[K], Ah[K];
 #pragma unroll
                 for (int q = 0; q < K / 4; ++q) {
@@ -421,8 +433,9 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                         const float2 outB = fma2(ya, rcpf2(sum), gshp2);
                         tmax = max3f(tmax, m.x, m.y);
                         const uint32_t mb0 = full_of[(2 * jh) * CL / K] + ob_mbar, mb1 = full_of[(2 * jh + 1) * CL / K] + ob_mbar;
-                        st_async_v2(push_b[i][2 * jh] + ob_off, outM.x, outB.x, mb0);
-                        st_async_v2(push_b[i][2 * jh + 1] + ob_off, outM.y, outB.y, mb1);
+                        const bool own = (2 * jh) * CL / K == (int)rank;         // both outputs of the pair go to the same CTA
+                        push_v2(own, push_b[i][2 * jh] + ob_off, outM.x, outB.x, mb0);
+                        push_v2(own, push_b[i][2 * jh + 1] + ob_off, outM.y, outB.y, mb1);
                         S0 = fma2(f, sum, S0);
                         S2 = fma2(f, fma2(Ahj, sum, ya), S2);
                         ZS = add2(ZS, zs);
@@ -436,12 +449,11 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
 #pragma unroll
                 for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
             }
-            TICK(tb0);
             __syncwarp();
-            TICK(tb1); TACC(1, tb0, tb1); TACC(0, tk0, tb1);
-            if (lane == 0 && !(drop_hook && t == n && blk == cid)) {   // this warp has read all its inputs
-#pragma unroll
-                for (int r = 0; r < CL; ++r) mbar_arrive_remote(full_of[r] + ob_mbar);
+            TICK(tb1); TACC(2, tk0, tb1);
+            if (lane == 0 && !(drop_hook && t == n && blk == cid)) {   // this warp has read all its inputs and written its outputs
+                mbar_arrive_local(mbar_full + ob_mbar);
+                mbar_arrive_remote(full_of[rank ^ 1u] + ob_mbar);
             }
             // the posterior sums follow the arrival: the phase cannot complete before their bytes have landed
             // (they are part of rank 0's expected count), and nobody waits for this warp's shuffles
@@ -477,8 +489,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         }
     }
 #ifdef BCJR_TIMING
-    if (blockIdx.x == 0 && warp == 1 && lane == 0)
-        for (int e = 0; e < 8; ++e) g_duo_timing[e] = tacc[e];
+    if (blockIdx.x < 2 && lane == 0)
+        for (int e = 0; e < 4; ++e) g_duo_timing[(blockIdx.x * 16 + warp) * 4 + e] = tacc[e];
 #endif
     if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
     asm volatile("cp.async.wait_all;" ::: "memory");           // no copy may be in flight at exit (a warp may have left the loop early)
