@@ -266,7 +266,9 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                     }
                 }
                 const uint32_t mb = push_a_mbar[i] + ob_mbar;
-                const bool own = (own_a >> i) & 1u;
+                // k = 2: the outputs of slot i go to CTA i & 1 whatever the thread (x*K mod NB = (i & 1)*NBC + 4 tid);
+                // said this way the choice is uniform for the compiler too
+                const bool own = BPT >= 2 ? (i & 1) == (int)rank : (own_a >> i) & 1u;
 #pragma unroll
                 for (int h = 0; h < K / 2; h += 2) {
                     push_v4(own, push_a[i] + ob_off + 8u * h, outL[h].x, outL[h].y, outL[h + 1].x, outL[h + 1].y, mb);
