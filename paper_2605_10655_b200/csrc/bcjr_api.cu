@@ -303,16 +303,21 @@ bcjr_status plan_cluster(bcjr_ctx *ctx, Kern kern, int CL, int threads, size_t s
 }
 
 // Lb = 16, 4 bits and 2 weights per step: one block per cluster of four CTAs, table slice in shared memory
-#ifndef VEC4_NBLK
-#define VEC4_NBLK 2
+// blocks in flight per cluster: three hide the exchange best in the forward kernel (6.6 -> 6.4 ms per 592 blocks),
+// the backward kernel has no registers for a third (9.55 -> 10.1 ms)
+#ifndef VEC4_FWD_NBLK
+#define VEC4_FWD_NBLK 3
+#endif
+#ifndef VEC4_BWD_NBLK
+#define VEC4_BWD_NBLK 2
 #endif
 bcjr_status launch_fwd_vec4(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
-    using C = Vec4Cfg<VEC4_NBLK>;
+    using C = Vec4Cfg<VEC4_FWD_NBLK>;
     if (p.n > C::MAX_N || ((uintptr_t)p.cb & 15u)) return BCJR_EUNSUPPORTED;
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1];
-    auto kern = fwd_vec4_kernel<VEC4_NBLK>;
+    auto kern = fwd_vec4_kernel<VEC4_FWD_NBLK>;
     bcjr_status rc = plan_cluster(ctx, kern, C::CL, C::THREADS, C::SMEM_BYTES, (p.B + C::NBLK - 1) / C::NBLK, &cfg, attr, st);
     if (rc) return rc;
     const int ncl = cfg.gridDim.x / C::CL, nt = p.n / C::V;
@@ -328,12 +333,12 @@ bcjr_status launch_fwd_vec4(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 
 bcjr_status launch_bwd_vec4(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
 {
-    using C = Vec4BwdCfg<VEC4_NBLK>;
+    using C = Vec4BwdCfg<VEC4_BWD_NBLK>;
     constexpr int S = C::F::S, V = 2, KB = 4;
     if (p.n > C::MAX_N || ((uintptr_t)p.cb & 15u)) return BCJR_EUNSUPPORTED;
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1];
-    auto kern = bwd_vec4_kernel<VEC4_NBLK>;
+    auto kern = bwd_vec4_kernel<VEC4_BWD_NBLK>;
     bcjr_status rc = plan_cluster(ctx, kern, C::CL, C::THREADS, C::SMEM_BYTES, (p.B + C::NBLK - 1) / C::NBLK, &cfg, attr, st);
     if (rc) return rc;
     const int ncl = cfg.gridDim.x / C::CL, nt = p.n / V;
