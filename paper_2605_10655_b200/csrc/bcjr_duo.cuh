@@ -345,7 +345,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         cluster_sync();                                          // beta start
         // rank 0, warp 0: turn the sums of step t (slots of parity b) into grad_W[t]
         auto finish_step = [&](int t, int b) {
-            if (rank == 0 && warp == 0) {
+            if (rank == 0 && warp == NWARP - 1) {                // the warps with the highest index finish a step first: slack
                 const float *pp = part + (b * 32 + lane) * 4;
                 float a0 = lane < SLOTS ? pp[0] : 0.f, a2 = lane < SLOTS ? pp[1] : 0.f, az = lane < SLOTS ? pp[2] : 0.f;
                 a0 = warp_sum(a0); a2 = warp_sum(a2); az = warp_sum(az);
@@ -494,7 +494,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     if (blockIdx.x < 2 && lane == 0)
         for (int e = 0; e < 4; ++e) g_duo_timing[(blockIdx.x * 16 + warp) * 4 + e] = tacc[e];
 #endif
-    if (tid == 0 && rank == 0) diag_max(&p.diag->max_defect, defect);
+    if (tid == CT - 32 && rank == 0) diag_max(&p.diag->max_defect, defect);
     asm volatile("cp.async.wait_all;" ::: "memory");           // no copy may be in flight at exit (a warp may have left the loop early)
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
