@@ -205,24 +205,27 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         for (int t = 1; t <= n; ++t) {
             const int ob = ib ^ 1;
             TICK(ta0);
+            // what does not depend on the step's inputs is requested before the wait for them: the first
+            // codebook unit from tensor memory and the step's scalars (their latency hides under the wait)
+            float2 cb[2][8];
+            tmem_ld16(tm_cb, cb[0]);
+            const float gt = __ldg(g_s + t - 1), wt = __ldg(w_s + t - 1);
+            const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
             if (t > 1) {
                 wait_inputs(ib);
                 TICK(ta1); TACC(1, ta0, ta1);
                 cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
                 off = rintf(cmax);
             }
-            if (!pr.warp_live()) break;                          // a wait ran out: this warp issues nothing more
+            if (!pr.warp_live()) { tmem_wait_ld(cb[0]); break; } // a wait ran out: this warp issues nothing more
             const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
             float4 *hrow = hist4 + ((size_t)(t - 1) * CL + rank) * (BPT * NCH * CT);      // (L_t, At_t) of this thread's butterflies
-            const float gt = __ldg(g_s + t - 1);
-            // shift for the consumers of this step's At (step t+1); unused at t = n
-            const float2 gshn2 = splat2(t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f);
-            const float2 w2 = splat2(__ldg(w_s + t - 1)), g2 = splat2(gt), off2 = splat2(off);
+            // gshn: shift for the consumers of this step's At (step t+1); unused at t = n
+            const float2 gshn2 = splat2(gshn);
+            const float2 w2 = splat2(wt), g2 = splat2(gt), off2 = splat2(off);
             float tmax = NEG_INF;
-            float2 cb[2][8];
-            tmem_ld16(tm_cb, cb[0]);
 #pragma unroll
             for (int i = 0; i < BPT; ++i) {
                 float2 outL[K / 2], outA[K / 2];
@@ -359,6 +362,14 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         for (int t = n; t >= 1; --t) {
             const int ob = ib ^ 1;
             TICK(tk0);
+            // requested before the wait for the step's inputs, like in the alpha sweep
+            float2 cb[2][8];
+            tmem_ld16(tm_cb, cb[0]);
+            const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1);
+            const float gsh = -gt * __ldg(sf_s + t - 1);                      // shift carried by the stored At
+            const float gshp = t > 1 ? -__ldg(g_s + t - 2) * __ldg(sf_s + t - 2) : 0.f;   // for step t-1
+            const int Ot = O_s[t];
+            asm volatile("cp.async.wait_group 0;" ::: "memory");    // this step's history, requested during the previous step
             if (t < n) {
                 wait_inputs(ib);
                 TICK(tk1); TACC(3, tk0, tk1);
@@ -367,20 +378,15 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 offM = rintf(cmax);
                 finish_step(t + 1, ib);
             }
-            if (!pr.warp_live()) break;                          // a wait ran out: this warp issues nothing more
+            if (!pr.warp_live()) { tmem_wait_ld(cb[0]); break; } // a wait ran out: this warp issues nothing more
             const float4 *MBin = reinterpret_cast<const float4 *>(msg + ib * 2 * QC);
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
-            const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1);
-            const float2 gsh2 = splat2(-gt * __ldg(sf_s + t - 1));            // shift carried by the stored At
-            const float2 gshp2 = splat2(t > 1 ? -__ldg(g_s + t - 2) * __ldg(sf_s + t - 2) : 0.f);   // for step t-1
+            const float2 gsh2 = splat2(gsh), gshp2 = splat2(gshp);
             const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT), offM2 = splat2(offM);
-            const float2 Dm2 = splat2((float)(Ofin - O_s[t] - P) + lsefin);
+            const float2 Dm2 = splat2((float)(Ofin - Ot - P) + lsefin);
             float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
             float tmax = NEG_INF;
-            float2 cb[2][8];
-            tmem_ld16(tm_cb, cb[0]);
-            asm volatile("cp.async.wait_group 0;" ::: "memory");    // this step's history, requested during the previous step
 #pragma unroll
             for (int i = 0; i < BPT; ++i, ++chunk) {
                 float Lh[K], Ah[K];
