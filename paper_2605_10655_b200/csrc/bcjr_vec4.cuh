@@ -170,6 +170,11 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
             for (int k = 0; k < NBLK; ++k) {
                 if (k < nact) {
                     const int si = ib * NBLK + k, so = ob * NBLK + k;
+                    // the first table unit and the step's weights do not depend on the step's inputs: requested before the wait
+                    float2 a[K], cb[2][8];
+                    tmem_ld16(tm, cb[0]);
+                    const float *wk = w_s + k * C::MAX_N + 2 * (t - 1);
+                    const float2 wx = splat2(wk[0]), wy = splat2(wk[1]);
                     if (t > 1) {
                         wait_inputs(ib, k);
                         cmax[k] = warp_max(slot_max(wmax + si * 64, lane, SLOTS)) - off[k];
@@ -177,10 +182,6 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
                     }
                     const float *Lin = msg + si * QC + (tid >> 3);            // [j][x], x = (q0 >> 4) & 63
                     if (tid == 0) pr.expect_tx(mbar_full + 8u * so, TX_MSG);
-                    const float *wk = w_s + k * C::MAX_N + 2 * (t - 1);
-                    const float2 wx = splat2(wk[0]), wy = splat2(wk[1]);
-                    float2 a[K], cb[2][8];
-                    tmem_ld16(tm, cb[0]);
 #pragma unroll
                     for (int u = 0; u < C::UNITS; ++u) {
                         tmem_wait_ld(cb[u & 1]);
@@ -277,6 +278,8 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
             for (int k = 0; k < NBLK; ++k) {
                 if (k < nact) {
                     const int si = ib * NBLK + k, so = ob * NBLK + k;
+                    float2 u[K], cb[2][8];
+                    tmem_ld16(tm, cb[0]);                                     // requested before the wait for the step's inputs
                     if (t < nt) {
                         wait_inputs(ib, k);
                         cmax[k] = warp_max(slot_max(wmax + si * 64, lane, SLOTS));
@@ -294,8 +297,6 @@ __global__ void __launch_bounds__(Vec4Cfg<NBLK_>::THREADS, 1) fwd_vec4_kernel(Fw
                     // the outputs are shifted by offM (once per group, below); D refers to the unshifted inputs
                     const float Dm = ((float)(Ofin[k] - O_s[k * OSTR + t] - P[k]) + lsefin[k]);
                     const float2 offM2 = splat2(offM[k]);
-                    float2 u[K], cb[2][8];
-                    tmem_ld16(tm, cb[0]);
 #pragma unroll
                     for (int un = 0; un < C::UNITS; ++un) {
                         tmem_wait_ld(cb[un & 1]);
