@@ -370,6 +370,14 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             const float gshp = t > 1 ? -__ldg(g_s + t - 2) * __ldg(sf_s + t - 2) : 0.f;   // for step t-1
             const int Ot = O_s[t];
             asm volatile("cp.async.wait_group 0;" ::: "memory");    // this step's history, requested during the previous step
+            float Lh0[K], Ah0[K];                                   // the first butterfly's, read before the wait as well
+#pragma unroll
+            for (int q = 0; q < K / 4; ++q) {
+                const float4 l4 = stage4[q * CT + tid], a4 = stage4[(K / 4 + q) * CT + tid];
+                Lh0[4 * q] = l4.x; Lh0[4 * q + 1] = l4.y; Lh0[4 * q + 2] = l4.z; Lh0[4 * q + 3] = l4.w;
+                Ah0[4 * q] = a4.x; Ah0[4 * q + 1] = a4.y; Ah0[4 * q + 2] = a4.z; Ah0[4 * q + 3] = a4.w;
+            }
+            issue_chunk(0);
             if (t < n) {
                 wait_inputs(ib);
                 TICK(tk1); TACC(3, tk0, tk1);
@@ -390,13 +398,18 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
 #pragma unroll
             for (int i = 0; i < BPT; ++i, ++chunk) {
                 float Lh[K], Ah[K];
+                if (i == 0) {
 #pragma unroll
-                for (int q = 0; q < K / 4; ++q) {
-                    const float4 l4 = stage4[(i * NCH + q) * CT + tid], a4 = stage4[(i * NCH + K / 4 + q) * CT + tid];
-                    Lh[4 * q] = l4.x; Lh[4 * q + 1] = l4.y; Lh[4 * q + 2] = l4.z; Lh[4 * q + 3] = l4.w;
-                    Ah[4 * q] = a4.x; Ah[4 * q + 1] = a4.y; Ah[4 * q + 2] = a4.z; Ah[4 * q + 3] = a4.w;
+                    for (int j = 0; j < K; ++j) { Lh[j] = Lh0[j]; Ah[j] = Ah0[j]; }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < K / 4; ++q) {
+                        const float4 l4 = stage4[(i * NCH + q) * CT + tid], a4 = stage4[(i * NCH + K / 4 + q) * CT + tid];
+                        Lh[4 * q] = l4.x; Lh[4 * q + 1] = l4.y; Lh[4 * q + 2] = l4.z; Lh[4 * q + 3] = l4.w;
+                        Ah[4 * q] = a4.x; Ah[4 * q + 1] = a4.y; Ah[4 * q + 2] = a4.z; Ah[4 * q + 3] = a4.w;
+                    }
+                    issue_chunk(i);                                  // this slot's entry for the next step (a whole step ahead)
                 }
-                issue_chunk(i);                                      // this slot's entry for the next step (a whole step ahead)
                 float Mb[K], Yb[K];
 #pragma unroll
                 for (int e = 0; e < K / 2; ++e) {
