@@ -186,6 +186,20 @@ def test_q_proj_shape_sampled_blocks(ctx, variant):
             ctx.set_option(k_, 0)
 
 
+@pytest.mark.parametrize("T", [0.3, 0.03, 0.01])
+def test_decoder_layer_temperature_range_sampled_blocks(ctx, T):
+    # the annealing range of the decoder-layer workload (0.3 -> 0.01) on its kernels: blocks of the down_proj-shaped
+    # matrix (rows of 8192 weights, 32 blocks per row), sampled
+    wl = synth.decoder_layer()
+    i = len(wl.matrices) - 1
+    Wm = wl.weights(i)
+    idx = synth.sample_blocks(Wm.shape[0], 4)
+    W, c = Wm[idx], wl.codebook()
+    g = np.random.default_rng(4242).standard_normal(W.shape).astype(np.float32)
+    got = _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"decoder layer sample, T={T}", viterbi=False)
+    assert got["diag"].last_path == 1
+
+
 @pytest.mark.parametrize("n,B", [(1, 3), (2, 2), (3, 1), (7, 5), (64, 2), (255, 1)])
 @pytest.mark.parametrize("variant", ["tmem", "cluster_registers"])
 def test_large_trellis_ragged_lengths_and_block_counts(ctx, variant, n, B):
