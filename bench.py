@@ -38,13 +38,17 @@ MUFU_PER_CLK_PER_SM = 16          # special-function results per clock per SM (C
 NUM_SMS = 148
 
 
-def mufu_ops_per_state_step(k: int, kernel: str, V: int = 1) -> float:
-    """Algorithmic special-function operations per state per step (one ex2 per state, plus per
-    group of K states: one lg2; the beta sweeps add one ex2 per group for the posterior; the
-    backward-pass sweeps add one rcp per group for the conditional expectation)."""
+def mufu_ops_per_state_step(k: int, kernel: str, V: int = 1, count: str = "algorithmic") -> float:
+    """Special-function operations per state per step, K = 2^(kV) states per group.
+
+    count="algorithmic": what the recursions need at the least -- one ex2 per state and one lg2 per group in
+    every sweep, plus one ex2 per group for the posterior in a beta sweep; the backward call repeats both
+    sweeps and reuses their exponentials for the gradient: forward 2 + 3/K, backward 2 + 3/K.
+    count="with_rcp": what the backward kernels in this library issue -- the same plus one rcp per group and
+    sweep (the conditional expectations carried next to the messages are normalised by the group sum)."""
     K = 1 << (k * V)
     fwd = (1 + 1 / K) + (1 + 2 / K)
-    bwd = (1 + 2 / K) + (1 + 3 / K)
+    bwd = fwd if count == "algorithmic" else (1 + 2 / K) + (1 + 3 / K)
     return {"fwd": fwd, "bwd": bwd, "both": fwd + bwd}[kernel]
 
 
@@ -144,6 +148,144 @@ def run_reference(args, wl):
     print(json.dumps(out))
 
 
+class Runner:
+    """Device buffers of one workload and the timed forward + backward step over all its matrices."""
+
+    def __init__(self, ctx, wl, dev, blocks_cap=0, rank=0, world=1, keep_host=False):
+        import torch
+        self.ctx, self.wl, self.dev, self.rank = ctx, wl, dev, rank
+        self.cb = torch.from_numpy(wl.codebook()).to(dev)
+        self.mats = []
+        for i, (name, _) in enumerate(wl.matrices):
+            W = wl.weights(i)
+            if blocks_cap:
+                W = W[:blocks_cap]
+            W = np.ascontiguousarray(W)
+            if world > 1:
+                W = np.roll(W, rank, axis=0)
+            m = {"name": name, "W": torch.from_numpy(W).to(dev)}
+            if keep_host:
+                m["W_host"] = torch.from_numpy(W).pin_memory()
+            m["soft"] = torch.empty_like(m["W"]); m["gW"] = torch.empty_like(m["W"]); m["g"] = torch.empty_like(m["W"])
+            self.mats.append(m)
+        self.nblocks = sum(m["W"].shape[0] for m in self.mats)
+        self.edges_per_step = 2 * self.nblocks * wl.steps * wl.S * wl.K
+        self.state_steps = self.nblocks * wl.steps * wl.S
+        self.gc = torch.empty(wl.S * wl.V, dtype=torch.float32, device=dev)
+        self.gc_total = torch.zeros(wl.S * wl.V, dtype=torch.float32, device=dev)
+        self.gen = torch.Generator(device=dev)
+
+    def fresh_g(self, step):
+        for i, m in enumerate(self.mats):
+            self.gen.manual_seed(self.wl.g_seed + 7919 * step + i + 104729 * self.rank)
+            m["g"].normal_(generator=self.gen)
+
+    def step(self, T, ev=None):
+        import torch
+        wl, ctx = self.wl, self.ctx
+        self.gc_total.zero_()
+        for m in self.mats:
+            if ev is not None:
+                ev["f0"].append(torch.cuda.Event(enable_timing=True)); ev["f0"][-1].record()
+            if wl.V == 1:
+                ctx.bcjr_soft_quantize(m["W"], self.cb, wl.Lb, wl.k, wl.n, T, soft=m["soft"])
+            else:
+                ctx.bcjr_soft_quantize_vec(m["W"], self.cb, wl.Lb, wl.k, wl.V, wl.n, T, soft=m["soft"])
+            if ev is not None:
+                ev["f1"].append(torch.cuda.Event(enable_timing=True)); ev["f1"][-1].record()
+            ctx.bcjr_backward(m["g"], grad_W=m["gW"], grad_codebook=self.gc)
+            if ev is not None:
+                ev["b1"].append(torch.cuda.Event(enable_timing=True)); ev["b1"][-1].record()
+            self.gc_total.add_(self.gc)
+        shard.allreduce_grad_codebook(self.gc_total)     # the one exchange of the data-parallel path
+
+    def timed(self, temps_warm, temps_timed, flush):
+        """Warm-up steps, then the timed ones (CUDA events per step on the launching stream, L2 evicted in
+        between).  Returns per-step ms, summed forward / backward ms and the launch count."""
+        import torch
+        for s, T in enumerate(temps_warm):
+            self.fresh_g(s); flush.zero_()
+            self.step(T)
+        d0 = self.ctx.sync_status()
+        evs = []
+        for s, T in enumerate(temps_timed):
+            self.fresh_g(len(temps_warm) + s)
+            flush.zero_()                                   # evict L2 between timed steps (not timed)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev = {"f0": [], "f1": [], "b1": []}
+            e0.record()
+            self.step(T, ev)
+            e1.record()
+            evs.append((e0, e1, ev))
+        torch.cuda.synchronize()
+        step_ms = [e0.elapsed_time(e1) for e0, e1, _ in evs]
+        fwd_ms = sum(a.elapsed_time(b) for _, _, ev in evs for a, b in zip(ev["f0"], ev["f1"]))
+        bwd_ms = sum(a.elapsed_time(b) for _, _, ev in evs for a, b in zip(ev["f1"], ev["b1"]))
+        diag = self.ctx.sync_status()
+        return step_ms, fwd_ms, bwd_ms, diag, diag.kernel_launches - d0.kernel_launches
+
+
+def mufu_fractions(wl, state_steps, fwd_ms, bwd_ms, step_ms, peak_gops):
+    """Fractions of the special-function peak, on both operation counts (see mufu_ops_per_state_step)."""
+    out = {}
+    for count, tag in (("algorithmic", "frac"), ("with_rcp", "frac_with_rcp")):
+        for kern, ms in (("fwd", fwd_ms), ("bwd", bwd_ms), ("both", step_ms)):
+            ops = mufu_ops_per_state_step(wl.k, kern, wl.V, count) * state_steps
+            out[f"{kern}_{tag}"] = ops / (ms * 1e-3) / 1e9 / peak_gops
+    return out
+
+
+def workload_leg(ctx, name, blocks_cap, dev, flush, peak_gops):
+    """A short measurement of another workload in the same run: one warm-up step, two timed steps."""
+    import torch
+    wl = WORKLOADS[name]()
+    r = Runner(ctx, wl, dev, blocks_cap)
+    step_ms, fwd_ms, bwd_ms, diag, _ = r.timed([wl.T], [wl.T, wl.T], flush)
+    ms = float(np.mean(step_ms))
+    leg = {"workload": wl.name, "blocks": r.nblocks, "Lb": wl.Lb, "k": wl.k, "V": wl.V, "n": wl.n, "T": wl.T,
+           "ms_per_step": ms, "fwd_ms": fwd_ms / 2, "bwd_ms": bwd_ms / 2, "edges_per_s": r.edges_per_step / (ms * 1e-3),
+           "path": "large-trellis kernels" if diag.last_path else "generic kernels",
+           "max_posterior_defect": diag.max_posterior_defect}
+    leg.update(mufu_fractions(wl, r.state_steps, fwd_ms / 2, bwd_ms / 2, ms, peak_gops))
+    del r
+    torch.cuda.empty_cache()
+    return leg
+
+
+def qat_loop_leg(ctx, dev, flush, steps=4):
+    """Algorithm 1 around the path, timed as a loop: at each step the forward call, a stand-in loss on the soft
+    codeword (mean squared distance to the initial weights: the layer-output loss of the paper needs a model and
+    calibration activations), then bcjr_backward_adam, which updates the latent weights and the table in
+    place.  q_proj-shaped matrix, T annealed 0.3 -> 0.01 over the steps."""
+    import torch
+    wl = WORKLOADS["q_proj"]()
+    W = torch.from_numpy(np.ascontiguousarray(wl.weights(0))).to(dev)
+    target = W.clone()
+    cb = torch.from_numpy(wl.codebook()).to(dev)
+    mW, vW, mc, vc = torch.zeros_like(W), torch.zeros_like(W), torch.zeros_like(cb), torch.zeros_like(cb)
+    soft = torch.empty_like(W)
+    temps = anneal_schedule(0.3, 0.01, steps)
+    losses, ms = [], []
+    for t in range(steps + 1):                                  # the first pass is the warm-up
+        T = temps[max(t - 1, 0)]
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.bcjr_soft_quantize(W, cb, wl.Lb, wl.k, wl.n, T, soft=soft)
+        diff = soft - target
+        loss = (diff * diff).mean()
+        g = diff * (2.0 / diff.numel())
+        ctx.bcjr_backward_adam(g, mW, vW, t + 1, 1e-3, m_c=mc, v_c=vc, lr_c=1e-4)
+        e1.record()
+        torch.cuda.synchronize()
+        if t > 0:
+            ms.append(e0.elapsed_time(e1)); losses.append(float(loss))
+    nb = W.shape[0]
+    return {"workload": wl.name, "blocks": nb, "steps": steps, "T": [temps[0], temps[-1]], "ms_per_step": float(np.mean(ms)),
+            "edges_per_s": 2 * nb * wl.steps * wl.S * wl.K / (float(np.mean(ms)) * 1e-3), "loss": losses,
+            "updates": "latent weights and codebook table, Adam, inside bcjr_backward_adam"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -155,9 +297,11 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 generic kernels, 2 cluster kernels")
     ap.add_argument("--fwd-variant", type=int, default=0)
     ap.add_argument("--bwd-variant", type=int, default=0)
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE", help="bcjr_set_option passthrough")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-viterbi", action="store_true")
+    ap.add_argument("--no-legs", action="store_true", help="skip the short legs over the other workloads")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]()
     if args.impl == "reference":
@@ -165,7 +309,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2605_10655_b200 import Context
+    from paper_2605_10655_b200 import Context, binding
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -181,6 +325,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # ---- pipe rates of this GPU, measured now (the roofline's denominator)
+    peaks = binding.measure_pipe_peaks(local)
+
     # Every rank processes the whole workload shape on its own seeded data (weak scaling over
     # independent blocks); the only exchange is the all-reduce of grad_codebook.
     ctx = Context(local)
@@ -190,79 +337,25 @@ def main():
         ctx.set_option("fwd_variant", args.fwd_variant)
     if args.bwd_variant:
         ctx.set_option("bwd_variant", args.bwd_variant)
-    cb = torch.from_numpy(wl.codebook()).to(dev)
-    mats = []
-    for i, (name, _) in enumerate(wl.matrices):
-        W = wl.weights(i)
-        if args.blocks:
-            W = W[:args.blocks]
-        W = np.ascontiguousarray(W)
-        if world > 1:
-            W = np.roll(W, rank, axis=0)
-        mats.append({"name": name, "W_host": torch.from_numpy(W).pin_memory(), "W": torch.from_numpy(W).to(dev)})
-    total_steps = args.warmup + args.steps
-    temps = anneal_schedule(0.3, 0.01, total_steps) if wl.name.startswith("llama32_1b_decoder") else [wl.T] * total_steps
-    nblocks = sum(m["W"].shape[0] for m in mats)
-    edges_per_step = 2 * nblocks * wl.steps * wl.S * wl.K
-    for m in mats:
-        m["soft"] = torch.empty_like(m["W"]); m["gW"] = torch.empty_like(m["W"])
-        m["g"] = torch.empty_like(m["W"])
-    gc = torch.empty(wl.S * wl.V, dtype=torch.float32, device=dev)
-    gc_total = torch.zeros(wl.S * wl.V, dtype=torch.float32, device=dev)
+    for kv in args.option:
+        name, _, val = kv.partition("=")
+        ctx.set_option(name, int(val))
+    run = Runner(ctx, wl, dev, args.blocks, rank, world, keep_host=not args.no_e2e)
+    mats, cb, nblocks, edges_per_step = run.mats, run.cb, run.nblocks, run.edges_per_step
+    # the decoder-layer workload anneals T geometrically from 0.3 to 0.01 over the timed steps (warm-up at T_0)
+    annealed = wl.name.startswith("llama32_1b_decoder")
+    temps_timed = anneal_schedule(0.3, 0.01, args.steps) if annealed else [wl.T] * args.steps
+    temps_warm = [temps_timed[0]] * args.warmup
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # > L2 (126 MB)
-    gen = torch.Generator(device=dev)
 
-    def fresh_g(step):
-        for i, m in enumerate(mats):
-            gen.manual_seed(wl.g_seed + 7919 * step + i + 104729 * rank)
-            m["g"].normal_(generator=gen)
-
-    def one_step(step, T, ev=None):
-        gc_total.zero_()
-        for m in mats:
-            if ev is not None:
-                ev["f0"].append(torch.cuda.Event(enable_timing=True)); ev["f0"][-1].record()
-            if wl.V == 1:
-                ctx.bcjr_soft_quantize(m["W"], cb, wl.Lb, wl.k, wl.n, T, soft=m["soft"])
-            else:
-                ctx.bcjr_soft_quantize_vec(m["W"], cb, wl.Lb, wl.k, wl.V, wl.n, T, soft=m["soft"])
-            if ev is not None:
-                ev["f1"].append(torch.cuda.Event(enable_timing=True)); ev["f1"][-1].record()
-            ctx.bcjr_backward(m["g"], grad_W=m["gW"], grad_codebook=gc)
-            if ev is not None:
-                ev["b1"].append(torch.cuda.Event(enable_timing=True)); ev["b1"][-1].record()
-            gc_total.add_(gc)
-        shard.allreduce_grad_codebook(gc_total)          # the one exchange of the data-parallel path
-
-    for s in range(args.warmup):
-        fresh_g(s); flush.zero_()
-        one_step(s, temps[s])
-    d0 = ctx.sync_status()
-    launches0 = d0.kernel_launches
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
     t_wall0 = time.time()
-    step_ms, fwd_ms, bwd_ms = [], 0.0, 0.0
-    evs = []
-    for s in range(args.steps):
-        fresh_g(args.warmup + s)
-        flush.zero_()                                   # evict L2 between timed steps (not timed)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev = {"f0": [], "f1": [], "b1": []}
-        e0.record()
-        one_step(args.warmup + s, temps[args.warmup + s], ev)
-        e1.record()
-        evs.append((e0, e1, ev))
+    step_ms, fwd_ms, bwd_ms, diag, launches = run.timed(temps_warm, temps_timed, flush)
     barrier()
     t_wall1 = time.time()
-    for e0, e1, ev in evs:
-        step_ms.append(e0.elapsed_time(e1))
-        fwd_ms += sum(a.elapsed_time(b) for a, b in zip(ev["f0"], ev["f1"]))
-        bwd_ms += sum(a.elapsed_time(b) for a, b in zip(ev["f1"], ev["b1"]))
     clocks = sampler.stop(t_wall0, t_wall1)
-    diag = ctx.sync_status()
-    launches = diag.kernel_launches - launches0
     total_ms = float(sum(step_ms))
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
@@ -324,7 +417,7 @@ def main():
             upd["rht"] = {"shape": [rows, cols], "ms": rms, "gbs": 8.0 * rows * cols / (rms * 1e-3) / 1e9}
             del W2, out2
 
-    # ---- end to end through the host-buffer entry point (pinned host memory both ways)
+    # ---- end to end through the host-buffer entry point (pinned host memory both ways), same schedule
     e2e = None
     if not args.no_e2e and wl.V == 1:          # the host-buffer entry point covers the scalar trellis
         host = []
@@ -333,42 +426,42 @@ def main():
                          "soft": torch.empty_like(m["W_host"]).pin_memory(),
                          "gW": torch.empty_like(m["W_host"]).pin_memory()})
         cb_h = cb.cpu().pin_memory(); gc_h = torch.empty(wl.S).pin_memory()
-        T_e = temps[-1]
 
-        def e2e_step():
+        def e2e_step(T_e):
             for h in host:
                 ctx.bcjr_step_host(h["W"], cb_h, h["g"], wl.Lb, wl.k, wl.n, T_e, soft=h["soft"], grad_W=h["gW"],
                                    grad_codebook=gc_h)
-        e2e_step()                                                  # warm-up (allocates staging buffers)
+        e2e_step(temps_timed[0])                                    # warm-up (allocates staging buffers)
         barrier()
-        reps = max(1, min(args.steps, 2))
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(reps):
-            e2e_step()
+        for T_e in temps_timed:
+            e2e_step(T_e)
         e1.record()
         barrier()
-        ems = e0.elapsed_time(e1) / reps
+        ems = e0.elapsed_time(e1) / len(temps_timed)
         t = torch.tensor([ems], dtype=torch.float64, device=dev)
         if world > 1:
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ems = float(t.item())
         wbytes = sum(h["W"].numel() * 4 for h in host)
-        e2e = {"value": edges_per_step * world / (ems * 1e-3), "unit": UNIT, "ms_per_step": ems,
+        e2e = {"value": edges_per_step * world / (ems * 1e-3), "unit": UNIT, "ms_per_step": ems, "steps": len(temps_timed),
                "h2d_bytes_per_step": 2 * wbytes + len(host) * wl.S * 4,
                "d2h_bytes_per_step": 2 * wbytes + len(host) * wl.S * 4}
+        del host
 
-    # ---- roofline of the dominant kernel (the backward-pass kernel): special-function pipe
-    state_steps = nblocks * wl.steps * wl.S
+    # ---- roofline of the dominant kernel: special-function pipe, peak measured in this run
+    state_steps = run.state_steps
     dom = "bwd" if bwd_ms >= fwd_ms else "fwd"
-    dom_ms = (bwd_ms if dom == "bwd" else fwd_ms) / (args.steps * len(mats))
-    ops = mufu_ops_per_state_step(wl.k, dom, wl.V) * state_steps / len(mats)
-    achieved = ops / (dom_ms * 1e-3) / 1e9
+    dom_ms = (bwd_ms if dom == "bwd" else fwd_ms) / (args.steps * len(mats))      # average launch
     sm_max = clocks.get("sm_max_mhz") or 1965.0
-    peak = NUM_SMS * MUFU_PER_CLK_PER_SM * sm_max * 1e6 / 1e9
-    # DRAM bytes per block of the dominant kernel, from the ncu captures summarised under profiles/
-    # (dram__bytes_read.sum + dram__bytes_write.sum of one launch / blocks of that launch, small
-    # case of the same kernel; traffic grows in proportion to the number of blocks)
+    peak = peaks["ex2_gops"]
+    nominal = NUM_SMS * MUFU_PER_CLK_PER_SM * sm_max * 1e6 / 1e9
+    fr = mufu_fractions(wl, state_steps, fwd_ms / args.steps, bwd_ms / args.steps, ms_per_step, peak)
+    ops = mufu_ops_per_state_step(wl.k, dom, wl.V, "algorithmic") * state_steps / len(mats)
+    achieved = ops / (dom_ms * 1e-3) / 1e9
+    # DRAM bytes per block of the dominant kernel: dram__bytes_read.sum + dram__bytes_write.sum of one launch of a
+    # small case under ncu (summaries under profiles/), divided by its blocks; traffic is proportional to blocks
     per_block = NCU_DRAM_BYTES_PER_BLOCK.get((wl.Lb, wl.k, dom)) if diag.last_path and wl.V == 1 else None
     traffic = per_block * nblocks / len(mats) if per_block else None
     hbm_peak = None
@@ -383,10 +476,33 @@ def main():
                "peak_source": "MEASURED_PEAKS.json (measured copy bandwidth)" if hbm_peak else "fallback 6.65 TB/s",
                "frac": gbs / (hbm_peak or 6650.0)}
     roofline = {"bound": "alu", "kernel": f"bcjr_{dom}", "achieved": achieved, "peak": peak, "unit": "Gop/s (MUFU)",
-                "frac": achieved / peak, "traffic": traffic,
-                "peak_source": f"{NUM_SMS} SMs x {MUFU_PER_CLK_PER_SM} MUFU/clk x {sm_max:.0f} MHz (derived)",
+                "frac": achieved / peak, "frac_with_rcp": fr[f"{dom}_frac_with_rcp"],
+                "count": "frac: algorithmic special-function operations per state-step (2 + 3/K per call: ex2 per state, "
+                         "lg2 per group, posterior ex2 per group); frac_with_rcp: operations the backward kernel issues "
+                         "(one rcp per group and sweep more)",
+                "traffic": traffic,
+                "traffic_source": "ncu dram bytes of a small-case launch, per block, scaled by this launch's blocks",
+                "peak_source": "measured in this run: ex2.approx chains on all SMs, CUDA events "
+                               f"({peaks['ex2_per_clk_sm']:.2f} per clock per SM at {peaks['sm_clock_mhz']:.0f} MHz)",
+                "peak_nominal": nominal,
+                "peak_nominal_source": f"{NUM_SMS} SMs x {MUFU_PER_CLK_PER_SM} per clock x {sm_max:.0f} MHz",
                 "avg_launch_ms": dom_ms, "hbm": hbm,
-                "whole_step_frac": mufu_ops_per_state_step(wl.k, "both", wl.V) * state_steps / (ms_per_step * 1e-3) / 1e9 / peak}
+                "fwd_frac": fr["fwd_frac"], "bwd_frac": fr["bwd_frac"], "whole_step_frac": fr["both_frac"],
+                "whole_step_frac_with_rcp": fr["both_frac_with_rcp"],
+                "binding_pipe": {"fwd": "special-function unit in both sweeps",
+                                 "bwd": "alpha sweep: special-function unit; beta sweep: FP32 pipe (16 lane-operations per "
+                                        "state-step) slightly ahead of the special-function unit"},
+                "pipe_peaks": peaks}
+
+    # ---- short legs over the other workloads, so that one line carries every configuration
+    legs = None
+    if not args.no_legs and world == 1 and not args.blocks and wl.name.startswith("llama32_1b_decoder"):
+        del run, mats
+        torch.cuda.empty_cache()
+        legs = {}
+        for name, cap in (("q_proj", 0), ("gate_k3", 32 * NUM_SMS), ("qtip_v2", 16 * NUM_SMS), ("mid", 0)):
+            legs[name] = workload_leg(ctx, name, cap, dev, flush, peak)
+        legs["qat_loop"] = qat_loop_leg(ctx, dev, flush)
 
     if rank == 0:
         base = None
@@ -395,13 +511,15 @@ def main():
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-               "config": {"workload": wl.name, "matrices": [m["name"] for m in mats], "blocks": nblocks, "n": wl.n,
-                          "Lb": wl.Lb, "k": wl.k, "V": wl.V, "T": [temps[args.warmup], temps[-1]],
+               "config": {"workload": wl.name, "matrices": [n for n, _ in wl.matrices], "blocks": nblocks, "n": wl.n,
+                          "Lb": wl.Lb, "k": wl.k, "V": wl.V, "T": [temps_timed[0], temps_timed[-1]],
+                          "T_schedule": "geometric over the timed steps, warm-up at the first value" if annealed else "constant",
                           "l2": "256 MB flush write between timed steps; per-step working set >> L2",
                           "path": "cluster" if diag.last_path else "generic"},
                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": base,
                "breakdown": {"fwd_ms_per_step": fwd_ms / args.steps, "bwd_ms_per_step": bwd_ms / args.steps,
-                             "viterbi": vit, "qat_update": upd, "max_posterior_defect": diag.max_posterior_defect}}
+                             "viterbi": vit, "qat_update": upd, "max_posterior_defect": diag.max_posterior_defect,
+                             "workloads": legs}}
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

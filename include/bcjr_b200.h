@@ -50,7 +50,16 @@ typedef struct {
     int32_t last_path;            /* 0 = generic kernels, 1 = cluster kernels used by the last call */
 } bcjr_diag;
 
-/* Limits: 1 <= k <= 4, k <= Lb <= 16, Lb - k <= 14, n >= 1, T > 0 and finite. */
+/* Limits: 1 <= k <= 4, k <= Lb <= 16, Lb - k <= 14, n >= 1, T > 0 and finite.
+ *
+ * Which kernel serves a shape (all give the same results within float32 tolerance; speed differs):
+ *   Lb = 16, k = 2 or 3:  tensor-memory kernels.  Forward and Viterbi for n <= 2048 / 4096; backward
+ *                         for n <= 1024.  Longer blocks step down: backward 1024 < n <= 2048 runs the
+ *                         four-CTA register kernel (about 1.7x slower per weight), and anything longer
+ *                         the generic one-CTA kernels (more than 10x slower per weight at Lb = 16).
+ *   Lb <= 14 (k = 1..4):  shared-memory kernels, one CTA per block, several blocks per SM.
+ *   everything else:      generic kernels.
+ * Block lengths of a few hundred weights (the paper uses 256) are the intended range. */
 
 /* Creates a context bound to CUDA device `device_ordinal`.  *out is owned by the caller
  * and released with bcjr_destroy.  Synchronous. */
@@ -67,6 +76,9 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *   "bwd_variant" large-trellis backward kernel: 0 = two-CTA clusters with codebook and gradient
  *                 accumulators in tensor memory (Lb = 16, k = 2 or 3), 1 = four-CTA clusters, registers
  *   "max_ctas"    cap on resident thread blocks (0 = fill the GPU)
+ *   "record_block_defect"  1: every scalar forward call also records, per block, max over steps of
+ *                 |sum_s gamma_t(s) - 1| (read back with bcjr_block_defects); 0 (default): only the
+ *                 maximum over the call is kept (bcjr_diag)
  *   "wait_limit_ms"  wall-time budget of one device-side wait (default 2000).  A wait that outlasts it
  *                 gives up: the kernel still runs to its end, the outputs of the call are
  *                 meaningless and bcjr_sync_status returns BCJR_ETIMEOUT; the context stays usable.
@@ -224,6 +236,13 @@ bcjr_status bcjr_step_host(bcjr_ctx *ctx, const float *W_host, const float *code
  * diagnostics.  Returns the device status (BCJR_OK when clean). */
 bcjr_status bcjr_sync_status(bcjr_ctx *ctx, void *cuda_stream, bcjr_diag *out);
 
+/* Per-block posterior defect of the last bcjr_soft_quantize made while "record_block_defect" was 1
+ * (Eq. 6: the marginals of a step sum to one; the deviation measures the float32 rounding a block's
+ * messages have accumulated).  Synchronises `cuda_stream`, then copies the first `count` values
+ * (count <= that call's num_blocks, else BCJR_ESTATE) to host_out (host, float32).  A block the
+ * kernel in use does not instrument reads NaN (the register-table cluster variant, vector emissions). */
+bcjr_status bcjr_block_defects(bcjr_ctx *ctx, float *host_out, int64_t count, void *cuda_stream);
+
 /* Scratch bytes currently held by the context. */
 int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx);
 
@@ -240,10 +259,12 @@ const char *bcjr_status_string(bcjr_status status);
  * Some callers may not call cudaMalloc or cudaFree at all: a latency-critical host loop that
  * cannot afford the device-wide synchronisation those calls imply, a process whose device
  * memory was handed to another allocator up front, a plug-in that may only launch work on the
- * buffers it is given.  This entry point computes exactly what bcjr_soft_quantize computes
- * (same kernel, same results) but needs no context and never allocates or frees: its scratch
- * is a fixed array of BCJR_STATIC_SCRATCH_BYTES that is part of the library image on every
- * GPU that loads the library, for the life of the process.
+ * buffers it is given.  This entry point computes what bcjr_soft_quantize computes (the same
+ * soft codeword and log Z within float32 tolerance; it always runs the one-CTA-per-block
+ * generic kernel, also for the shapes where bcjr_soft_quantize picks a tensor-memory kernel,
+ * so the two are not bit-identical there) but needs no context and never allocates or frees:
+ * its scratch is a fixed array of BCJR_STATIC_SCRATCH_BYTES that is part of the library image
+ * on every GPU that loads the library, for the life of the process.
  *
  *   W, codebook, soft, logZ, cuda_stream: as for bcjr_soft_quantize (device pointers of the
  *   CURRENT device; logZ may be NULL).  Nothing is saved for a backward pass.
@@ -251,7 +272,14 @@ const char *bcjr_status_string(bcjr_status status);
  * Limits: the messages must fit shared memory (Lb - k <= 14) and one block's history must fit
  * the scratch: n * 2^(Lb-k) * 4 + (n+2) * 4 bytes (rounded up to 256) <= BCJR_STATIC_SCRATCH_BYTES
  * - 256.  Larger problems are refused with BCJR_ETOOLARGE before anything is launched.  The
- * number of blocks is unlimited; fewer thread blocks run at once when the scratch is tight.
+ * number of blocks is unlimited; the scratch caps how many thread blocks run at once: at
+ * Lb = 16, k = 2, n = 256 one block's history is 16 MiB, so a single thread block works through
+ * all blocks in turn (one SM of the GPU); at Lb = 12 the same scratch feeds 127 thread blocks.
+ * Throughput-critical callers that can allocate should use bcjr_soft_quantize.
+ *
+ * Not reported: there is no context to query, so device-side diagnostics (a non-finite input
+ * that bcjr_sync_status would report as BCJR_ENUMERIC, the posterior defect) are not available
+ * from this call; a block with non-finite input yields non-finite output for that block only.
  *
  * Set-up: the first call on each device looks up the device address of the scratch array
  * (once, under a lock; that device must be current, as it is for the call itself).  Make that

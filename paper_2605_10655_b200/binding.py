@@ -14,15 +14,23 @@ LIB_PATH = _PKG / "libbcjr_b200.so"
 
 EXPORTS = ["bcjr_create", "bcjr_destroy", "bcjr_set_option", "bcjr_soft_quantize", "bcjr_backward",
            "viterbi_hard", "bcjr_soft_quantize_vec", "viterbi_hard_vec", "bcjr_ste_forward", "bcjr_temperature", "bcjr_gaussian_codebook", "bcjr_adam_update",
-           "bcjr_backward_adam", "bcjr_rht", "bcjr_group_scale", "bcjr_group_unscale", "bcjr_step_host", "bcjr_sync_status", "bcjr_workspace_bytes",
+           "bcjr_backward_adam", "bcjr_rht", "bcjr_group_scale", "bcjr_group_unscale", "bcjr_step_host", "bcjr_sync_status", "bcjr_block_defects", "bcjr_workspace_bytes",
            "bcjr_last_cuda_error", "bcjr_status_string", "bcjr_soft_quantize_static",
-           "bcjr_static_scratch_bytes"]
+           "bcjr_static_scratch_bytes", "bcjr_measure_pipe_peaks"]
 
 
 class BcjrError(RuntimeError):
     def __init__(self, code, where, detail=""):
         self.code = code
         super().__init__(f"{where}: {status_string(code)} ({code}){(' - ' + detail) if detail else ''}")
+
+
+class PipePeaks(ctypes.Structure):
+    """Mirror of bcjr_pipe_peaks (include/bcjr_microbench.h)."""
+    _fields_ = [("num_sms", ctypes.c_int32), ("pad", ctypes.c_int32)] + [(n, ctypes.c_double) for n in (
+        "sm_clock_mhz", "ex2_per_clk_sm", "lg2_per_clk_sm", "rcp_per_clk_sm", "fma_f32_per_clk_sm",
+        "fma_f32x2_per_clk_sm", "ex2_gops", "fma_f32x2_gops", "st_async_bytes_per_clk_sm", "cta_barrier_clk",
+        "mbarrier_round_clk")]
 
 
 class Diag(ctypes.Structure):
@@ -70,14 +78,25 @@ def load_library() -> ctypes.CDLL:
     lib.bcjr_step_host.restype = i
     lib.bcjr_step_host.argtypes = [vp, vp, vp, vp, i, i, i, i64, f, vp, vp, vp, vp]
     lib.bcjr_sync_status.restype = i; lib.bcjr_sync_status.argtypes = [vp, vp, ctypes.POINTER(Diag)]
+    lib.bcjr_block_defects.restype = i; lib.bcjr_block_defects.argtypes = [vp, vp, i64, vp]
     lib.bcjr_workspace_bytes.restype = i64; lib.bcjr_workspace_bytes.argtypes = [vp]
     lib.bcjr_last_cuda_error.restype = ctypes.c_char_p; lib.bcjr_last_cuda_error.argtypes = [vp]
     lib.bcjr_status_string.restype = ctypes.c_char_p; lib.bcjr_status_string.argtypes = [i]
     lib.bcjr_soft_quantize_static.restype = i
     lib.bcjr_soft_quantize_static.argtypes = [vp, vp, i, i, i, i64, f, vp, vp, vp]
     lib.bcjr_static_scratch_bytes.restype = i64; lib.bcjr_static_scratch_bytes.argtypes = []
+    lib.bcjr_measure_pipe_peaks.restype = i; lib.bcjr_measure_pipe_peaks.argtypes = [i, ctypes.POINTER(PipePeaks), vp]
     _lib = lib
     return lib
+
+
+def measure_pipe_peaks(device: int = 0, stream=None) -> dict:
+    """Measured special-function, FP32 and cluster-exchange rates of the device (see include/bcjr_microbench.h)."""
+    pk = PipePeaks()
+    rc = load_library().bcjr_measure_pipe_peaks(int(device), ctypes.byref(pk), _stream_ptr(stream))
+    if rc != 0:
+        raise BcjrError(rc, "bcjr_measure_pipe_peaks")
+    return {name: getattr(pk, name) for name, _ in PipePeaks._fields_ if name != "pad"}
 
 
 def temperature(T0: float, T_end: float, t: int, n_steps: int) -> float:
@@ -358,6 +377,15 @@ class Context:
         if check:
             self._check(rc, "bcjr_sync_status")
         return d
+
+    def block_defects(self, count: int, stream=None):
+        """Per-block posterior defect of the last forward call made with option record_block_defect = 1
+        (numpy float32 array of `count` values)."""
+        import numpy as np
+        out = np.empty(int(count), dtype=np.float32)
+        rc = self._lib.bcjr_block_defects(self._h, out.ctypes.data_as(ctypes.c_void_p), int(count), _stream_ptr(stream))
+        self._check(rc, "bcjr_block_defects")
+        return out
 
     def workspace_bytes(self) -> int:
         return int(self._lib.bcjr_workspace_bytes(self._h))

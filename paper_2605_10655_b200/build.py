@@ -11,8 +11,8 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libbcjr_b200.so"
-SOURCES = [CSRC / "bcjr_api.cu", CSRC / "bcjr_static.cu"]
-HEADERS = sorted(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "bcjr_b200.h"]
+SOURCES = [CSRC / "bcjr_api.cu", CSRC / "bcjr_static.cu", CSRC / "bcjr_microbench.cu"]
+HEADERS = sorted(CSRC.glob("*.cuh")) + sorted((PKG.parent / "include").glob("*.h"))
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "-cudart", "static"]

@@ -38,7 +38,7 @@ struct bcjr_ctx {
     int device = 0;
     int num_sms = 0;
     int max_smem_optin = 0;
-    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, cb_beta, grad_w, grad_c, staging[6];
+    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, cb_beta, grad_w, grad_c, blk_defect, staging[6];
     DeviceDiag *diag = nullptr;
     // saved by bcjr_soft_quantize for bcjr_backward
     bool have_fwd = false;
@@ -52,6 +52,8 @@ struct bcjr_ctx {
     int opt_max_ctas = 0;
     int opt_bwd_variant = 0;   // 0 = TMEM two-CTA backward kernel where it applies, 1 = register-accumulator cluster kernel
     int opt_fwd_variant = 0;   // 0 = TMEM single-CTA forward kernel where it applies, 1 = cluster forward kernel
+    int opt_record_defect = 0; // forward calls record the posterior defect of every block
+    int64_t defect_blocks = 0; // blocks covered by the last recording
     int launches = 0;
     int last_path = 0;
     std::string cuda_error;
@@ -111,7 +113,7 @@ bcjr_status plan_generic(bcjr_ctx *ctx, Kern kern, int Q, size_t msg_bytes, int6
     const size_t budget = (size_t)ctx->max_smem_optin - 1024;
     out->msg_global = header + msg_bytes > budget;
     out->smem = out->msg_global ? header : header + msg_bytes;
-    CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)out->smem));
+    CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
     int occ = 0;
     CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, out->threads, out->smem));
     if (occ < 1) occ = 1;
@@ -282,7 +284,7 @@ template <typename Kern>
 bcjr_status plan_cluster(bcjr_ctx *ctx, Kern kern, int CL, int threads, size_t smem, int64_t B,
                          cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attr, cudaStream_t st)
 {
-    CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CL;
     attr[0].val.clusterDim.y = 1;
@@ -443,7 +445,7 @@ bcjr_status launch_vit_solo(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
 {
     using C = VitSoloCfg<KB>;
     if (p.n > C::MAX_N) return BCJR_EUNSUPPORTED;
-    CU(cudaFuncSetAttribute(viterbi_solo_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    CU(cudaFuncSetAttribute(viterbi_solo_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
     int64_t grid = ctx->num_sms;
     if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
     if (grid > p.B) grid = p.B;
@@ -463,7 +465,7 @@ bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
     using C = SoloCfg<KB>;
     if (p.n > C::MAX_N) return BCJR_EUNSUPPORTED;
-    CU(cudaFuncSetAttribute(fwd_solo_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    CU(cudaFuncSetAttribute(fwd_solo_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
     int64_t grid = ctx->num_sms;
     if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
     if (grid > p.B) grid = p.B;
@@ -519,11 +521,6 @@ void launch_fwht_rows(const float *in, float *out, const float *s, int m, float 
 
 extern "C" {
 
-#ifdef BCJR_TIMING
-// development aid, not part of the ABI: per-warp cycle counters of the backward kernel's sweeps (CTA 0)
-void bcjr_debug_duo_timing(unsigned long long *out128) { cudaMemcpyFromSymbol(out128, g_duo_timing, 1024); }
-#endif
-
 bcjr_status bcjr_create(bcjr_ctx **out, int device_ordinal)
 {
     if (!out) return BCJR_EINVAL;
@@ -558,7 +555,7 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx)
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
     Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp, &ctx->path_ws,
-                     &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
+                     &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->blk_defect, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
                      &ctx->staging[5]};
     for (Buffer *b : all)
         if (b->ptr) cudaFree(b->ptr);
@@ -600,6 +597,11 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
         }
         return BCJR_OK;
     }
+    if (!strcmp(name, "record_block_defect")) {
+        if (value < 0 || value > 1) return BCJR_EINVAL;
+        ctx->opt_record_defect = (int)value;
+        return BCJR_OK;
+    }
     if (!strcmp(name, "max_ctas")) {
         if (value < 0 || value > (1 << 20)) return BCJR_EINVAL;
         ctx->opt_max_ctas = (int)value;
@@ -631,6 +633,13 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
     p.W = W; p.cb = codebook; p.soft = soft; p.soft_copy = (float *)ctx->soft_copy.ptr; p.logZ = logZ;
     p.diag = ctx->diag; p.B = num_blocks; p.Lb = Lb; p.n = n;
     p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)T));
+    ctx->defect_blocks = 0;
+    if (ctx->opt_record_defect) {
+        if ((rc = ensure(ctx, ctx->blk_defect, (size_t)num_blocks * 4))) return rc;
+        CU(cudaMemsetAsync(ctx->blk_defect.ptr, 0xff, (size_t)num_blocks * 4, st));   // NaN = not recorded by this kernel
+        p.blk_defect = (float *)ctx->blk_defect.ptr;
+        ctx->defect_blocks = num_blocks;
+    }
     bool use_cluster = false;
 #ifndef BCJR_NO_CLUSTER
     use_cluster = ctx->opt_path != 1 && cluster_supported(Lb, k);
@@ -1045,11 +1054,23 @@ bcjr_status bcjr_sync_status(bcjr_ctx *ctx, void *cuda_stream, bcjr_diag *out)
     return (bcjr_status)h.status;
 }
 
+bcjr_status bcjr_block_defects(bcjr_ctx *ctx, float *host_out, int64_t count, void *cuda_stream)
+{
+    if (!ctx || count < 0 || (count > 0 && !host_out)) return BCJR_EINVAL;
+    if (count > ctx->defect_blocks) return BCJR_ESTATE;
+    if (count == 0) return BCJR_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return BCJR_ECUDA;
+    CU(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    CU(cudaMemcpy(host_out, ctx->blk_defect.ptr, (size_t)count * 4, cudaMemcpyDeviceToHost));
+    return BCJR_OK;
+}
+
 int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx)
 {
     if (!ctx) return 0;
     const Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp,
-                           &ctx->path_ws, &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
+                           &ctx->path_ws, &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->blk_defect, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
                            &ctx->staging[4], &ctx->staging[5]};
     int64_t tot = 0;
     for (const Buffer *b : all) tot += (int64_t)b->bytes;

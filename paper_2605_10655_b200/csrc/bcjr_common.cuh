@@ -102,6 +102,7 @@ struct FwdParams {
     float *hist;             // [grid][n*Q] gauge-fixed L_t, t = 1..n
     int *stepO;              // [grid][n+2] cumulative integer offsets O_t
     float *msg;              // [grid][2*Q] message ping-pong in global memory, or null (shared)
+    float *blk_defect;       // [B] max_t |sum_s gamma_t(s) - 1| of every block, or null (not recorded)
     DeviceDiag *diag;
     int64_t B;
     int Lb, n;

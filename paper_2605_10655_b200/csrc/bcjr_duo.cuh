@@ -37,14 +37,6 @@
 namespace bcjr {
 
 
-#ifdef BCJR_TIMING
-__device__ unsigned long long g_duo_timing[128]; // CTAs 0 and 1, per warp: alpha step, alpha input wait, beta step, beta input wait (cycles, summed)
-#define TICK(var) const long long var = clock64()
-#define TACC(slot, a, b) do { if (blockIdx.x < 2 && lane == 0) tacc[slot] += (unsigned long long)((b) - (a)); } while (0)
-#else
-#define TICK(var)
-#define TACC(slot, a, b)
-#endif
 
 template <int KB_>
 struct DuoCfg {
@@ -177,9 +169,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         for (int g = 0; g < NU; ++g) tmem_st16(tm_acc + 16u * g, z);
         tmem_wait_st();
     }
-#ifdef BCJR_TIMING
-    unsigned long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#endif
     // test hook for the waits' abort path: one warp of CTA 0 withholds an arrival of its first block
     const bool drop_hook = blockIdx.x == 0 && warp == 1 && p.diag->drop_history_load != 0;
     float defect = 0.f;
@@ -204,7 +193,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         // ================= alpha sweep carrying (L, At)
         for (int t = 1; t <= n; ++t) {
             const int ob = ib ^ 1;
-            TICK(ta0);
             // what does not depend on the step's inputs is requested before the wait for them: the first
             // codebook unit from tensor memory and the step's scalars (their latency hides under the wait)
             float2 cb[2][8];
@@ -213,7 +201,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
             if (t > 1) {
                 wait_inputs(ib);
-                TICK(ta1); TACC(1, ta0, ta1);
                 cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
                 off = rintf(cmax);
             }
@@ -291,7 +278,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 mbar_arrive_local(mbar_full + ob_mbar);
                 mbar_arrive_remote(full_of[rank ^ 1u] + ob_mbar);
             }
-            TICK(ta2); TACC(0, ta0, ta2);
             ib = ob;
         }
         // ================= log2 Z
@@ -362,7 +348,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         };
         for (int t = n; t >= 1; --t) {
             const int ob = ib ^ 1;
-            TICK(tk0);
             // requested before the wait for the step's inputs, like in the alpha sweep
             float2 cb[2][8];
             tmem_ld16(tm_cb, cb[0]);
@@ -381,7 +366,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             issue_chunk(0);
             if (t < n) {
                 wait_inputs(ib);
-                TICK(tk1); TACC(3, tk0, tk1);
                 cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF);
                 P += (int)offM;
                 offM = rintf(cmax);
@@ -472,7 +456,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
             }
             __syncwarp();
-            TICK(tb1); TACC(2, tk0, tb1);
             if (lane == 0 && !(drop_hook && t == n && blk == cid)) {   // this warp has read all its inputs and written its outputs
                 mbar_arrive_local(mbar_full + ob_mbar);
                 mbar_arrive_remote(full_of[rank ^ 1u] + ob_mbar);
@@ -510,10 +493,6 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             }
         }
     }
-#ifdef BCJR_TIMING
-    if (blockIdx.x < 2 && lane == 0)
-        for (int e = 0; e < 4; ++e) g_duo_timing[(blockIdx.x * 16 + warp) * 4 + e] = tacc[e];
-#endif
     if (tid == CT - 32 && rank == 0) diag_max(&p.diag->max_defect, defect);
     asm volatile("cp.async.wait_all;" ::: "memory");           // no copy may be in flight at exit (a warp may have left the loop early)
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

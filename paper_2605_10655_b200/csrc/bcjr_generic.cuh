@@ -41,7 +41,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
         for (int q = tid; q < Q; q += nthr) { Lin[q] = 0.f; hist[q] = 0.f; }   // L_1 = 0: free first state
         if (tid == 0) stepO[1] = 0;
         int O = 0;
-        float off = 0.f, cmax = 0.f;
+        float off = 0.f, cmax = 0.f, bdef = 0.f;
         __syncthreads();
         // ---- alpha: from L_t to L_{t+1}, t = 1..n (the last one only feeds log Z)
         for (int t = 1; t <= n; ++t) {
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
                     const float sw = a / b;
                     p.soft[blk * n + t - 1] = sw;
                     if (p.soft_copy) p.soft_copy[blk * n + t - 1] = sw;
-                    defect = fmaxf(defect, fabsf(b - 1.f));
+                    bdef = fmaxf(bdef, fabsf(b - 1.f));
                 }
             }
             float *sw = Min; Min = Mout; Mout = sw;
@@ -150,6 +150,8 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
         if (lane == 0) lzpart[warp] = ssum;
         __syncthreads();
         if (tid == 0) {
+            defect = fmaxf(defect, bdef);
+            if (p.blk_defect) p.blk_defect[blk] = bdef;
             float t2 = 0.f;
             for (int i = 0; i < nwarp; ++i) t2 += lzpart[i];
             const float lz_beta = cmax + lg2f(t2);

@@ -18,7 +18,7 @@
 // staging slots, RD - 1 butterflies ahead (cp.async.wait_group: no mbarrier, no copy warp, no
 // branch in the butterfly loop).  No thread of this kernel spins on anything.
 #pragma once
-#include "bcjr_cluster.cuh"
+#include "bcjr_ptx.cuh"
 
 
 namespace bcjr {
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), false);
             tmem_wait_st();
             int O = 0;
-            float off = 0.f, cmax = 0.f;
+            float off = 0.f, cmax = 0.f, bdef = 0.f;
             compute_barrier(CT);
             // ================= alpha sweep
             for (int t = 1; t <= n; ++t) {
@@ -305,7 +305,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                             const float sw = a / c;
                             p.soft[blk * n + t] = sw;
                             if (p.soft_copy) p.soft_copy[blk * n + t] = sw;
-                            defect = fmaxf(defect, fabsf(c - 1.f));
+                            bdef = fmaxf(bdef, fabsf(c - 1.f));
                         }
                     }
                 }
@@ -386,7 +386,9 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                         const float sw = a / c;
                         p.soft[blk * n] = sw;
                         if (p.soft_copy) p.soft_copy[blk * n] = sw;
-                        defect = fmaxf(defect, fabsf(c - 1.f));
+                        bdef = fmaxf(bdef, fabsf(c - 1.f));
+                        defect = fmaxf(defect, bdef);
+                        if (p.blk_defect) p.blk_defect[blk] = bdef;
                     }
                 }
                 // consistency: P_0 + LSE_q M_0(q) against log2 Z

@@ -72,11 +72,13 @@ bcjr_status launch_static(int dev, unsigned char *scratch, FwdParams p, cudaStre
     if (smem + 1024 > (size_t)g_smem_optin[dev]) return BCJR_EUNSUPPORTED;   // messages must fit shared memory
     // per CTA: n*Q floats of history, n+2 ints of step offsets (rounded up to 256 bytes)
     const size_t hist_bytes = (size_t)p.n * Q * 4;
-    const size_t step_bytes = ((size_t)(p.n + 2) * 4 + 255) / 256 * 256;
+    const size_t step_bytes = (((size_t)p.n + 2) * 4 + 255) / 256 * 256;
     const size_t per_cta = hist_bytes + step_bytes;
     const size_t room = kStaticScratchBytes - kHeaderBytes;
     if (per_cta > room) return BCJR_ETOOLARGE;                               // one block alone does not fit
-    if (cudaFuncSetAttribute(fwd_generic_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    // always the device's opt-in maximum, never this call's own size: the attribute belongs to the kernel, not to a
+    // call, and a smaller value set here could undercut a launch another host thread is about to make
+    if (cudaFuncSetAttribute(fwd_generic_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, g_smem_optin[dev]) != cudaSuccess) {
         cudaGetLastError();
         return BCJR_ECUDA;
     }
@@ -91,7 +93,7 @@ bcjr_status launch_static(int dev, unsigned char *scratch, FwdParams p, cudaStre
     if ((size_t)grid > room / per_cta) grid = (int64_t)(room / per_cta);
     if (grid < 1) return BCJR_ETOOLARGE;
     // layout: [header][grid x (n+2) ints, padded to 256 bytes][grid x n*Q floats]
-    const size_t step_total = ((size_t)grid * (p.n + 2) * 4 + 255) / 256 * 256;
+    const size_t step_total = ((size_t)grid * ((size_t)p.n + 2) * 4 + 255) / 256 * 256;
     p.diag = reinterpret_cast<DeviceDiag *>(scratch);
     p.stepO = reinterpret_cast<int *>(scratch + kHeaderBytes);
     p.hist = reinterpret_cast<float *>(scratch + kHeaderBytes + step_total);

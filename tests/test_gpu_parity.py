@@ -141,27 +141,55 @@ def test_empty_input_and_argument_errors(ctx):
 @pytest.mark.parametrize("T", [1.0, 0.1, 0.01])
 def test_mid_trellis_temperature_sweep(ctx, T):
     wl = synth.mid()
-    idx = synth.sample_blocks(wl.num_blocks(), 24)
+    idx = synth.sample_blocks(wl.num_blocks(), 512)
     W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
     _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"mid T={T}", viterbi=(T == 1.0))
 
 
+def _cold_limit_statistics(soft_gpu, soft_ref, W, c, Lb, k, T, what):
+    """Section 3.3, identity 1 (as T -> 0 the soft codeword tends to the Viterbi hard code), stated for a
+    finite T.  A block has converged when no other path comes close to the best one: its margin
+    (squared error of the best path that leaves the Viterbi path somewhere, minus the Viterbi path's)
+    exceeds 20 T / kappa with kappa = 1/2, so that every other path carries less than e^-20 of the
+    Viterbi path's weight.  On those blocks the soft codeword, decoded to the nearest table entry, must
+    BE the hard code at every position, for the oracle and for the GPU alike.  Over all blocks the
+    agreement is reported as the fraction of positions within 1e-3 of the hard code."""
+    import minsum
+    B = W.shape[0]
+    margin = np.empty(B); hard = np.empty(W.shape)
+    for b in range(B):
+        st, _, margin[b] = minsum.best_and_margin(W[b], c, Lb, k)
+        hard[b] = c.astype(np.float64)[st]
+    conv = margin > 20.0 * T / 0.5
+    dec_ref = np.stack([minsum.decode_nearest(soft_ref[b], c) for b in range(B)])
+    dec_gpu = np.stack([minsum.decode_nearest(soft_gpu[b], c) for b in range(B)])
+    ref_blocks_differ = [int(b) for b in range(B) if not np.array_equal(dec_ref[b], hard[b])]
+    frac_ref = float((np.abs(soft_ref - hard) <= 1e-3).mean())
+    frac_gpu = float((np.abs(soft_gpu - hard) <= 1e-3).mean())
+    worst_conv = float(np.abs(soft_gpu[conv] - hard[conv]).max()) if conv.any() else 0.0
+    print(f"\n{what}: T={T}: {int(conv.sum())}/{B} blocks past the margin 20T/kappa; positions within 1e-3 of the hard "
+          f"code: oracle {frac_ref:.4f}, GPU {frac_gpu:.4f}; max |soft - hard| on converged blocks {worst_conv:.2e}; "
+          f"blocks whose decoded oracle soft codeword differs from the hard code: {len(ref_blocks_differ)} "
+          f"(none of them converged: {not any(conv[b] for b in ref_blocks_differ)})")
+    assert not any(conv[b] for b in ref_blocks_differ), what + ": the oracle itself disagrees on a converged block"
+    for b in np.nonzero(conv)[0]:
+        np.testing.assert_array_equal(dec_gpu[b], hard[b], err_msg=f"{what}: block {b} (margin {margin[b]:.3g})")
+    assert worst_conv <= 1e-3
+    assert abs(frac_gpu - frac_ref) <= 2e-3
+    return conv
+
+
 def test_mid_trellis_cold_limit_matches_viterbi(ctx):
-    # Section 3.3, identity 1: as T -> 0 the soft codeword tends to the hard Viterbi output.
-    # Compared where the float64 oracle itself has converged (its argmax equals its Viterbi).
     wl = synth.mid()
-    idx = synth.sample_blocks(wl.num_blocks(), 16, seed=5)
+    idx = synth.sample_blocks(wl.num_blocks(), 256, seed=5)
     W, c = wl.weights()[idx], wl.codebook()
     T = 1e-4
     got = parity.gpu_forward_backward(ctx, W, c, None, wl.Lb, wl.k, T)
     ref = oracle.soft_quantize(W, c, wl.Lb, wl.k, T)
-    vit = oracle.viterbi(W, c, wl.Lb, wl.k)
     assert parity.rel_inf(got["soft"], ref["soft"]) <= parity.SOFT_TOL
-    c64 = c.astype(np.float64)
-    # nearest table entry to the soft value = the state the posterior has collapsed onto
-    conv = np.abs(ref["soft"] - vit["hard"]) < 1e-3
-    assert conv.mean() > 0.9
-    assert np.abs(got["soft"][conv] - vit["hard"][conv]).max() < 2e-3
+    conv = _cold_limit_statistics(got["soft"], ref["soft"], W, c, wl.Lb, wl.k, T, "mid trellis")
+    assert conv.mean() > 0.5                       # at T = 1e-4 most blocks have a clear winner
+    vit = oracle.viterbi(W, c, wl.Lb, wl.k)
     gvit = parity.gpu_viterbi(ctx, W, c, wl.Lb, wl.k)
     parity.assert_viterbi(gvit, vit, "mid viterbi")
 
@@ -186,18 +214,38 @@ def test_q_proj_shape_sampled_blocks(ctx, variant):
             ctx.set_option(k_, 0)
 
 
-@pytest.mark.parametrize("T", [0.3, 0.03, 0.01])
-def test_decoder_layer_temperature_range_sampled_blocks(ctx, T):
-    # the annealing range of the decoder-layer workload (0.3 -> 0.01) on its kernels: blocks of the down_proj-shaped
-    # matrix (rows of 8192 weights, 32 blocks per row), sampled
+@pytest.fixture(scope="module")
+def decoder_sample():
+    # four blocks (first, last, two seeded) from each of the seven matrices of the decoder-layer workload
     wl = synth.decoder_layer()
-    i = len(wl.matrices) - 1
-    Wm = wl.weights(i)
-    idx = synth.sample_blocks(Wm.shape[0], 4)
-    W, c = Wm[idx], wl.codebook()
+    Ws = []
+    for i in range(len(wl.matrices)):
+        Wm = wl.weights(i)
+        Ws.append(Wm[synth.sample_blocks(Wm.shape[0], 4, seed=40 + i)])
+    W = np.ascontiguousarray(np.concatenate(Ws))
     g = np.random.default_rng(4242).standard_normal(W.shape).astype(np.float32)
+    return wl, W, wl.codebook(), g
+
+
+@pytest.mark.parametrize("T", [0.3, 0.03, 0.01])
+def test_decoder_layer_temperature_range_sampled_blocks(ctx, decoder_sample, T):
+    # the annealing range of the decoder-layer workload (0.3 -> 0.01) on its kernels
+    wl, W, c, g = decoder_sample
+    assert W.shape[0] == 28
     got = _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"decoder layer sample, T={T}", viterbi=False)
     assert got["diag"].last_path == 1
+
+
+@pytest.mark.parametrize("k", [2, 3])
+def test_large_trellis_viterbi_full_length_many_blocks(ctx, k):
+    # 256 blocks of 256 weights: near-ties between paths are what a wrong metric precision or
+    # operation order would flip, and they only show in a sample of this size
+    wl = synth.q_proj() if k == 2 else synth.gate_k3()
+    idx = synth.sample_blocks(wl.num_blocks(), 256, seed=60 + k)
+    W, c = wl.weights()[idx], wl.codebook()
+    ref = oracle.viterbi(W, c, wl.Lb, k)
+    got = parity.gpu_viterbi(ctx, W, c, wl.Lb, k)
+    parity.assert_viterbi(got, ref, f"viterbi 256 blocks k={k}")
 
 
 @pytest.mark.parametrize("n,B", [(1, 3), (2, 2), (3, 1), (7, 5), (64, 2), (255, 1)])
@@ -341,7 +389,7 @@ def test_q_proj_full_size_sampled_outputs_and_invariants(ctx):
     assert got["diag"].last_path == 1 and got["diag"].device_status == 0
     assert got["diag"].max_posterior_defect < 1e-3
     assert np.all(np.isfinite(got["soft"])) and np.all(np.isfinite(got["grad_W"]))
-    idx = synth.sample_blocks(wl.num_blocks(), 8, seed=123)
+    idx = synth.sample_blocks(wl.num_blocks(), 64, seed=123)
     ref_f = oracle.soft_quantize(W[idx], c, wl.Lb, wl.k, wl.T)
     ref_b = oracle.backward(W[idx], c, g[idx], wl.Lb, wl.k, wl.T)
     assert parity.rel_inf(got["soft"][idx], ref_f["soft"]) <= parity.SOFT_TOL
@@ -354,21 +402,68 @@ def test_q_proj_full_size_sampled_outputs_and_invariants(ctx):
     assert got["soft"].min() >= c.min() - 1e-4 and got["soft"].max() <= c.max() + 1e-4
 
 
-@pytest.mark.parametrize("T,variant", [(0.01, "tmem"), (0.001, "tmem"), (0.01, "cluster_registers")])
-def test_three_bit_student_t_low_temperature(ctx, T, variant):
+def test_three_bit_student_t_register_variant(ctx):
     wl = synth.gate_k3()
     idx = synth.sample_blocks(wl.num_blocks(), 4)
     W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
-    v = int(variant != "tmem")
     try:
-        ctx.set_option("fwd_variant", v); ctx.set_option("bwd_variant", v)
-        got = _check_all(ctx, W, c, g, wl.Lb, wl.k, T, f"k=3 student-t T={T} [{variant}]", viterbi=(T == 0.01 and v == 0))
+        ctx.set_option("fwd_variant", 1); ctx.set_option("bwd_variant", 1)
+        got = _check_all(ctx, W, c, g, wl.Lb, wl.k, 0.01, "k=3 student-t T=0.01 [cluster_registers]", viterbi=False)
     finally:
         ctx.set_option("fwd_variant", 0); ctx.set_option("bwd_variant", 0)
     assert got["diag"].last_path == 1
-    assert np.all(np.isfinite(got["soft"])) and np.all(np.isfinite(got["grad_W"]))
+
+
+def defect_bound(W, c, T, n):
+    """Bound on |sum_s gamma_t(s) - 1| from float32 rounding.  Every message of step t is rounded at the
+    magnitude of that step's log2-potentials, E_t = log2(e) min_s (w_t - c[s])^2 / (2T) (the gauge removes
+    the rest); an error common to all states shifts the computed sum of the marginals and nothing else
+    (soft codeword and gradients are normalised by that same sum).  Half an ulp per message, one message per
+    step on each side, accumulated as a random walk with a factor 4 for the tail:
+        4 ln2 2^-24 sqrt(sum_t (1 + E_t)^2)   per block, floored at 1e-4."""
+    d2 = np.min((W[:, :, None].astype(np.float64) - np.sort(c.astype(np.float64))[None, None, [0, -1]]) ** 2, axis=2)
+    inside = (W >= c.min()) & (W <= c.max())
+    d2 = np.where(inside, 0.0, d2)              # inside the table's range some entry is close: E_t ~ 0 on this scale
+    E = 1.4426950408889634 * d2 / (2.0 * T)
+    return np.maximum(1e-4, 4.0 * 0.6931 * 2.0 ** -24 * np.sqrt(((1.0 + E) ** 2).sum(axis=1)))
+
+
+@pytest.mark.parametrize("T", [0.01, 0.001])
+def test_three_bit_student_t_low_temperature(ctx, T):
+    """592 blocks of the heavy-tailed 3-bit workload in one call, the posterior defect of every block recorded.
+    Compared with the oracle: the sixteen blocks with the largest defect and sixteen seeded ones, taken from
+    that call (soft, log Z, grad_W depend on their block alone); grad_codebook from a second call on those
+    blocks only; Viterbi on them; the cold-limit statistics."""
+    wl = synth.gate_k3()
+    NB = 592
+    W, c, g = wl.weights()[:NB], wl.codebook(), wl.upstream()[:NB]
+    ctx.set_option("record_block_defect", 1)
+    try:
+        got = parity.gpu_forward_backward(ctx, W, c, g, wl.Lb, wl.k, T)
+        defects = ctx.block_defects(NB)
+    finally:
+        ctx.set_option("record_block_defect", 0)
+    assert got["diag"].last_path == 1 and got["diag"].device_status == 0
+    assert np.all(np.isfinite(defects)) and np.all(np.isfinite(got["soft"])) and np.all(np.isfinite(got["grad_W"]))
+    bound = defect_bound(W, c, T, wl.n)
+    worst = np.argsort(defects)[::-1][:16]
+    print(f"\nk=3 student-t T={T}: posterior defect max {defects.max():.2e} (block {int(defects.argmax())}, "
+          f"max |w| there {np.abs(W[defects.argmax()]).max():.1f}), median {np.median(defects):.2e}; "
+          f"largest defect / bound {float((defects / bound).max()):.2f}")
+    assert np.all(defects <= bound), f"defect above the rounding bound: {(defects / bound).max():.2f}x"
+    idx = np.array(sorted(set(worst.tolist()) | set(synth.sample_blocks(NB, 16, seed=7).tolist())), dtype=np.int64)
+    ref_f = oracle.soft_quantize(W[idx], c, wl.Lb, wl.k, T)
+    ref_b = oracle.backward(W[idx], c, g[idx], wl.Lb, wl.k, T)
+    for j, b in enumerate(idx):                        # block by block: a large block must not hide a small one
+        assert parity.rel_inf(got["soft"][b], ref_f["soft"][j]) <= parity.SOFT_TOL, f"soft, block {b} (defect {defects[b]:.2e})"
+        assert parity.rel_inf(got["grad_W"][b], ref_b["grad_W"][j]) <= parity.GRAD_TOL, f"grad_W, block {b}"
+    np.testing.assert_allclose(got["logZ"][idx], ref_f["logZ"], rtol=1e-5, atol=1e-3)
+    sub = parity.gpu_forward_backward(ctx, W[idx], c, g[idx], wl.Lb, wl.k, T)
+    parity.assert_forward_backward(sub, ref_f, ref_b, f"k=3 student-t T={T}, sampled blocks")
     tot = got["grad_W"].astype(np.float64).sum() + got["grad_codebook"].astype(np.float64).sum()
     assert abs(tot - g.astype(np.float64).sum()) < 1e-2 * np.abs(g).sum()
+    parity.assert_viterbi(parity.gpu_viterbi(ctx, W[idx], c, wl.Lb, wl.k), oracle.viterbi(W[idx], c, wl.Lb, wl.k), "k=3")
+    _cold_limit_statistics(got["soft"][idx], ref_f["soft"], W[idx], c, wl.Lb, wl.k, T, "3-bit student-t")
 
 
 @pytest.mark.parametrize("n,B", [(1, 2), (5, 3), (33, 1)])

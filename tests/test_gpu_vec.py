@@ -94,11 +94,15 @@ def test_full_block_length_sampled_blocks(ctx):
     Lb, k, V, nt, T = 16, 2, 2, 128, 0.1
     W, c, g = _case(Lb, V, nt, 150, seed=8300)
     got = _run(ctx, W, c, g, Lb, k, V, T, viterbi=True)
-    pick = [0, 71, 149]
+    pick = [0, 17, 38, 71, 99, 120, 133, 149]
     ref_f = oracle.soft_quantize_vec(W[pick], c, Lb, k * V, V, T)
     assert parity.rel_inf(got["soft"][pick], ref_f["soft"]) <= parity.SOFT_TOL
     ref_b = oracle.backward_vec(W[pick], c, g[pick], Lb, k * V, V, T)
     assert parity.rel_inf(got["grad_W"][pick], ref_b["grad_W"]) <= parity.GRAD_TOL
+    # grad_codebook sums over the blocks of a call: compare it on a call of its own over the picked blocks
+    sub = _run(ctx, W[pick], c, g[pick], Lb, k, V, T)
+    assert parity.rel_inf(sub["grad_codebook"], ref_b["grad_codebook"]) <= parity.GRAD_TOL
+    assert parity.rel_inf(sub["grad_W"], ref_b["grad_W"]) <= parity.GRAD_TOL
     ref_v = oracle.viterbi_vec(W[pick], c, Lb, k * V, V)
     np.testing.assert_array_equal(got["states"][pick], ref_v["states"])
     np.testing.assert_array_equal(got["hard"][pick].view(np.uint32), ref_v["hard"].view(np.uint32))

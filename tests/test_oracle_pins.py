@@ -275,3 +275,26 @@ def test_invalid_arguments_are_rejected():
         oracle.soft_quantize(W, c, 4, 2, 0.0)
     with pytest.raises(RuntimeError):
         oracle.soft_quantize(W, c[:4], 2, 3, 1.0)      # k > Lb
+
+
+# ---------------------------------------------------------------- min-sum helper of the cold-limit tests
+@pytest.mark.parametrize("Lb,k,n", [(4, 2, 6), (3, 1, 7), (5, 3, 4), (4, 2, 1)])
+def test_minsum_margin_against_enumeration_and_oracle_viterbi(Lb, k, n):
+    import minsum
+    rng = np.random.default_rng(900 + Lb + n)
+    c = rng.standard_normal(1 << Lb).astype(np.float32)
+    for trial in range(4):
+        w = rng.standard_normal(n).astype(np.float32)
+        states, cost, gap = bf.best_path(w, c, Lb, k)
+        s2, cost2, margin = minsum.best_and_margin(w, c, Lb, k)
+        np.testing.assert_array_equal(s2, states)
+        assert abs(cost2 - cost) < 1e-12 and abs(margin - gap) < 1e-12
+        ref = oracle.viterbi(w[None], c, Lb, k)
+        np.testing.assert_array_equal(ref["states"][0], states)
+        assert abs(ref["cost"][0] - cost) < 1e-12
+
+
+def test_nearest_entry_decoding():
+    import minsum
+    c = np.array([0.5, -1.0, 2.0, 0.75], dtype=np.float32)
+    np.testing.assert_array_equal(minsum.decode_nearest([0.6, 0.7, -3.0, 9.0, 1.3, 1.4], c), [0.5, 0.75, -1.0, 2.0, 0.75, 2.0])

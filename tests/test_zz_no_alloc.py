@@ -16,6 +16,7 @@ import ctypes
 import numpy as np
 import pytest
 
+import oracle
 import parity
 from paper_2605_10655_b200 import synth
 
@@ -50,6 +51,10 @@ def test_static_entry_point_matches_regular_one_twice_in_a_row():
             torch.cuda.synchronize()
             assert parity.rel_inf(soft.cpu().numpy(), ref_soft.cpu().numpy()) <= parity.SOFT_TOL
             np.testing.assert_allclose(logZ.cpu().numpy(), ref_logZ.cpu().numpy(), rtol=1e-5, atol=1e-3)
+            # and against the float64 oracle, which shares nothing with either CUDA entry point
+            ref = oracle.soft_quantize(Wd.cpu().numpy(), cd.cpu().numpy(), wl.Lb, wl.k, wl.T)
+            assert parity.rel_inf(soft.cpu().numpy(), ref["soft"]) <= parity.SOFT_TOL
+            np.testing.assert_allclose(logZ.cpu().numpy(), ref["logZ"], rtol=1e-5, atol=1e-3)
         # the same inputs again, straight after a different problem has used the scratch
         wl = synth.tiny()
         Wd, cd = _device_inputs(wl, 64)
@@ -60,6 +65,40 @@ def test_static_entry_point_matches_regular_one_twice_in_a_row():
         ref, _ = ctx.bcjr_soft_quantize(Wd, cd, wl.Lb, wl.k, wl.n, wl.T)
         ctx.sync_status()
         assert parity.rel_inf(a.cpu().numpy(), ref.cpu().numpy()) <= parity.SOFT_TOL
+    finally:
+        ctx.close()
+
+
+def test_static_entry_point_largest_trellis_one_resident_block_and_no_allocation():
+    # Lb = 16, k = 2, n = 256: one block's history is 16 MiB, so the 32 MiB scratch holds exactly one
+    # thread block, which must work through all three weight blocks reusing the same history slot.
+    # The regular call runs a different (tensor-memory) kernel here, so this also compares two
+    # implementations; the oracle decides.  With caller-supplied outputs the second call must leave
+    # the device's free memory untouched.
+    import torch
+    from paper_2605_10655_b200 import Context, binding
+    wl = synth.q_proj()
+    nblk = 3
+    Wd, cd = _device_inputs(wl, nblk)
+    soft = torch.full_like(Wd, float("nan"))
+    logZ = torch.full((nblk,), float("nan"), device=Wd.device)
+    binding.bcjr_soft_quantize_static(Wd, cd, wl.Lb, wl.k, wl.n, wl.T, soft=soft, logZ=logZ)
+    torch.cuda.synchronize()
+    first = soft.clone()
+    free0, _ = torch.cuda.mem_get_info()
+    binding.bcjr_soft_quantize_static(Wd, cd, wl.Lb, wl.k, wl.n, wl.T, soft=soft, logZ=logZ)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, "the static entry point changed the device's free memory"
+    assert torch.equal(first, soft)
+    ref = oracle.soft_quantize(Wd.cpu().numpy(), cd.cpu().numpy(), wl.Lb, wl.k, wl.T)
+    assert parity.rel_inf(soft.cpu().numpy(), ref["soft"]) <= parity.SOFT_TOL
+    np.testing.assert_allclose(logZ.cpu().numpy(), ref["logZ"], rtol=1e-5, atol=1e-3)
+    ctx = Context(0)
+    try:
+        reg, _ = ctx.bcjr_soft_quantize(Wd, cd, wl.Lb, wl.k, wl.n, wl.T)
+        assert ctx.sync_status().last_path == 1
+        assert parity.rel_inf(soft.cpu().numpy(), reg.cpu().numpy()) <= parity.SOFT_TOL
     finally:
         ctx.close()
 
