@@ -74,7 +74,14 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *   "fwd_variant" large-trellis forward kernel: 0 = one CTA per block with the codebook in tensor
  *                 memory (Lb = 16, k = 2 or 3), 1 = two-CTA cluster kernel with the codebook in registers
  *   "bwd_variant" large-trellis backward kernel: 0 = two-CTA clusters with codebook and gradient
- *                 accumulators in tensor memory (Lb = 16, k = 2 or 3), 1 = four-CTA clusters, registers
+ *                 accumulators in tensor memory (Lb = 16, k = 2 or 3; at k = 2 with the butterflies ordered so
+ *                 that a step starts before the whole cluster has finished the previous one), 1 = four-CTA
+ *                 clusters, registers, 2 = the two-CTA tensor-memory kernel with one barrier per step at k = 2 too
+ *   "history_every_m"  1 (default): the large-trellis forward kernel stores the forward messages of every step
+ *                 for its beta sweep; m = 2..16: it keeps them for every m-th step only and recomputes the
+ *                 m - 1 steps in between inside the beta sweep (1/m of the history traffic to HBM for
+ *                 (m-1)/m of an alpha sweep more arithmetic; same results within float32 rounding; Lb = 16, k = 2 or 3,
+ *                 n <= 512, otherwise the option has no effect)
  *   "max_ctas"    cap on resident thread blocks (0 = fill the GPU)
  *   "record_block_defect"  1: every scalar forward call also records, per block, max over steps of
  *                 |sum_s gamma_t(s) - 1| (read back with bcjr_block_defects); 0 (default): only the
@@ -93,7 +100,11 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value);
  * marginals from the temperature-T forward-backward recursions of Eq. 5-6 carried in the
  * log domain.
  *   W         device in   [num_blocks * n] float32
- *   codebook  device in   [2^Lb] float32
+ *   codebook  device in   [2^Lb] float32, or NULL for the computed Gaussian emission of Section 3.1,
+ *                         codebook[s] = Phi^-1((s + 1/2) / 2^Lb) (what bcjr_gaussian_codebook writes out): at
+ *                         Lb = 16, k = 2 or 3 the kernels then evaluate the entries themselves while filling
+ *                         their tensor-memory slices and no table is read; other shapes use a table the
+ *                         context keeps.  viterbi_hard and bcjr_ste_forward take NULL the same way.
  *   soft      device out  [num_blocks * n] float32
  *   logZ      device out  [num_blocks] float32, natural log of Z_T per block (sum over legal
  *                         paths of exp(-E/T), no prior constant); may be NULL
@@ -111,7 +122,10 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
  *   grad_soft      device in   [num_blocks * n]
  *   grad_W         device out  [num_blocks * n]
  *   grad_codebook  device out  [2^Lb], OVERWRITTEN with the sum over all blocks (direct term
- *                  through the emitted value plus the term through the energies); may be NULL
+ *                  through the emitted value plus the term through the energies); may be NULL: the table is
+ *                  then treated as fixed, as in the paper's experiments, and the 2^16-state kernel runs
+ *                  without its accumulator half.  Must be NULL after a forward call with a NULL codebook
+ *                  (BCJR_EINVAL otherwise: a computed emission has no table to differentiate).
  * Uses the state saved by the last bcjr_soft_quantize on this context; BCJR_ESTATE if none.
  */
 bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft,

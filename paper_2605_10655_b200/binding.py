@@ -184,7 +184,8 @@ class Context:
         self._check(self._lib.bcjr_set_option(self._h, name.encode(), int(value)), "bcjr_set_option")
 
     def bcjr_soft_quantize(self, W, codebook, Lb, k, n, T, soft=None, logZ=None, stream=None):
-        """W: [num_blocks*n] (any shape with that many elements) float32 CUDA.  Returns (soft, logZ)."""
+        """W: [num_blocks*n] (any shape with that many elements) float32 CUDA.  Returns (soft, logZ).
+        codebook=None selects the computed Gaussian emission of Section 3.1 (no table)."""
         import torch
         B = W.numel() // n
         if B * n != W.numel():
@@ -201,18 +202,23 @@ class Context:
         self._saved = (W, codebook, Lb, B * n)       # keep the borrowed tensors alive
         return soft, logZ
 
-    def bcjr_backward(self, grad_soft, grad_W=None, grad_codebook=None, stream=None):
+    def bcjr_backward(self, grad_soft, grad_W=None, grad_codebook=None, stream=None, want_grad_codebook=True):
+        """Returns (grad_W, grad_codebook); with want_grad_codebook=False the table's gradient is not formed
+        (NULL is passed; the second value is None)."""
         import torch
         if self._saved is None:
             raise BcjrError(-4, "bcjr_backward")
         W, codebook, Lb, numel = self._saved
         if grad_W is None:
             grad_W = torch.empty_like(W)
-        if grad_codebook is None:
+        if codebook is None:                          # computed emission: there is no table to differentiate
+            want_grad_codebook = False
+        if grad_codebook is None and want_grad_codebook:
             grad_codebook = torch.empty(codebook.numel(), dtype=torch.float32, device=W.device)
         rc = self._lib.bcjr_backward(self._h, _dev(grad_soft, torch.float32, numel, "grad_soft"),
                                      _dev(grad_W, torch.float32, numel, "grad_W"),
-                                     _dev(grad_codebook, torch.float32, codebook.numel(), "grad_codebook"),
+                                     _dev(grad_codebook, torch.float32, name="grad_codebook")
+                                     if grad_codebook is not None else None,
                                      _stream_ptr(stream))
         self._check(rc, "bcjr_backward")
         return grad_W, grad_codebook

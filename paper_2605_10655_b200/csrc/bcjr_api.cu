@@ -18,6 +18,8 @@
 #include "bcjr_rht.cuh"
 #include "bcjr_solo.cuh"
 #include "bcjr_duo.cuh"
+#include "bcjr_skew.cuh"
+#include "bcjr_ckpt.cuh"
 #include "bcjr_viterbi.cuh"
 #endif
 
@@ -38,10 +40,11 @@ struct bcjr_ctx {
     int device = 0;
     int num_sms = 0;
     int max_smem_optin = 0;
-    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, cb_beta, grad_w, grad_c, blk_defect, staging[6];
+    Buffer hist, stepO, msg, gc_part, soft_copy, bp, path_ws, cb_beta, grad_w, grad_c, blk_defect, gauss_cb, staging[6];
     DeviceDiag *diag = nullptr;
     // saved by bcjr_soft_quantize for bcjr_backward
     bool have_fwd = false;
+    bool cb_computed = false;  // the call in flight (and the saved forward state) uses the computed Gaussian emission
     const float *W = nullptr, *cb = nullptr;
     int Lb = 0, k = 0, n = 0;
     int V = 1;                 // numbers emitted per state and step by the saved forward call
@@ -50,9 +53,11 @@ struct bcjr_ctx {
     // options
     int opt_path = 0;
     int opt_max_ctas = 0;
-    int opt_bwd_variant = 0;   // 0 = TMEM two-CTA backward kernel where it applies, 1 = register-accumulator cluster kernel
+    int opt_bwd_variant = 0;   // 0 = TMEM two-CTA backward kernels (k = 2: skewed slot order), 1 = register-accumulator cluster kernel,
+                               // 2 = TMEM two-CTA kernel with one barrier per step also at k = 2
     int opt_fwd_variant = 0;   // 0 = TMEM single-CTA forward kernel where it applies, 1 = cluster forward kernel
     int opt_record_defect = 0; // forward calls record the posterior defect of every block
+    int opt_hist_every = 1;    // large-trellis forward call: keep L_t of every m-th step, recompute the others in the beta sweep
     int64_t defect_blocks = 0; // blocks covered by the last recording
     int launches = 0;
     int last_path = 0;
@@ -80,6 +85,20 @@ bcjr_status ensure(bcjr_ctx *ctx, Buffer &b, size_t bytes)
     if (b.ptr) { CU(cudaFree(b.ptr)); b.ptr = nullptr; b.bytes = 0; }
     CU(cudaMalloc(&b.ptr, bytes));
     b.bytes = bytes;
+    return BCJR_OK;
+}
+
+// Computed Gaussian emission (a NULL codebook): the tensor-memory kernels evaluate the entries themselves while
+// staging; every other kernel reads a table, so the context keeps one written by gaussian_table_kernel.
+bcjr_status computed_table(bcjr_ctx *ctx, int Lb, cudaStream_t st, const float **table)
+{
+    const int S = 1 << Lb;
+    bcjr_status rc = ensure(ctx, ctx->gauss_cb, (size_t)(1 << 16) * 4);
+    if (rc) return rc;
+    gaussian_table_kernel<<<(S + 255) / 256, 256, 0, st>>>((float *)ctx->gauss_cb.ptr, S);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    *table = (const float *)ctx->gauss_cb.ptr;
     return BCJR_OK;
 }
 
@@ -419,6 +438,7 @@ bcjr_status launch_bwd_duo(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cud
     if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * C::S * 4))) return rc;
     p.hist = (float *)ctx->hist.ptr;
     p.gc_part = (float *)ctx->gc_part.ptr;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
     CU(cudaLaunchKernelEx(&cfg, bwd_duo_kernel<KB>, p));
     ctx->launches += 1;
     if (grad_codebook) {
@@ -429,9 +449,37 @@ bcjr_status launch_bwd_duo(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cud
     return BCJR_OK;
 }
 
+// Backward call for k = 2: the two-CTA tensor-memory kernel with the skewed slot order; without grad_codebook the
+// accumulator half of the kernel is compiled out.
+template <bool ACC>
+bcjr_status launch_bwd_skew(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    using C = SkewCfg;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    bcjr_status rc = plan_cluster(ctx, bwd_skew_kernel<ACC>, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    if (rc) return rc;
+    const int ncl = cfg.gridDim.x / C::CL;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * p.n * 2 * C::Q * 4))) return rc;
+    if (ACC && (rc = ensure(ctx, ctx->gc_part, (size_t)ncl * C::S * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.gc_part = ACC ? (float *)ctx->gc_part.ptr : nullptr;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
+    CU(cudaLaunchKernelEx(&cfg, bwd_skew_kernel<ACC>, p));
+    ctx->launches += 1;
+    if (ACC) {
+        reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, C::S, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
 bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_codebook, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
+    if (k == 2 && ctx->opt_bwd_variant == 0 && p.n <= SkewCfg::MAX_N)
+        return grad_codebook ? launch_bwd_skew<true>(ctx, p, grad_codebook, st) : launch_bwd_skew<false>(ctx, p, nullptr, st);
     if (k == 2 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<2>::MAX_N) return launch_bwd_duo<2>(ctx, p, grad_codebook, st);
     if (k == 3 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<3>::MAX_N) return launch_bwd_duo<3>(ctx, p, grad_codebook, st);
     if (k == 2) return launch_bwd_cluster_t<16, 2, 4, 512>(ctx, p, grad_codebook, st);
@@ -453,6 +501,7 @@ bcjr_status launch_vit_solo(bcjr_ctx *ctx, VitParams p, cudaStream_t st)
     if (rc) return rc;
     p.bp = (uint8_t *)ctx->bp.ptr;
     p.diag = ctx->diag;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
     viterbi_solo_kernel<KB><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
     ctx->launches += 1;
     CU(cudaGetLastError());
@@ -472,7 +521,28 @@ bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
     bcjr_status rc = ensure(ctx, ctx->hist, (size_t)grid * p.n * C::Q * 4);
     if (rc) return rc;
     p.hist = (float *)ctx->hist.ptr;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
     fwd_solo_kernel<KB><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+// Forward call with checkpointed history (option history_every_m > 1; Lb = 16; k = 2, 3; n <= 512).
+template <int KB>
+bcjr_status launch_fwd_ckpt(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    using C = CkptCfg<KB>;
+    CU(cudaFuncSetAttribute(fwd_ckpt_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
+    int64_t grid = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    if (grid > p.B) grid = p.B;
+    p.hist_every = ctx->opt_hist_every;
+    bcjr_status rc = ensure(ctx, ctx->hist, (size_t)grid * C::rows(p.n, p.hist_every) * C::Q * 4);
+    if (rc) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
+    fwd_ckpt_kernel<KB><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
     ctx->launches += 1;
     CU(cudaGetLastError());
     return BCJR_OK;
@@ -481,6 +551,10 @@ bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
+    if (ctx->opt_hist_every > 1 && ctx->opt_fwd_variant != 1 && p.n <= CkptCfg<2>::MAX_N) {
+        if (k == 2) return launch_fwd_ckpt<2>(ctx, p, st);
+        if (k == 3) return launch_fwd_ckpt<3>(ctx, p, st);
+    }
     if (k == 2 && ctx->opt_fwd_variant != 1) return launch_fwd_solo<2>(ctx, p, st);
     if (k == 3 && ctx->opt_fwd_variant != 1) return launch_fwd_solo<3>(ctx, p, st);
     if (k == 2) return launch_fwd_cluster_t<16, 2, FWD_CL_K2, FWD_THREADS_K2>(ctx, p, st);
@@ -555,7 +629,7 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx)
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
     Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp, &ctx->path_ws,
-                     &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->blk_defect, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
+                     &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->blk_defect, &ctx->gauss_cb, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3], &ctx->staging[4],
                      &ctx->staging[5]};
     for (Buffer *b : all)
         if (b->ptr) cudaFree(b->ptr);
@@ -574,7 +648,7 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
         return BCJR_OK;
     }
     if (!strcmp(name, "bwd_variant")) {
-        if (value < 0 || value > 1) return BCJR_EINVAL;
+        if (value < 0 || value > 2) return BCJR_EINVAL;
         ctx->opt_bwd_variant = (int)value;
         return BCJR_OK;
     }
@@ -597,6 +671,11 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
         }
         return BCJR_OK;
     }
+    if (!strcmp(name, "history_every_m")) {
+        if (value < 1 || value > 16) return BCJR_EINVAL;
+        ctx->opt_hist_every = (int)value;
+        return BCJR_OK;
+    }
     if (!strcmp(name, "record_block_defect")) {
         if (value < 0 || value > 1) return BCJR_EINVAL;
         ctx->opt_record_defect = (int)value;
@@ -617,22 +696,26 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
     if (!(T > 0.f) || !std::isfinite(T)) return BCJR_EINVAL;
     bcjr_status rc = check_dims(Lb, k, n, num_blocks);
     if (rc) return rc;
-    if (num_blocks > 0 && (!W || !codebook || !soft)) return BCJR_EINVAL;   // empty input: pointers unused
+    if (num_blocks > 0 && (!W || !soft)) return BCJR_EINVAL;   // empty input: pointers unused; codebook NULL = computed emission
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return BCJR_ECUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     ctx->have_fwd = false;
+    ctx->cb_computed = codebook == nullptr;
     if (num_blocks == 0) {
         ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = 0; ctx->T = T;
         ctx->V = 1;
         ctx->have_fwd = true;
         return BCJR_OK;
     }
+    if (ctx->cb_computed && (rc = computed_table(ctx, Lb, st, &codebook))) return rc;
     if ((rc = ensure(ctx, ctx->soft_copy, (size_t)num_blocks * n * 4))) return rc;
     FwdParams p{};
     p.W = W; p.cb = codebook; p.soft = soft; p.soft_copy = (float *)ctx->soft_copy.ptr; p.logZ = logZ;
     p.diag = ctx->diag; p.B = num_blocks; p.Lb = Lb; p.n = n;
     p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)T));
+    table_range_kernel<<<1, 1024, 0, st>>>(codebook, 1 << Lb, ctx->diag);     // c_lo, c_hi for step_energy
+    ctx->launches += 1;
     ctx->defect_blocks = 0;
     if (ctx->opt_record_defect) {
         if ((rc = ensure(ctx, ctx->blk_defect, (size_t)num_blocks * 4))) return rc;
@@ -673,6 +756,7 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
     if (!ctx) return BCJR_EINVAL;
     if (!ctx->have_fwd) return BCJR_ESTATE;
     if (ctx->B > 0 && (!grad_soft || !grad_W)) return BCJR_EINVAL;
+    if (ctx->cb_computed && ctx->V == 1 && grad_codebook) return BCJR_EINVAL;   // a computed emission has no table to differentiate
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return BCJR_ECUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -687,6 +771,10 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
     p.lam2 = (float)(1.4426950408889634 / (2.0 * (double)ctx->T));
     p.invT = (float)(1.0 / (double)ctx->T);
     bcjr_status rc = BCJR_OK;
+    if (ctx->V == 1) {
+        table_range_kernel<<<1, 1024, 0, st>>>(ctx->cb, S, ctx->diag);          // c_lo, c_hi for step_energy
+        ctx->launches += 1;
+    }
     if (ctx->V == 2) {                                   // saved by bcjr_soft_quantize_vec: k bits per weight
         if (!aligned8(grad_soft) || !aligned8(grad_W)) return BCJR_EINVAL;
         bool large = false;
@@ -737,13 +825,21 @@ bcjr_status viterbi_hard(bcjr_ctx *ctx, const float *W, const float *codebook, i
     if (!ctx) return BCJR_EINVAL;
     bcjr_status rc = check_dims(Lb, k, n, num_blocks);
     if (rc) return rc;
-    if (num_blocks > 0 && (!W || !codebook)) return BCJR_EINVAL;
+    if (num_blocks > 0 && !W) return BCJR_EINVAL;                // codebook NULL = computed emission
     const int64_t nbits = Lb + (int64_t)k * (n - 1);
     if (path_bits && path_stride_bytes < (nbits + 7) / 8) return BCJR_EINVAL;
     if (num_blocks == 0) return BCJR_OK;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return BCJR_ECUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    const bool saved_computed = ctx->cb_computed;                // belongs to the saved forward state: restored below
+    struct Restore { bcjr_ctx *c; bool v; ~Restore() { c->cb_computed = v; } } restore{ctx, saved_computed};
+    ctx->cb_computed = codebook == nullptr;
+    if (ctx->cb_computed) {
+        // the context has one computed table: a saved forward state that relies on another size of it ends here
+        if (ctx->have_fwd && saved_computed && ctx->Lb != Lb) ctx->have_fwd = false;
+        if ((rc = computed_table(ctx, Lb, st, &codebook))) return rc;
+    }
     VitParams p{};
     p.W = W; p.cb = codebook; p.path_bits = path_bits; p.path_stride = path_stride_bytes;
     p.states = states; p.hard = hard; p.B = num_blocks; p.Lb = Lb; p.n = n;
@@ -846,7 +942,7 @@ bcjr_status bcjr_ste_forward(bcjr_ctx *ctx, const float *W, const float *codeboo
     if (!(T > 0.f) || !std::isfinite(T)) return BCJR_EINVAL;
     bcjr_status rc = check_dims(Lb, k, n, num_blocks);
     if (rc) return rc;
-    if (num_blocks > 0 && (!W || !codebook || !hard)) return BCJR_EINVAL;
+    if (num_blocks > 0 && (!W || !hard)) return BCJR_EINVAL;
     float *soft_out = soft;
     if (!soft_out && num_blocks > 0) {
         // the relaxation's output is only needed as saved state: let it land in the context's own copy
@@ -1070,7 +1166,7 @@ int64_t bcjr_workspace_bytes(const bcjr_ctx *ctx)
 {
     if (!ctx) return 0;
     const Buffer *all[] = {&ctx->hist, &ctx->stepO, &ctx->msg, &ctx->gc_part, &ctx->soft_copy, &ctx->bp,
-                           &ctx->path_ws, &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->blk_defect, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
+                           &ctx->path_ws, &ctx->cb_beta, &ctx->grad_w, &ctx->grad_c, &ctx->blk_defect, &ctx->gauss_cb, &ctx->staging[0], &ctx->staging[1], &ctx->staging[2], &ctx->staging[3],
                            &ctx->staging[4], &ctx->staging[5]};
     int64_t tot = 0;
     for (const Buffer *b : all) tot += (int64_t)b->bytes;

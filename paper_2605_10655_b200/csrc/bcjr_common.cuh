@@ -76,6 +76,7 @@ struct DeviceDiag {
     unsigned long long wait_limit_ns;   // budget of one device-side wait before it gives up
     int drop_history_load;              // test hook: CTA 0 never requests its first history chunk
     int pad2;
+    float c_lo, c_hi;                   // smallest and largest table entry of the call in flight (table_range_kernel)
 };
 constexpr size_t DIAG_STATUS_BYTES = 16;   // the part bcjr_sync_status reads and clears
 
@@ -90,6 +91,66 @@ __device__ __forceinline__ void diag_max(unsigned int *slot, float v) {
 __device__ __forceinline__ void diag_check_finite(DeviceDiag *diag, float v)
 {
     if (!(fabsf(v) <= 3.0e38f)) atomicCAS(&diag->status, 0, -7);
+}
+
+// Energies without the step's common part.  A weight far outside the table's range (heavy-tailed inputs) puts
+// lam2 (w - c)^2 in the tens of thousands for EVERY state, and a float32 rounded at that magnitude has lost the
+// differences between states that the posterior is made of.  A constant of the step is a gauge (it shifts log Z
+// and nothing else), so the kernels subtract one: with wc = w clamped to [c_lo, c_hi] and delta = w - wc,
+//     (w - c)^2 - delta^2 = du (du - 2 delta),   du = c - wc,
+// and the log2-potential is  e'(s) = du * (du * (-lam2) + kap),  kap = 2 lam2 delta -- two fused multiply-adds, as
+// many operations as the plain square, small wherever c is near the weight (or near the end of the table the
+// weight lies beyond).  Inside the range delta = 0 and this IS the plain square.  log Z gets lam2 delta^2 back.
+struct StepEnergy {
+    float wc;       // clamped weight
+    float kap;      // 2 lam2 delta
+    float delta;    // w - wc
+};
+__device__ __forceinline__ StepEnergy step_energy(float w, float lo, float hi, float lam2)
+{
+    StepEnergy e;
+    e.wc = fminf(fmaxf(w, lo), hi);
+    e.delta = w - e.wc;
+    e.kap = 2.f * lam2 * e.delta;
+    return e;
+}
+
+// Computed Gaussian emission of Section 3.1: c(s) = Phi^-1((s + 1/2) / S).  The cell centre is formed in double
+// (exact), the inverse CDF in single precision; antisymmetric by construction (lower half evaluated, upper half
+// mirrored).  A kernel given a null table pointer uses this instead of a load.
+// (not inlined: the staging loops that call it are fully unrolled)
+__device__ __noinline__ static float gaussian_entry(int s, int S)
+{
+    const int lo = s < S / 2 ? s : S - 1 - s;
+    const float x = normcdfinvf((float)(((double)lo + 0.5) / (double)S));
+    return s < S / 2 ? x : -x;
+}
+__device__ __forceinline__ float table_entry(const float *cb, int s, int S) { return cb ? __ldg(cb + s) : gaussian_entry(s, S); }
+
+// smallest and largest entry of the table, for step_energy: one small block, launched ahead of the sweeps
+static __global__ void __launch_bounds__(1024) table_range_kernel(const float *__restrict__ cb, int S, DeviceDiag *diag)
+{
+    __shared__ float lo_s[32], hi_s[32];
+    float lo = __int_as_float(0x7f800000), hi = __int_as_float(0xff800000);
+    if (!cb) {                                   // computed emission: monotone in s
+        if (threadIdx.x == 0) { diag->c_lo = gaussian_entry(0, S); diag->c_hi = gaussian_entry(S - 1, S); }
+        return;
+    }
+    for (int s = threadIdx.x; s < S; s += blockDim.x) {
+        const float c = __ldg(cb + s);
+        lo = fminf(lo, c); hi = fmaxf(hi, c);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if ((threadIdx.x & 31) == 0) { lo_s[threadIdx.x >> 5] = lo; hi_s[threadIdx.x >> 5] = hi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < (int)(blockDim.x >> 5); ++i) { lo = fminf(lo, lo_s[i]); hi = fmaxf(hi, hi_s[i]); }
+        diag->c_lo = lo; diag->c_hi = hi;
+    }
 }
 
 struct FwdParams {
@@ -107,6 +168,7 @@ struct FwdParams {
     int64_t B;
     int Lb, n;
     float lam2;              // log2(e) / (2T)
+    int hist_every;          // checkpointing kernels: L_t is kept for every hist_every-th step (1 = every step)
 };
 
 struct BwdParams {

@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
     const float NEG_INF = __int_as_float(0xff800000);
     const float invT = p.invT;
     const float2 nl2 = splat2(-p.lam2);
+    const float c_lo = p.diag->c_lo, c_hi = p.diag->c_hi;
 
     float *msg = smem + C::OFF_MSG;
     float4 *stage4 = reinterpret_cast<float4 *>(smem + C::OFF_RING);      // [RD][NCH][CT], thread-private entries
@@ -211,7 +212,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             float4 *hrow = hist4 + ((size_t)(t - 1) * CL + rank) * (BPT * NCH * CT);      // (L_t, At_t) of this thread's butterflies
             // gshn: shift for the consumers of this step's At (step t+1); unused at t = n
             const float2 gshn2 = splat2(gshn);
-            const float2 w2 = splat2(wt), g2 = splat2(gt), off2 = splat2(off);
+            const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
+            const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt), off2 = splat2(off);
             float tmax = NEG_INF;
 #pragma unroll
             for (int i = 0; i < BPT; ++i) {
@@ -238,8 +240,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                         float2 a[K];
 #pragma unroll
                         for (int j = 0; j < K; ++j) {
-                            const float2 d = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
-                            a[j] = fma2(mul2(d, d), nl2, splat2(Lj[j]));
+                            const float2 du = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
+                            a[j] = energy2(du, nl2, kap2, splat2(Lj[j]));
                         }
                         const float2 m = max_pairs<K>(a);
                         float2 pj = ex2f2(sub2(a[0], m));
@@ -376,7 +378,8 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, rank == 0 ? TX_MSG + TX_PART : TX_MSG);
             const float2 gsh2 = splat2(gsh), gshp2 = splat2(gshp);
-            const float2 w2 = splat2(wt), g2 = splat2(gt), gi2 = splat2(invT), offM2 = splat2(offM);
+            const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
+            const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt), ngi2 = splat2(-invT), gid2 = splat2(invT * se.delta), offM2 = splat2(offM);
             const float2 Dm2 = splat2((float)(Ofin - Ot - P) + lsefin);
             float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
             float tmax = NEG_INF;
@@ -415,21 +418,22 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                         float2 uu[K], d[K];
 #pragma unroll
                         for (int b = 0; b < K; ++b) {
-                            d[b] = sub2(w2, cb[g & 1][C::b_idx(hh, b)]);
-                            uu[b] = fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
+                            d[b] = sub2(cb[g & 1][C::b_idx(hh, b)], w2);            // du = c - wc
+                            uu[b] = energy2(d[b], nl2, kap2, splat2(Mb[b]));
                         }
                         const float2 m = max_pairs<K>(uu);
                         const float2 Ahj = sub2(make_float2(Ah[2 * jh], Ah[2 * jh + 1]), gsh2);
                         const float2 Lhj = make_float2(Lh[2 * jh], Lh[2 * jh + 1]);
                         const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
-                        const float2 fg = mul2(f, g2), fi = mul2(f, gi2);
+                        // f (w - c) / T = f delta / T - (f / T) du
+                        const float2 fg = mul2(f, g2), nfi = mul2(f, ngi2), fid = mul2(f, gid2);
                         if (!acc_ready) { tmem_wait_ld(acc); acc_ready = true; }
                         float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
 #pragma unroll
                         for (int b = 0; b < K; ++b) {
                             const float2 pb = ex2f2(sub2(uu[b], m));
                             const float2 y = fma2(g2, cb[g & 1][C::b_idx(hh, b)], splat2(Yb[b]));   // h + Bt
-                            const float2 z = fma2(mul2(fi, d[b]), add2(y, Ahj), fg);                  // f (g + (w - c) r / T)
+                            const float2 z = fma2(fma2(nfi, d[b], fid), add2(y, Ahj), fg);            // f (g + (w - c) r / T)
                             sum = add2(sum, pb);
                             ya = fma2(pb, y, ya);
                             zs = fma2(pb, z, zs);

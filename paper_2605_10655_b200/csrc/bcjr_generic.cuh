@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
     float *hist = p.hist + (size_t)blockIdx.x * n * Q;
     int *stepO = p.stepO + (size_t)blockIdx.x * (n + 2);
     const float lam2 = p.lam2;
+    const float c_lo = p.diag->c_lo, c_hi = p.diag->c_hi;
     float defect = 0.f, zgap = 0.f;
 
     for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
@@ -42,18 +43,20 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
         if (tid == 0) stepO[1] = 0;
         int O = 0;
         float off = 0.f, cmax = 0.f, bdef = 0.f;
+        double zshift = 0.0;                     // sum_t lam2 delta_t^2: what step_energy leaves out of log2 Z
         __syncthreads();
         // ---- alpha: from L_t to L_{t+1}, t = 1..n (the last one only feeds log Z)
         for (int t = 1; t <= n; ++t) {
-            const float wt = __ldg(w + t - 1);
+            const StepEnergy se = step_energy(__ldg(w + t - 1), c_lo, c_hi, lam2);
+            zshift += (double)lam2 * (double)se.delta * (double)se.delta;
             float tmax = NEG_INF;
             for (int q = tid; q < Q; q += nthr) {
                 float a[K], m = NEG_INF;
 #pragma unroll
                 for (int j = 0; j < K; ++j) {
                     const int s = q + j * Q;
-                    const float d = wt - __ldg(p.cb + s);
-                    a[j] = fmaf(d * d, -lam2, Lin[s >> KB]);
+                    const float du = __ldg(p.cb + s) - se.wc;
+                    a[j] = fmaf(du, fmaf(du, -lam2, se.kap), Lin[s >> KB]);
                     m = fmaxf(m, a[j]);
                 }
                 float sum = 0.f;
@@ -84,7 +87,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
         const float lsefin = cmax + lg2f(tot);
         if (tid == 0) diag_check_finite(p.diag, lsefin);
         const int Ofin = O;
-        if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
+        if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin - zshift) * 0.6931471805599453);
         // ---- beta sweep fused with the posterior and the expectation
         float *Min = msgbuf, *Mout = msgbuf + Q;
         for (int q = tid; q < Q; q += nthr) Min[q] = 0.f;                      // M_n = 0: free last state
@@ -92,7 +95,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
         float offM = 0.f;
         __syncthreads();
         for (int t = n; t >= 1; --t) {
-            const float wt = __ldg(w + t - 1);
+            const StepEnergy se = step_energy(__ldg(w + t - 1), c_lo, c_hi, lam2);
             const float D = (float)(Ofin - stepO[t] - P) + lsefin;
             float num = 0.f, den = 0.f, tmax = NEG_INF;
             for (int q = tid; q < Q; q += nthr) {
@@ -102,8 +105,8 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
                 for (int b = 0; b < K; ++b) {
                     const int s = q * K + b;
                     c[b] = __ldg(p.cb + s);
-                    const float d = wt - c[b];
-                    u[b] = fmaf(d * d, -lam2, Min[s & (Q - 1)]);
+                    const float du = c[b] - se.wc;
+                    u[b] = fmaf(du, fmaf(du, -lam2, se.kap), Min[s & (Q - 1)]);
                     m = fmaxf(m, u[b]);
                 }
                 float sum = 0.f, craw = 0.f;
@@ -192,6 +195,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams 
     int *stepO = p.stepO + (size_t)blockIdx.x * (n + 2);
     float *gc = p.gc_part + (size_t)blockIdx.x * S;
     const float lam2 = p.lam2, invT = p.invT;
+    const float c_lo = p.diag->c_lo, c_hi = p.diag->c_hi;
     float defect = 0.f;
 
     for (int q = tid; q < Q; q += nthr)
@@ -207,7 +211,8 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams 
         float off = 0.f, cmax = 0.f;
         __syncthreads();
         for (int t = 1; t <= n; ++t) {
-            const float wt = __ldg(w + t - 1), gt = __ldg(g + t - 1), st = __ldg(sf + t - 1);
+            const float gt = __ldg(g + t - 1), st = __ldg(sf + t - 1);
+            const StepEnergy se = step_energy(__ldg(w + t - 1), c_lo, c_hi, lam2);
             float tmax = NEG_INF;
             for (int q = tid; q < Q; q += nthr) {
                 float a[K], x[K], m = NEG_INF;
@@ -215,8 +220,8 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams 
                 for (int j = 0; j < K; ++j) {
                     const int s = q + j * Q;
                     const float c = __ldg(p.cb + s);
-                    const float d = wt - c;
-                    a[j] = fmaf(d * d, -lam2, Lin[s >> KB]);
+                    const float du = c - se.wc;
+                    a[j] = fmaf(du, fmaf(du, -lam2, se.kap), Lin[s >> KB]);
                     x[j] = fmaf(gt, c - st, Ain[s >> KB]);
                     m = fmaxf(m, a[j]);
                 }
@@ -259,7 +264,8 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams 
         float offM = 0.f;
         __syncthreads();
         for (int t = n; t >= 1; --t) {
-            const float wt = __ldg(w + t - 1), gt = __ldg(g + t - 1), st = __ldg(sf + t - 1);
+            const float gt = __ldg(g + t - 1), st = __ldg(sf + t - 1);
+            const StepEnergy se = step_energy(__ldg(w + t - 1), c_lo, c_hi, lam2);
             const float D = (float)(Ofin - stepO[t] - P) + lsefin;
             float S0 = 0.f, S1 = 0.f, S2 = 0.f, S3 = 0.f, tmax = NEG_INF;
             for (int q = tid; q < Q; q += nthr) {
@@ -270,9 +276,10 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams 
                 for (int b = 0; b < K; ++b) {
                     const int s = q * K + b;
                     const float c = __ldg(p.cb + s);
-                    d[b] = wt - c;
+                    const float du = c - se.wc;
+                    d[b] = se.delta - du;                       // w - c
                     cm[b] = c - st;
-                    u[b] = fmaf(d[b] * d[b], -lam2, Min[s & (Q - 1)]);
+                    u[b] = fmaf(du, fmaf(du, -lam2, se.kap), Min[s & (Q - 1)]);
                     y[b] = fmaf(gt, cm[b], Bin[s & (Q - 1)]);
                     m = fmaxf(m, u[b]);
                 }

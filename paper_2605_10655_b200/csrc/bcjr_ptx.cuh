@@ -259,6 +259,15 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
     return d;
 }
 __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+// log2-potential of a pair of states plus a message: du (du (-lam2) + kap) + msg, see step_energy
+__device__ __forceinline__ float2 energy2(float2 du, float2 nl2, float2 kap2, float2 msg)
+{
+#ifdef BCJR_AB_PLAIN_ENERGY
+    return fma2(mul2(du, du), nl2, msg);          // timing experiment only: the plain square (exact when delta = 0)
+#else
+    return fma2(du, fma2(du, nl2, kap2), msg);
+#endif
+}
 __device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
 __device__ __forceinline__ float2 lg2f2(float2 a) { return make_float2(lg2f(a.x), lg2f(a.y)); }
 __device__ __forceinline__ float2 rcpf2(float2 a) { return make_float2(rcpf(a.x), rcpf(a.y)); }

@@ -2,22 +2,15 @@
 // update of the continuous pre-image (and, optionally, of the table) and the computed Gaussian
 // emission table of Section 3.1.  Element-wise, bound by HBM: 16-byte accesses, one pass.
 #pragma once
-#include <cuda_runtime.h>
-#include <stdint.h>
+#include "bcjr_common.cuh"
 
 namespace bcjr {
 
-// c(s) = Phi^-1((s + 1/2) / S): evaluated in double on the argument (the cell centre is exact in
-// double), inverse CDF in single precision
+// c(s) = Phi^-1((s + 1/2) / S) written out as a table (the same routine the kernels use for a null table)
 __global__ void gaussian_table_kernel(float *c, int S)
 {
     const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= S) return;
-    // antisymmetric by construction: evaluate on the lower half, mirror
-    const int lo = s < S / 2 ? s : S - 1 - s;
-    const float u = (float)(((double)lo + 0.5) / (double)S);
-    const float x = normcdfinvf(u);
-    c[s] = s < S / 2 ? x : -x;
+    if (s < S) c[s] = gaussian_entry(s, S);
 }
 
 struct AdamParams {

