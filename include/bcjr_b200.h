@@ -80,7 +80,7 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *   "history_every_m"  1 (default): the large-trellis forward kernel stores the forward messages of every step
  *                 for its beta sweep; m = 2..16: it keeps them for every m-th step only and recomputes the
  *                 m - 1 steps in between inside the beta sweep (1/m of the history traffic to HBM for
- *                 (m-1)/m of an alpha sweep more arithmetic; same results within float32 rounding; Lb = 16, k = 2 or 3,
+ *                 (m-1)/m of an alpha sweep more arithmetic; same results within float32 rounding; Lb = 16, k = 2,
  *                 n <= 512, otherwise the option has no effect)
  *   "max_ctas"    cap on resident thread blocks (0 = fill the GPU)
  *   "record_block_defect"  1: every scalar forward call also records, per block, max over steps of

@@ -19,6 +19,7 @@
 #include "bcjr_solo.cuh"
 #include "bcjr_duo.cuh"
 #include "bcjr_skew.cuh"
+#include "bcjr_alpha.cuh"
 #include "bcjr_ckpt.cuh"
 #include "bcjr_viterbi.cuh"
 #endif
@@ -457,7 +458,7 @@ bcjr_status launch_bwd_skew(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cu
     using C = SkewCfg;
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1];
-    bcjr_status rc = plan_cluster(ctx, bwd_skew_kernel<ACC>, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    bcjr_status rc = plan_cluster(ctx, bwd_skew_kernel<ACC, false>, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
     if (rc) return rc;
     const int ncl = cfg.gridDim.x / C::CL;
     if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * p.n * 2 * C::Q * 4))) return rc;
@@ -465,8 +466,56 @@ bcjr_status launch_bwd_skew(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cu
     p.hist = (float *)ctx->hist.ptr;
     p.gc_part = ACC ? (float *)ctx->gc_part.ptr : nullptr;
     if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
-    CU(cudaLaunchKernelEx(&cfg, bwd_skew_kernel<ACC>, p));
+    CU(cudaLaunchKernelEx(&cfg, bwd_skew_kernel<ACC, false>, p));
     ctx->launches += 1;
+    if (ACC) {
+        reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, C::S, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
+// Backward call for k = 2 in two kernels per chunk of blocks: the alpha sweeps on one CTA per block (bwd_alpha_kernel),
+// then the beta sweeps of the same blocks on two-CTA clusters (bwd_skew_kernel<ACC, true>).  A chunk is as many blocks
+// as the GPU has SMs; the history of a chunk (32 MB per block at n = 256) is the hand-over between the two.
+template <bool ACC>
+bcjr_status launch_bwd_split(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    using C = SkewCfg;
+    using A = AlphaCfg;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    bcjr_status rc = plan_cluster(ctx, bwd_skew_kernel<ACC, true>, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    if (rc) return rc;
+    CU(cudaFuncSetAttribute(bwd_alpha_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
+    const int ncl = cfg.gridDim.x / C::CL;
+    int64_t chunk = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && chunk > ctx->opt_max_ctas) chunk = ctx->opt_max_ctas;
+    if (chunk > p.B) chunk = p.B;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)chunk * p.n * 2 * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, (size_t)chunk * A::AUX_INTS * 4))) return rc;
+    if (ACC) {
+        if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * C::S * 4))) return rc;
+        CU(cudaMemsetAsync(ctx->gc_part.ptr, 0, (size_t)ncl * C::S * 4, st));     // the beta launches add into it
+    }
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    p.gc_part = ACC ? (float *)ctx->gc_part.ptr : nullptr;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
+    const int64_t B = p.B;
+    const float *W = p.W, *g = p.g, *soft = p.soft;
+    float *gW = p.gW;
+    for (int64_t b0 = 0; b0 < B; b0 += chunk) {
+        const int64_t nb = B - b0 < chunk ? B - b0 : chunk;
+        p.B = nb;
+        p.W = W + b0 * p.n; p.g = g + b0 * p.n; p.soft = soft + b0 * p.n; p.gW = gW + b0 * p.n;
+        bwd_alpha_kernel<false><<<(int)nb, A::THREADS, A::SMEM_BYTES, st>>>(p);
+        CU(cudaGetLastError());
+        cfg.gridDim = dim3((unsigned)(C::CL * (nb < ncl ? nb : ncl)), 1, 1);
+        CU(cudaLaunchKernelEx(&cfg, bwd_skew_kernel<ACC, true>, p));
+        ctx->launches += 2;
+    }
     if (ACC) {
         reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, C::S, grad_codebook);
         ctx->launches += 1;
@@ -479,6 +528,8 @@ bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_co
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
     if (k == 2 && ctx->opt_bwd_variant == 0 && p.n <= SkewCfg::MAX_N)
+        return grad_codebook ? launch_bwd_split<true>(ctx, p, grad_codebook, st) : launch_bwd_split<false>(ctx, p, nullptr, st);
+    if (k == 2 && ctx->opt_bwd_variant == 3 && p.n <= SkewCfg::MAX_N)
         return grad_codebook ? launch_bwd_skew<true>(ctx, p, grad_codebook, st) : launch_bwd_skew<false>(ctx, p, nullptr, st);
     if (k == 2 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<2>::MAX_N) return launch_bwd_duo<2>(ctx, p, grad_codebook, st);
     if (k == 3 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<3>::MAX_N) return launch_bwd_duo<3>(ctx, p, grad_codebook, st);
@@ -528,7 +579,7 @@ bcjr_status launch_fwd_solo(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
     return BCJR_OK;
 }
 
-// Forward call with checkpointed history (option history_every_m > 1; Lb = 16; k = 2, 3; n <= 512).
+// Forward call with checkpointed history (option history_every_m > 1; Lb = 16, k = 2, n <= 512).
 template <int KB>
 bcjr_status launch_fwd_ckpt(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
@@ -551,10 +602,7 @@ bcjr_status launch_fwd_ckpt(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
-    if (ctx->opt_hist_every > 1 && ctx->opt_fwd_variant != 1 && p.n <= CkptCfg<2>::MAX_N) {
-        if (k == 2) return launch_fwd_ckpt<2>(ctx, p, st);
-        if (k == 3) return launch_fwd_ckpt<3>(ctx, p, st);
-    }
+    if (ctx->opt_hist_every > 1 && ctx->opt_fwd_variant != 1 && k == 2 && p.n <= CkptCfg<2>::MAX_N) return launch_fwd_ckpt<2>(ctx, p, st);
     if (k == 2 && ctx->opt_fwd_variant != 1) return launch_fwd_solo<2>(ctx, p, st);
     if (k == 3 && ctx->opt_fwd_variant != 1) return launch_fwd_solo<3>(ctx, p, st);
     if (k == 2) return launch_fwd_cluster_t<16, 2, FWD_CL_K2, FWD_THREADS_K2>(ctx, p, st);
@@ -648,7 +696,7 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
         return BCJR_OK;
     }
     if (!strcmp(name, "bwd_variant")) {
-        if (value < 0 || value > 2) return BCJR_EINVAL;
+        if (value < 0 || value > 3) return BCJR_EINVAL;
         ctx->opt_bwd_variant = (int)value;
         return BCJR_OK;
     }

@@ -1,4 +1,4 @@
-// Forward call with checkpointed forward messages (Lb = 16; k = 2, 3): the one-CTA tensor-memory kernel of
+// Forward call with checkpointed forward messages (Lb = 16, k = 2): the one-CTA tensor-memory kernel of
 // bcjr_solo.cuh, except that the alpha sweep keeps L_t only for every m-th step and the beta sweep recomputes
 // the m - 1 steps in between.
 //
@@ -39,6 +39,7 @@ struct CkptCfg {
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static_assert(OFF_RING % 4 == 0, "staging alignment");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
+    static_assert(KB_ == 2 && NCH == 1, "the alpha step on the beta-paired table is written for K = 4");
     __host__ __device__ static constexpr int a_idx(int j, int h) { return B::a_idx(j, h); }
     __host__ __device__ static constexpr int b_idx(int jh, int b) { return B::b_idx(jh, b); }
     // history rows per CTA: the checkpoints, then the segment scratch
@@ -88,10 +89,13 @@ __global__ void __launch_bounds__(CkptCfg<KB>::THREADS, 1) fwd_ckpt_kernel(FwdPa
     }
     float defect = 0.f, zgap = 0.f;
 
-    // one alpha step: L_{t+1} from L_t (Lin, thread-private entries) into Lout (the consumers' entries); the inputs are
-    // stored to hrow when it is not null.  Used by the alpha sweep and, unchanged, by the recomputation.
+    // One alpha step: L_{t+1} from L_t (Lin, thread-private entries) into Lout (the consumers' entries); the inputs are
+    // stored to hrow when it is not null.  Used by the alpha sweep and, unchanged, by the recomputation, so both give
+    // the same bits.  It works on the table as the BETA sweep pairs it -- (c[2jh|x|b], c[2jh+1|x|b]) -- so that the
+    // table is staged once per block and never re-paired: the sum over the predecessors j of output b is then a sum
+    // over the two halves of two packed values instead of over four packed values.
     auto alpha_step = [&](const float *Lin, float *Lout, float4 *hrow, float wc, float kap, float off) -> float {
-        const float2 w2 = splat2(wc), kap2 = splat2(kap), off2 = splat2(off);
+        const float2 w2 = splat2(wc), kap2 = splat2(kap);
         float tmax = NEG_INF;
         float2 cb[2][8];
         tmem_ld16(tm, cb[0]);
@@ -100,37 +104,22 @@ __global__ void __launch_bounds__(CkptCfg<KB>::THREADS, 1) fwd_ckpt_kernel(FwdPa
             float Lj[K];
 #pragma unroll
             for (int j = 0; j < K; ++j) Lj[j] = Lin[(i * K + j) * CT + tid];
-            if (hrow) {
+            if (hrow) hrow[i * CT] = make_float4(Lj[0], Lj[1], Lj[2], Lj[3]);
+            tmem_wait_ld(cb[i & 1]);
+            if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
+            const float2 L01 = make_float2(Lj[0], Lj[1]), L23 = make_float2(Lj[2], Lj[3]);
+            float out[K];
 #pragma unroll
-                for (int q = 0; q < NCH; ++q)
-                    hrow[(i * NCH + q) * CT] = make_float4(Lj[4 * q], Lj[4 * q + 1], Lj[4 * q + 2], Lj[4 * q + 3]);
+            for (int b = 0; b < K; ++b) {
+                const float2 d0 = sub2(cb[i & 1][C::b_idx(0, b)], w2), d1 = sub2(cb[i & 1][C::b_idx(1, b)], w2);
+                const float2 a0 = energy2(d0, nl2, kap2, L01), a1 = energy2(d1, nl2, kap2, L23);
+                const float mx = fmaxf(max3f(a0.x, a0.y, a1.x), a1.y);
+                const float2 m2 = splat2(mx);
+                const float2 s2 = add2(ex2f2(sub2(a0, m2)), ex2f2(sub2(a1, m2)));
+                out[b] = (mx - off) + lg2f(s2.x + s2.y);
+                tmax = fmaxf(tmax, mx);
             }
-            float2 out[K / 2];
-#pragma unroll
-            for (int u = 0; u < UNITS; ++u) {
-                const int g = i * UNITS + u;
-                tmem_wait_ld(cb[g & 1]);
-                if (g + 1 < NU) tmem_ld16(tm + 16u * (g + 1), cb[(g + 1) & 1]);
-#pragma unroll
-                for (int hh = 0; hh < HPU; ++hh) {
-                    const int h = u * HPU + hh;
-                    float2 a[K];
-#pragma unroll
-                    for (int j = 0; j < K; ++j) {
-                        const float2 du = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
-                        a[j] = energy2(du, nl2, kap2, splat2(Lj[j]));
-                    }
-                    const float2 mx = max_pairs<K>(a);
-                    float2 sum = ex2f2(sub2(a[0], mx));
-#pragma unroll
-                    for (int j = 1; j < K; ++j) sum = add2(sum, ex2f2(sub2(a[j], mx)));
-                    out[h] = add2(sub2(mx, off2), lg2f2(sum));
-                    tmax = max3f(tmax, mx.x, mx.y);
-                }
-            }
-#pragma unroll
-            for (int h = 0; h < K / 2; h += 2)
-                *reinterpret_cast<float4 *>(Lout + push_a[i] + 2 * h) = make_float4(out[h].x, out[h].y, out[h + 1].x, out[h + 1].y);
+            *reinterpret_cast<float4 *>(Lout + push_a[i]) = make_float4(out[0], out[1], out[2], out[3]);
         }
         return tmax;
     };
@@ -144,7 +133,7 @@ __global__ void __launch_bounds__(CkptCfg<KB>::THREADS, 1) fwd_ckpt_kernel(FwdPa
         for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // L_1 = 0 in buffer 0
         if (tid == 0) O_s[1] = 0;
 #pragma unroll
-        for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), false);
+        for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), true);   // beta pairing, for both sweeps
         tmem_wait_st();
         int O = 0;
         float off = 0.f, cmax = 0.f, bdef = 0.f;
@@ -190,9 +179,6 @@ __global__ void __launch_bounds__(CkptCfg<KB>::THREADS, 1) fwd_ckpt_kernel(FwdPa
         }
         // ================= beta sweep, segment by segment
         for (int q = tid; q < Q; q += CT) msg[q] = 0.f;                      // M_n = 0 in buffer 0
-#pragma unroll
-        for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), true);
-        tmem_wait_st();
         int P = 0, mb = 0;                                                   // mb: buffer that holds the current M
         float offM = 0.f;
         int par = 0;                                                         // parity of the wmax / part slots
@@ -204,9 +190,6 @@ __global__ void __launch_bounds__(CkptCfg<KB>::THREADS, 1) fwd_ckpt_kernel(FwdPa
             if (len > 1) {
                 // ---- recompute L_{t0+1} .. L_{t_end} from the checkpoint, in the two buffers that do not hold M
                 const int a0 = mb == 0 ? 1 : 0, a1 = 3 - mb - a0;
-#pragma unroll
-                for (int i = 0; i < BPT; ++i)                                // alpha pairing of the table
-                    stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), false);
                 {
                     float *A = msg + a0 * Q;
                     const float4 *ck = hist4 + (size_t)c * ROW;
@@ -219,7 +202,6 @@ __global__ void __launch_bounds__(CkptCfg<KB>::THREADS, 1) fwd_ckpt_kernel(FwdPa
                             A[(i * K + 4 * q + 2) * CT + tid] = v.z; A[(i * K + 4 * q + 3) * CT + tid] = v.w;
                         }
                 }
-                tmem_wait_st();
                 for (int s = 0; s + 1 < len; ++s) {
                     const int t = t0 + s;
                     const float *Lin = msg + ((s & 1) ? a1 : a0) * Q;
@@ -237,10 +219,6 @@ __global__ void __launch_bounds__(CkptCfg<KB>::THREADS, 1) fwd_ckpt_kernel(FwdPa
                             hrow[(i * NCH + q) * CT] = make_float4(Lin[(i * K + 4 * q) * CT + tid], Lin[(i * K + 4 * q + 1) * CT + tid],
                                                                    Lin[(i * K + 4 * q + 2) * CT + tid], Lin[(i * K + 4 * q + 3) * CT + tid]);
                 }
-#pragma unroll
-                for (int i = 0; i < BPT; ++i)                                // back to the beta pairing
-                    stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), true);
-                tmem_wait_st();
                 compute_barrier(CT);                                         // the recomputation's buffers are free for M again
             }
             // ---- the segment's beta steps, t = t_end .. t0; L_t from the scratch (row t - t0) or the checkpoint (t = t0)

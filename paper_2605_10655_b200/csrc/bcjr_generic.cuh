@@ -19,7 +19,7 @@ constexpr int GEN_MAX_THREADS = 512;
 // Forward call: alpha sweep (Eq. 5, log domain) then beta sweep fused with Eq. 6-7.
 // --------------------------------------------------------------------------------------
 template <int KB>
-__global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams p)
+__global__ void __launch_bounds__(GEN_MAX_THREADS, (KB == 2 || KB == 3) ? 2 : 1) fwd_generic_kernel(FwdParams p)
 {
     constexpr int K = 1 << KB;
     extern __shared__ float smem[];
@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(GEN_MAX_THREADS) fwd_generic_kernel(FwdParams 
 //   grad_c[u] += gamma_t(u) [ g_t + (w_t - c[u]) r_t(u) / T ]
 // --------------------------------------------------------------------------------------
 template <int KB>
-__global__ void __launch_bounds__(GEN_MAX_THREADS) bwd_generic_kernel(BwdParams p)
+__global__ void __launch_bounds__(GEN_MAX_THREADS, KB == 2 ? 2 : 1) bwd_generic_kernel(BwdParams p)
 {
     constexpr int K = 1 << KB;
     extern __shared__ float smem[];

@@ -262,15 +262,29 @@ __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
 // log2-potential of a pair of states plus a message: du (du (-lam2) + kap) + msg, see step_energy
 __device__ __forceinline__ float2 energy2(float2 du, float2 nl2, float2 kap2, float2 msg)
 {
-#ifdef BCJR_AB_PLAIN_ENERGY
+#if defined(BCJR_AB_PLAIN_ENERGY)
     return fma2(mul2(du, du), nl2, msg);          // timing experiment only: the plain square (exact when delta = 0)
+#elif defined(BCJR_AB_AAF_ENERGY)
+    return fma2(du, sub2(kap2, du), msg);         // timing experiment only: add, add, fma (needs a pre-scaled table)
 #else
     return fma2(du, fma2(du, nl2, kap2), msg);
 #endif
 }
 __device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
 __device__ __forceinline__ float2 lg2f2(float2 a) { return make_float2(lg2f(a.x), lg2f(a.y)); }
+#ifdef BCJR_AB_RCP_NR
+// timing experiment: 1/x for x in [1, K] on the FP32 pipe: linear seed in the exponent domain + three Newton steps
+__device__ __forceinline__ float2 rcpf2(float2 a)
+{
+    float2 y = make_float2(__int_as_float(0x7EF311C7 - __float_as_int(a.x)), __int_as_float(0x7EF311C7 - __float_as_int(a.y)));
+    const float2 one = make_float2(1.f, 1.f), na = make_float2(-a.x, -a.y);
+#pragma unroll
+    for (int it = 0; it < 3; ++it) y = fma2(y, fma2(na, y, one), y);
+    return y;
+}
+#else
 __device__ __forceinline__ float2 rcpf2(float2 a) { return make_float2(rcpf(a.x), rcpf(a.y)); }
+#endif
 // 2^x for x <= 0 on the FP32 pipe (no special-function instruction): x = n + f with n the nearest
 // integer and |f| <= 1/2, 2^f by the degree-5 interpolant at the Chebyshev nodes of [-1/2, 1/2] (relative
 // error 2.4e-7 evaluated in float32, about that of ex2.approx), the

@@ -29,8 +29,13 @@
 //
 // Everything else -- tensor-memory tables and accumulators, thread-private history, bounded waits, the
 // arithmetic itself -- is that of bcjr_duo.cuh.  ACC = false leaves out the gradient accumulators (a call
-// that does not ask for grad_codebook).
+// that does not ask for grad_codebook).  BETA_ONLY = true runs the beta sweeps alone, on the history, gauge
+// offsets and log Z that bwd_alpha_kernel (bcjr_alpha.cuh) wrote for the same blocks; block b of the call then
+// has its history at p.hist + b n 2Q and its offsets at p.stepO + b (MAX_N + 4), and the partial codebook
+// gradient is ADDED to p.gc_part (several launches share it).
 #pragma once
+#include <type_traits>
+
 #include "bcjr_duo.cuh"
 
 namespace bcjr {
@@ -75,7 +80,7 @@ struct SkewCfg {
     }
 };
 
-template <bool ACC>
+template <bool ACC, bool BETA_ONLY>
 __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams p)
 {
     using C = SkewCfg;
@@ -111,7 +116,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
     const uint32_t msg_u32 = smem_u32(msg), stage_u32 = smem_u32(stage4) + (uint32_t)tid * 16u;
     const uint32_t wmax_u32 = smem_u32(wmax), part_u32 = smem_u32(part), lz_u32 = smem_u32(lz);
 
-    // history of this cluster: float4 [n][CL][BPT][NCH][CT]; this thread's entries
+    // history of this cluster (BETA_ONLY: of the block at hand): float4 [n][CL][BPT][NCH][CT]; this thread's entries
     float4 *hist4 = reinterpret_cast<float4 *>(p.hist + (size_t)cid * n * 2 * C::Q) + tid;
     constexpr ptrdiff_t HSTEP = (ptrdiff_t)CL * BPT * NCH * CT;     // float4 per step
 
@@ -178,135 +183,158 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
     for (int64_t blk = cid; blk < p.B; blk += ncl) {
         int ib = 0;
         const float *w_s = p.W + blk * n, *g_s = p.g + blk * n, *sf_s = p.soft + blk * n;
-        // L_1 = 0; the At array carries At + gsh (gsh_t = -g_t soft_t centres h_t = g_t c - g_t soft_t)
-        {
+        if (BETA_ONLY) {
+            // the alpha sweep of this block was run by bwd_alpha_kernel: its history, gauge offsets and log Z tail
+            hist4 = reinterpret_cast<float4 *>(p.hist + (size_t)blk * n * 2 * C::Q) + tid;
+            const int *aux = p.stepO + (size_t)blk * (C::MAX_N + 4);
+            for (int t = 1 + tid; t <= n + 1; t += CT) O_s[t] = aux[t];
+        } else {
+            // L_1 = 0; the At array carries At + gsh (gsh_t = -g_t soft_t centres h_t = g_t c - g_t soft_t)
             const float gsh1 = -__ldg(g_s) * __ldg(sf_s);
             for (int q = tid; q < QC; q += CT) { msg[q] = 0.f; msg[QC + q] = gsh1; }
+            if (tid == 0) O_s[1] = 0;
         }
-        if (tid == 0) O_s[1] = 0;
-#pragma unroll
-        for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, alpha pairing
-            stage_codebook<C>(p.cb, C::x_of((int)rank, tid, i), tm_cb + (uint32_t)(16 * i), false);
-        tmem_wait_st();
-        int O = 0;
-        float off = 0.f, cmax = 0.f;
+        // a block whose weights all lie inside the table's range (nearly every block of Gaussian weights) takes the
+        // sweeps with the plain square; any other block the form of step_energy (both CTAs decide alike)
+        int outside = 0;
+        for (int t = tid; t < n; t += CT) {
+            const float wv = __ldg(w_s + t);
+            outside |= !(wv >= c_lo && wv <= c_hi);
+        }
+        const bool recentre = __syncthreads_or(outside) != 0;
+        int O = 0, Ofin = 0;
+        float off = 0.f, cmax = 0.f, lsefin = 0.f;
         bool dead = false;
-        cluster_sync();                                          // block start
-        // ================= alpha sweep carrying (L, At)
-        for (int t = 1; t <= n; ++t) {
-            const int ob = ib ^ 1;
-            float2 cb[2][8];
-            tmem_ld16(tm_cb, cb[0]);
-            const float gt = __ldg(g_s + t - 1), wt = __ldg(w_s + t - 1);
-            const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
-            if (t > 1) wait_early(ib);
-            if (!pr.warp_live()) { tmem_wait_ld(cb[0]); dead = true; break; }
-            const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
-            const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
-            if (tid == 0) {
-                mbar_expect_tx(mb_early + ob_mbar, TX_A_EARLY);
-                mbar_expect_tx(mb_late + ob_mbar, TX_A_LATE);
-            }
-            float4 *hrow = hist4 + (size_t)(t - 1) * HSTEP + (size_t)rank * (BPT * NCH * CT);   // (L_t, At_t) of this thread's butterflies
-            const float2 gshn2 = splat2(gshn);
-            const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
-            const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt);
-            float2 off2 = splat2(off);
-            float tmax = NEG_INF;
+        if constexpr (!BETA_ONLY) {
 #pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                float2 outL[K / 2], outA[K / 2];
-                float Lj[K], Aj[K];
-#pragma unroll
-                for (int j = 0; j < K; ++j) {
-                    Lj[j] = Lin[(i * K + j) * CT + tid];
-                    Aj[j] = Ain[(i * K + j) * CT + tid];
+            for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, alpha pairing
+                stage_codebook<C>(p.cb, C::x_of((int)rank, tid, i), tm_cb + (uint32_t)(16 * i), false);
+            tmem_wait_st();
+            cluster_sync();                                          // block start
+            // ================= alpha sweep carrying (L, At)
+            auto alpha_sweep = [&](auto rc_tag) {
+            constexpr bool RC = decltype(rc_tag)::value;
+            for (int t = 1; t <= n; ++t) {
+                const int ob = ib ^ 1;
+                float2 cb[2][8];
+                tmem_ld16(tm_cb, cb[0]);
+                const float gt = __ldg(g_s + t - 1), wt = __ldg(w_s + t - 1);
+                const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
+                if (t > 1) wait_early(ib);
+                if (!pr.warp_live()) { tmem_wait_ld(cb[0]); dead = true; break; }
+                const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
+                const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
+                if (tid == 0) {
+                    mbar_expect_tx(mb_early + ob_mbar, TX_A_EARLY);
+                    mbar_expect_tx(mb_late + ob_mbar, TX_A_LATE);
                 }
-                hrow[(i * NCH) * CT] = make_float4(Lj[0], Lj[1], Lj[2], Lj[3]);
-                hrow[(i * NCH + 1) * CT] = make_float4(Aj[0], Aj[1], Aj[2], Aj[3]);
-                tmem_wait_ld(cb[i & 1]);
-                if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
+                float4 *hrow = hist4 + (size_t)(t - 1) * HSTEP + (size_t)rank * (BPT * NCH * CT);   // (L_t, At_t) of this thread's butterflies
+                const float2 gshn2 = splat2(gshn);
+                const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
+                const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt);
+                float2 off2 = splat2(off);
+                float tmax = NEG_INF;
 #pragma unroll
-                for (int h = 0; h < K / 2; ++h) {
-                    float2 a[K];
+                for (int i = 0; i < BPT; ++i) {
+                    float2 outL[K / 2], outA[K / 2];
+                    float Lj[K], Aj[K];
 #pragma unroll
                     for (int j = 0; j < K; ++j) {
-                        const float2 du = sub2(cb[i & 1][C::a_idx(j, h)], w2);
-                        a[j] = energy2(du, nl2, kap2, splat2(Lj[j]));
+                        Lj[j] = Lin[(i * K + j) * CT + tid];
+                        Aj[j] = Ain[(i * K + j) * CT + tid];
                     }
-                    const float2 m = max_pairs<K>(a);
-                    float2 pj = ex2f2(sub2(a[0], m));
-                    float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][C::a_idx(0, h)], splat2(Aj[0])));
+                    hrow[(i * NCH) * CT] = make_float4(Lj[0], Lj[1], Lj[2], Lj[3]);
+                    hrow[(i * NCH + 1) * CT] = make_float4(Aj[0], Aj[1], Aj[2], Aj[3]);
+                    tmem_wait_ld(cb[i & 1]);
+                    if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
 #pragma unroll
-                    for (int j = 1; j < K; ++j) {
-                        pj = (j == 3 && (h & 1)) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));   // one in eight on the FP32 pipe
-                        sum = add2(sum, pj);
-                        ax = fma2(pj, fma2(g2, cb[i & 1][C::a_idx(j, h)], splat2(Aj[j])), ax);
-                    }
-                    outL[h] = add2(m, lg2f2(sum));               // the gauge offset is subtracted below
-                    outA[h] = fma2(ax, rcpf2(sum), gshn2);
-                    tmax = max3f(tmax, m.x, m.y);
-                }
-                if (i == 0) {
-                    // everything of the previous step has arrived and every warp of the cluster is done with it:
-                    // the gauge of this step's outputs, and leave to overwrite the buffer that step read
-                    if (t > 1) {
-                        wait_late(ib);
-                        cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
-                        off = rintf(cmax);
-                        off2 = splat2(off);
-                    }
-                    if (!pr.warp_live()) { dead = true; break; }
-                }
-                outL[0] = sub2(outL[0], off2); outL[1] = sub2(outL[1], off2);
-                if (i < 2) {
-                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(push_a[i] + ob_off), "f"(outL[0].x), "f"(outL[0].y),
-                                 "f"(outL[1].x), "f"(outL[1].y) : "memory");
-                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(push_a[i] + ob_off + QC * 4u), "f"(outA[0].x),
-                                 "f"(outA[0].y), "f"(outA[1].x), "f"(outA[1].y) : "memory");
-                } else {
-                    const uint32_t mb = (i == 2 ? peer_early : peer_late) + ob_mbar;
-                    st_async_v4(push_a[i] + ob_off, outL[0].x, outL[0].y, outL[1].x, outL[1].y, mb);
-                    st_async_v4(push_a[i] + ob_off + QC * 4u, outA[0].x, outA[0].y, outA[1].x, outA[1].y, mb);
-                }
-                if (i == 1) {                                     // slots 0 and 1 are in this CTA's buffer: publish them
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_local(mb_early + ob_mbar);
-                }
-            }
-            if (dead) { tmem_wait_ld(cb[0]); tmem_wait_ld(cb[1]); break; }
-            tmax = warp_max(tmax);
-            if (lane == 0) {
+                    for (int h = 0; h < K / 2; ++h) {
+                        float2 a[K];
 #pragma unroll
-                for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, late_of[r] + ob_mbar);
+                        for (int j = 0; j < K; ++j) {
+                            const float2 du = sub2(cb[i & 1][C::a_idx(j, h)], w2);
+                            a[j] = RC ? energy2(du, nl2, kap2, splat2(Lj[j])) : fma2(mul2(du, du), nl2, splat2(Lj[j]));
+                        }
+                        const float2 m = max_pairs<K>(a);
+                        float2 pj = ex2f2(sub2(a[0], m));
+                        float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][C::a_idx(0, h)], splat2(Aj[0])));
+#pragma unroll
+                        for (int j = 1; j < K; ++j) {
+                            pj = (j == 3 && (h & 1)) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));   // one in eight on the FP32 pipe
+                            sum = add2(sum, pj);
+                            ax = fma2(pj, fma2(g2, cb[i & 1][C::a_idx(j, h)], splat2(Aj[j])), ax);
+                        }
+                        outL[h] = add2(m, lg2f2(sum));               // the gauge offset is subtracted below
+                        outA[h] = fma2(ax, rcpf2(sum), gshn2);
+                        tmax = max3f(tmax, m.x, m.y);
+                    }
+                    if (i == 0) {
+                        // everything of the previous step has arrived and every warp of the cluster is done with it:
+                        // the gauge of this step's outputs, and leave to overwrite the buffer that step read
+                        if (t > 1) {
+                            wait_late(ib);
+                            cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
+                            off = rintf(cmax);
+                            off2 = splat2(off);
+                        }
+                        if (!pr.warp_live()) { dead = true; break; }
+                    }
+                    outL[0] = sub2(outL[0], off2); outL[1] = sub2(outL[1], off2);
+                    if (i < 2) {
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(push_a[i] + ob_off), "f"(outL[0].x), "f"(outL[0].y),
+                                     "f"(outL[1].x), "f"(outL[1].y) : "memory");
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(push_a[i] + ob_off + QC * 4u), "f"(outA[0].x),
+                                     "f"(outA[0].y), "f"(outA[1].x), "f"(outA[1].y) : "memory");
+                    } else {
+                        const uint32_t mb = (i == 2 ? peer_early : peer_late) + ob_mbar;
+                        st_async_v4(push_a[i] + ob_off, outL[0].x, outL[0].y, outL[1].x, outL[1].y, mb);
+                        st_async_v4(push_a[i] + ob_off + QC * 4u, outA[0].x, outA[0].y, outA[1].x, outA[1].y, mb);
+                    }
+                    if (i == 1) {                                     // slots 0 and 1 are in this CTA's buffer: publish them
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_local(mb_early + ob_mbar);
+                    }
+                }
+                if (dead) { tmem_wait_ld(cb[0]); tmem_wait_ld(cb[1]); break; }
+                tmax = warp_max(tmax);
+                if (lane == 0) {
+#pragma unroll
+                    for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, late_of[r] + ob_mbar);
+                }
+                O += (int)off;
+                if (tid == 0) O_s[t + 1] = O;
+                __syncwarp();
+                if (lane == 0) {                                     // this warp has read all its inputs and written its outputs
+                    mbar_arrive_local(mb_late + ob_mbar);
+                    mbar_arrive_remote(peer_late + ob_mbar);
+                }
+                ib = ob;
             }
-            O += (int)off;
-            if (tid == 0) O_s[t + 1] = O;
-            __syncwarp();
-            if (lane == 0) {                                     // this warp has read all its inputs and written its outputs
-                mbar_arrive_local(mb_late + ob_mbar);
-                mbar_arrive_remote(peer_late + ob_mbar);
+            };
+            if (recentre) alpha_sweep(std::true_type{}); else alpha_sweep(std::false_type{});
+            // ================= log2 Z
+            wait_early(ib);
+            wait_late(ib);
+            cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
+            {
+                const float *Lfin = msg + ib * 2 * QC;
+                float ssum = 0.f;
+                for (int q = tid; q < QC; q += CT) ssum += ex2f(Lfin[q] - cmax);
+                ssum = warp_sum(ssum);
+                if (lane == 0) {
+#pragma unroll
+                    for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
+                }
+                cluster_sync();                                      // log Z exchange
             }
-            ib = ob;
+            lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
+            if (tid == 0) diag_check_finite(p.diag, lsefin);
+            Ofin = O;
+        } else {
+            __syncthreads();                                     // the offsets loaded above
+            Ofin = O_s[n + 1];
+            lsefin = __int_as_float(p.stepO[(size_t)blk * (C::MAX_N + 4) + n + 2]);
         }
-        // ================= log2 Z
-        wait_early(ib);
-        wait_late(ib);
-        cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
-        {
-            const float *Lfin = msg + ib * 2 * QC;
-            float ssum = 0.f;
-            for (int q = tid; q < QC; q += CT) ssum += ex2f(Lfin[q] - cmax);
-            ssum = warp_sum(ssum);
-            if (lane == 0) {
-#pragma unroll
-                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
-            }
-            cluster_sync();                                      // log Z exchange
-        }
-        const float lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
-        if (tid == 0) diag_check_finite(p.diag, lsefin);
-        const int Ofin = O;
         // ================= beta sweep carrying (M, Bt), with the gradient contraction
         {
             const float gshn = -__ldg(g_s + n - 1) * __ldg(sf_s + n - 1);     // M_n = 0, Bt_n = 0 (+ centring shift)
@@ -343,6 +371,8 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                 }
             }
         };
+        auto beta_sweep = [&](auto rc_tag) {
+        constexpr bool RC = decltype(rc_tag)::value;
         for (int t = n; t >= 1 && !dead; --t) {
             const int ob = ib ^ 1;
             float2 cb[2][8];
@@ -399,21 +429,21 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
 #pragma unroll
                     for (int b = 0; b < K; ++b) {
                         d[b] = sub2(cb[pos & 1][C::b_idx(jh, b)], w2);              // du = c - wc
-                        uu[b] = energy2(d[b], nl2, kap2, splat2(Mb[b]));
+                        uu[b] = RC ? energy2(d[b], nl2, kap2, splat2(Mb[b])) : fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
                     }
                     const float2 m = max_pairs<K>(uu);
                     const float2 Ahj = sub2(make_float2(Ah[2 * jh], Ah[2 * jh + 1]), gsh2);
                     const float2 Lhj = make_float2(Lh[2 * jh], Lh[2 * jh + 1]);
                     const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
                     // f (w - c) / T = f delta / T - (f / T) du
-                    const float2 fg = mul2(f, g2), nfi = mul2(f, ngi2), fid = mul2(f, gid2);
+                    const float2 fg = mul2(f, g2), nfi = mul2(f, ngi2), fid = RC ? mul2(f, gid2) : make_float2(0.f, 0.f);
                     if (!acc_ready) { tmem_wait_ld(acc); acc_ready = true; }
                     float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
 #pragma unroll
                     for (int b = 0; b < K; ++b) {
                         const float2 pb = ex2f2(sub2(uu[b], m));
                         const float2 y = fma2(g2, cb[pos & 1][C::b_idx(jh, b)], splat2(Yb[b]));   // h + Bt
-                        const float2 z = fma2(fma2(nfi, d[b], fid), add2(y, Ahj), fg);            // f (g + (w - c) r / T)
+                        const float2 z = fma2(RC ? fma2(nfi, d[b], fid) : mul2(nfi, d[b]), add2(y, Ahj), fg);   // f (g + (w - c) r / T)
                         sum = add2(sum, pb);
                         ya = fma2(pb, y, ya);
                         zs = fma2(pb, z, zs);
@@ -474,6 +504,8 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                 st_async_f32(part_dst + (uint32_t)(ob * 128 + (lane >> 3)) * 4u, s3, late_of[0] + ob_mbar);
             ib = ob;
         }
+        };
+        if (recentre) beta_sweep(std::true_type{}); else beta_sweep(std::false_type{});
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         if (!dead) {
             wait_early(ib);
@@ -496,8 +528,9 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
             for (int jh = 0; jh < K / 2; ++jh)
 #pragma unroll
                 for (int b = 0; b < K; ++b) {
-                    gc[(size_t)(2 * jh) * C::Q + (size_t)x * K + b] = acc[C::b_idx(jh, b)].x;
-                    gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[C::b_idx(jh, b)].y;
+                    float *g0 = gc + (size_t)(2 * jh) * C::Q + (size_t)x * K + b, *g1 = gc + (size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b;
+                    *g0 = BETA_ONLY ? *g0 + acc[C::b_idx(jh, b)].x : acc[C::b_idx(jh, b)].x;
+                    *g1 = BETA_ONLY ? *g1 + acc[C::b_idx(jh, b)].y : acc[C::b_idx(jh, b)].y;
                 }
         }
     }
