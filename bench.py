@@ -282,7 +282,8 @@ def qat_loop_leg(ctx, dev, flush, steps=4):
             ms.append(e0.elapsed_time(e1)); losses.append(float(loss))
     nb = W.shape[0]
     return {"workload": wl.name, "blocks": nb, "steps": steps, "T": [temps[0], temps[-1]], "ms_per_step": float(np.mean(ms)),
-            "edges_per_s": 2 * nb * wl.steps * wl.S * wl.K / (float(np.mean(ms)) * 1e-3), "loss": losses,
+            "edges_per_s": 2 * nb * wl.steps * wl.S * wl.K / (float(np.mean(ms)) * 1e-3),
+            "stand_in_loss_per_step": losses, "note": "T falls from step to step, so the losses of different steps are not comparable",
             "updates": "latent weights and codebook table, Adam, inside bcjr_backward_adam"}
 
 

@@ -22,7 +22,6 @@ typedef struct {
     double sm_clock_mhz;              /* clock the register-only chains ran at (events vs. cycle counter) */
     double ex2_per_clk_sm;            /* ex2.approx results per clock per SM */
     double lg2_per_clk_sm;
-    double rcp_per_clk_sm;
     double fma_f32_per_clk_sm;        /* scalar fma.f32 thread-instructions per clock per SM */
     double fma_f32x2_per_clk_sm;      /* packed fma.f32x2 thread-instructions (pairs) per clock per SM */
     double ex2_gops;                  /* ex2 results per second over the whole GPU, 1e9/s */

@@ -115,6 +115,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity)
         : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
     return ok != 0;
 }
+// The same probe, but the thread may be parked by the hardware for up to `ns` nanoseconds while the phase is
+// incomplete: a waiting warp then costs the SM's schedulers a handful of instructions instead of a busy loop.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t mbar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(mbar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
 // Device-side waits are bounded by wall time (the context's wait budget, default 2 s): a wait that
 // runs out raises BCJR_ETIMEOUT (-6) in the diagnostics and sets the CTA-wide abort flag; the kernel
 // then runs to its end on meaningless numbers instead of hanging (see Proto below).
@@ -175,9 +185,9 @@ struct Proto {
         if (!live) return;
         if (*abort_flag) { live = 0u; return; }
         unsigned long long t0 = 0;
-        for (int i = 0; i < (1 << 24); ++i) {                    // hard cap besides the time budget
-            if (mbar_try_wait(mbar, parity)) return;
-            if ((i & 1023) == 1023) {
+        for (int i = 0; i < (1 << 22); ++i) {                    // hard cap besides the time budget
+            if (mbar_try_wait_parked(mbar, parity, 4000u)) return;
+            if ((i & 63) == 63) {
                 const unsigned long long now = global_timer_ns();
                 if (t0 == 0) t0 = now;
                 if (*abort_flag || now - t0 > diag->wait_limit_ns) break;
@@ -262,29 +272,11 @@ __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
 // log2-potential of a pair of states plus a message: du (du (-lam2) + kap) + msg, see step_energy
 __device__ __forceinline__ float2 energy2(float2 du, float2 nl2, float2 kap2, float2 msg)
 {
-#if defined(BCJR_AB_PLAIN_ENERGY)
-    return fma2(mul2(du, du), nl2, msg);          // timing experiment only: the plain square (exact when delta = 0)
-#elif defined(BCJR_AB_AAF_ENERGY)
-    return fma2(du, sub2(kap2, du), msg);         // timing experiment only: add, add, fma (needs a pre-scaled table)
-#else
     return fma2(du, fma2(du, nl2, kap2), msg);
-#endif
 }
 __device__ __forceinline__ float2 ex2f2(float2 a) { return make_float2(ex2f(a.x), ex2f(a.y)); }
 __device__ __forceinline__ float2 lg2f2(float2 a) { return make_float2(lg2f(a.x), lg2f(a.y)); }
-#ifdef BCJR_AB_RCP_NR
-// timing experiment: 1/x for x in [1, K] on the FP32 pipe: linear seed in the exponent domain + three Newton steps
-__device__ __forceinline__ float2 rcpf2(float2 a)
-{
-    float2 y = make_float2(__int_as_float(0x7EF311C7 - __float_as_int(a.x)), __int_as_float(0x7EF311C7 - __float_as_int(a.y)));
-    const float2 one = make_float2(1.f, 1.f), na = make_float2(-a.x, -a.y);
-#pragma unroll
-    for (int it = 0; it < 3; ++it) y = fma2(y, fma2(na, y, one), y);
-    return y;
-}
-#else
 __device__ __forceinline__ float2 rcpf2(float2 a) { return make_float2(rcpf(a.x), rcpf(a.y)); }
-#endif
 // 2^x for x <= 0 on the FP32 pipe (no special-function instruction): x = n + f with n the nearest
 // integer and |f| <= 1/2, 2^f by the degree-5 interpolant at the Chebyshev nodes of [-1/2, 1/2] (relative
 // error 2.4e-7 evaluated in float32, about that of ex2.approx), the

@@ -48,8 +48,10 @@ struct SkewCfg {
     static constexpr int SLOTS = CL * NWARP;
     static constexpr int NCH = 2 * K / 4;                      // 16-byte chunks per butterfly and thread: K values of L, K of At
     static constexpr int MAX_N = 1024;
-    static constexpr int OFF_MSG = 0;                          // [2 parity][2 arrays][QC]
-    static constexpr int OFF_RING = OFF_MSG + 4 * QC;          // float4 [BPT][NCH][THREADS]
+    static constexpr int BUF = 2 * QC + 16;                    // floats of one message buffer: (L, At), or the two planes of (M, Bt) pairs + padding
+    static constexpr int PLANE = NBC + 4;                      // float4 between the planes: a half-warp's 8-byte stores then reach all 32 banks
+    static constexpr int OFF_MSG = 0;                          // [2 parity][BUF]
+    static constexpr int OFF_RING = OFF_MSG + 2 * BUF;         // float4 [BPT][NCH][THREADS]
     static constexpr int OFF_O = OFF_RING + BPT * NCH * THREADS * 4;   // int [MAX_N + 2]
     static constexpr int OFF_WMAX = OFF_O + MAX_N + 2 + 2;     // [2][32]
     static constexpr int OFF_PART = OFF_WMAX + 64;             // [2][32][4]
@@ -86,7 +88,8 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
     using C = SkewCfg;
     constexpr int K = C::K, NBC = C::NBC, QC = C::QC, BPT = C::BPT, NWARP = C::NWARP, CT = C::THREADS;
     constexpr int CL = C::CL, SLOTS = C::SLOTS, NCH = C::NCH;
-    constexpr uint32_t BUF_BYTES = 2u * QC * 4u;                 // (L, At) of one parity
+    constexpr uint32_t BUF_BYTES = (uint32_t)C::BUF * 4u;        // one parity
+    constexpr int PLANE = C::PLANE;
     // bytes the peer sends into a buffer of this CTA per step: alpha, one slot = 512 threads x (16 + 16) bytes;
     // beta, one slot = 512 threads x 2 outputs x 8 bytes; the gauge slots (32 x 4) and, on CTA 0, the posterior
     // sums (32 x 12) travel with the "late" part
@@ -154,8 +157,8 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
         {
             const int bin = x & 3;
             const int xl = ((int)rank << 11) | (x >> 2), xr = ((int)peer << 11) | (x >> 2);     // consumer butterflies of outputs j = (CTA, 0)
-            const uint32_t al = msg_u32 + (uint32_t)(((bin >> 1) * NBC + C::slot_of(xl) * CT + C::tid_of(xl)) * 4 + (bin & 1) * 2) * 4u;
-            const uint32_t ar = msg_u32 + (uint32_t)(((bin >> 1) * NBC + C::slot_of(xr) * CT + C::tid_of(xr)) * 4 + (bin & 1) * 2) * 4u;
+            const uint32_t al = msg_u32 + (uint32_t)(((bin >> 1) * PLANE + C::slot_of(xl) * CT + C::tid_of(xl)) * 4 + (bin & 1) * 2) * 4u;
+            const uint32_t ar = msg_u32 + (uint32_t)(((bin >> 1) * PLANE + C::slot_of(xr) * CT + C::tid_of(xr)) * 4 + (bin & 1) * 2) * 4u;
             push_bl[i] = al;
             push_br[i] = mapa_u32(ar, peer);
         }
@@ -222,7 +225,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                 const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
                 if (t > 1) wait_early(ib);
                 if (!pr.warp_live()) { tmem_wait_ld(cb[0]); dead = true; break; }
-                const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
+                const float *Lin = msg + ib * C::BUF, *Ain = Lin + QC;
                 const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
                 if (tid == 0) {
                     mbar_expect_tx(mb_early + ob_mbar, TX_A_EARLY);
@@ -317,7 +320,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
             wait_late(ib);
             cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
             {
-                const float *Lfin = msg + ib * 2 * QC;
+                const float *Lfin = msg + ib * C::BUF;
                 float ssum = 0.f;
                 for (int q = tid; q < QC; q += CT) ssum += ex2f(Lfin[q] - cmax);
                 ssum = warp_sum(ssum);
@@ -338,7 +341,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
         // ================= beta sweep carrying (M, Bt), with the gradient contraction
         {
             const float gshn = -__ldg(g_s + n - 1) * __ldg(sf_s + n - 1);     // M_n = 0, Bt_n = 0 (+ centring shift)
-            for (int f = tid; f < 2 * QC; f += CT) msg[ib * 2 * QC + f] = (f & 1) ? gshn : 0.f;
+            for (int f = tid; f < C::BUF; f += CT) msg[ib * C::BUF + f] = (f & 1) ? gshn : 0.f;
         }
 #pragma unroll
         for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, beta pairing
@@ -386,7 +389,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
             if (t < n) wait_early(ib);
             if (!pr.warp_live()) { tmem_wait_ld(cb[0]); dead = true; break; }
             P += (int)offM;                                         // offsets carried by this step's inputs M_t
-            const float4 *MBin = reinterpret_cast<const float4 *>(msg + ib * 2 * QC);
+            const float4 *MBin = reinterpret_cast<const float4 *>(msg + ib * C::BUF);
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
             if (tid == 0) {
                 mbar_expect_tx(mb_early + ob_mbar, TX_B_EARLY);
@@ -414,7 +417,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                 float Mb[K], Yb[K];
 #pragma unroll
                 for (int e = 0; e < K / 2; ++e) {
-                    const float4 v = MBin[e * NBC + i * CT + tid];
+                    const float4 v = MBin[e * PLANE + i * CT + tid];
                     Mb[2 * e] = v.x; Yb[2 * e] = v.y; Mb[2 * e + 1] = v.z; Yb[2 * e + 1] = v.w;
                 }
                 float2 acc[8];
