@@ -244,7 +244,7 @@ def workload_leg(ctx, name, blocks_cap, dev, flush, peak_gops):
     ms = float(np.mean(step_ms))
     leg = {"workload": wl.name, "blocks": r.nblocks, "Lb": wl.Lb, "k": wl.k, "V": wl.V, "n": wl.n, "T": wl.T,
            "ms_per_step": ms, "fwd_ms": fwd_ms / 2, "bwd_ms": bwd_ms / 2, "edges_per_s": r.edges_per_step / (ms * 1e-3),
-           "path": "large-trellis kernels" if diag.last_path else "generic kernels",
+           "path": {0: "generic kernels", 1: "large-trellis kernels", 2: "one warp per block"}[diag.last_path],
            "max_posterior_defect": diag.max_posterior_defect}
     leg.update(mufu_fractions(wl, r.state_steps, fwd_ms / 2, bwd_ms / 2, ms, peak_gops))
     del r
@@ -516,7 +516,7 @@ def main():
                           "Lb": wl.Lb, "k": wl.k, "V": wl.V, "T": [temps_timed[0], temps_timed[-1]],
                           "T_schedule": "geometric over the timed steps, warm-up at the first value" if annealed else "constant",
                           "l2": "256 MB flush write between timed steps; per-step working set >> L2",
-                          "path": "cluster" if diag.last_path else "generic"},
+                          "path": {0: "generic", 1: "cluster", 2: "warp"}[diag.last_path]},
                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": base,
                "breakdown": {"fwd_ms_per_step": fwd_ms / args.steps, "bwd_ms_per_step": bwd_ms / args.steps,
                              "viterbi": vit, "qat_update": upd, "max_posterior_defect": diag.max_posterior_defect,

@@ -47,7 +47,7 @@ typedef struct {
     float max_posterior_defect;   /* max over blocks and steps of |sum_s gamma_t(s) - 1| (Eq. 6) */
     float max_logz_mismatch;      /* max |log Z (alpha side) - log Z (beta side)|, natural log */
     int32_t kernel_launches;      /* kernels launched by this context since creation */
-    int32_t last_path;            /* 0 = generic kernels, 1 = cluster kernels used by the last call */
+    int32_t last_path;            /* kernels used by the last call: 0 = generic, 1 = large-trellis (Lb = 16), 2 = one warp per block (Lb = 11..13, k = 2) */
 } bcjr_diag;
 
 /* Limits: 1 <= k <= 4, k <= Lb <= 16, Lb - k <= 14, n >= 1, T > 0 and finite.
@@ -57,8 +57,9 @@ typedef struct {
  *                         for n <= 1024.  Longer blocks step down: backward 1024 < n <= 2048 runs the
  *                         four-CTA register kernel (about 1.7x slower per weight), and anything longer
  *                         the generic one-CTA kernels (more than 10x slower per weight at Lb = 16).
- *   Lb <= 14 (k = 1..4):  shared-memory kernels, one CTA per block, several blocks per SM.
- *   everything else:      generic kernels.
+ *   Lb = 11..13, k = 2:   one warp per block, sixteen (forward) or eight (backward) blocks per SM at Lb = 12, table in
+ *                         tensor memory; any n.
+ *   everything else:      generic kernels, one CTA per block (also "path" = 1).
  * Block lengths of a few hundred weights (the paper uses 256) are the intended range. */
 
 /* Creates a context bound to CUDA device `device_ordinal`.  *out is owned by the caller

@@ -21,6 +21,7 @@
 #include "bcjr_skew.cuh"
 #include "bcjr_alpha.cuh"
 #include "bcjr_ckpt.cuh"
+#include "bcjr_warp.cuh"
 #include "bcjr_viterbi.cuh"
 #endif
 
@@ -599,6 +600,78 @@ bcjr_status launch_fwd_ckpt(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
     return BCJR_OK;
 }
 
+// Mid-size trellises (Lb = 11 .. 13, k = 2): one warp per block, table (and accumulators) in tensor memory.
+inline bool warp_supported(int Lb, int k) { return k == 2 && Lb >= 11 && Lb <= 13; }
+
+template <int LB>
+bcjr_status launch_fwd_warp(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    using C = WarpCfg<LB, false>;
+    CU(cudaFuncSetAttribute(fwd_warp_kernel<LB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
+    int64_t grid = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    const int64_t need = (p.B + C::NWARP - 1) / C::NWARP;
+    if (grid > need) grid = need;
+    const size_t warps = (size_t)grid * C::NWARP;
+    bcjr_status rc;
+    if ((rc = ensure(ctx, ctx->hist, warps * p.n * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, warps * ((size_t)p.n + 2) * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
+    fwd_warp_kernel<LB><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
+template <int LB, bool ACC>
+bcjr_status launch_bwd_warp(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    using C = WarpCfg<LB, true>;
+    CU(cudaFuncSetAttribute(bwd_warp_kernel<LB, ACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
+    int64_t grid = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    const int64_t need = (p.B + C::NWARP - 1) / C::NWARP;
+    if (grid > need) grid = need;
+    const size_t warps = (size_t)grid * C::NWARP;
+    bcjr_status rc;
+    if ((rc = ensure(ctx, ctx->hist, warps * p.n * 2 * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, warps * ((size_t)p.n + 2) * 4))) return rc;
+    if (ACC && (rc = ensure(ctx, ctx->gc_part, warps * C::S * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    p.gc_part = ACC ? (float *)ctx->gc_part.ptr : nullptr;
+    if (ctx->cb_computed) p.cb = nullptr;
+    bwd_warp_kernel<LB, ACC><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    if (ACC) {
+        reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, (int)warps, C::S, grad_codebook);
+        ctx->launches += 1;
+        CU(cudaGetLastError());
+    }
+    return BCJR_OK;
+}
+
+bcjr_status launch_fwd_warp_any(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    switch (p.Lb) {
+        case 11: return launch_fwd_warp<11>(ctx, p, st);
+        case 12: return launch_fwd_warp<12>(ctx, p, st);
+        default: return launch_fwd_warp<13>(ctx, p, st);
+    }
+}
+
+bcjr_status launch_bwd_warp_any(bcjr_ctx *ctx, BwdParams p, float *gc, cudaStream_t st)
+{
+    switch (p.Lb) {
+        case 11: return gc ? launch_bwd_warp<11, true>(ctx, p, gc, st) : launch_bwd_warp<11, false>(ctx, p, gc, st);
+        case 12: return gc ? launch_bwd_warp<12, true>(ctx, p, gc, st) : launch_bwd_warp<12, false>(ctx, p, gc, st);
+        default: return gc ? launch_bwd_warp<13, true>(ctx, p, gc, st) : launch_bwd_warp<13, false>(ctx, p, gc, st);
+    }
+}
+
 bcjr_status launch_fwd_cluster(bcjr_ctx *ctx, FwdParams p, int k, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
@@ -779,10 +852,13 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
         rc = launch_fwd_cluster(ctx, p, k, st);
         if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { use_cluster = false; rc = BCJR_OK; }   // e.g. n too long
     }
+    bool use_warp = !use_cluster && ctx->opt_path == 0 && warp_supported(Lb, k);
+    if (use_warp) rc = launch_fwd_warp_any(ctx, p, st);
 #else
     if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
+    const bool use_warp = false;
 #endif
-    if (!use_cluster) {
+    if (!use_cluster && !use_warp) {
         switch (k) {
             case 1: rc = launch_fwd_generic<1>(ctx, p, st); break;
             case 2: rc = launch_fwd_generic<2>(ctx, p, st); break;
@@ -791,7 +867,7 @@ bcjr_status bcjr_soft_quantize(bcjr_ctx *ctx, const float *W, const float *codeb
         }
     }
     if (rc) return rc;
-    ctx->last_path = use_cluster ? 1 : 0;
+    ctx->last_path = use_cluster ? 1 : use_warp ? 2 : 0;
     ctx->W = W; ctx->cb = codebook; ctx->Lb = Lb; ctx->k = k; ctx->n = n; ctx->B = num_blocks; ctx->T = T;
     ctx->V = 1;
     ctx->have_fwd = true;
@@ -850,10 +926,13 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
         rc = launch_bwd_cluster(ctx, p, ctx->k, grad_codebook, st);
         if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { use_cluster = false; rc = BCJR_OK; }
     }
+    const bool use_warp = !use_cluster && ctx->opt_path == 0 && warp_supported(ctx->Lb, ctx->k);
+    if (use_warp) rc = launch_bwd_warp_any(ctx, p, grad_codebook, st);
 #else
     if (ctx->opt_path == 2) return BCJR_EUNSUPPORTED;
+    const bool use_warp = false;
 #endif
-    if (!use_cluster) {
+    if (!use_cluster && !use_warp) {
         switch (ctx->k) {
             case 1: rc = launch_bwd_generic<1>(ctx, p, grad_codebook, st); break;
             case 2: rc = launch_bwd_generic<2>(ctx, p, grad_codebook, st); break;
@@ -862,7 +941,7 @@ bcjr_status bcjr_backward(bcjr_ctx *ctx, const float *grad_soft, float *grad_W, 
         }
     }
     if (rc) return rc;
-    ctx->last_path = use_cluster ? 1 : 0;
+    ctx->last_path = use_cluster ? 1 : use_warp ? 2 : 0;
     return BCJR_OK;
 }
 

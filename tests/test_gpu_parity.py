@@ -92,6 +92,25 @@ def test_shapes_generic_path(ctx, Lb, k, n, B, T):
         ctx.set_option("path", 0)
 
 
+@pytest.mark.parametrize("Lb,n,B,T", [(11, 33, 37, 0.3), (12, 1, 3, 0.5), (12, 2, 70, 0.2), (12, 256, 40, 0.1), (13, 50, 9, 0.05),
+                                      (13, 7, 1, 0.3), (12, 1500, 2, 0.2), (11, 64, 300, 0.02)])
+def test_one_warp_per_block_kernels(ctx, Lb, n, B, T):
+    # Lb = 11..13, k = 2: a warp runs a block alone (no CTA barrier in the sweeps), sixteen or eight blocks per CTA;
+    # ragged block counts leave warps without work, long blocks exercise the history stream
+    k = 2
+    W, c, g = _rand(n, Lb, B, seed=1300 + Lb + n)
+    got = _check_all(ctx, W, c, g, Lb, k, T, f"warp per block Lb={Lb} n={n} B={B}")
+    assert got["diag"].last_path == 2 and got["diag"].device_status == 0
+    ctx.set_option("max_ctas", 2)                       # fewer CTAs than the work needs: every warp loops over blocks
+    try:
+        again = parity.gpu_forward_backward(ctx, W, c, g, Lb, k, T)
+    finally:
+        ctx.set_option("max_ctas", 0)
+    np.testing.assert_array_equal(again["soft"], got["soft"])
+    np.testing.assert_array_equal(again["grad_W"], got["grad_W"])
+    assert parity.rel_inf(again["grad_codebook"], got["grad_codebook"]) < 1e-5
+
+
 def test_more_blocks_than_resident_ctas(ctx):
     # the persistent loop must visit every block exactly once, whatever the grid size
     Lb, k, n, T = 8, 2, 16, 0.3
@@ -386,7 +405,7 @@ def test_checkpointed_history_matches_the_oracle(ctx, k, n, B, m):
     assert parity.rel_inf(got["soft"], plain["soft"]) <= 1e-5
 
 
-@pytest.mark.parametrize("Lb,k,n,B", [(16, 2, 64, 5), (16, 3, 40, 3), (16, 2, 1100, 1), (8, 2, 64, 9), (12, 3, 30, 4)])
+@pytest.mark.parametrize("Lb,k,n,B", [(16, 2, 64, 5), (16, 3, 40, 3), (16, 2, 1100, 1), (8, 2, 64, 9), (12, 3, 30, 4), (12, 2, 30, 21)])
 def test_computed_gaussian_emission(ctx, Lb, k, n, B):
     """codebook = NULL: the emission of Section 3.1, c(s) = Phi^-1((s + 1/2) / S), evaluated by the kernels
     themselves (2^16 states) or read from a table the context writes (other shapes).  The oracle is fed the
