@@ -1,4 +1,4 @@
-// Backward call, first half (2^16 states, k = 2): the alpha sweep carrying (L, At) on ONE CTA per block.
+// Backward call, first half (2^16 states; k = 2, 3): the alpha sweep carrying (L, At) on ONE CTA per block.
 //
 // The backward pass needs gradient accumulators next to the codebook only in its beta sweep.  Its alpha sweep
 // -- the forward messages L_t and the conditional expectations At_t of every step, which the beta sweep reads
@@ -6,8 +6,8 @@
 // one CTA barrier instead of a cluster handshake and a thread has eight butterflies per step instead of four to
 // hide it behind, which is why the forward kernel reaches a higher fraction of the special-function peak than
 // the two-CTA backward kernel.  So the backward call is split: this kernel writes the history of a chunk of
-// blocks (one block per SM), bwd_skew_kernel<ACC, true> then runs the beta sweeps of the same chunk on
-// two-CTA clusters.
+// blocks (one block per SM), bwd_skew_kernel<ACC, true> (k = 2) or bwd_duo_kernel<3, true> (k = 3) then runs the beta
+// sweeps of the same chunk on two-CTA clusters.
 //
 // Messages in place.  (L, At) double-buffered would be 256 KB; here each array has ONE buffer of Q floats.  A
 // butterfly's four inputs have no other reader, so its four outputs overwrite them (output [x|l] takes the place
@@ -26,39 +26,55 @@
 
 namespace bcjr {
 
+template <int KB_>
 struct AlphaCfg {
-    static constexpr int LB = 16, KB = 2, K = 4, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB), QB = LB - KB;
-    static constexpr int CTHREADS = 512, THREADS = 512, NWARP = 16, BPT = NB / CTHREADS;   // 8 butterflies per thread: x = i * 512 + tid
-    static constexpr int UNITS = 1, HPU = 2;
-    static constexpr int MAX_N = SkewCfg::MAX_N, NROT = QB / KB;   // 7 rotations
+    static constexpr int LB = 16, KB = KB_, K = 1 << KB, S = 1 << LB, Q = S >> KB, NB = S >> (2 * KB), QB = LB - KB;
+    static constexpr int CTHREADS = 512, THREADS = 512, NWARP = 16, BPT = NB / CTHREADS;   // butterflies per thread: x = i * 512 + tid
+    static constexpr int UNITS = K * K / 16, HPU = (K / 2) / UNITS;                       // 16-column table units per butterfly
+    static constexpr int MAX_N = 1024, NROT = QB;              // rotations: k (t-1) mod (Lb - k) takes 7 values at k = 2, all 13 at k = 3
     static constexpr int OFF_L = 0;                            // [Q]
     static constexpr int OFF_A = OFF_L + Q;                    // [Q]
-    static constexpr int OFF_TAB = OFF_A + Q;                  // uint32 [NROT][16]: T_i (8), T_j (4)
+    static constexpr int OFF_TAB = OFF_A + Q;                  // uint32 [NROT][16]: T_i (BPT), T_j (K) from entry 8
     static constexpr int OFF_WMAX = OFF_TAB + NROT * 16;       // [2][32]
     static constexpr int OFF_LZ = OFF_WMAX + 64;               // [32]
     static constexpr int OFF_TMEM = OFF_LZ + 32;
     static constexpr int SMEM_FLOATS = OFF_TMEM + 4;
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static constexpr int AUX_INTS = MAX_N + 4;                 // per block: O_t (t = 1 .. n+1), then the bits of the log2 Z tail
-    __host__ __device__ static constexpr int a_idx(int j, int h) { return 2 * j + h; }
-    __host__ __device__ static constexpr int b_idx(int jh, int b) { return 4 * jh + b; }
+    static_assert(BPT * K * K == 128 && BPT <= 8 && K <= 8, "a thread's table slice fills its 128 tensor-memory columns");
+    __host__ __device__ static constexpr int a_idx(int j, int h) { return K == 4 ? 2 * j + h : j; }
+    __host__ __device__ static constexpr int b_idx(int jh, int b) { return K == 4 ? 4 * jh + b : b; }
     __host__ __device__ static constexpr uint32_t rotr(uint32_t v, int r) { return ((v >> r) | (v << (QB - r))) & ((1u << QB) - 1u); }
-    // bank bits ^= M * (upper bits): columns e0..e4 for index bits 5..9, then e0+e1, e2, e0+e3, e4 for bits 10..13
+    // bank bits ^= M * (upper index bits).  The columns of M were chosen (by hand at k = 2, by search at k = 3; both
+    // checked exhaustively) so that at every rotation the five index bits that vary across a warp reach five
+    // independent vectors: e0..e4 for index bits 5..9, then e0+e1, e2, e0+e3, e4 for bits 10..13 (k = 2, 14 index bits)
+    // or e0+e2, e1+e3, e0+e1+e4 for bits 10..12 (k = 3, 13 index bits).
     __host__ __device__ static constexpr uint32_t swz(uint32_t v)
     {
         const uint32_t h = v >> 10;
-        return v ^ ((v >> 5) & 31u) ^ ((h & 1u) * 3u) ^ ((h & 2u) << 1) ^ (((h >> 2) & 1u) * 9u) ^ ((h & 8u) << 1);
+        const uint32_t top = KB == 2 ? ((h & 1u) * 3u) ^ ((h & 2u) << 1) ^ (((h >> 2) & 1u) * 9u) ^ ((h & 8u) << 1)
+                                     : ((h & 1u) * 5u) ^ (((h >> 1) & 1u) * 10u) ^ (((h >> 2) & 1u) * 19u);
+        return v ^ ((v >> 5) & 31u) ^ top;
     }
     __host__ __device__ static constexpr uint32_t slot(uint32_t q, int r) { return swz(rotr(q, r)); }
 };
 
-template <bool UNUSED = false>
-__global__ void __launch_bounds__(AlphaCfg::THREADS, 1) bwd_alpha_kernel(BwdParams p)
+// HL: the beta kernel's history layout (SkewCfg at k = 2, DuoCfg<3> at k = 3): float4 index of chunk 0 of butterfly x inside a step
+template <int KB>
+__device__ __forceinline__ int beta_history_pos(int x)
 {
-    using C = AlphaCfg;
-    using SK = SkewCfg;
-    constexpr int K = C::K, Q = C::Q, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS;
-    constexpr ptrdiff_t HSTEP = (ptrdiff_t)SK::CL * SK::BPT * SK::NCH * SK::THREADS;     // float4 per step of the beta kernel's layout
+    if (KB == 2) return SkewCfg::rank_of(x) * (SkewCfg::BPT * SkewCfg::NCH * SkewCfg::THREADS) + SkewCfg::slot_of(x) * SkewCfg::NCH * SkewCfg::THREADS + SkewCfg::tid_of(x);
+    using D = DuoCfg<3>;                                        // x = rank * NBC + tid, one butterfly per thread
+    return (x / D::NBC) * (D::BPT * D::NCH * D::THREADS) + (x % D::NBC);
+}
+
+template <int KB>
+__global__ void __launch_bounds__(AlphaCfg<KB>::THREADS, 1) bwd_alpha_kernel(BwdParams p)
+{
+    using C = AlphaCfg<KB>;
+    constexpr int K = C::K, Q = C::Q, BPT = C::BPT, NWARP = C::NWARP, CT = C::CTHREADS, UNITS = C::UNITS, HPU = C::HPU, NU = BPT * UNITS;
+    constexpr ptrdiff_t HSTEP = 2 * Q / 4;                      // float4 per step: (L, At) of every group
+    constexpr int HCH = CT;                                     // float4 between the 16-byte chunks of a butterfly (both layouts: 512 threads)
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = p.n;
@@ -73,10 +89,10 @@ __global__ void __launch_bounds__(AlphaCfg::THREADS, 1) bwd_alpha_kernel(BwdPara
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
 
     if (tid < C::NROT * 16) {
-        const int ri = tid >> 4, e = tid & 15, r = C::KB * ri;
+        const int r = tid >> 4, e = tid & 15;                            // table row = the rotation itself
         uint32_t v = 0;
-        if (e < 8) v = C::slot((uint32_t)e << 9, r);                    // T_i: butterfly bits above the thread index
-        else if (e < 12) v = C::slot((uint32_t)(e - 8) << 12, r);       // T_j: the input's branch bits
+        if (e < BPT) v = C::slot((uint32_t)e << 9, r);                   // T_i: butterfly bits above the thread index
+        else if (e >= 8 && e < 8 + K) v = C::slot((uint32_t)(e - 8) << (C::QB - KB), r);   // T_j: the input's branch bits
         tab[tid] = v;
     }
     if (warp == 0) tmem_alloc_512(smem_u32(const_cast<uint32_t *>(tmem_slot)));
@@ -89,7 +105,7 @@ __global__ void __launch_bounds__(AlphaCfg::THREADS, 1) bwd_alpha_kernel(BwdPara
 #pragma unroll
     for (int i = 0; i < BPT; ++i) {
         const int x = i * CT + tid;
-        hpos[i] = SK::rank_of(x) * (SK::BPT * SK::NCH * SK::THREADS) + SK::slot_of(x) * SK::NCH * SK::THREADS + SK::tid_of(x);
+        hpos[i] = beta_history_pos<KB>(x);
     }
 
     for (int64_t blk = blockIdx.x; blk < p.B; blk += gridDim.x) {
@@ -108,14 +124,14 @@ __global__ void __launch_bounds__(AlphaCfg::THREADS, 1) bwd_alpha_kernel(BwdPara
         }
         const bool recentre = __syncthreads_or(outside) != 0;
 #pragma unroll
-        for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(16 * i), false);
+        for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, i * CT + tid, tm + (uint32_t)(K * K * i), false);
         tmem_wait_st();
         int O = 0;
         float off = 0.f, cmax = 0.f;
         compute_barrier(CT);
         auto alpha_sweep = [&](auto rc_tag) {
             constexpr bool RC = decltype(rc_tag)::value;
-            int ri = 0;                                               // (t - 1) mod 7
+            int r = 0;                                                // k (t - 1) mod (Lb - k)
             for (int t = 1; t <= n; ++t) {
                 const int cur = (t - 1) & 1;
                 float2 cb[2][8];
@@ -128,8 +144,8 @@ __global__ void __launch_bounds__(AlphaCfg::THREADS, 1) bwd_alpha_kernel(BwdPara
                 }
                 const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
                 const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt), off2 = splat2(off), gshn2 = splat2(gshn);
-                const uint32_t *tb = tab + ri * 16;
-                const uint32_t st = C::slot((uint32_t)tid, C::KB * ri);
+                const uint32_t *tb = tab + r * 16;
+                const uint32_t st = C::slot((uint32_t)tid, r);
                 uint32_t TJ[K];
 #pragma unroll
                 for (int j = 0; j < K; ++j) TJ[j] = tb[8 + j] ^ st;
@@ -144,41 +160,52 @@ __global__ void __launch_bounds__(AlphaCfg::THREADS, 1) bwd_alpha_kernel(BwdPara
                         Lj[j] = Ls[ti ^ TJ[j]];
                         Aj[j] = As[ti ^ TJ[j]];
                     }
-                    hrow[hpos[i]] = make_float4(Lj[0], Lj[1], Lj[2], Lj[3]);
-                    hrow[hpos[i] + SK::THREADS] = make_float4(Aj[0], Aj[1], Aj[2], Aj[3]);
-                    tmem_wait_ld(cb[i & 1]);
-                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
+#pragma unroll
+                    for (int q = 0; q < K / 4; ++q) {
+                        hrow[hpos[i] + q * HCH] = make_float4(Lj[4 * q], Lj[4 * q + 1], Lj[4 * q + 2], Lj[4 * q + 3]);
+                        hrow[hpos[i] + (K / 4 + q) * HCH] = make_float4(Aj[4 * q], Aj[4 * q + 1], Aj[4 * q + 2], Aj[4 * q + 3]);
+                    }
                     float2 outL[K / 2], outA[K / 2];
 #pragma unroll
-                    for (int h = 0; h < K / 2; ++h) {
-                        float2 a[K];
+                    for (int u = 0; u < UNITS; ++u) {
+                        const int g = i * UNITS + u;
+                        tmem_wait_ld(cb[g & 1]);
+                        if (g + 1 < NU) tmem_ld16(tm + 16u * (g + 1), cb[(g + 1) & 1]);
 #pragma unroll
-                        for (int j = 0; j < K; ++j) {
-                            const float2 du = sub2(cb[i & 1][C::a_idx(j, h)], w2);
-                            a[j] = RC ? energy2(du, nl2, kap2, splat2(Lj[j])) : fma2(mul2(du, du), nl2, splat2(Lj[j]));
-                        }
-                        const float2 m = max_pairs<K>(a);
-                        float2 pj = ex2f2(sub2(a[0], m));
-                        float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][C::a_idx(0, h)], splat2(Aj[0])));
+                        for (int hh = 0; hh < HPU; ++hh) {
+                            const int h = u * HPU + hh;
+                            float2 a[K];
 #pragma unroll
-                        for (int j = 1; j < K; ++j) {
-                            pj = (j == 3) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));   // one in four on the FP32 pipe
-                            sum = add2(sum, pj);
-                            ax = fma2(pj, fma2(g2, cb[i & 1][C::a_idx(j, h)], splat2(Aj[j])), ax);
+                            for (int j = 0; j < K; ++j) {
+                                const float2 du = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
+                                a[j] = RC ? energy2(du, nl2, kap2, splat2(Lj[j])) : fma2(mul2(du, du), nl2, splat2(Lj[j]));
+                            }
+                            const float2 m = max_pairs<K>(a);
+                            float2 pj = ex2f2(sub2(a[0], m));
+                            float2 sum = pj, ax = mul2(pj, fma2(g2, cb[g & 1][C::a_idx(0, hh)], splat2(Aj[0])));
+#pragma unroll
+                            for (int j = 1; j < K; ++j) {
+                                pj = (KB == 2 && j == 3) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));   // k = 2: one in four on the FP32 pipe
+                                sum = add2(sum, pj);
+                                ax = fma2(pj, fma2(g2, cb[g & 1][C::a_idx(j, hh)], splat2(Aj[j])), ax);
+                            }
+                            outL[h] = add2(sub2(m, off2), lg2f2(sum));
+                            outA[h] = fma2(ax, rcpf2(sum), gshn2);
+                            tmax = max3f(tmax, m.x, m.y);
                         }
-                        outL[h] = add2(sub2(m, off2), lg2f2(sum));
-                        outA[h] = fma2(ax, rcpf2(sum), gshn2);
-                        tmax = max3f(tmax, m.x, m.y);
                     }
                     // output [x|l] takes the place of input [l|x]
-                    Ls[ti ^ TJ[0]] = outL[0].x; Ls[ti ^ TJ[1]] = outL[0].y; Ls[ti ^ TJ[2]] = outL[1].x; Ls[ti ^ TJ[3]] = outL[1].y;
-                    As[ti ^ TJ[0]] = outA[0].x; As[ti ^ TJ[1]] = outA[0].y; As[ti ^ TJ[2]] = outA[1].x; As[ti ^ TJ[3]] = outA[1].y;
+#pragma unroll
+                    for (int h = 0; h < K / 2; ++h) {
+                        Ls[ti ^ TJ[2 * h]] = outL[h].x; Ls[ti ^ TJ[2 * h + 1]] = outL[h].y;
+                        As[ti ^ TJ[2 * h]] = outA[h].x; As[ti ^ TJ[2 * h + 1]] = outA[h].y;
+                    }
                 }
                 tmax = warp_max(tmax);
                 if (lane == 0) wmax[(cur ^ 1) * 32 + warp] = tmax;
                 O += (int)off;
                 if (tid == 0) aux[t + 1] = O;
-                ri = ri + 1 == C::NROT ? 0 : ri + 1;
+                r += KB; r = r >= C::QB ? r - C::QB : r;
                 compute_barrier(CT);
             }
         };

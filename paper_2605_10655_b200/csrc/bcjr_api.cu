@@ -477,28 +477,28 @@ bcjr_status launch_bwd_skew(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cu
     return BCJR_OK;
 }
 
-// Backward call for k = 2 in two kernels per chunk of blocks: the alpha sweeps on one CTA per block (bwd_alpha_kernel),
-// then the beta sweeps of the same blocks on two-CTA clusters (bwd_skew_kernel<ACC, true>).  A chunk is as many blocks
-// as the GPU has SMs; the history of a chunk (32 MB per block at n = 256) is the hand-over between the two.
-template <bool ACC>
-bcjr_status launch_bwd_split(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+// Backward call in two kernels per chunk of blocks: the alpha sweeps on one CTA per block (bwd_alpha_kernel), then the
+// beta sweeps of the same blocks on two-CTA clusters (k = 2: bwd_skew_kernel<ACC, true>; k = 3: bwd_duo_kernel<3, true>).
+// A chunk is as many blocks as the GPU has SMs; the history of a chunk (32 MB per block at n = 256) is the hand-over.
+template <int KB, bool ACC, typename BetaKernel>
+bcjr_status launch_bwd_split(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st, BetaKernel beta, size_t beta_smem)
 {
-    using C = SkewCfg;
-    using A = AlphaCfg;
+    using A = AlphaCfg<KB>;
+    constexpr int CL = 2, THREADS = 512;
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1];
-    bcjr_status rc = plan_cluster(ctx, bwd_skew_kernel<ACC, true>, C::CL, C::THREADS, C::SMEM_BYTES, p.B, &cfg, attr, st);
+    bcjr_status rc = plan_cluster(ctx, beta, CL, THREADS, beta_smem, p.B, &cfg, attr, st);
     if (rc) return rc;
-    CU(cudaFuncSetAttribute(bwd_alpha_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
-    const int ncl = cfg.gridDim.x / C::CL;
+    CU(cudaFuncSetAttribute(bwd_alpha_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
+    const int ncl = cfg.gridDim.x / CL;
     int64_t chunk = ctx->num_sms;
     if (ctx->opt_max_ctas > 0 && chunk > ctx->opt_max_ctas) chunk = ctx->opt_max_ctas;
     if (chunk > p.B) chunk = p.B;
-    if ((rc = ensure(ctx, ctx->hist, (size_t)chunk * p.n * 2 * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)chunk * p.n * 2 * A::Q * 4))) return rc;
     if ((rc = ensure(ctx, ctx->stepO, (size_t)chunk * A::AUX_INTS * 4))) return rc;
     if (ACC) {
-        if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * C::S * 4))) return rc;
-        CU(cudaMemsetAsync(ctx->gc_part.ptr, 0, (size_t)ncl * C::S * 4, st));     // the beta launches add into it
+        if ((rc = ensure(ctx, ctx->gc_part, (size_t)ncl * A::S * 4))) return rc;
+        CU(cudaMemsetAsync(ctx->gc_part.ptr, 0, (size_t)ncl * A::S * 4, st));     // the beta launches add into it
     }
     p.hist = (float *)ctx->hist.ptr;
     p.stepO = (int *)ctx->stepO.ptr;
@@ -511,14 +511,14 @@ bcjr_status launch_bwd_split(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, c
         const int64_t nb = B - b0 < chunk ? B - b0 : chunk;
         p.B = nb;
         p.W = W + b0 * p.n; p.g = g + b0 * p.n; p.soft = soft + b0 * p.n; p.gW = gW + b0 * p.n;
-        bwd_alpha_kernel<false><<<(int)nb, A::THREADS, A::SMEM_BYTES, st>>>(p);
+        bwd_alpha_kernel<KB><<<(int)nb, A::THREADS, A::SMEM_BYTES, st>>>(p);
         CU(cudaGetLastError());
-        cfg.gridDim = dim3((unsigned)(C::CL * (nb < ncl ? nb : ncl)), 1, 1);
-        CU(cudaLaunchKernelEx(&cfg, bwd_skew_kernel<ACC, true>, p));
+        cfg.gridDim = dim3((unsigned)(CL * (nb < ncl ? nb : ncl)), 1, 1);
+        CU(cudaLaunchKernelEx(&cfg, beta, p));
         ctx->launches += 2;
     }
     if (ACC) {
-        reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, C::S, grad_codebook);
+        reduce_gc_kernel<<<(A::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, A::S, grad_codebook);
         ctx->launches += 1;
         CU(cudaGetLastError());
     }
@@ -529,11 +529,14 @@ bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_co
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
     if (k == 2 && ctx->opt_bwd_variant == 0 && p.n <= SkewCfg::MAX_N)
-        return grad_codebook ? launch_bwd_split<true>(ctx, p, grad_codebook, st) : launch_bwd_split<false>(ctx, p, nullptr, st);
+        return grad_codebook ? launch_bwd_split<2, true>(ctx, p, grad_codebook, st, bwd_skew_kernel<true, true>, SkewCfg::SMEM_BYTES)
+                             : launch_bwd_split<2, false>(ctx, p, nullptr, st, bwd_skew_kernel<false, true>, SkewCfg::SMEM_BYTES);
+    if (k == 3 && ctx->opt_bwd_variant == 0 && p.n <= DuoCfg<3>::MAX_N && grad_codebook)
+        return launch_bwd_split<3, true>(ctx, p, grad_codebook, st, bwd_duo_kernel<3, true>, DuoCfg<3>::SMEM_BYTES);
     if (k == 2 && ctx->opt_bwd_variant == 3 && p.n <= SkewCfg::MAX_N)
         return grad_codebook ? launch_bwd_skew<true>(ctx, p, grad_codebook, st) : launch_bwd_skew<false>(ctx, p, nullptr, st);
     if (k == 2 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<2>::MAX_N) return launch_bwd_duo<2>(ctx, p, grad_codebook, st);
-    if (k == 3 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<3>::MAX_N) return launch_bwd_duo<3>(ctx, p, grad_codebook, st);
+    if (k == 3 && ctx->opt_bwd_variant != 1 && p.n <= DuoCfg<3>::MAX_N) return launch_bwd_duo<3>(ctx, p, grad_codebook, st);   // variants 2, 3; no grad_codebook
     if (k == 2) return launch_bwd_cluster_t<16, 2, 4, 512>(ctx, p, grad_codebook, st);
     if (k == 3) return launch_bwd_cluster_t<16, 3, 4, 256>(ctx, p, grad_codebook, st);
     return BCJR_EUNSUPPORTED;

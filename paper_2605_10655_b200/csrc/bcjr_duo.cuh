@@ -72,7 +72,10 @@ struct DuoCfg {
     __host__ __device__ static constexpr int b_idx(int jh, int b) { return K == 4 ? 4 * jh + b : b; }
 };
 
-template <int KB>
+// BETA_ONLY = true: the beta sweeps alone, on the history, gauge offsets and log Z tail that bwd_alpha_kernel
+// (bcjr_alpha.cuh) wrote for the same blocks (block b of the call: history at p.hist + b n 2Q, offsets at
+// p.stepO + b (MAX_N + 4)); the partial codebook gradient is then ADDED to p.gc_part.
+template <int KB, bool BETA_ONLY = false>
 __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdParams p)
 {
     using C = DuoCfg<KB>;
@@ -178,127 +181,136 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
         int ib = 0;
         // per-step scalars of this block (read through the read-only cache, one line per warp)
         const float *w_s = p.W + blk * n, *g_s = p.g + blk * n, *sf_s = p.soft + blk * n;
-        // L_1 = 0; the At array carries At + gsh (gsh_t = -g_t soft_t centres h_t = g_t c - g_t soft_t)
-        {
-            const float gsh1 = -__ldg(g_s) * __ldg(sf_s);
-            for (int q = tid; q < QC; q += CT) { msg[q] = 0.f; msg[QC + q] = gsh1; }
-        }
-        if (tid == 0) O_s[1] = 0;
-#pragma unroll
-        for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, alpha pairing
-            stage_codebook<C>(p.cb, (int)rank * NBC + i * CT + tid, tm_cb + (uint32_t)(KK * i), false);
-        tmem_wait_st();
-        int O = 0;
-        float off = 0.f, cmax = 0.f;
-        cluster_sync();                                          // block start
-        // ================= alpha sweep carrying (L, At)
-        for (int t = 1; t <= n; ++t) {
-            const int ob = ib ^ 1;
-            // what does not depend on the step's inputs is requested before the wait for them: the first
-            // codebook unit from tensor memory and the step's scalars (their latency hides under the wait)
-            float2 cb[2][8];
-            tmem_ld16(tm_cb, cb[0]);
-            const float gt = __ldg(g_s + t - 1), wt = __ldg(w_s + t - 1);
-            const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
-            if (t > 1) {
-                wait_inputs(ib);
-                cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
-                off = rintf(cmax);
+        int O = 0, Ofin = 0;
+        float off = 0.f, cmax = 0.f, lsefin = 0.f;
+        if constexpr (BETA_ONLY) {
+            hist4 = reinterpret_cast<float4 *>(p.hist + (size_t)blk * n * 2 * C::Q) + tid;
+            const int *aux = p.stepO + (size_t)blk * (C::MAX_N + 4);
+            for (int t = 1 + tid; t <= n + 1; t += CT) O_s[t] = aux[t];
+            __syncthreads();
+            Ofin = O_s[n + 1];
+            lsefin = __int_as_float(aux[n + 2]);
+        } else {
+            // L_1 = 0; the At array carries At + gsh (gsh_t = -g_t soft_t centres h_t = g_t c - g_t soft_t)
+            {
+                const float gsh1 = -__ldg(g_s) * __ldg(sf_s);
+                for (int q = tid; q < QC; q += CT) { msg[q] = 0.f; msg[QC + q] = gsh1; }
             }
-            if (!pr.warp_live()) { tmem_wait_ld(cb[0]); break; } // a wait ran out: this warp issues nothing more
-            const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
-            const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
-            if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
-            float4 *hrow = hist4 + ((size_t)(t - 1) * CL + rank) * (BPT * NCH * CT);      // (L_t, At_t) of this thread's butterflies
-            // gshn: shift for the consumers of this step's At (step t+1); unused at t = n
-            const float2 gshn2 = splat2(gshn);
-            const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
-            const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt), off2 = splat2(off);
-            float tmax = NEG_INF;
+            if (tid == 0) O_s[1] = 0;
 #pragma unroll
-            for (int i = 0; i < BPT; ++i) {
-                float2 outL[K / 2], outA[K / 2];
-                float Lj[K], Aj[K];
-#pragma unroll
-                for (int j = 0; j < K; ++j) {
-                    Lj[j] = Lin[(i * K + j) * CT + tid];
-                    Aj[j] = Ain[(i * K + j) * CT + tid];
+            for (int i = 0; i < BPT; ++i)                             // codebook -> TMEM, alpha pairing
+                stage_codebook<C>(p.cb, (int)rank * NBC + i * CT + tid, tm_cb + (uint32_t)(KK * i), false);
+            tmem_wait_st();
+            cluster_sync();                                          // block start
+            // ================= alpha sweep carrying (L, At)
+            for (int t = 1; t <= n; ++t) {
+                const int ob = ib ^ 1;
+                // what does not depend on the step's inputs is requested before the wait for them: the first
+                // codebook unit from tensor memory and the step's scalars (their latency hides under the wait)
+                float2 cb[2][8];
+                tmem_ld16(tm_cb, cb[0]);
+                const float gt = __ldg(g_s + t - 1), wt = __ldg(w_s + t - 1);
+                const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
+                if (t > 1) {
+                    wait_inputs(ib);
+                    cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
+                    off = rintf(cmax);
                 }
+                if (!pr.warp_live()) { tmem_wait_ld(cb[0]); break; } // a wait ran out: this warp issues nothing more
+                const float *Lin = msg + ib * 2 * QC, *Ain = Lin + QC;
+                const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
+                if (tid == 0) mbar_expect_tx(mbar_full + ob_mbar, TX_MSG);
+                float4 *hrow = hist4 + ((size_t)(t - 1) * CL + rank) * (BPT * NCH * CT);      // (L_t, At_t) of this thread's butterflies
+                // gshn: shift for the consumers of this step's At (step t+1); unused at t = n
+                const float2 gshn2 = splat2(gshn);
+                const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
+                const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt), off2 = splat2(off);
+                float tmax = NEG_INF;
 #pragma unroll
-                for (int q = 0; q < K / 4; ++q) {
-                    hrow[(i * NCH + q) * CT] = make_float4(Lj[4 * q], Lj[4 * q + 1], Lj[4 * q + 2], Lj[4 * q + 3]);
-                    hrow[(i * NCH + K / 4 + q) * CT] = make_float4(Aj[4 * q], Aj[4 * q + 1], Aj[4 * q + 2], Aj[4 * q + 3]);
-                }
+                for (int i = 0; i < BPT; ++i) {
+                    float2 outL[K / 2], outA[K / 2];
+                    float Lj[K], Aj[K];
 #pragma unroll
-                for (int u = 0; u < UNITS; ++u) {
-                    const int g = i * UNITS + u;
-                    tmem_wait_ld(cb[g & 1]);
-                    if (g + 1 < NU) tmem_ld16(tm_cb + 16u * (g + 1), cb[(g + 1) & 1]);
+                    for (int j = 0; j < K; ++j) {
+                        Lj[j] = Lin[(i * K + j) * CT + tid];
+                        Aj[j] = Ain[(i * K + j) * CT + tid];
+                    }
 #pragma unroll
-                    for (int hh = 0; hh < HPU; ++hh) {
-                        const int h = u * HPU + hh;
-                        float2 a[K];
+                    for (int q = 0; q < K / 4; ++q) {
+                        hrow[(i * NCH + q) * CT] = make_float4(Lj[4 * q], Lj[4 * q + 1], Lj[4 * q + 2], Lj[4 * q + 3]);
+                        hrow[(i * NCH + K / 4 + q) * CT] = make_float4(Aj[4 * q], Aj[4 * q + 1], Aj[4 * q + 2], Aj[4 * q + 3]);
+                    }
 #pragma unroll
-                        for (int j = 0; j < K; ++j) {
-                            const float2 du = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
-                            a[j] = energy2(du, nl2, kap2, splat2(Lj[j]));
+                    for (int u = 0; u < UNITS; ++u) {
+                        const int g = i * UNITS + u;
+                        tmem_wait_ld(cb[g & 1]);
+                        if (g + 1 < NU) tmem_ld16(tm_cb + 16u * (g + 1), cb[(g + 1) & 1]);
+#pragma unroll
+                        for (int hh = 0; hh < HPU; ++hh) {
+                            const int h = u * HPU + hh;
+                            float2 a[K];
+#pragma unroll
+                            for (int j = 0; j < K; ++j) {
+                                const float2 du = sub2(cb[g & 1][C::a_idx(j, hh)], w2);
+                                a[j] = energy2(du, nl2, kap2, splat2(Lj[j]));
+                            }
+                            const float2 m = max_pairs<K>(a);
+                            float2 pj = ex2f2(sub2(a[0], m));
+                            float2 sum = pj, ax = mul2(pj, fma2(g2, cb[g & 1][C::a_idx(0, hh)], splat2(Aj[0])));
+#pragma unroll
+                            for (int j = 1; j < K; ++j) {
+                                // one in eight exponentials on the FP32 pipe (none: 13.17 ms, one in four: 13.14, one in eight: 13.04 per 592 blocks); no gain at K = 8
+                                pj = (KB == 2 && j % 4 == 3 && (hh & 1)) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));
+                                sum = add2(sum, pj);
+                                ax = fma2(pj, fma2(g2, cb[g & 1][C::a_idx(j, hh)], splat2(Aj[j])), ax);
+                            }
+                            outL[h] = add2(sub2(m, off2), lg2f2(sum));
+                            outA[h] = fma2(ax, rcpf2(sum), gshn2);
+                            tmax = max3f(tmax, m.x, m.y);
                         }
-                        const float2 m = max_pairs<K>(a);
-                        float2 pj = ex2f2(sub2(a[0], m));
-                        float2 sum = pj, ax = mul2(pj, fma2(g2, cb[g & 1][C::a_idx(0, hh)], splat2(Aj[0])));
+                    }
+                    const uint32_t mb = push_a_mbar[i] + ob_mbar;
+                    // k = 2: the outputs of slot i go to CTA i & 1 whatever the thread (x*K mod NB = (i & 1)*NBC + 4 tid);
+                    // said this way the choice is uniform for the compiler too
+                    const bool own = BPT >= 2 ? (i & 1) == (int)rank : (own_a >> i) & 1u;
 #pragma unroll
-                        for (int j = 1; j < K; ++j) {
-                            // one in eight exponentials on the FP32 pipe (none: 13.17 ms, one in four: 13.14, one in eight: 13.04 per 592 blocks); no gain at K = 8
-                            pj = (KB == 2 && j % 4 == 3 && (hh & 1)) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));
-                            sum = add2(sum, pj);
-                            ax = fma2(pj, fma2(g2, cb[g & 1][C::a_idx(j, hh)], splat2(Aj[j])), ax);
-                        }
-                        outL[h] = add2(sub2(m, off2), lg2f2(sum));
-                        outA[h] = fma2(ax, rcpf2(sum), gshn2);
-                        tmax = max3f(tmax, m.x, m.y);
+                    for (int h = 0; h < K / 2; h += 2) {
+                        push_v4(own, push_a[i] + ob_off + 8u * h, outL[h].x, outL[h].y, outL[h + 1].x, outL[h + 1].y, mb);
+                        push_v4(own, push_a[i] + ob_off + QC * 4u + 8u * h, outA[h].x, outA[h].y, outA[h + 1].x, outA[h + 1].y, mb);
                     }
                 }
-                const uint32_t mb = push_a_mbar[i] + ob_mbar;
-                // k = 2: the outputs of slot i go to CTA i & 1 whatever the thread (x*K mod NB = (i & 1)*NBC + 4 tid);
-                // said this way the choice is uniform for the compiler too
-                const bool own = BPT >= 2 ? (i & 1) == (int)rank : (own_a >> i) & 1u;
+                tmax = warp_max(tmax);
+                if (lane == 0) {
 #pragma unroll
-                for (int h = 0; h < K / 2; h += 2) {
-                    push_v4(own, push_a[i] + ob_off + 8u * h, outL[h].x, outL[h].y, outL[h + 1].x, outL[h + 1].y, mb);
-                    push_v4(own, push_a[i] + ob_off + QC * 4u + 8u * h, outA[h].x, outA[h].y, outA[h + 1].x, outA[h + 1].y, mb);
+                    for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
                 }
+                O += (int)off;
+                if (tid == 0) O_s[t + 1] = O;
+                __syncwarp();
+                if (lane == 0) {                                     // this warp has read all its inputs and written its outputs
+                    mbar_arrive_local(mbar_full + ob_mbar);
+                    mbar_arrive_remote(full_of[rank ^ 1u] + ob_mbar);
+                }
+                ib = ob;
             }
-            tmax = warp_max(tmax);
-            if (lane == 0) {
+            // ================= log2 Z
+            wait_inputs(ib);
+            cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
+            {
+                const float *Lfin = msg + ib * 2 * QC;
+                float ssum = 0.f;
+                for (int q = tid; q < QC; q += CT) ssum += ex2f(Lfin[q] - cmax);
+                ssum = warp_sum(ssum);
+                if (lane == 0) {
 #pragma unroll
-                for (int r = 0; r < CL; ++r) st_async_f32(wmax_dst[r] + (uint32_t)(ob * 32) * 4u, tmax, full_of[r] + ob_mbar);
+                    for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
+                }
+                cluster_sync();                                      // log Z exchange
             }
-            O += (int)off;
-            if (tid == 0) O_s[t + 1] = O;
-            __syncwarp();
-            if (lane == 0) {                                     // this warp has read all its inputs and written its outputs
-                mbar_arrive_local(mbar_full + ob_mbar);
-                mbar_arrive_remote(full_of[rank ^ 1u] + ob_mbar);
-            }
-            ib = ob;
+            lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
+            if (tid == 0) diag_check_finite(p.diag, lsefin);
+            Ofin = O;
         }
-        // ================= log2 Z
-        wait_inputs(ib);
-        cmax = warp_max(lane < SLOTS ? wmax[ib * 32 + lane] : NEG_INF) - off;
-        {
-            const float *Lfin = msg + ib * 2 * QC;
-            float ssum = 0.f;
-            for (int q = tid; q < QC; q += CT) ssum += ex2f(Lfin[q] - cmax);
-            ssum = warp_sum(ssum);
-            if (lane == 0) {
-#pragma unroll
-                for (int r = 0; r < CL; ++r) st_cluster_f32(lz_dst[r], ssum);
-            }
-            cluster_sync();                                      // log Z exchange
-        }
-        const float lsefin = cmax + lg2f(warp_sum(lane < SLOTS ? lz[lane] : 0.f));
-        if (tid == 0) diag_check_finite(p.diag, lsefin);
-        const int Ofin = O;
         // ================= beta sweep carrying (M, Bt), with the gradient contraction
         {
             const float gshn = -__ldg(g_s + n - 1) * __ldg(sf_s + n - 1);     // M_n = 0, Bt_n = 0 (+ centring shift)
@@ -491,8 +503,9 @@ __global__ void __launch_bounds__(DuoCfg<KB>::THREADS, 1) bwd_duo_kernel(BwdPara
                 const int jh = u * HPU + hh;
 #pragma unroll
                 for (int b = 0; b < K; ++b) {
-                    gc[(size_t)(2 * jh) * C::Q + (size_t)x * K + b] = acc[C::b_idx(hh, b)].x;
-                    gc[(size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b] = acc[C::b_idx(hh, b)].y;
+                    float *g0 = gc + (size_t)(2 * jh) * C::Q + (size_t)x * K + b, *g1 = gc + (size_t)(2 * jh + 1) * C::Q + (size_t)x * K + b;
+                    *g0 = BETA_ONLY ? *g0 + acc[C::b_idx(hh, b)].x : acc[C::b_idx(hh, b)].x;
+                    *g1 = BETA_ONLY ? *g1 + acc[C::b_idx(hh, b)].y : acc[C::b_idx(hh, b)].y;
                 }
             }
         }
