@@ -1,0 +1,96 @@
+// Host-side check of the index arithmetic the 2^16-state backward kernels rely on (no GPU needed): the
+// functions below are the kernels' own (constexpr, host and device), compiled here for the host.
+//   1. bwd_skew_kernel: (CTA, thread, slot) <-> butterfly is a bijection; every output has one destination entry;
+//      the butterfly a thread computes FIRST in a step depends on none of those computed LAST in the step before
+//      (alpha order 0,1,2,3; beta order 2,0,3,1); alpha slots 0,1 feed the own CTA, slots 2,3 the peer.
+//   2. bwd_alpha_kernel<2>, <3>: the in-place slot function is a bijection, XOR-linear over the bit fields the
+//      kernel combines, consistent from one step to the next (output [x|l] takes the slot of input [l|x]), and a
+//      warp's 32 lanes always reach 32 different banks.
+#include <cstdio>
+#include <set>
+#include <vector>
+
+#include "../paper_2605_10655_b200/csrc/bcjr_alpha.cuh"
+
+using namespace bcjr;
+
+static int fails = 0;
+#define CHECK(cond, ...) do { if (!(cond)) { if (fails < 20) { std::printf("FAIL %s:%d: ", __FILE__, __LINE__); std::printf(__VA_ARGS__); std::printf("\n"); } ++fails; } } while (0)
+
+static void check_skew()
+{
+    using C = SkewCfg;
+    std::set<int> seen;
+    for (int r = 0; r < 2; ++r)
+        for (int t = 0; t < 512; ++t)
+            for (int s = 0; s < 4; ++s) {
+                const int x = C::x_of(r, t, s);
+                CHECK(x >= 0 && x < C::NB && seen.insert(x).second, "x_of not injective at (%d,%d,%d)", r, t, s);
+                CHECK(C::rank_of(x) == r && C::slot_of(x) == s && C::tid_of(x) == t, "inverse of x_of at %d", x);
+            }
+    const int beta_pos[4] = {1, 3, 0, 2};                 // position of slot s in the beta order 2,0,3,1
+    std::set<long> dest_a, dest_b;
+    for (int x = 0; x < C::NB; ++x) {
+        const int r = C::rank_of(x), s = C::slot_of(x);
+        for (int l = 0; l < 4; ++l) {                     // alpha: L'([x|l]) is input x >> 10 of butterfly ((x & 1023) << 2) | l
+            const int x2 = ((x & 1023) << 2) | l, j2 = x >> 10;
+            CHECK((C::rank_of(x2) == r) == (s < 2), "alpha destination CTA of slot %d", s);
+            dest_a.insert((long)C::rank_of(x2) * 65536 + (C::slot_of(x2) * 4 + j2) * 512 + C::tid_of(x2));
+            CHECK(!(C::slot_of(x2) == 0 && s == 3), "alpha: first butterfly depends on a last one (x=%d)", x);
+            CHECK(C::tid_of((x & 1023) << 2) % 4 == 0 && C::tid_of(x2) == C::tid_of((x & 1023) << 2) + l, "alpha outputs not one 16-byte entry");
+        }
+        for (int j = 0; j < 4; ++j) {                     // beta: M'([j|x]) is input x & 3 of butterfly (j << 10) | (x >> 2)
+            const int x1 = (j << 10) | (x >> 2);
+            CHECK(C::rank_of(x1) == (j >> 1), "beta destination CTA");
+            dest_b.insert((long)C::rank_of(x1) * 65536 + ((x & 3) * 2048 + C::slot_of(x1) * 512 + C::tid_of(x1)));
+            CHECK(!(beta_pos[C::slot_of(x1)] == 0 && beta_pos[s] == 3), "beta: first butterfly depends on a last one (x=%d)", x);
+            // what the kernel assumes about the two outputs of a pair: next slot (own CTA) / upper half of the threads (peer)
+            if ((j & 1) == 0) {
+                const int y = ((j + 1) << 10) | (x >> 2);
+                if (C::rank_of(x1) == r) CHECK(C::slot_of(y) == C::slot_of(x1) + 1 && C::tid_of(y) == C::tid_of(x1), "beta own-CTA pair");
+                else CHECK(C::slot_of(y) == C::slot_of(x1) && C::tid_of(y) == C::tid_of(x1) + 256, "beta peer pair");
+            }
+        }
+    }
+    CHECK(dest_a.size() == 2u * 8192u && dest_b.size() == 2u * 8192u, "destinations not a bijection");
+}
+
+template <int KB>
+static void check_alpha()
+{
+    using C = AlphaCfg<KB>;
+    constexpr int QB = C::QB, K = C::K;
+    for (int step = 0; step < 3 * QB; ++step) {
+        const int r = (KB * step) % QB, r2 = (KB * (step + 1)) % QB;
+        std::vector<char> used(1 << QB, 0);
+        for (uint32_t q = 0; q < (1u << QB); ++q) {
+            const uint32_t s = C::slot(q, r);
+            CHECK(s < (1u << QB) && !used[s], "slot not a bijection (k=%d r=%d)", KB, r);
+            used[s] = 1;
+        }
+        for (int i = 0; i < C::BPT; ++i)
+            for (int j = 0; j < K; ++j)
+                for (int w = 0; w < 16; ++w) {
+                    std::set<uint32_t> banks;
+                    for (int l = 0; l < 32; ++l) {
+                        const uint32_t tid = w * 32 + l, x = ((uint32_t)i << 9) | tid, q = ((uint32_t)j << (QB - KB)) | x;
+                        const uint32_t s = C::slot(q, r);
+                        CHECK(s == (C::slot((uint32_t)i << 9, r) ^ C::slot(tid, r) ^ C::slot((uint32_t)j << (QB - KB), r)), "slot not XOR-linear");
+                        banks.insert(s & 31u);
+                        // in place: output [x|l'] of this step is found next step where input [l'|x] was
+                        CHECK(C::slot(((x << KB) | (uint32_t)j) & ((1u << QB) - 1u), r2) == s, "in-place slots inconsistent (k=%d)", KB);
+                    }
+                    CHECK(banks.size() == 32u, "bank conflict (k=%d r=%d)", KB, r);
+                }
+    }
+}
+
+int main()
+{
+    check_skew();
+    check_alpha<2>();
+    check_alpha<3>();
+    if (fails) std::printf("%d checks failed\n", fails);
+    else std::printf("layouts ok\n");
+    return fails ? 1 : 0;
+}
