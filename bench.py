@@ -151,9 +151,10 @@ def run_reference(args, wl):
 class Runner:
     """Device buffers of one workload and the timed forward + backward step over all its matrices."""
 
-    def __init__(self, ctx, wl, dev, blocks_cap=0, rank=0, world=1, keep_host=False):
+    def __init__(self, ctx, wl, dev, blocks_cap=0, rank=0, world=1, keep_host=False, fixed_table=False):
         import torch
         self.ctx, self.wl, self.dev, self.rank = ctx, wl, dev, rank
+        self.fixed_table = fixed_table                      # backward without grad_codebook (the paper's setting: the table is not trained)
         self.cb = torch.from_numpy(wl.codebook()).to(dev)
         self.mats = []
         for i, (name, _) in enumerate(wl.matrices):
@@ -193,11 +194,16 @@ class Runner:
                 ctx.bcjr_soft_quantize_vec(m["W"], self.cb, wl.Lb, wl.k, wl.V, wl.n, T, soft=m["soft"])
             if ev is not None:
                 ev["f1"].append(torch.cuda.Event(enable_timing=True)); ev["f1"][-1].record()
-            ctx.bcjr_backward(m["g"], grad_W=m["gW"], grad_codebook=self.gc)
+            if self.fixed_table:
+                ctx.bcjr_backward(m["g"], grad_W=m["gW"], want_grad_codebook=False)
+            else:
+                ctx.bcjr_backward(m["g"], grad_W=m["gW"], grad_codebook=self.gc)
             if ev is not None:
                 ev["b1"].append(torch.cuda.Event(enable_timing=True)); ev["b1"][-1].record()
-            self.gc_total.add_(self.gc)
-        shard.allreduce_grad_codebook(self.gc_total)     # the one exchange of the data-parallel path
+            if not self.fixed_table:
+                self.gc_total.add_(self.gc)
+        if not self.fixed_table:
+            shard.allreduce_grad_codebook(self.gc_total)     # the one exchange of the data-parallel path
 
     def timed(self, temps_warm, temps_timed, flush):
         """Warm-up steps, then the timed ones (CUDA events per step on the launching stream, L2 evicted in
@@ -235,17 +241,19 @@ def mufu_fractions(wl, state_steps, fwd_ms, bwd_ms, step_ms, peak_gops):
     return out
 
 
-def workload_leg(ctx, name, blocks_cap, dev, flush, peak_gops):
+def workload_leg(ctx, name, blocks_cap, dev, flush, peak_gops, fixed_table=False):
     """A short measurement of another workload in the same run: one warm-up step, two timed steps."""
     import torch
     wl = WORKLOADS[name]()
-    r = Runner(ctx, wl, dev, blocks_cap)
+    r = Runner(ctx, wl, dev, blocks_cap, fixed_table=fixed_table)
     step_ms, fwd_ms, bwd_ms, diag, _ = r.timed([wl.T], [wl.T, wl.T], flush)
     ms = float(np.mean(step_ms))
     leg = {"workload": wl.name, "blocks": r.nblocks, "Lb": wl.Lb, "k": wl.k, "V": wl.V, "n": wl.n, "T": wl.T,
            "ms_per_step": ms, "fwd_ms": fwd_ms / 2, "bwd_ms": bwd_ms / 2, "edges_per_s": r.edges_per_step / (ms * 1e-3),
            "path": {0: "generic kernels", 1: "large-trellis kernels", 2: "one warp per block"}[diag.last_path],
            "max_posterior_defect": diag.max_posterior_defect}
+    if fixed_table:
+        leg["backward"] = "grad_W only (table not trained)"
     leg.update(mufu_fractions(wl, r.state_steps, fwd_ms / 2, bwd_ms / 2, ms, peak_gops))
     del r
     torch.cuda.empty_cache()
@@ -303,7 +311,11 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-viterbi", action="store_true")
     ap.add_argument("--no-legs", action="store_true", help="skip the short legs over the other workloads")
+    ap.add_argument("--fixed-table", action="store_true",
+                    help="backward calls without grad_codebook (not the headline configuration, which trains the table)")
     args = ap.parse_args()
+    if args.fixed_table:
+        args.no_e2e = True                                  # the host-buffer call always forms grad_codebook
     wl = WORKLOADS[args.workload]()
     if args.impl == "reference":
         return run_reference(args, wl)
@@ -341,7 +353,7 @@ def main():
     for kv in args.option:
         name, _, val = kv.partition("=")
         ctx.set_option(name, int(val))
-    run = Runner(ctx, wl, dev, args.blocks, rank, world, keep_host=not args.no_e2e)
+    run = Runner(ctx, wl, dev, args.blocks, rank, world, keep_host=not args.no_e2e, fixed_table=args.fixed_table)
     mats, cb, nblocks, edges_per_step = run.mats, run.cb, run.nblocks, run.edges_per_step
     # the decoder-layer workload anneals T geometrically from 0.3 to 0.01 over the timed steps (warm-up at T_0)
     annealed = wl.name.startswith("llama32_1b_decoder")
@@ -503,6 +515,7 @@ def main():
         legs = {}
         for name, cap in (("q_proj", 0), ("gate_k3", 32 * NUM_SMS), ("qtip_v2", 16 * NUM_SMS), ("mid", 0)):
             legs[name] = workload_leg(ctx, name, cap, dev, flush, peak)
+        legs["q_proj_fixed_table"] = workload_leg(ctx, "q_proj", 32 * NUM_SMS, dev, flush, peak, fixed_table=True)
         legs["qat_loop"] = qat_loop_leg(ctx, dev, flush)
 
     if rank == 0:
@@ -516,7 +529,8 @@ def main():
                           "Lb": wl.Lb, "k": wl.k, "V": wl.V, "T": [temps_timed[0], temps_timed[-1]],
                           "T_schedule": "geometric over the timed steps, warm-up at the first value" if annealed else "constant",
                           "l2": "256 MB flush write between timed steps; per-step working set >> L2",
-                          "path": {0: "generic", 1: "cluster", 2: "warp"}[diag.last_path]},
+                          "path": {0: "generic", 1: "cluster", 2: "warp"}[diag.last_path],
+                          **({"backward": "grad_W only (--fixed-table)"} if args.fixed_table else {})},
                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": base,
                "breakdown": {"fwd_ms_per_step": fwd_ms / args.steps, "bwd_ms_per_step": bwd_ms / args.steps,
                              "viterbi": vit, "qat_update": upd, "max_posterior_defect": diag.max_posterior_defect,

@@ -74,10 +74,14 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *                 (BCJR_EUNSUPPORTED at call time when they do not cover the shape)
  *   "fwd_variant" large-trellis forward kernel: 0 = one CTA per block with the codebook in tensor
  *                 memory (Lb = 16, k = 2 or 3), 1 = two-CTA cluster kernel with the codebook in registers
- *   "bwd_variant" large-trellis backward kernel: 0 = two-CTA clusters with codebook and gradient
- *                 accumulators in tensor memory (Lb = 16, k = 2 or 3; at k = 2 with the butterflies ordered so
- *                 that a step starts before the whole cluster has finished the previous one), 1 = four-CTA
- *                 clusters, registers, 2 = the two-CTA tensor-memory kernel with one barrier per step at k = 2 too
+ *   "bwd_variant" large-trellis backward call (Lb = 16, k = 2 or 3).  0 (default): with grad_codebook, two
+ *                 kernels per chunk of as many blocks as the GPU has SMs -- the alpha sweeps on one CTA per
+ *                 block, then the beta sweeps on two-CTA clusters with codebook and gradient accumulators in
+ *                 tensor memory; without grad_codebook at k = 2, one kernel with both sweeps on one CTA per
+ *                 block.  1 = four-CTA clusters, registers.  2 = one two-CTA tensor-memory kernel for both
+ *                 sweeps, one cluster barrier per step.  3 = the same with the butterflies ordered so that a
+ *                 step starts before the whole cluster has finished the previous one (k = 2; k = 3 as 2).
+ *                 4 = as 0, but the two-kernel call also without grad_codebook.
  *   "history_every_m"  1 (default): the large-trellis forward kernel stores the forward messages of every step
  *                 for its beta sweep; m = 2..16: it keeps them for every m-th step only and recomputes the
  *                 m - 1 steps in between inside the beta sweep (1/m of the history traffic to HBM for

@@ -20,6 +20,7 @@
 #include "bcjr_duo.cuh"
 #include "bcjr_skew.cuh"
 #include "bcjr_alpha.cuh"
+#include "bcjr_bsolo.cuh"
 #include "bcjr_ckpt.cuh"
 #include "bcjr_warp.cuh"
 #include "bcjr_viterbi.cuh"
@@ -55,8 +56,8 @@ struct bcjr_ctx {
     // options
     int opt_path = 0;
     int opt_max_ctas = 0;
-    int opt_bwd_variant = 0;   // 0 = TMEM two-CTA backward kernels (k = 2: skewed slot order), 1 = register-accumulator cluster kernel,
-                               // 2 = TMEM two-CTA kernel with one barrier per step also at k = 2
+    int opt_bwd_variant = 0;   // 0 = alpha kernel + two-CTA beta kernel (without grad_codebook at k = 2: one-CTA kernel), 1 = register-accumulator
+                               // cluster kernel, 2 = fused two-CTA TMEM kernel, 3 = fused with skewed slot order, 4 = two-kernel call always
     int opt_fwd_variant = 0;   // 0 = TMEM single-CTA forward kernel where it applies, 1 = cluster forward kernel
     int opt_record_defect = 0; // forward calls record the posterior defect of every block
     int opt_hist_every = 1;    // large-trellis forward call: keep L_t of every m-th step, recompute the others in the beta sweep
@@ -525,13 +526,33 @@ bcjr_status launch_bwd_split(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, c
     return BCJR_OK;
 }
 
+// Backward call without grad_codebook (Lb = 16, k = 2): both sweeps on one CTA per block.
+bcjr_status launch_bwd_solo(bcjr_ctx *ctx, BwdParams p, cudaStream_t st)
+{
+    using C = BSoloCfg;
+    CU(cudaFuncSetAttribute(bwd_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
+    int64_t grid = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    if (grid > p.B) grid = p.B;
+    bcjr_status rc = ensure(ctx, ctx->hist, (size_t)grid * p.n * 2 * C::Q * 4);
+    if (rc) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.gc_part = nullptr;
+    if (ctx->cb_computed) p.cb = nullptr;                    // entries are evaluated while staging
+    bwd_solo_kernel<<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
 bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_codebook, cudaStream_t st)
 {
     if (p.Lb != 16) return BCJR_EUNSUPPORTED;
-    if (k == 2 && ctx->opt_bwd_variant == 0 && p.n <= SkewCfg::MAX_N)
+    if (k == 2 && ctx->opt_bwd_variant == 0 && !grad_codebook && p.n <= BSoloCfg::MAX_N) return launch_bwd_solo(ctx, p, st);
+    if (k == 2 && (ctx->opt_bwd_variant == 0 || ctx->opt_bwd_variant == 4) && p.n <= SkewCfg::MAX_N)
         return grad_codebook ? launch_bwd_split<2, true>(ctx, p, grad_codebook, st, bwd_skew_kernel<true, true>, SkewCfg::SMEM_BYTES)
                              : launch_bwd_split<2, false>(ctx, p, nullptr, st, bwd_skew_kernel<false, true>, SkewCfg::SMEM_BYTES);
-    if (k == 3 && ctx->opt_bwd_variant == 0 && p.n <= DuoCfg<3>::MAX_N && grad_codebook)
+    if (k == 3 && (ctx->opt_bwd_variant == 0 || ctx->opt_bwd_variant == 4) && p.n <= DuoCfg<3>::MAX_N && grad_codebook)
         return launch_bwd_split<3, true>(ctx, p, grad_codebook, st, bwd_duo_kernel<3, true>, DuoCfg<3>::SMEM_BYTES);
     if (k == 2 && ctx->opt_bwd_variant == 3 && p.n <= SkewCfg::MAX_N)
         return grad_codebook ? launch_bwd_skew<true>(ctx, p, grad_codebook, st) : launch_bwd_skew<false>(ctx, p, nullptr, st);
@@ -772,7 +793,7 @@ bcjr_status bcjr_set_option(bcjr_ctx *ctx, const char *name, int64_t value)
         return BCJR_OK;
     }
     if (!strcmp(name, "bwd_variant")) {
-        if (value < 0 || value > 3) return BCJR_EINVAL;
+        if (value < 0 || value > 4) return BCJR_EINVAL;
         ctx->opt_bwd_variant = (int)value;
         return BCJR_OK;
     }

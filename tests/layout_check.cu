@@ -3,14 +3,14 @@
 //   1. bwd_skew_kernel: (CTA, thread, slot) <-> butterfly is a bijection; every output has one destination entry;
 //      the butterfly a thread computes FIRST in a step depends on none of those computed LAST in the step before
 //      (alpha order 0,1,2,3; beta order 2,0,3,1); alpha slots 0,1 feed the own CTA, slots 2,3 the peer.
-//   2. bwd_alpha_kernel<2>, <3>: the in-place slot function is a bijection, XOR-linear over the bit fields the
+//   2. bwd_alpha_kernel<2>, <3> (and the same sweeps inside bwd_solo_kernel, whose in-place beta sweep is checked too): the in-place slot function is a bijection, XOR-linear over the bit fields the
 //      kernel combines, consistent from one step to the next (output [x|l] takes the slot of input [l|x]), and a
 //      warp's 32 lanes always reach 32 different banks.
 #include <cstdio>
 #include <set>
 #include <vector>
 
-#include "../paper_2605_10655_b200/csrc/bcjr_alpha.cuh"
+#include "../paper_2605_10655_b200/csrc/bcjr_bsolo.cuh"
 
 using namespace bcjr;
 
@@ -85,8 +85,36 @@ static void check_alpha()
     }
 }
 
+// bwd_solo_kernel's in-place beta sweep: input b of butterfly x is group (x << k) | b at rotation rr; output j takes
+// the slot of input j and must be where the next step (rotation rr - k) looks for group (j << (QB - k)) | x.
+static void check_beta_in_place()
+{
+    using C = BSoloCfg;
+    constexpr int QB = C::QB, K = C::K, KB = C::KB;
+    int rr = 0;
+    for (int step = 0; step < 3 * QB; ++step) {
+        const int rr2 = rr == 0 ? QB - KB : rr - KB;
+        for (int i = 0; i < C::BPT; ++i)
+            for (int b = 0; b < K; ++b)
+                for (int w = 0; w < 16; ++w) {
+                    std::set<uint32_t> banks;
+                    for (int l = 0; l < 32; ++l) {
+                        const int tid = w * 32 + l;
+                        const uint32_t x = (uint32_t)(i * C::THREADS + tid), q = C::beta_q(i, tid, b);
+                        const uint32_t s = C::slot(q, rr);
+                        CHECK(s == (C::slot(C::beta_q(i, 0, 0), rr) ^ C::slot(C::beta_q(0, tid, 0), rr) ^ C::slot((uint32_t)b, rr)), "beta slot not XOR-linear");
+                        banks.insert(s & 31u);
+                        CHECK(C::slot(((uint32_t)b << (QB - KB)) | x, rr2) == s, "beta in-place slots inconsistent (rr=%d)", rr);
+                    }
+                    CHECK(banks.size() == 32u, "beta bank conflict (rr=%d)", rr);
+                }
+        rr = rr2;
+    }
+}
+
 int main()
 {
+    check_beta_in_place();
     check_skew();
     check_alpha<2>();
     check_alpha<3>();
