@@ -14,6 +14,7 @@
 #include "bcjr_cluster.cuh"
 #include "bcjr_vec.cuh"
 #include "bcjr_vec4.cuh"
+#include "bcjr_vec2.cuh"
 #include "bcjr_qat.cuh"
 #include "bcjr_rht.cuh"
 #include "bcjr_solo.cuh"
@@ -332,6 +333,9 @@ bcjr_status plan_cluster(bcjr_ctx *ctx, Kern kern, int CL, int threads, size_t s
 #ifndef VEC4_FWD_NBLK
 #define VEC4_FWD_NBLK 3
 #endif
+#ifndef VEC2_FWD_NBLK
+#define VEC2_FWD_NBLK 3
+#endif
 #ifndef VEC4_BWD_NBLK
 #define VEC4_BWD_NBLK 2
 #endif
@@ -342,6 +346,27 @@ bcjr_status launch_fwd_vec4(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1];
     auto kern = fwd_vec4_kernel<VEC4_FWD_NBLK>;
+    bcjr_status rc = plan_cluster(ctx, kern, C::CL, C::THREADS, C::SMEM_BYTES, (p.B + C::NBLK - 1) / C::NBLK, &cfg, attr, st);
+    if (rc) return rc;
+    const int ncl = cfg.gridDim.x / C::CL, nt = p.n / C::V;
+    if ((rc = ensure(ctx, ctx->hist, (size_t)ncl * C::NBLK * nt * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->cb_beta, (size_t)C::S * C::V * 4))) return rc;
+    regroup_table_kernel<<<(C::S * C::V + 255) / 256, 256, 0, st>>>(p.cb, (float *)ctx->cb_beta.ptr, C::S, C::KB, C::V);
+    p.hist = (float *)ctx->hist.ptr;
+    p.cb_beta = (const float *)ctx->cb_beta.ptr;
+    CU(cudaLaunchKernelEx(&cfg, kern, p));
+    ctx->launches += 2;
+    return BCJR_OK;
+}
+
+// Forward call of the same trellis on clusters of two CTAs (the table alone fits two tensor memories): the default.
+bcjr_status launch_fwd_vec2(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
+{
+    using C = Vec2Cfg<VEC2_FWD_NBLK>;
+    if (p.n > C::MAX_N || ((uintptr_t)p.cb & 15u)) return BCJR_EUNSUPPORTED;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    auto kern = fwd_vec2_kernel<VEC2_FWD_NBLK>;
     bcjr_status rc = plan_cluster(ctx, kern, C::CL, C::THREADS, C::SMEM_BYTES, (p.B + C::NBLK - 1) / C::NBLK, &cfg, attr, st);
     if (rc) return rc;
     const int ncl = cfg.gridDim.x / C::CL, nt = p.n / C::V;
@@ -1043,7 +1068,7 @@ bcjr_status bcjr_soft_quantize_vec(bcjr_ctx *ctx, const float *W, const float *c
         large = ctx->opt_path != 1 && Lb == 16 && k == 2;
         if (ctx->opt_path == 2 && !large) return BCJR_EUNSUPPORTED;
         if (large) {
-            rc = launch_fwd_vec4(ctx, p, st);
+            rc = ctx->opt_fwd_variant == 1 ? launch_fwd_vec4(ctx, p, st) : launch_fwd_vec2(ctx, p, st);
             if (rc == BCJR_EUNSUPPORTED && ctx->opt_path != 2) { large = false; rc = BCJR_OK; }   // e.g. n too long
         }
 #else

@@ -3,6 +3,7 @@
 //   1. bwd_skew_kernel: (CTA, thread, slot) <-> butterfly is a bijection; every output has one destination entry;
 //      the butterfly a thread computes FIRST in a step depends on none of those computed LAST in the step before
 //      (alpha order 0,1,2,3; beta order 2,0,3,1); alpha slots 0,1 feed the own CTA, slots 2,3 the peer.
+//   3. fwd_vec2_kernel: production, consumer CTA and reader's address of every group in both sweeps.
 //   2. bwd_alpha_kernel<2>, <3> (and the same sweeps inside bwd_solo_kernel, whose in-place beta sweep is checked too): the in-place slot function is a bijection, XOR-linear over the bit fields the
 //      kernel combines, consistent from one step to the next (output [x|l] takes the slot of input [l|x]), and a
 //      warp's 32 lanes always reach 32 different banks.
@@ -11,6 +12,7 @@
 #include <vector>
 
 #include "../paper_2605_10655_b200/csrc/bcjr_bsolo.cuh"
+#include "../paper_2605_10655_b200/csrc/bcjr_vec2.cuh"
 
 using namespace bcjr;
 
@@ -112,8 +114,53 @@ static void check_beta_in_place()
     }
 }
 
+// fwd_vec2_kernel: every group is produced once per sweep, lands in the CTA that reads it, at the place its reader looks
+static void check_vec2()
+{
+    using C = Vec2Cfg<3>;
+    // alpha: entry i = j * 256 + x of L is read by the threads of butterfly x as input j
+    std::vector<int> seen(C::Q, 0);
+    for (int rank = 0; rank < 2; ++rank)
+        for (int tid = 0; tid < C::THREADS; ++tid) {
+            const int q0 = C::alpha_q0(rank, tid);
+            for (int e = 0; e < 4; ++e) {
+                const int i = q0 + e, j = i >> 8, x = i & 255, rc = x >> 7;
+                ++seen[i];
+                CHECK(C::alpha_dst_rank(q0) == rc, "alpha: consumer CTA of group %d", i);
+                // a reader of butterfly x in CTA rc: tid' with (rc * 2048 + 4 tid') >> 4 == x
+                const int tidr = (x & 127) << 2;
+                CHECK((C::alpha_q0(rc, tidr) >> 4) == x && C::alpha_dst_off(q0) + e == C::alpha_in(tidr) + 128 * j, "alpha: group %d not where its reader looks", i);
+            }
+            CHECK(C::alpha_dst_off(q0) % 4 == 0, "alpha push not 16-byte aligned");
+        }
+    for (int i = 0; i < C::Q; ++i) CHECK(seen[i] == 1, "alpha: group %d produced %d times", i, seen[i]);
+    // beta: entry i = (x << 4) | b of M is read by the thread that owns butterflies 2 xp, 2 xp + 1 (x >> 1 == xp) as part of one float4
+    std::fill(seen.begin(), seen.end(), 0);
+    for (int rank = 0; rank < 2; ++rank)
+        for (int warp = 0; warp < 16; ++warp)
+            for (int lane = 0; lane < 32; ++lane)
+                for (int pp = 0; pp < 2; ++pp) {
+                    const int q = C::beta_q0(rank, warp, lane, pp);
+                    CHECK(q == C::beta_q0(rank, warp, lane, 0) + 256 * pp && ((q & 255) >> 7) == rank && q % 2 == 0, "beta: ownership of group %d", q);
+                    CHECK(C::beta_dst_rank(q) == C::beta_dst_rank(C::beta_q0(rank, warp, lane, 0)), "beta: the two pairs of a thread go to different CTAs");
+                    CHECK(C::beta_dst_off(q) - C::beta_dst_off(C::beta_q0(rank, warp, lane, 0)) == pp * (C::beta_dst_off(256) - C::beta_dst_off(0)), "beta: pair offset");
+                    for (int e = 0; e < 2; ++e) {
+                        const int i = q + e, x = i >> 4, b = i & 15, rc = x >> 7;
+                        ++seen[i];
+                        CHECK(C::beta_dst_rank(q) == rc && C::beta_dst_off(q) + e == C::beta_dst_off(i), "beta: consumer of group %d", i);
+                        // the reader: CTA rc, xp = (x & 127) >> 1 -> lane' = xp & 31, warp' & 1 = xp >> 5
+                        const int xp = (x & 127) >> 1;
+                        const int want = C::beta_in(xp >> 5, xp & 31) + 256 * (b >> 1) + 2 * (x & 1) + (b & 1);
+                        CHECK(C::beta_dst_off(i) == want, "beta: group %d not where its reader looks", i);
+                    }
+                    CHECK(C::beta_dst_off(q) % 2 == 0, "beta push not 8-byte aligned");
+                }
+    for (int i = 0; i < C::Q; ++i) CHECK(seen[i] == 1, "beta: group %d produced %d times", i, seen[i]);
+}
+
 int main()
 {
+    check_vec2();
     check_beta_in_place();
     check_skew();
     check_alpha<2>();
