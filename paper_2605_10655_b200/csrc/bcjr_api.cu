@@ -334,7 +334,7 @@ bcjr_status plan_cluster(bcjr_ctx *ctx, Kern kern, int CL, int threads, size_t s
 #define VEC4_FWD_NBLK 3
 #endif
 #ifndef VEC2_FWD_NBLK
-#define VEC2_FWD_NBLK 3
+#define VEC2_FWD_NBLK 4
 #endif
 #ifndef VEC4_BWD_NBLK
 #define VEC4_BWD_NBLK 2

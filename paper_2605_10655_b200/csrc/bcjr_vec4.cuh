@@ -722,11 +722,10 @@ __global__ void __launch_bounds__(Vec4BwdCfg<NBLK_>::THREADS, 1) bwd_vec4_kernel
                                 ya = fma2(pb, y, ya);
                                 const float2 rT = mul2(add2(y, Ahj), iT2);                 // r / T
                                 const float2 gam = mul2(pb, f);                            // gamma
-                                const float2 zx = mul2(gam, fma2(rT, sub2(wx, cx), gx));   // gamma (g_v + (w_v - c_v) r / T)
-                                const float2 zy = mul2(gam, fma2(rT, sub2(wy, cy), gy));
-                                Z0 = add2(Z0, zx); Z1 = add2(Z1, zy);
-                                acc[2 * (e + bb)] = add2(acc[2 * (e + bb)], zx);
-                                acc[2 * (e + bb) + 1] = add2(acc[2 * (e + bb) + 1], zy);
+                                const float2 ix = fma2(rT, sub2(wx, cx), gx), iy = fma2(rT, sub2(wy, cy), gy);   // g_v + (w_v - c_v) r / T
+                                Z0 = fma2(gam, ix, Z0); Z1 = fma2(gam, iy, Z1);                                  // z_v = gamma (g_v + (w_v - c_v) r / T)
+                                acc[2 * (e + bb)] = fma2(gam, ix, acc[2 * (e + bb)]);
+                                acc[2 * (e + bb) + 1] = fma2(gam, iy, acc[2 * (e + bb) + 1]);
                             }
                         }
                         tmem_st16(tm_acc + 16u * un, acc);
