@@ -71,7 +71,7 @@ def test_two_weights_per_step_small_and_mid_trellises(ctx, Lb, k, nt, B, T):
 @pytest.mark.parametrize("T", [0.3, 0.05])
 def test_sixteen_bit_state_sixteen_predecessors(ctx, T, path):
     # the paper's own configuration: Lb = 16, 2 bits per weight, 2 weights per step; on the
-    # four-CTA cluster kernels (default) and on the one-CTA-per-block kernels
+    # cluster kernels (default) and on the one-CTA-per-block kernels
     ctx.set_option("path", path)
     try:
         got = _check(ctx, 16, 2, 2, 24, 3, T, seed=8100, what=f"V=2 Lb=16 k=2 T={T} path={path}")
@@ -83,6 +83,20 @@ def test_sixteen_bit_state_sixteen_predecessors(ctx, T, path):
 @pytest.mark.parametrize("nt,B", [(1, 2), (2, 5), (3, 1), (37, 70)])
 def test_cluster_kernels_ragged_step_counts_and_more_blocks_than_clusters(ctx, nt, B):
     _check(ctx, 16, 2, 2, nt, B, 0.2, seed=8500 + nt, what=f"V=2 Lb=16 nt={nt} B={B}")
+
+
+@pytest.mark.parametrize("fwd_variant", [0, 1], ids=["clusters_of_two", "clusters_of_four"])
+def test_cluster_forward_kernels_several_batches_per_cluster(ctx, fwd_variant):
+    # both forward kernels (two-CTA clusters, the default, and four-CTA clusters) with the resident CTAs capped so
+    # that every cluster works through several batches of blocks in flight, the last one ragged
+    ctx.set_option("fwd_variant", fwd_variant)
+    ctx.set_option("max_ctas", 8)
+    try:
+        got = _check(ctx, 16, 2, 2, 9, 19, 0.15, seed=8600 + fwd_variant, what=f"V=2 Lb=16 B=19 capped, fwd_variant={fwd_variant}")
+        assert got["fwd_path"] == 1
+    finally:
+        ctx.set_option("fwd_variant", 0)
+        ctx.set_option("max_ctas", 0)
 
 
 def test_sixteen_bit_state_one_bit_per_weight(ctx):
