@@ -59,6 +59,9 @@ typedef struct {
  *                         the generic one-CTA kernels (more than 10x slower per weight at Lb = 16).
  *   Lb = 11..13, k = 2:   one warp per block, sixteen (forward) or eight (backward) blocks per SM at Lb = 12, table in
  *                         tensor memory; any n.
+ *   V = 2, Lb = 16, k = 2: forward on clusters of two CTAs (n <= 2048), backward on clusters of four (table and
+ *                         gradient accumulators are 1 MB of tensor memory; n <= 1024); longer blocks and every
+ *                         other V = 2 shape run the one-CTA vector kernels.
  *   everything else:      generic kernels, one CTA per block (also "path" = 1).
  * Block lengths of a few hundred weights (the paper uses 256) are the intended range. */
 
@@ -73,7 +76,9 @@ bcjr_status bcjr_destroy(bcjr_ctx *ctx);
  *   "path"        0 auto, 1 force the generic kernels, 2 force the large-trellis kernels
  *                 (BCJR_EUNSUPPORTED at call time when they do not cover the shape)
  *   "fwd_variant" large-trellis forward kernel: 0 = one CTA per block with the codebook in tensor
- *                 memory (Lb = 16, k = 2 or 3), 1 = two-CTA cluster kernel with the codebook in registers
+ *                 memory (Lb = 16, k = 2 or 3), 1 = two-CTA cluster kernel with the codebook in registers.
+ *                 Vector emissions (V = 2, Lb = 16, k = 2): 0 = clusters of two CTAs (the table whole in two
+ *                 tensor memories, all SMs), 1 = clusters of four (the backward kernel's shape)
  *   "bwd_variant" large-trellis backward call (Lb = 16, k = 2 or 3).  0 (default): with grad_codebook, two
  *                 kernels per chunk of as many blocks as the GPU has SMs -- the alpha sweeps on one CTA per
  *                 block, then the beta sweeps on two-CTA clusters with codebook and gradient accumulators in
