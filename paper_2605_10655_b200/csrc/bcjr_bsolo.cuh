@@ -297,12 +297,13 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
                         const float2 f = ex2f2(add2(sub2(m, Dm2), Lhj));
                         // f (w - c) / T = f delta / T - (f / T) du
                         const float2 fg = mul2(f, g2), nfi = mul2(f, ngi2), fid = RC ? mul2(f, gid2) : make_float2(0.f, 0.f);
+                        const float2 nfiA = mul2(nfi, Ahj);                 // plain square: f (w - c) r / T = du (nfi y + nfi At)
                         float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
 #pragma unroll
                         for (int b = 0; b < K; ++b) {
                             const float2 pb = ex2f2(sub2(uu[b], m));
                             const float2 y = fma2(g2, cb[i & 1][C::b_idx(jh, b)], splat2(Yb[b]));   // h + Bt
-                            const float2 z = fma2(RC ? fma2(nfi, d[b], fid) : mul2(nfi, d[b]), add2(y, Ahj), fg);   // f (g + (w - c) r / T)
+                            const float2 z = RC ? fma2(fma2(nfi, d[b], fid), add2(y, Ahj), fg) : fma2(d[b], fma2(nfi, y, nfiA), fg);   // f (g + (w - c) r / T)
                             sum = add2(sum, pb);
                             ya = fma2(pb, y, ya);
                             zs = fma2(pb, z, zs);
