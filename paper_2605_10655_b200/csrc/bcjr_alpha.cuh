@@ -185,7 +185,9 @@ __global__ void __launch_bounds__(AlphaCfg<KB>::THREADS, 1) bwd_alpha_kernel(Bwd
                             float2 sum = pj, ax = mul2(pj, fma2(g2, cb[g & 1][C::a_idx(0, hh)], splat2(Aj[0])));
 #pragma unroll
                             for (int j = 1; j < K; ++j) {
-                                pj = (KB == 2 && j == 3) ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));   // k = 2: one in four on the FP32 pipe
+                                // (no exponential goes to the FP32 pipe here, unlike the forward kernel's alpha sweep: with the
+                                // conditional expectations riding along this sweep is short of issue slots, not of the special-function unit)
+                                pj = ex2f2(sub2(a[j], m));
                                 sum = add2(sum, pj);
                                 ax = fma2(pj, fma2(g2, cb[g & 1][C::a_idx(j, hh)], splat2(Aj[j])), ax);
                             }

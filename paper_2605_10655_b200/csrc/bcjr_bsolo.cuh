@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
                         float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][C::a_idx(0, h)], splat2(Aj[0])));
 #pragma unroll
                         for (int j = 1; j < K; ++j) {
-                            pj = j == 3 ? ex2_poly2(sub2(a[j], m)) : ex2f2(sub2(a[j], m));   // one in four on the FP32 pipe
+                            pj = ex2f2(sub2(a[j], m));
                             sum = add2(sum, pj);
                             ax = fma2(pj, fma2(g2, cb[i & 1][C::a_idx(j, h)], splat2(Aj[j])), ax);
                         }
