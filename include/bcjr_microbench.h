@@ -29,6 +29,9 @@ typedef struct {
     double st_async_bytes_per_clk_sm; /* st.async.v4 to the peer CTA of a two-CTA cluster, both sending, landed */
     double cta_barrier_clk;           /* one named-barrier round of 512 threads, clocks */
     double mbarrier_round_clk;        /* one mbarrier round: an arrival per warp, 16 warps polling, clocks */
+    double fma_f32x2_with_alu_per_clk_sm; /* packed pairs per clock per SM when every packed instruction has an integer
+                                         instruction (another pipe) beside it: equal to fma_f32x2_per_clk_sm if a packed
+                                         instruction takes one issue slot, two thirds of it if it takes two */
 } bcjr_pipe_peaks;
 
 /*

@@ -7,7 +7,8 @@
 // cycles), so bcjr_measure_pipe_peaks measures them on the device the benchmark runs on, in
 // well under a second:
 //   - register-only chains (512 threads per SM, 8 independent chains per thread) for ex2, lg2,
-//     fma.f32 and fma.f32x2 (rcp shares the unit with ex2 and lg2; a chain of reciprocals is not measured
+//     fma.f32, fma.f32x2 and fma.f32x2 with one integer instruction beside each (does a packed instruction, two
+//     cycles on the FP32 pipe, also hold the issue port for two?) (rcp shares the unit with ex2 and lg2; a chain of reciprocals is not measured
 //     because the assembler simplifies it): results per clock per SM (clock64) and per second (CUDA events
 //     over the whole grid, so the clock the GPU actually ran at is part of the number);
 //   - st.async.v4 between the two CTAs of a cluster, both sending, on every SM: bytes landed per
@@ -27,17 +28,19 @@ namespace {
 
 constexpr int MB_THREADS = 512, MB_CHAINS = 8;
 
-enum { OP_EX2 = 0, OP_LG2, OP_FMA, OP_FMA2, OP_COUNT };
+enum { OP_EX2 = 0, OP_LG2, OP_FMA, OP_FMA2, OP_FMA2_ALU, OP_COUNT };
 
 template <int OP>
 __global__ void __launch_bounds__(MB_THREADS, 1) chain_kernel(float *sink, unsigned long long *clk, int iters)
 {
     float x[MB_CHAINS];
     float2 p[MB_CHAINS];
+    unsigned u[MB_CHAINS];
 #pragma unroll
     for (int i = 0; i < MB_CHAINS; ++i) {
         x[i] = 1.0f + threadIdx.x * 1e-3f + i;
         p[i] = make_float2(x[i], x[i] + 1.f);
+        u[i] = threadIdx.x * 2654435761u + i;
     }
     const float2 c1 = make_float2(1.0001f, 0.9999f), c2 = make_float2(1e-3f, 2e-3f);
     __syncthreads();
@@ -48,7 +51,8 @@ __global__ void __launch_bounds__(MB_THREADS, 1) chain_kernel(float *sink, unsig
             if (OP == OP_EX2) asm volatile("ex2.approx.ftz.f32 %0, %0;" : "+f"(x[i]));
             if (OP == OP_LG2) asm volatile("lg2.approx.ftz.f32 %0, %0;" : "+f"(x[i]));
             if (OP == OP_FMA) asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(x[i]) : "f"(c1.x), "f"(c2.x));
-            if (OP == OP_FMA2)
+            if (OP == OP_FMA2_ALU) asm volatile("xor.b32 %0, %0, %1;" : "+r"(u[i]) : "r"(0x9e3779b9u + (unsigned)it));   // an integer instruction per packed one
+            if (OP == OP_FMA2 || OP == OP_FMA2_ALU)
                 asm volatile("{ .reg .b64 ra, rb, rc; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %3}; mov.b64 rc, {%4, %5}; "
                              "fma.rn.f32x2 ra, ra, rb, rc; mov.b64 {%0, %1}, ra; }"
                              : "+f"(p[i].x), "+f"(p[i].y) : "f"(c1.x), "f"(c1.y), "f"(c2.x), "f"(c2.y));
@@ -57,7 +61,7 @@ __global__ void __launch_bounds__(MB_THREADS, 1) chain_kernel(float *sink, unsig
     const long long t1 = clock64();
     float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < MB_CHAINS; ++i) s += x[i] + p[i].x + p[i].y;
+    for (int i = 0; i < MB_CHAINS; ++i) s += x[i] + p[i].x + p[i].y + (float)(u[i] & 255u);
     sink[blockIdx.x * MB_THREADS + threadIdx.x] = s;
     if (threadIdx.x == 0 && blockIdx.x == 0) clk[OP] = (unsigned long long)(t1 - t0);
 }
@@ -196,6 +200,9 @@ extern "C" bcjr_status bcjr_measure_pipe_peaks(int device, bcjr_pipe_peaks *out,
     ok = ok && run_chain<OP_FMA>(sms, iters, sink, clk, st, &out->fma_f32_per_clk_sm, &dummy);
     ok = ok && run_chain<OP_FMA2>(sms, iters, sink, clk, st, &out->fma_f32x2_per_clk_sm, &per_s);
     out->fma_f32x2_gops = per_s * 1e-9;
+    // one integer instruction (another pipe) beside every packed one: pairs per clock per SM again.  The same figure as
+    // without them says a packed instruction leaves the issue port free for a cycle; two thirds of it says it does not.
+    ok = ok && run_chain<OP_FMA2_ALU>(sms, iters, sink, clk, st, &out->fma_f32x2_with_alu_per_clk_sm, &dummy);
     // the clock the chains ran at: results per second / (results per clock per SM * SMs)
     if (ok && out->ex2_per_clk_sm > 0.0) out->sm_clock_mhz = out->ex2_gops * 1e3 / (out->ex2_per_clk_sm * sms);
     out->num_sms = sms;
