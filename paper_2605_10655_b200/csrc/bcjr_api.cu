@@ -543,7 +543,7 @@ bcjr_status launch_bwd_split(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, c
         CU(cudaLaunchKernelEx(&cfg, beta, p));
         ctx->launches += 2;
     }
-    if (ACC) {
+    if (ACC && grad_codebook) {
         reduce_gc_kernel<<<(A::S + 255) / 256, 256, 0, st>>>(p.gc_part, ncl, A::S, grad_codebook);
         ctx->launches += 1;
         CU(cudaGetLastError());
@@ -577,7 +577,7 @@ bcjr_status launch_bwd_cluster(bcjr_ctx *ctx, BwdParams p, int k, float *grad_co
     if (k == 2 && (ctx->opt_bwd_variant == 0 || ctx->opt_bwd_variant == 4) && p.n <= SkewCfg::MAX_N)
         return grad_codebook ? launch_bwd_split<2, true>(ctx, p, grad_codebook, st, bwd_skew_kernel<true, true>, SkewCfg::SMEM_BYTES)
                              : launch_bwd_split<2, false>(ctx, p, nullptr, st, bwd_skew_kernel<false, true>, SkewCfg::SMEM_BYTES);
-    if (k == 3 && (ctx->opt_bwd_variant == 0 || ctx->opt_bwd_variant == 4) && p.n <= DuoCfg<3>::MAX_N && grad_codebook)
+    if (k == 3 && (ctx->opt_bwd_variant == 0 || ctx->opt_bwd_variant == 4) && p.n <= DuoCfg<3>::MAX_N)   // without grad_codebook the partial sums are formed and dropped
         return launch_bwd_split<3, true>(ctx, p, grad_codebook, st, bwd_duo_kernel<3, true>, DuoCfg<3>::SMEM_BYTES);
     if (k == 2 && ctx->opt_bwd_variant == 3 && p.n <= SkewCfg::MAX_N)
         return grad_codebook ? launch_bwd_skew<true>(ctx, p, grad_codebook, st) : launch_bwd_skew<false>(ctx, p, nullptr, st);
