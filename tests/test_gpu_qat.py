@@ -73,8 +73,8 @@ def test_annealed_qat_loop_follows_the_oracle_loop(ctx):
     W0 = rng.standard_normal((B, n)).astype(np.float32)
     target = (W0 + 0.3 * rng.standard_normal((B, n))).astype(np.float32)
     dev = torch.device("cuda", ctx.device)
-    c_dev = ctx.bcjr_gaussian_codebook(Lb)
-    c0 = c_dev.cpu().numpy()
+    c0 = qo.gaussian_codebook(Lb).astype(np.float32)          # both sides start from the oracle's table
+    c_dev = torch.from_numpy(c0.copy()).to(dev)
     W = torch.from_numpy(W0.copy()).to(dev); tgt = torch.from_numpy(target).to(dev)
     mW = torch.zeros_like(W); vW = torch.zeros_like(W); mc = torch.zeros_like(c_dev); vc = torch.zeros_like(c_dev)
     rW, rc = W0.astype(np.float64), c0.astype(np.float64)
