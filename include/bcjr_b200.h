@@ -58,7 +58,8 @@ typedef struct {
  *                         four-CTA register kernel (about 1.7x slower per weight), and anything longer
  *                         the generic one-CTA kernels (more than 10x slower per weight at Lb = 16).
  *   Lb = 11..13, k = 2:   one warp per block, sixteen (forward) or eight (backward) blocks per SM at Lb = 12, table in
- *                         tensor memory; any n.
+ *                         tensor memory; any n.  The backward call with grad_codebook at Lb = 12, 13 gives a block to
+ *                         two warps ("bwd_variant" = 1: one warp).
  *   V = 2, Lb = 16, k = 2: forward on clusters of two CTAs (n <= 2048), backward on clusters of four (table and
  *                         gradient accumulators are 1 MB of tensor memory; n <= 1024); longer blocks and every
  *                         other V = 2 shape run the one-CTA vector kernels.

@@ -703,6 +703,33 @@ bcjr_status launch_bwd_warp(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cu
     return BCJR_OK;
 }
 
+// Backward call with grad_codebook at Lb = 12, 13: two warps per block (twice the warps per SM for the same tensor memory).
+template <int LB>
+bcjr_status launch_bwd_warp2(bcjr_ctx *ctx, BwdParams p, float *grad_codebook, cudaStream_t st)
+{
+    using C = Warp2Cfg<LB>;
+    CU(cudaFuncSetAttribute(bwd_warp2_kernel<LB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin));
+    int64_t grid = ctx->num_sms;
+    if (ctx->opt_max_ctas > 0 && grid > ctx->opt_max_ctas) grid = ctx->opt_max_ctas;
+    const int64_t need = (p.B + C::NPAIR - 1) / C::NPAIR;
+    if (grid > need) grid = need;
+    const size_t pairs = (size_t)grid * C::NPAIR;
+    bcjr_status rc;
+    if ((rc = ensure(ctx, ctx->hist, pairs * p.n * 2 * C::Q * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->stepO, pairs * ((size_t)p.n + 2) * 4))) return rc;
+    if ((rc = ensure(ctx, ctx->gc_part, pairs * C::S * 4))) return rc;
+    p.hist = (float *)ctx->hist.ptr;
+    p.stepO = (int *)ctx->stepO.ptr;
+    p.gc_part = (float *)ctx->gc_part.ptr;
+    if (ctx->cb_computed) p.cb = nullptr;
+    bwd_warp2_kernel<LB><<<(int)grid, C::THREADS, C::SMEM_BYTES, st>>>(p);
+    CU(cudaGetLastError());
+    reduce_gc_kernel<<<(C::S + 255) / 256, 256, 0, st>>>(p.gc_part, (int)pairs, C::S, grad_codebook);
+    ctx->launches += 2;
+    CU(cudaGetLastError());
+    return BCJR_OK;
+}
+
 bcjr_status launch_fwd_warp_any(bcjr_ctx *ctx, FwdParams p, cudaStream_t st)
 {
     switch (p.Lb) {
@@ -716,8 +743,12 @@ bcjr_status launch_bwd_warp_any(bcjr_ctx *ctx, BwdParams p, float *gc, cudaStrea
 {
     switch (p.Lb) {
         case 11: return gc ? launch_bwd_warp<11, true>(ctx, p, gc, st) : launch_bwd_warp<11, false>(ctx, p, gc, st);
-        case 12: return gc ? launch_bwd_warp<12, true>(ctx, p, gc, st) : launch_bwd_warp<12, false>(ctx, p, gc, st);
-        default: return gc ? launch_bwd_warp<13, true>(ctx, p, gc, st) : launch_bwd_warp<13, false>(ctx, p, gc, st);
+        case 12:
+            if (gc && ctx->opt_bwd_variant != 1) return launch_bwd_warp2<12>(ctx, p, gc, st);
+            return gc ? launch_bwd_warp<12, true>(ctx, p, gc, st) : launch_bwd_warp<12, false>(ctx, p, gc, st);
+        default:
+            if (gc && ctx->opt_bwd_variant != 1) return launch_bwd_warp2<13>(ctx, p, gc, st);
+            return gc ? launch_bwd_warp<13, true>(ctx, p, gc, st) : launch_bwd_warp<13, false>(ctx, p, gc, st);
     }
 }
 

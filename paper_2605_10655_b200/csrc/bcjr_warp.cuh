@@ -488,4 +488,317 @@ __global__ void __launch_bounds__(WarpCfg<LB, true>::THREADS, 1) bwd_warp_kernel
     if (warp == 0) tmem_dealloc_512(tmem_base);
 }
 
+// Backward call with grad_codebook at Lb = 12, 13: TWO warps per weight block.
+//
+// Table plus accumulators are 2 x 2^Lb floats per block; with one warp per block that is 256 (Lb = 12) or 512 (Lb = 13)
+// columns per lane, so only eight or four warps fit an SM and the schedulers run short of warps to pick from (issue
+// slots two thirds used).  Here the butterflies of a block are split between two warps -- half the columns each, twice
+// the warps per SM for the same number of resident blocks.  The pair shares the block's message buffers; one named
+// barrier of 64 threads per step orders them (the gauge maximum and the posterior sums of the two warps meet in a few
+// words of shared memory, read after that barrier).  Everything else is bwd_warp_kernel.
+template <int LB_>
+struct Warp2Cfg {
+    using W = WarpCfg<LB_, true>;
+    static constexpr int LB = LB_, KB = 2, K = 4, S = W::S, Q = W::Q, NB = W::NB;
+    static constexpr int BPT = W::BPT / 2;                     // butterflies per lane and warp: 4 (Lb = 12), 8 (Lb = 13)
+    static constexpr int UNITS = 1, HPU = 2;
+    static constexpr int COLS = 32 * BPT;                      // table + accumulators
+    static constexpr int NWARP = 2048 / COLS < 16 ? 2048 / COLS : 16;
+    static constexpr int NPAIR = NWARP / 2, THREADS = 32 * NWARP;
+    static constexpr int RD = BPT < 8 ? BPT : 8;
+    static constexpr int MSG = 4 * Q;                          // floats per pair: two parities of (L, At)
+    static constexpr int RING = RD * 2 * 32 * 4;               // floats per warp
+    static constexpr int XCH = 32;                             // floats per pair: gauge maxima [2][2], sums [2][2][4], log Z partials [2]
+    static constexpr int PER_PAIR = MSG + 2 * RING + XCH;
+    static constexpr int OFF_TMEM = NPAIR * PER_PAIR;
+    static constexpr int SMEM_FLOATS = OFF_TMEM + 4;
+    static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
+    static_assert(LB == 12 || LB == 13, "two warps per block: 2^12 and 2^13 states");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
+    static_assert(NPAIR + 1 <= 15, "one named barrier per pair");
+    __host__ __device__ static constexpr int a_idx(int j, int h) { return 2 * j + h; }
+    __host__ __device__ static constexpr int b_idx(int jh, int b) { return 4 * jh + b; }
+};
+
+__device__ __forceinline__ void pair_barrier(int pair)
+{
+    asm volatile("bar.sync %0, 64;" ::"r"(pair + 1) : "memory");
+}
+
+// p.gc_part: [pairs][S]; p.hist: [pairs][n][2 warps][BPT][2][32] float4; p.stepO: [pairs][n + 2].
+template <int LB>
+__global__ void __launch_bounds__(Warp2Cfg<LB>::THREADS, 1) bwd_warp2_kernel(BwdParams p)
+{
+    using C = Warp2Cfg<LB>;
+    constexpr int K = C::K, NB = C::NB, Q = C::Q, BPT = C::BPT, RD = C::RD;
+    extern __shared__ __align__(16) float smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, pw = warp & 1, pair = warp >> 1;
+    const int n = p.n;
+    const float NEG_INF = __int_as_float(0xff800000);
+    const float invT = p.invT;
+    const float2 nl2 = splat2(-p.lam2);
+    const float c_lo = p.diag->c_lo, c_hi = p.diag->c_hi;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + C::OFF_TMEM);
+
+    float *msg = smem + pair * C::PER_PAIR;                               // [2 parities][L | At][Q], shared by the pair
+    float4 *stage4 = reinterpret_cast<float4 *>(msg + C::MSG + pw * C::RING);   // [RD][2][32], thread-private entries
+    float *xch = msg + C::MSG + 2 * C::RING;
+    float *wm = xch;                                                      // [2 parities][2 warps]
+    float *part = xch + 4;                                                // [2 parities][2 warps][4]
+    float *lzp = xch + 20;                                                // [2 warps]
+    const uint32_t stage_u32 = smem_u32(stage4) + (uint32_t)lane * 16u;
+    const int64_t pg = (int64_t)blockIdx.x * C::NPAIR + pair, npg = (int64_t)gridDim.x * C::NPAIR;
+    const int x0 = pw * BPT * 32 + lane;                                  // this thread's butterflies: x0 + 32 i
+    float4 *hist4 = reinterpret_cast<float4 *>(p.hist + (size_t)pg * n * 2 * Q) + pw * (BPT * 2 * 32) + lane;   // row t: [2][BPT][2][32]
+    constexpr int HROW = 2 * BPT * 2 * 32;
+    int *O_g = p.stepO + (size_t)pg * (n + 2);
+
+    if (warp == 0) tmem_alloc_512(smem_u32(const_cast<uint32_t *>(tmem_slot)));
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tm_cb = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * C::COLS);
+    const uint32_t tm_acc = tm_cb + 16u * BPT;
+    {
+        float2 z[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z[e] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) tmem_st16(tm_acc + 16u * i, z);
+        tmem_wait_st();
+    }
+    float defect = 0.f;
+
+    for (int64_t blk = pg; blk < p.B; blk += npg) {
+        const float *w_s = p.W + blk * n, *g_s = p.g + blk * n, *sf_s = p.soft + blk * n;
+        {
+            const float gsh1 = -__ldg(g_s) * __ldg(sf_s);                 // L_1 = 0; the At array carries At + gsh (see bcjr_duo.cuh)
+            for (int q = pw * 32 + lane; q < Q; q += 64) { msg[q] = 0.f; msg[Q + q] = gsh1; }
+        }
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, x0 + 32 * i, tm_cb + (uint32_t)(16 * i), false);
+        tmem_wait_st();
+        int O = 0;
+        float off = 0.f, cmax = 0.f;
+        if (pw == 0 && lane == 0) O_g[1] = 0;
+        pair_barrier(pair);
+        // ================= alpha sweep carrying (L, At)
+        for (int t = 1; t <= n; ++t) {
+            const int cur = (t - 1) & 1;
+            const float *Lin = msg + cur * 2 * Q, *Ain = Lin + Q;
+            float *Lout = msg + (cur ^ 1) * 2 * Q, *Aout = Lout + Q;
+            float2 cb[2][8];
+            tmem_ld16(tm_cb, cb[0]);
+            const float gt = __ldg(g_s + t - 1);
+            const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
+            const StepEnergy se = step_energy(__ldg(w_s + t - 1), c_lo, c_hi, p.lam2);
+            if (t > 1) {
+                cmax = fmaxf(wm[cur * 2], wm[cur * 2 + 1]) - off;            // maximum of this step's inputs as stored
+                off = rintf(cmax);
+            }
+            const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt), off2 = splat2(off), gshn2 = splat2(gshn);
+            float4 *hrow = hist4 + (size_t)(t - 1) * HROW;
+            float tmax = NEG_INF;
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                const int x = x0 + 32 * i;
+                float Lj[K], Aj[K];
+#pragma unroll
+                for (int j = 0; j < K; ++j) {
+                    Lj[j] = Lin[j * NB + x];
+                    Aj[j] = Ain[j * NB + x];
+                }
+                hrow[(i * 2) * 32] = make_float4(Lj[0], Lj[1], Lj[2], Lj[3]);
+                hrow[(i * 2 + 1) * 32] = make_float4(Aj[0], Aj[1], Aj[2], Aj[3]);
+                tmem_wait_ld(cb[i & 1]);
+                if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
+                float2 outL[K / 2], outA[K / 2];
+#pragma unroll
+                for (int h = 0; h < K / 2; ++h) {
+                    float2 a[K];
+#pragma unroll
+                    for (int j = 0; j < K; ++j) a[j] = energy2(sub2(cb[i & 1][C::a_idx(j, h)], w2), nl2, kap2, splat2(Lj[j]));
+                    const float2 m = max_pairs<K>(a);
+                    float2 pj = ex2f2(sub2(a[0], m));
+                    float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][C::a_idx(0, h)], splat2(Aj[0])));
+#pragma unroll
+                    for (int j = 1; j < K; ++j) {
+                        pj = ex2f2(sub2(a[j], m));
+                        sum = add2(sum, pj);
+                        ax = fma2(pj, fma2(g2, cb[i & 1][C::a_idx(j, h)], splat2(Aj[j])), ax);
+                    }
+                    outL[h] = add2(sub2(m, off2), lg2f2(sum));
+                    outA[h] = fma2(ax, rcpf2(sum), gshn2);
+                    tmax = max3f(tmax, m.x, m.y);
+                }
+                *reinterpret_cast<float4 *>(Lout + x * K) = make_float4(outL[0].x, outL[0].y, outL[1].x, outL[1].y);
+                *reinterpret_cast<float4 *>(Aout + x * K) = make_float4(outA[0].x, outA[0].y, outA[1].x, outA[1].y);
+            }
+            tmax = warp_max(tmax);
+            if (lane == 0) wm[(cur ^ 1) * 2 + pw] = tmax;
+            O += (int)off;
+            if (pw == 0 && lane == 0) O_g[t + 1] = O;
+            pair_barrier(pair);
+        }
+        // ================= log2 Z
+        cmax = fmaxf(wm[(n & 1) * 2], wm[(n & 1) * 2 + 1]) - off;
+        float lsefin;
+        {
+            const float *Lfin = msg + (n & 1) * 2 * Q;
+            float ssum = 0.f;
+            for (int q = pw * 32 + lane; q < Q; q += 64) ssum += ex2f(Lfin[q] - cmax);
+            ssum = warp_sum(ssum);
+            if (lane == 0) lzp[pw] = ssum;
+            pair_barrier(pair);
+            lsefin = cmax + lg2f(lzp[0] + lzp[1]);
+        }
+        if (pw == 0 && lane == 0) diag_check_finite(p.diag, lsefin);
+        const int Ofin = O;
+        pair_barrier(pair);                                               // everybody has read the last alpha messages and lzp
+        // ================= beta sweep carrying (M, Bt), with the gradient contraction
+        {
+            const float gshn = -__ldg(g_s + n - 1) * __ldg(sf_s + n - 1);   // M_n = 0, Bt_n = 0 (+ centring shift)
+            for (int q = pw * 32 + lane; q < Q; q += 64) { msg[q] = 0.f; msg[Q + q] = gshn; }
+        }
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) stage_codebook<C>(p.cb, x0 + 32 * i, tm_cb + (uint32_t)(16 * i), true);
+        tmem_wait_st();
+        int P = 0;
+        float offM = 0.f;
+        int nt = n, ni = 0;
+        auto issue_chunk = [&](uint32_t slot) {
+            const float4 *src = hist4 + (size_t)(nt - 1) * HROW + ni * 64;
+            const uint32_t dst = stage_u32 + slot * 1024u;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 512u), "l"(src + 32) : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            if (++ni == BPT) { ni = 0; if (nt > 1) --nt; }
+        };
+#pragma unroll
+        for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c);
+        uint32_t slot = 0;
+        int Ot = O_g[n];
+        // pair, warp 0, lane 0: turn the sums of step t (slots of parity b) into grad_W[t]
+        auto finish_step = [&](int t, int b) {
+            if (pw == 0 && lane == 0) {
+                const float *pp = part + b * 8;
+                const float a0 = pp[0] + pp[4], a2 = pp[1] + pp[5], az = pp[2] + pp[6];
+                const float i0 = 1.f / a0;
+                p.gW[blk * n + t - 1] = (__ldg(g_s + t - 1) - az * i0) + (a2 * i0) * (__ldg(w_s + t - 1) - __ldg(sf_s + t - 1)) * invT;
+                defect = fmaxf(defect, fabsf(a0 - 1.f));
+            }
+        };
+        pair_barrier(pair);
+        for (int t = n; t >= 1; --t) {
+            const int cur = (n - t) & 1;
+            const float *Min = msg + cur * 2 * Q, *Bin = Min + Q;
+            float *Mout = msg + (cur ^ 1) * 2 * Q, *Bout = Mout + Q;
+            const int Onext = t > 1 ? O_g[t - 1] : 0;
+            if (t < n) {
+                P += (int)offM;
+                cmax = fmaxf(wm[cur * 2], wm[cur * 2 + 1]);
+                offM = rintf(cmax);
+                finish_step(t + 1, cur);
+            }
+            const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1), st = __ldg(sf_s + t - 1);
+            const float gsh = -gt * st;                                     // shift carried by the stored At
+            const float gshp = t > 1 ? -__ldg(g_s + t - 2) * __ldg(sf_s + t - 2) : 0.f;   // for step t-1
+            const StepEnergy se = step_energy(wt, c_lo, c_hi, p.lam2);
+            const float2 w2 = splat2(se.wc), kap2 = splat2(se.kap), g2 = splat2(gt), ngi2 = splat2(-invT), gid2 = splat2(invT * se.delta);
+            const float2 gsh2 = splat2(gsh), gshp2 = splat2(gshp), offM2 = splat2(offM);
+            const float2 Dm2 = splat2((float)(Ofin - Ot - P) + lsefin);
+            float2 S0 = make_float2(0.f, 0.f), S2 = S0, ZS = S0;
+            float tmax = NEG_INF;
+            float2 cb[2][8];
+            tmem_ld16(tm_cb, cb[0]);
+#pragma unroll
+            for (int i = 0; i < BPT; ++i) {
+                const int x = x0 + 32 * i;
+                issue_chunk(slot == 0 ? RD - 1 : slot - 1);
+                asm volatile("cp.async.wait_group %0;" ::"n"(RD - 1) : "memory");
+                const float4 l4 = stage4[slot * 64 + lane], a4 = stage4[slot * 64 + 32 + lane];
+                const float Lh[K] = {l4.x, l4.y, l4.z, l4.w}, Ah[K] = {a4.x, a4.y, a4.z, a4.w};
+                slot = slot + 1 == RD ? 0 : slot + 1;
+                const float4 mv = *reinterpret_cast<const float4 *>(Min + x * K);
+                const float4 bv = *reinterpret_cast<const float4 *>(Bin + x * K);
+                const float Mb[K] = {mv.x, mv.y, mv.z, mv.w}, Yb[K] = {bv.x, bv.y, bv.z, bv.w};
+                float2 acc[8];
+                tmem_wait_ld(cb[i & 1]);
+                tmem_ld16(tm_acc + 16u * i, acc);
+                if (i + 1 < BPT) tmem_ld16(tm_cb + 16u * (i + 1), cb[(i + 1) & 1]);
+                bool acc_ready = false;
+#pragma unroll
+                for (int jh = 0; jh < K / 2; ++jh) {
+                    float2 uu[K], d[K];
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        d[b] = sub2(cb[i & 1][C::b_idx(jh, b)], w2);        // du = c - wc
+                        uu[b] = energy2(d[b], nl2, kap2, splat2(Mb[b]));
+                    }
+                    const float2 m = max_pairs<K>(uu);
+                    const float2 Ahj = sub2(make_float2(Ah[2 * jh], Ah[2 * jh + 1]), gsh2);
+                    const float2 f = ex2f2(add2(sub2(m, Dm2), make_float2(Lh[2 * jh], Lh[2 * jh + 1])));
+                    const float2 fg = mul2(f, g2), nfi = mul2(f, ngi2), fid = mul2(f, gid2);   // f (w - c) / T = f delta / T - (f / T) du
+                    if (!acc_ready) { tmem_wait_ld(acc); acc_ready = true; }
+                    float2 sum = make_float2(0.f, 0.f), ya = sum, zs = sum;
+#pragma unroll
+                    for (int b = 0; b < K; ++b) {
+                        const float2 pb = ex2f2(sub2(uu[b], m));
+                        const float2 y = fma2(g2, cb[i & 1][C::b_idx(jh, b)], splat2(Yb[b]));   // h + Bt
+                        const float2 z = fma2(fma2(nfi, d[b], fid), add2(y, Ahj), fg);            // f (g + (w - c) r / T)
+                        sum = add2(sum, pb);
+                        ya = fma2(pb, y, ya);
+                        zs = fma2(pb, z, zs);
+                        acc[C::b_idx(jh, b)] = fma2(pb, z, acc[C::b_idx(jh, b)]);
+                    }
+                    const float2 outM = add2(sub2(m, offM2), lg2f2(sum));
+                    const float2 outB = fma2(ya, rcpf2(sum), gshp2);
+                    tmax = max3f(tmax, m.x, m.y);
+                    Mout[(2 * jh) * NB + x] = outM.x; Mout[(2 * jh + 1) * NB + x] = outM.y;
+                    Bout[(2 * jh) * NB + x] = outB.x; Bout[(2 * jh + 1) * NB + x] = outB.y;
+                    S0 = fma2(f, sum, S0);
+                    S2 = fma2(f, fma2(Ahj, sum, ya), S2);
+                    ZS = add2(ZS, zs);
+                }
+                tmem_st16(tm_acc + 16u * i, acc);
+            }
+            tmem_wait_st();
+            tmax = warp_max(tmax) - offM;
+            // lanes 0-7 hold sum gamma, 8-15 sum gamma r, 16-23 sum gamma z
+            const float s3 = warp_sum3_split(S0.x + S0.y, S2.x + S2.y, ZS.x + ZS.y, lane);
+            if (lane == 0) wm[(cur ^ 1) * 2 + pw] = tmax;
+            if ((lane & 7) == 0 && lane < 24) part[(cur ^ 1) * 8 + pw * 4 + (lane >> 3)] = s3;
+            Ot = Onext;
+            pair_barrier(pair);
+        }
+        finish_step(1, n & 1);
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        pair_barrier(pair);                                               // the exchange words are free for the next block
+    }
+    {
+        // this pair's partial of grad_codebook: beta pair (jh, b) of butterfly x holds states [2jh | x | b], [2jh+1 | x | b]
+        float *gc = p.gc_part + (size_t)pg * C::S;
+        tmem_wait_st();
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) {
+            const int x = x0 + 32 * i;
+            float2 acc[8];
+            tmem_ld16(tm_acc + 16u * i, acc);
+            tmem_wait_ld(acc);
+#pragma unroll
+            for (int jh = 0; jh < K / 2; ++jh)
+#pragma unroll
+                for (int b = 0; b < K; ++b) {
+                    gc[(size_t)(2 * jh) * Q + (size_t)x * K + b] = acc[C::b_idx(jh, b)].x;
+                    gc[(size_t)(2 * jh + 1) * Q + (size_t)x * K + b] = acc[C::b_idx(jh, b)].y;
+                }
+        }
+    }
+    if (pw == 0 && lane == 0) diag_max(&p.diag->max_defect, defect);
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) tmem_dealloc_512(tmem_base);
+}
+
 }  // namespace bcjr

@@ -110,6 +110,14 @@ def test_one_warp_per_block_kernels(ctx, Lb, n, B, T):
     np.testing.assert_array_equal(again["soft"], got["soft"])
     np.testing.assert_array_equal(again["grad_W"], got["grad_W"])
     assert parity.rel_inf(again["grad_codebook"], got["grad_codebook"]) < 1e-5
+    if Lb >= 12:
+        # with grad_codebook the default at Lb = 12, 13 gives a block to two warps; the one-warp kernel stays selectable
+        ctx.set_option("bwd_variant", 1)
+        try:
+            one = _check_all(ctx, W, c, g, Lb, k, T, f"one warp per block (backward) Lb={Lb} n={n} B={B}", viterbi=False)
+        finally:
+            ctx.set_option("bwd_variant", 0)
+        assert one["diag"].last_path == 2 and parity.rel_inf(one["grad_W"], got["grad_W"]) < 2e-5
 
 
 def test_more_blocks_than_resident_ctas(ctx):
