@@ -34,10 +34,6 @@ WORKLOADS = {"tiny": synth.tiny, "mid": synth.mid, "q_proj": synth.q_proj, "laye
              "gate_k3": synth.gate_k3, "qtip_v2": synth.qtip_v2}
 # (Lb, k, kernel) -> measured DRAM bytes per weight block (n = 256), see profiles/*.md
 NCU_DRAM_BYTES_PER_BLOCK = {(16, 2, "bwd"): 66.3e6, (16, 2, "fwd"): 33.1e6}
-# (Lb, k, kernel) -> issue slots per state-step and thread of the kernels that serve it: warp instructions of a small-case
-# launch under ncu (smsp__inst_executed, profiles/*.md), packed f32x2 instructions counted twice, x 32 threads,
-# / (blocks x steps x states).  Backward = alpha kernel 12.2 + beta kernel 22.8.
-NCU_ISSUE_SLOTS_PER_STATE_STEP = {(16, 2, "fwd"): 22.1, (16, 2, "bwd"): 35.0}
 MUFU_PER_CLK_PER_SM = 16          # special-function results per clock per SM (CUDA throughput table, cc 10.0)
 NUM_SMS = 148
 
@@ -492,21 +488,6 @@ def main():
         hbm = {"achieved_gbs": gbs, "peak_gbs": hbm_peak or 6650.0,
                "peak_source": "MEASURED_PEAKS.json (measured copy bandwidth)" if hbm_peak else "fallback 6.65 TB/s",
                "frac": gbs / (hbm_peak or 6650.0)}
-    # Second view: the warp schedulers' issue ports.  A packed f32x2 instruction holds its scheduler's port for two
-    # cycles (the in-run micro-benchmark: packed instructions with an integer instruction beside each run at two
-    # thirds of the rate of packed instructions alone), so a kernel's demand is scalar instructions + 2 x packed ones.
-    issue = None
-    s_f, s_b = (NCU_ISSUE_SLOTS_PER_STATE_STEP.get((wl.Lb, wl.k, kk)) for kk in ("fwd", "bwd"))
-    if s_f and s_b and diag.last_path == 1 and wl.V == 1 and not args.fixed_table:
-        slot_peak = NUM_SMS * 4 * 32 * peaks["sm_clock_mhz"] * 1e6            # thread-slots per second: 4 schedulers x 32 lanes per SM
-        issue = {"slots_per_state_step": {"fwd": s_f, "bwd": s_b},
-                 "source": "ncu warp-instruction counts of small-case launches (profiles/), packed f32x2 counted twice",
-                 "packed_rate_alone_per_clk_sm": peaks["fma_f32x2_per_clk_sm"],
-                 "packed_rate_with_integer_instruction_beside_per_clk_sm": peaks["fma_f32x2_with_alu_per_clk_sm"],
-                 "peak_thread_slots_per_s": slot_peak,
-                 "fwd_frac": s_f * state_steps / (fwd_ms / args.steps * 1e-3) / slot_peak,
-                 "bwd_frac": s_b * state_steps / (bwd_ms / args.steps * 1e-3) / slot_peak,
-                 "whole_step_frac": (s_f + s_b) * state_steps / (ms_per_step * 1e-3) / slot_peak}
     roofline = {"bound": "alu", "kernel": f"bcjr_{dom}", "achieved": achieved, "peak": peak, "unit": "Gop/s (MUFU)",
                 "frac": achieved / peak, "frac_with_rcp": fr[f"{dom}_frac_with_rcp"],
                 "count": "frac: algorithmic special-function operations per state-step (2 + 3/K per call: ex2 per state, "
@@ -521,11 +502,12 @@ def main():
                 "avg_launch_ms": dom_ms, "hbm": hbm,
                 "fwd_frac": fr["fwd_frac"], "bwd_frac": fr["bwd_frac"], "whole_step_frac": fr["both_frac"],
                 "whole_step_frac_with_rcp": fr["both_frac_with_rcp"],
-                "binding_pipe": {"fwd": "special-function unit (75 % busy) with the issue ports at 83 %",
-                                 "bwd": "the warp schedulers' issue ports (alpha kernel 75 %, beta kernel 85 % of the slots, "
-                                        "packed f32x2 instructions taking two): the gradient recursion needs 35 slots per "
-                                        "state-step against the 26 that 3.25 special-function operations leave room for"},
-                "issue": issue,
+                "binding_pipe": {"fwd": "special-function unit 76 % busy; FP32 pipe 55 % + integer pipe 24 % of the cycles "
+                                        "(ncu sm__pipe_fma_cycles_active, sm__pipe_alu_cycles_active)",
+                                 "bwd": "alpha kernel: special-function unit 74 %; beta kernel: FP32 pipe 57 % + integer pipe 21 % of "
+                                        "the cycles, special-function unit 53 %.  Integer-pipe instructions do not overlap with "
+                                        "packed f32x2 ones (pipe_peaks: packed pairs per clock alone and with an integer "
+                                        "instruction beside each), so the two pipes act as one resource 78 % busy"},
                 "pipe_peaks": peaks}
 
     # ---- short legs over the other workloads, so that one line carries every configuration
