@@ -30,8 +30,11 @@ typedef struct {
     double cta_barrier_clk;           /* one named-barrier round of 512 threads, clocks */
     double mbarrier_round_clk;        /* one mbarrier round: an arrival per warp, 16 warps polling, clocks */
     double fma_f32x2_with_alu_per_clk_sm; /* packed pairs per clock per SM when every packed instruction has an integer
-                                         instruction (another pipe) beside it: equal to fma_f32x2_per_clk_sm if a packed
-                                         instruction takes one issue slot, two thirds of it if it takes two */
+                                         instruction (the ALU pipe) beside it: equal to fma_f32x2_per_clk_sm if the two
+                                         pipes overlap, two thirds of it if they take turns */
+    double fma_f32x2_with_max_per_clk_sm; /* the same with a max.f32 (also the ALU pipe) beside every packed instruction */
+    double fma_f32x2_with_ex2_per_clk_sm; /* the same with one ex2.approx (special-function unit) per four packed instructions */
+    double fma_f32x2_with_f64_per_clk_sm; /* the same with one fma.f64 (fp64 pipe) per two packed instructions */
 } bcjr_pipe_peaks;
 
 /*

@@ -30,7 +30,8 @@ class PipePeaks(ctypes.Structure):
     _fields_ = [("num_sms", ctypes.c_int32), ("pad", ctypes.c_int32)] + [(n, ctypes.c_double) for n in (
         "sm_clock_mhz", "ex2_per_clk_sm", "lg2_per_clk_sm", "fma_f32_per_clk_sm",
         "fma_f32x2_per_clk_sm", "ex2_gops", "fma_f32x2_gops", "st_async_bytes_per_clk_sm", "cta_barrier_clk",
-        "mbarrier_round_clk", "fma_f32x2_with_alu_per_clk_sm")]
+        "mbarrier_round_clk", "fma_f32x2_with_alu_per_clk_sm", "fma_f32x2_with_max_per_clk_sm",
+        "fma_f32x2_with_ex2_per_clk_sm", "fma_f32x2_with_f64_per_clk_sm")]
 
 
 class Diag(ctypes.Structure):

@@ -28,7 +28,7 @@ namespace {
 
 constexpr int MB_THREADS = 512, MB_CHAINS = 8;
 
-enum { OP_EX2 = 0, OP_LG2, OP_FMA, OP_FMA2, OP_FMA2_ALU, OP_COUNT };
+enum { OP_EX2 = 0, OP_LG2, OP_FMA, OP_FMA2, OP_FMA2_ALU, OP_FMA2_MAX, OP_FMA2_EX2, OP_FMA2_F64, OP_COUNT };
 
 template <int OP>
 __global__ void __launch_bounds__(MB_THREADS, 1) chain_kernel(float *sink, unsigned long long *clk, int iters)
@@ -36,6 +36,9 @@ __global__ void __launch_bounds__(MB_THREADS, 1) chain_kernel(float *sink, unsig
     float x[MB_CHAINS];
     float2 p[MB_CHAINS];
     unsigned u[MB_CHAINS];
+    double dd[MB_CHAINS / 2];
+#pragma unroll
+    for (int i = 0; i < MB_CHAINS / 2; ++i) dd[i] = 1.0 + threadIdx.x * 1e-6 + i;
 #pragma unroll
     for (int i = 0; i < MB_CHAINS; ++i) {
         x[i] = 1.0f + threadIdx.x * 1e-3f + i;
@@ -46,13 +49,17 @@ __global__ void __launch_bounds__(MB_THREADS, 1) chain_kernel(float *sink, unsig
     __syncthreads();
     const long long t0 = clock64();
     for (int it = 0; it < iters; ++it) {
+        const float vary = 1.0f + 1e-3f * (float)it;               // an operand that changes every iteration, so that nothing folds
 #pragma unroll
         for (int i = 0; i < MB_CHAINS; ++i) {
             if (OP == OP_EX2) asm volatile("ex2.approx.ftz.f32 %0, %0;" : "+f"(x[i]));
             if (OP == OP_LG2) asm volatile("lg2.approx.ftz.f32 %0, %0;" : "+f"(x[i]));
             if (OP == OP_FMA) asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(x[i]) : "f"(c1.x), "f"(c2.x));
             if (OP == OP_FMA2_ALU) asm volatile("xor.b32 %0, %0, %1;" : "+r"(u[i]) : "r"(0x9e3779b9u + (unsigned)it));   // an integer instruction per packed one
-            if (OP == OP_FMA2 || OP == OP_FMA2_ALU)
+            if (OP == OP_FMA2_MAX) asm volatile("max.f32 %0, %0, %1;" : "+f"(x[i]) : "f"(vary));                          // a float maximum (integer pipe) per packed one
+            if (OP == OP_FMA2_EX2 && (i & 3) == 0) asm volatile("ex2.approx.ftz.f32 %0, %0;" : "+f"(x[i]));                // a special-function instruction per four packed ones
+            if (OP == OP_FMA2_F64 && (i & 1) == 0) asm volatile("fma.rn.f64 %0, %0, %1, %2;" : "+d"(dd[i >> 1]) : "d"(1.0000001), "d"(1e-9));   // an fp64 instruction per two packed ones
+            if (OP >= OP_FMA2)
                 asm volatile("{ .reg .b64 ra, rb, rc; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %3}; mov.b64 rc, {%4, %5}; "
                              "fma.rn.f32x2 ra, ra, rb, rc; mov.b64 {%0, %1}, ra; }"
                              : "+f"(p[i].x), "+f"(p[i].y) : "f"(c1.x), "f"(c1.y), "f"(c2.x), "f"(c2.y));
@@ -61,7 +68,7 @@ __global__ void __launch_bounds__(MB_THREADS, 1) chain_kernel(float *sink, unsig
     const long long t1 = clock64();
     float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < MB_CHAINS; ++i) s += x[i] + p[i].x + p[i].y + (float)(u[i] & 255u);
+    for (int i = 0; i < MB_CHAINS; ++i) s += x[i] + p[i].x + p[i].y + (float)(u[i] & 255u) + (float)dd[i >> 1];
     sink[blockIdx.x * MB_THREADS + threadIdx.x] = s;
     if (threadIdx.x == 0 && blockIdx.x == 0) clk[OP] = (unsigned long long)(t1 - t0);
 }
@@ -201,8 +208,13 @@ extern "C" bcjr_status bcjr_measure_pipe_peaks(int device, bcjr_pipe_peaks *out,
     ok = ok && run_chain<OP_FMA2>(sms, iters, sink, clk, st, &out->fma_f32x2_per_clk_sm, &per_s);
     out->fma_f32x2_gops = per_s * 1e-9;
     // one integer instruction (another pipe) beside every packed one: pairs per clock per SM again.  The same figure as
-    // without them says a packed instruction leaves the issue port free for a cycle; two thirds of it says it does not.
+    // without them says the two pipes overlap; two thirds of it says they do not.
     ok = ok && run_chain<OP_FMA2_ALU>(sms, iters, sink, clk, st, &out->fma_f32x2_with_alu_per_clk_sm, &dummy);
+    // the same question for a float maximum (integer pipe), a special-function instruction per four packed ones and
+    // an fp64 instruction per two: packed pairs per clock per SM in each mix
+    ok = ok && run_chain<OP_FMA2_MAX>(sms, iters, sink, clk, st, &out->fma_f32x2_with_max_per_clk_sm, &dummy);
+    ok = ok && run_chain<OP_FMA2_EX2>(sms, iters, sink, clk, st, &out->fma_f32x2_with_ex2_per_clk_sm, &dummy);
+    ok = ok && run_chain<OP_FMA2_F64>(sms, iters, sink, clk, st, &out->fma_f32x2_with_f64_per_clk_sm, &dummy);
     // the clock the chains ran at: results per second / (results per clock per SM * SMs)
     if (ok && out->ex2_per_clk_sm > 0.0) out->sm_clock_mhz = out->ex2_gops * 1e3 / (out->ex2_per_clk_sm * sms);
     out->num_sms = sms;
