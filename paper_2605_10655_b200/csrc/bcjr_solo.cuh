@@ -306,8 +306,21 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                 ni = wrap ? 0 : ni + 1;
                 nleft -= more ? 1u : 0u;
             };
+            // RD == BPT (k = 2): the ring slot of a butterfly is its index in the step, and everything about a request is
+            // known at compile time but the step
+            constexpr bool STATIC_RING = RD == BPT;
+            constexpr ptrdiff_t HROW = (ptrdiff_t)BPT * NCH * CT;
+            auto issue_static = [&](const float4 *row, int i) {           // butterfly i of the step whose history starts at row
+                const uint32_t dst = stage_u32 + (uint32_t)i * (uint32_t)(NCH * CT * 16);
 #pragma unroll
-            for (uint32_t c = 0; c + 1 < RD; ++c) issue_chunk(c);
+                for (int q = 0; q < NCH; ++q)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(q * CT * 16)), "l"(row + (i * NCH + q) * CT) : "memory");
+            };
+#pragma unroll
+            for (uint32_t c = 0; c + 1 < RD; ++c) {
+                if (STATIC_RING) { issue_static(hist4 + (size_t)(n - 1) * HROW, (int)c); asm volatile("cp.async.commit_group;" ::: "memory"); }
+                else issue_chunk(c);
+            }
             uint32_t chunk = 0, slot = 0;
             compute_barrier(CT);
             auto beta_sweep = [&](auto rc_tag) {
@@ -341,12 +354,20 @@ __global__ void __launch_bounds__(SoloCfg<KB>::THREADS, 1) fwd_solo_kernel(FwdPa
                 tmem_ld16(tm, cb[0]);
 #pragma unroll
                 for (int i = 0; i < BPT; ++i, ++chunk) {
-                    issue_chunk(slot == 0 ? RD - 1 : slot - 1);      // refill the slot consumed last
+                    if (STATIC_RING) {                               // RD - 1 butterflies ahead, into the slot consumed last
+                        const float4 *hrow = hist4 + (size_t)(t - 1) * HROW;
+                        if (i == 0) issue_static(hrow, BPT - 1);
+                        else if (t > 1) issue_static(hrow - HROW, i - 1);
+                        asm volatile("cp.async.commit_group;" ::: "memory");
+                    } else {
+                        issue_chunk(slot == 0 ? RD - 1 : slot - 1);  // refill the slot consumed last
+                    }
                     asm volatile("cp.async.wait_group %0;" ::"n"(RD - 1) : "memory"); // chunk `chunk` has landed
+                    const uint32_t sl = STATIC_RING ? (uint32_t)i : slot;
                     float Lh[K];
 #pragma unroll
                     for (int q = 0; q < NCH; ++q) {
-                        const float4 l4 = stage4[(slot * NCH + q) * CT + tid];
+                        const float4 l4 = stage4[(sl * NCH + q) * CT + tid];
                         Lh[4 * q] = l4.x; Lh[4 * q + 1] = l4.y; Lh[4 * q + 2] = l4.z; Lh[4 * q + 3] = l4.w;
                     }
                     slot = slot + 1 == RD ? 0 : slot + 1;
