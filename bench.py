@@ -100,15 +100,15 @@ class ClockSampler:
                 "power_w_max": max(float(r[3]) for r in rows), "samples": len(rows), "reasons": sorted(reasons)}
 
 
-def cpu_baseline(wl, seconds_hint: float = 20.0):
+def cpu_baseline(wl, blocks_per_core: int = 4):
     """The float64 oracle, as it stands, on the host cores: forward + backward of a bounded
-    sample of blocks of the same workload (one block per core)."""
+    sample of blocks of the same workload (blocks_per_core blocks per core)."""
     import oracle
     cores = oracle.host_cores()
     # ~5 core-seconds per block at S = 2^16, n = 256 (forward + backward); four blocks per core
     # keep the sample near 20 s; smaller trellises take proportionally more blocks
     scale = max(1, int((1 << 16) * 256 / (wl.S * wl.n)))
-    nblk = max(1, min(wl.num_blocks(), 4 * cores * min(scale, 64)))
+    nblk = max(1, min(wl.num_blocks(), blocks_per_core * cores * min(scale, 64)))
     W, c, g = wl.weights(0)[:nblk], wl.codebook(), wl.upstream(0)[:nblk]
     t0 = time.time()
     if wl.V == 1:
@@ -133,8 +133,10 @@ def run_reference(args, wl):
     for _ in range(args.warmup):
         pass                                    # the oracle has no warm-up state
     base = None
-    for _ in range(max(1, args.steps)):
-        base, dt = cpu_baseline(wl)
+    steps = max(1, args.steps)
+    per_core = 4 if steps <= 6 else 2 if steps <= 12 else 1    # keeps the whole run near two minutes (~5 core-seconds per block)
+    for _ in range(steps):
+        base, dt = cpu_baseline(wl, per_core)
         vals.append((base["value"], dt))
     value = float(np.mean([v for v, _ in vals]))
     base["value"] = value
