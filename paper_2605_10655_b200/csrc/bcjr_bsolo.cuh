@@ -113,8 +113,8 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
             int r = 0;                                                // k (t - 1) mod (Lb - k)
             for (int t = 1; t <= n; ++t) {
                 const int cur = (t - 1) & 1;
-                float2 cb[2][8];
-                tmem_ld16(tm, cb[0]);
+                float2 cb[8];
+                tmem_ld16(tm, cb);
                 const float gt = __ldg(g_s + t - 1), wt = __ldg(w_s + t - 1);
                 const float gshn = t < n ? -__ldg(g_s + t) * __ldg(sf_s + t) : 0.f;
                 if (t > 1) {
@@ -141,30 +141,30 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
                     }
                     hrow[(i * NCH) * CT] = make_float4(Lj[0], Lj[1], Lj[2], Lj[3]);
                     hrow[(i * NCH + 1) * CT] = make_float4(Aj[0], Aj[1], Aj[2], Aj[3]);
-                    tmem_wait_ld(cb[i & 1]);
-                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
+                    tmem_wait_ld(cb);
                     float2 outL[K / 2], outA[K / 2];
 #pragma unroll
                     for (int h = 0; h < K / 2; ++h) {
                         float2 a[K];
 #pragma unroll
                         for (int j = 0; j < K; ++j) {
-                            const float2 du = sub2(cb[i & 1][C::a_idx(j, h)], w2);
+                            const float2 du = sub2(cb[C::a_idx(j, h)], w2);
                             a[j] = RC ? energy2(du, nl2, kap2, splat2(Lj[j])) : fma2(mul2(du, du), nl2, splat2(Lj[j]));
                         }
                         const float2 m = max_pairs<K>(a);
                         float2 pj = ex2f2(sub2(a[0], m));
-                        float2 sum = pj, ax = mul2(pj, fma2(g2, cb[i & 1][C::a_idx(0, h)], splat2(Aj[0])));
+                        float2 sum = pj, ax = mul2(pj, fma2(g2, cb[C::a_idx(0, h)], splat2(Aj[0])));
 #pragma unroll
                         for (int j = 1; j < K; ++j) {
                             pj = ex2f2(sub2(a[j], m));
                             sum = add2(sum, pj);
-                            ax = fma2(pj, fma2(g2, cb[i & 1][C::a_idx(j, h)], splat2(Aj[j])), ax);
+                            ax = fma2(pj, fma2(g2, cb[C::a_idx(j, h)], splat2(Aj[j])), ax);
                         }
                         outL[h] = add2(sub2(m, off2), lg2f2(sum));
                         outA[h] = fma2(ax, rcpf2(sum), gshn2);
                         tmax = max3f(tmax, m.x, m.y);
                     }
+                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb);
                     // output [x|l] takes the place of input [l|x]
 #pragma unroll
                     for (int h = 0; h < K / 2; ++h) {
@@ -234,8 +234,8 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
             int rr = 0;                                               // -k (n - t) mod (Lb - k)
             for (int t = n; t >= 1; --t) {
                 const int par = t & 1;
-                float2 cb[2][8];
-                tmem_ld16(tm, cb[0]);
+                float2 cb[8];                                     // one set of table registers (see bcjr_skew.cuh)
+                tmem_ld16(tm, cb);
                 const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1);
                 const float gsh = -gt * __ldg(sf_s + t - 1);                      // shift carried by the stored At
                 const float gshp = t > 1 ? -__ldg(g_s + t - 2) * __ldg(sf_s + t - 2) : 0.f;   // for step t-1
@@ -280,15 +280,14 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
                         Mb[b] = Ms[ti ^ TB[b]];
                         Yb[b] = Bs[ti ^ TB[b]];
                     }
-                    tmem_wait_ld(cb[i & 1]);
-                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb[(i + 1) & 1]);
+                    tmem_wait_ld(cb);
                     float2 outM[K / 2], outB[K / 2];
 #pragma unroll
                     for (int jh = 0; jh < K / 2; ++jh) {
                         float2 uu[K], d[K];
 #pragma unroll
                         for (int b = 0; b < K; ++b) {
-                            d[b] = sub2(cb[i & 1][C::b_idx(jh, b)], w2);              // du = c - wc
+                            d[b] = sub2(cb[C::b_idx(jh, b)], w2);              // du = c - wc
                             uu[b] = RC ? energy2(d[b], nl2, kap2, splat2(Mb[b])) : fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
                         }
                         const float2 m = max_pairs<K>(uu);
@@ -302,7 +301,7 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
 #pragma unroll
                         for (int b = 0; b < K; ++b) {
                             const float2 pb = ex2f2(sub2(uu[b], m));
-                            const float2 y = fma2(g2, cb[i & 1][C::b_idx(jh, b)], splat2(Yb[b]));   // h + Bt
+                            const float2 y = fma2(g2, cb[C::b_idx(jh, b)], splat2(Yb[b]));   // h + Bt
                             const float2 z = RC ? fma2(fma2(nfi, d[b], fid), add2(y, Ahj), fg) : fma2(d[b], fma2(nfi, y, nfiA), fg);   // f (g + (w - c) r / T)
                             sum = add2(sum, pb);
                             ya = fma2(pb, y, ya);
@@ -315,6 +314,7 @@ __global__ void __launch_bounds__(BSoloCfg::THREADS, 1) bwd_solo_kernel(BwdParam
                         S2 = fma2(f, fma2(Ahj, sum, ya), S2);
                         ZS = add2(ZS, zs);
                     }
+                    if (i + 1 < BPT) tmem_ld16(tm + 16u * (i + 1), cb);
                     // output [j|x] takes the place of input [x|j]
 #pragma unroll
                     for (int jh = 0; jh < K / 2; ++jh) {

@@ -59,7 +59,8 @@ struct SkewCfg {
     static constexpr int OFF_MBAR = OFF_LZ + 32;               // uint64: early[2], late[2]
     static constexpr int OFF_TMEM = OFF_MBAR + 8;
     static constexpr int OFF_FLAG = OFF_TMEM + 2;
-    static constexpr int SMEM_FLOATS = OFF_FLAG + 2;
+    static constexpr int OFF_PUSH = OFF_FLAG + 2;              // uint32 [2 BPT][THREADS]: beta push addresses of every thread and slot
+    static constexpr int SMEM_FLOATS = OFF_PUSH + 2 * BPT * THREADS;
     static constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * 4;
     static_assert(OFF_MBAR % 2 == 0, "mbarrier alignment");
     static_assert(BPT == 4 && K == 4, "slot scheme is written for four butterflies of sixteen states per thread");
@@ -161,8 +162,13 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
             const uint32_t ar = msg_u32 + (uint32_t)(((bin >> 1) * PLANE + C::slot_of(xr) * CT + C::tid_of(xr)) * 4 + (bin & 1) * 2) * 4u;
             push_bl[i] = al;
             push_br[i] = mapa_u32(ar, peer);
+            if (BETA_ONLY) {
+                reinterpret_cast<uint32_t *>(smem + C::OFF_PUSH)[(2 * i) * CT + tid] = push_bl[i];
+                reinterpret_cast<uint32_t *>(smem + C::OFF_PUSH)[(2 * i + 1) * CT + tid] = push_br[i];
+            }
         }
     }
+    const uint32_t *pushtab = reinterpret_cast<const uint32_t *>(smem + C::OFF_PUSH) + tid;
     constexpr uint32_t BL_STEP = CT * 16u, BR_STEP = 256u * 16u;     // j0 = 1: next slot (own CTA) / upper half of the threads (peer)
     uint32_t wmax_dst[CL], lz_dst[CL];
 #pragma unroll
@@ -378,8 +384,10 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
         constexpr bool RC = decltype(rc_tag)::value;
         for (int t = n; t >= 1 && !dead; --t) {
             const int ob = ib ^ 1;
-            float2 cb[2][8];
-            tmem_ld16(tm_cb + 16u * ORD_B0, cb[0]);
+            // one set of table registers: the next butterfly's entries are requested when this one's arithmetic is done
+            // (a second set, loaded a butterfly ahead, costs sixteen registers the scheduler makes better use of: 11.74 -> 11.63 ms)
+            float2 cb[8];
+            tmem_ld16(tm_cb + 16u * ORD_B0, cb);
             const float wt = __ldg(w_s + t - 1), gt = __ldg(g_s + t - 1);
             const float gsh = -gt * __ldg(sf_s + t - 1);                      // shift carried by the stored At
             const float gshp = t > 1 ? -__ldg(g_s + t - 2) * __ldg(sf_s + t - 2) : 0.f;   // for step t-1
@@ -387,7 +395,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
             asm volatile("cp.async.wait_group 0;" ::: "memory");    // this step's history, requested during the previous step
             hsrc -= t > 1 ? HSTEP : 0;                              // next requests: step t - 1 (at t = 1: step 1 again, unread)
             if (t < n) wait_early(ib);
-            if (!pr.warp_live()) { tmem_wait_ld(cb[0]); dead = true; break; }
+            if (!pr.warp_live()) { tmem_wait_ld(cb); dead = true; break; }
             P += (int)offM;                                         // offsets carried by this step's inputs M_t
             const float4 *MBin = reinterpret_cast<const float4 *>(msg + ib * C::BUF);
             const uint32_t ob_off = (uint32_t)ob * BUF_BYTES, ob_mbar = 8u * ob;
@@ -421,9 +429,8 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                     Mb[2 * e] = v.x; Yb[2 * e] = v.y; Mb[2 * e + 1] = v.z; Yb[2 * e + 1] = v.w;
                 }
                 float2 acc[8];
-                tmem_wait_ld(cb[pos & 1]);
+                tmem_wait_ld(cb);
                 if (ACC) tmem_ld16(tm_acc + 16u * i, acc);
-                if (pos + 1 < BPT) tmem_ld16(tm_cb + 16u * inext, cb[(pos + 1) & 1]);
                 bool acc_ready = !ACC;
                 float2 outM[K / 2], outB[K / 2];
 #pragma unroll
@@ -431,7 +438,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                     float2 uu[K], d[K];
 #pragma unroll
                     for (int b = 0; b < K; ++b) {
-                        d[b] = sub2(cb[pos & 1][C::b_idx(jh, b)], w2);              // du = c - wc
+                        d[b] = sub2(cb[C::b_idx(jh, b)], w2);              // du = c - wc
                         uu[b] = RC ? energy2(d[b], nl2, kap2, splat2(Mb[b])) : fma2(mul2(d[b], d[b]), nl2, splat2(Mb[b]));
                     }
                     const float2 m = max_pairs<K>(uu);
@@ -446,7 +453,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
 #pragma unroll
                     for (int b = 0; b < K; ++b) {
                         const float2 pb = ex2f2(sub2(uu[b], m));
-                        const float2 y = fma2(g2, cb[pos & 1][C::b_idx(jh, b)], splat2(Yb[b]));   // h + Bt
+                        const float2 y = fma2(g2, cb[C::b_idx(jh, b)], splat2(Yb[b]));   // h + Bt
                         const float2 z = RC ? fma2(fma2(nfi, d[b], fid), add2(y, Ahj), fg) : fma2(d[b], fma2(nfi, y, nfiA), fg);   // f (g + (w - c) r / T)
                         sum = add2(sum, pb);
                         ya = fma2(pb, y, ya);
@@ -471,17 +478,20 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                     }
                     if (!pr.warp_live()) { dead = true; break; }
                 }
+                if (pos + 1 < BPT) tmem_ld16(tm_cb + 16u * inext, cb);
                 // outputs j = 2 jh, 2 jh + 1 go to CTA jh: own CTA by plain stores, the peer by st.async
                 const uint32_t mbp = (pos == BPT - 1 ? peer_late : peer_early) + ob_mbar;
 #pragma unroll
                 for (int jh = 0; jh < K / 2; ++jh) {
                     const float2 oM = sub2(outM[jh], offM2);
                     if (jh == (int)rank) {
-                        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(push_bl[i] + ob_off), "f"(oM.x), "f"(outB[jh].x) : "memory");
-                        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(push_bl[i] + ob_off + BL_STEP), "f"(oM.y), "f"(outB[jh].y) : "memory");
+                        const uint32_t pl = (BETA_ONLY ? pushtab[(2 * i) * CT] : push_bl[i]) + ob_off;
+                        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(pl), "f"(oM.x), "f"(outB[jh].x) : "memory");
+                        asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(pl + BL_STEP), "f"(oM.y), "f"(outB[jh].y) : "memory");
                     } else {
-                        st_async_v2(push_br[i] + ob_off, oM.x, outB[jh].x, mbp);
-                        st_async_v2(push_br[i] + ob_off + BR_STEP, oM.y, outB[jh].y, mbp);
+                        const uint32_t prm = (BETA_ONLY ? pushtab[(2 * i + 1) * CT] : push_br[i]) + ob_off;
+                        st_async_v2(prm, oM.x, outB[jh].x, mbp);
+                        st_async_v2(prm + BR_STEP, oM.y, outB[jh].y, mbp);
                     }
                 }
                 if (pos == BPT - 2) {                             // "early" also counts the local warps (its arrival count is fixed)
@@ -489,7 +499,7 @@ __global__ void __launch_bounds__(SkewCfg::THREADS, 1) bwd_skew_kernel(BwdParams
                     if (lane == 0) mbar_arrive_local(mb_early + ob_mbar);
                 }
             }
-            if (dead) { tmem_wait_ld(cb[0]); tmem_wait_ld(cb[1]); break; }
+            if (dead) { tmem_wait_ld(cb); break; }
             if (ACC) tmem_wait_st();
             tmax = warp_max(tmax) - offM;
             if (lane == 0) {
